@@ -1,0 +1,520 @@
+"""CPU oracle for the DREAM draft-and-verify loop.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, step-by-step implementation of what the hot path computes,
+written from the paper's method section with plain PyTorch CPU tensor ops
+(matmul, softmax, sort are used as library steps; no blocking, no fusion).
+It shares no code with the CUDA path and imports nothing from it.  Only the
+tests, the smoke check and the benchmark's CPU-baseline leg may call it.
+
+Precision: `dtype` is the arithmetic and activation/KV storage type.  float64 is
+used for the pins and the toy model; float32 is used for the bf16 model shapes
+(weights are taken as given, i.e. bf16-rounded values, and up-converted).
+
+Readings taken where the paper is silent (each is listed in the design notes):
+pre-norm decoder blocks with RMSNorm, rotary positions (half-split pairing) on
+self-attention only, gated SiLU MLP, no biases, softmax scale 1/sqrt(head_dim),
+grouped KV heads, causal mask in the entropy and importance sums, natural log,
+ties broken toward the lower index everywhere.
+
+Paper anchors: Section 2.1 (draft-then-verify, acceptance), Section 3.1 and
+Eq. 1 (cross-attention fusion, growing key/value memory, tree drafting),
+Section 3.2 and Eq. 2 (average attention entropy, layer selection),
+Section 3.3 (visual-token importance and top-k subsampling), Section 4 setup
+(tree depth/width, bonus token, KV caching).
+
+Parity unpinned: acceptance length tau and speedup S (need trained weights).
+
+Weight layout: every matrix is [out_features, in_features]; wqkv stacks the
+query/key/value projections by rows, wgu stacks gate then up, xkv stacks the
+cross-attention key then value projections.
+"""
+from dataclasses import dataclass, field
+import math
+import torch
+
+TAP_FIXED, TAP_ENTROPY_MIN, TAP_ENTROPY_MAX = 0, 1, 2
+
+
+@dataclass
+class OracleConfig:
+    n_layers: int
+    d_model: int
+    n_heads: int
+    n_kv_heads: int
+    head_dim: int
+    d_ff: int
+    vocab: int
+    rms_eps: float = 1e-5
+    rope_theta: float = 10000.0
+    tree_depth: int = 3
+    tree_topk: int = 2
+    tree_beam: int = 2
+    tree_max_nodes: int = 14
+    tap_mode: int = TAP_FIXED
+    tap_layer: int = 1          # 1-based: S^l is the residual stream after block l
+    tap_lo: int = 1
+    tap_hi: int = 1
+    score_include_self: int = 0
+    xattn_full_memory: int = 0
+
+    @staticmethod
+    def from_preset(p):
+        names = ("n_layers d_model n_heads n_kv_heads head_dim d_ff vocab rms_eps rope_theta "
+                 "tree_depth tree_topk tree_beam tree_max_nodes tap_mode tap_layer tap_lo tap_hi "
+                 "score_include_self xattn_full_memory").split()
+        return OracleConfig(**{k: p[k] for k in names})
+
+
+# --------------------------------------------------------------------------- primitives
+
+def rmsnorm(x, g, eps):
+    """x * g / sqrt(mean(x^2) + eps) over the last axis."""
+    ms = (x * x).mean(dim=-1, keepdim=True)
+    return x / torch.sqrt(ms + eps) * g.to(x.dtype)
+
+
+def rope(x, pos, theta):
+    """Rotary position embedding on x [rows, heads, hd] at integer positions pos [rows].
+
+    Pair (i, i + hd/2) is rotated by the angle pos * theta^(-2i/hd).
+    """
+    hd = x.shape[-1]
+    half = hd // 2
+    i = torch.arange(half, dtype=torch.float64)
+    inv = theta ** (-2.0 * i / hd)
+    ang = pos.to(torch.float64)[:, None] * inv[None, :]
+    c = torch.cos(ang).to(x.dtype)[:, None, :]
+    s = torch.sin(ang).to(x.dtype)[:, None, :]
+    a, b = x[..., :half], x[..., half:]
+    return torch.cat([a * c - b * s, b * c + a * s], dim=-1)
+
+
+def linear(x, w):
+    """x [rows, in] times W^T for W [out, in]."""
+    return x @ w.to(x.dtype).t()
+
+
+def attention(q, K, V, mask):
+    """softmax(q K^T / sqrt(hd)) V with a boolean mask (Eq. 1 with several heads).
+
+    q [m, H, hd]; K, V [r, Hkv, hd]; mask [m, r] True = visible.  Query head h reads
+    KV head h // (H / Hkv).  Returns (out [m, H*hd], probs [H, m, r]).
+    """
+    m, H, hd = q.shape
+    Hkv = K.shape[1]
+    g = H // Hkv
+    outs, probs = [], []
+    for h in range(H):
+        kh, vh = K[:, h // g, :], V[:, h // g, :]
+        s = (q[:, h, :] @ kh.t()) / math.sqrt(hd)
+        s = s.masked_fill(~mask, float("-inf"))
+        p = torch.softmax(s, dim=-1)
+        outs.append(p @ vh)
+        probs.append(p)
+    return torch.cat(outs, dim=-1), torch.stack(probs, 0)
+
+
+def mlp(b, wgu, wd, ff):
+    gu = linear(b, wgu)
+    gate, up = gu[:, :ff], gu[:, ff:]
+    return linear(torch.nn.functional.silu(gate) * up, wd)
+
+
+def row_entropy(p):
+    """-sum_j p_j ln p_j per row with 0 ln 0 = 0 (inner sum of Eq. 2)."""
+    t = torch.where(p > 0, p * torch.log(torch.where(p > 0, p, torch.ones_like(p))),
+                    torch.zeros_like(p))
+    return -t.sum(dim=-1)
+
+
+def argmax_low(x):
+    """Index of the maximum, ties to the lower index; also the top-1 minus top-2 margin."""
+    v, i = torch.sort(x, descending=True, stable=True)
+    return int(i[0]), float(v[0] - v[1]) if x.numel() > 1 else float("inf")
+
+
+def topk_low(x, k):
+    """The k largest entries, ties to the lower index, in descending order."""
+    v, i = torch.sort(x, descending=True, stable=True)
+    return v[:k], i[:k]
+
+
+# --------------------------------------------------------------------------- state
+
+@dataclass
+class SeqState:
+    """Everything the loop keeps for one sequence."""
+    K: list = field(default_factory=list)       # per target layer [rows, Hkv, hd]
+    V: list = field(default_factory=list)
+    P: int = 0                                  # verified length: positions 0..P-1 are in K/V
+    pending: int = -1                           # token at position P, not yet run through the target
+    n_prompt_total: int = 0                     # n = q + v
+    taps: dict = field(default_factory=dict)    # layer -> S^layer over the prompt [n, d]
+    x0: torch.Tensor = None                     # input embeddings of the prompt [n, d]
+    entropy: torch.Tensor = None                # AE per layer [L]
+    scores: dict = field(default_factory=dict)  # layer -> importance of visual tokens [v]
+    vis_start: int = 0
+    n_visual: int = 0
+    tap: int = 0                                # selected layer l*
+    kept: torch.Tensor = None                   # kept visual indices, ascending, relative to vis_start
+    ctx_pos: torch.Tensor = None                # positions of the compressed context C
+    dK: torch.Tensor = None                     # draft self-attention K rows [rows, Hkv, hd]
+    dV: torch.Tensor = None
+    mK: torch.Tensor = None                     # cross-attention memory K rows
+    mV: torch.Tensor = None
+    new_tokens: list = field(default_factory=list)   # tokens verified since the last draft call
+    new_pos: list = field(default_factory=list)
+
+
+class DreamOracle:
+    def __init__(self, cfg, tw, dw, dtype=torch.float64):
+        self.cfg, self.tw, self.dw, self.dtype = cfg, tw, dw, dtype
+
+    # ------------------------------------------------------------------ target block
+    def _block(self, x, l, pos, Kc, Vc, mask, want_probs=False):
+        """One pre-norm decoder block of the target on rows x at positions pos.
+
+        Kc/Vc are the cached rows visible to these queries (may be empty); the new
+        rows' K/V are appended after them and mask [m, cached + m] covers both.
+        """
+        c, w = self.cfg, self.tw
+        H, Hkv, hd = c.n_heads, c.n_kv_heads, c.head_dim
+        a = rmsnorm(x, w["ln1"][l], c.rms_eps)
+        qkv = linear(a, w["wqkv"][l])
+        q = qkv[:, :H * hd].reshape(-1, H, hd)
+        k = qkv[:, H * hd:(H + Hkv) * hd].reshape(-1, Hkv, hd)
+        v = qkv[:, (H + Hkv) * hd:].reshape(-1, Hkv, hd)
+        q, k = rope(q, pos, c.rope_theta), rope(k, pos, c.rope_theta)
+        Kall = torch.cat([Kc, k], 0) if Kc is not None and Kc.shape[0] else k
+        Vall = torch.cat([Vc, v], 0) if Vc is not None and Vc.shape[0] else v
+        o, probs = attention(q, Kall, Vall, mask)
+        x = x + linear(o, w["wo"][l])
+        b = rmsnorm(x, w["ln2"][l], c.rms_eps)
+        x = x + mlp(b, w["wgu"][l], w["wd"][l], c.d_ff)
+        return x, k, v, (probs if want_probs else None)
+
+    def _logits(self, x):
+        return linear(rmsnorm(x, self.tw["ln_f"], self.cfg.rms_eps), self.tw["lm_head"])
+
+    def embed_rows(self, ids):
+        return self.tw["embed"][torch.as_tensor(ids, dtype=torch.long)].to(self.dtype)
+
+    # ------------------------------------------------------------------ O1 + O2 + scores
+    def prefill(self, visual, vis_start, ids, extra_ids=(), keep_all_taps=False):
+        """Causal forward of the n = q + v prompt tokens (Section 3, inference).
+
+        The sequence holds the visual embeddings at [vis_start, vis_start+v) and
+        embed[id] elsewhere; `extra_ids` are further text tokens appended at the end.
+        Keeps per-layer K/V, S^l for every layer, the per-layer average attention
+        entropy (Eq. 2) and, per layer, the importance of each visual token
+        (Section 3.3).  Returns the state and (first token, margin).
+        """
+        c = self.cfg
+        ids = [int(t) for t in ids] + [int(t) for t in extra_ids]
+        v = visual.shape[0]
+        n = v + len(ids)
+        x = torch.empty(n, c.d_model, dtype=self.dtype)
+        emb = self.embed_rows(ids) if ids else torch.empty(0, c.d_model, dtype=self.dtype)
+        x[:vis_start] = emb[:vis_start]
+        x[vis_start:vis_start + v] = visual.to(self.dtype)
+        x[vis_start + v:] = emb[vis_start:]
+        st = SeqState(P=n, n_prompt_total=n, vis_start=vis_start, n_visual=v, x0=x.clone())
+        pos = torch.arange(n)
+        causal = torch.ones(n, n, dtype=torch.bool).tril()
+        ent = torch.zeros(c.n_layers, dtype=torch.float64)
+        for l in range(c.n_layers):
+            x, k, vv, probs = self._block(x, l, pos, None, None, causal, want_probs=True)
+            st.K.append(k)
+            st.V.append(vv)
+            if keep_all_taps or c.tap_mode != TAP_FIXED and c.tap_lo <= l + 1 <= c.tap_hi \
+                    or c.tap_mode == TAP_FIXED and l + 1 == c.tap_layer:
+                st.taps[l + 1] = x.clone()
+            ent[l] = row_entropy(probs).to(torch.float64).mean()       # mean over rows and heads
+            col = probs.sum(dim=0)                                      # sum over heads [n, n]
+            if not c.score_include_self:
+                col = col - torch.diag(torch.diagonal(col))
+            st.scores[l + 1] = col.sum(dim=0)[vis_start:vis_start + v].clone()
+        st.entropy = ent
+        tok, margin = argmax_low(self._logits(x[n - 1:n])[0])
+        st.pending = tok
+        st.tap, st.tap_margin = self.select_tap(ent)
+        self._last_hidden = x
+        return st, tok, margin
+
+    # ------------------------------------------------------------------ O3
+    def select_tap(self, ent):
+        """l* = argmin (or argmax) of AE over [tap_lo, tap_hi], ties to the lower layer."""
+        c = self.cfg
+        if c.tap_mode == TAP_FIXED:
+            return c.tap_layer, float("inf")
+        e = ent[c.tap_lo - 1:c.tap_hi].clone()
+        if c.tap_mode == TAP_ENTROPY_MIN:
+            e = -e
+        i, margin = argmax_low(e)
+        return c.tap_lo + i, margin
+
+    # ------------------------------------------------------------------ O4 + O5
+    def compress_visual(self, st, k, forced_idx=None):
+        """Keep the k most important visual tokens and build the draft's context.
+
+        Importance of visual token j = attention it receives from later tokens at
+        layer l*, summed over heads (Section 3.3).  The compressed context C is the
+        kept visual positions plus every text position, ascending.  Draft
+        self-attention K/V rows come from the input embeddings at C with rotary
+        angles of the original positions; cross-attention memory rows are
+        S^{l*}_c W_K, S^{l*}_c W_V (Eq. 1, no norm on the memory side).
+        Returns (kept indices ascending, scores, margin at the cut).
+        """
+        c, dw = self.cfg, self.dw
+        sc = st.scores[st.tap]
+        v = st.n_visual
+        if forced_idx is None:
+            vals, idx = topk_low(sc, k)
+            margin = float("inf")
+            if k < v:
+                allv, _ = torch.sort(sc, descending=True, stable=True)
+                margin = float(allv[k - 1] - allv[k])
+            kept = torch.sort(idx).values
+        else:
+            kept, margin = torch.as_tensor(forced_idx, dtype=torch.long), float("inf")
+        st.kept = kept
+        n = st.n_prompt_total
+        is_vis = torch.zeros(n, dtype=torch.bool)
+        is_vis[st.vis_start:st.vis_start + v] = True
+        keep = ~is_vis
+        keep[st.vis_start + kept] = True
+        C = torch.nonzero(keep).flatten()
+        st.ctx_pos = C
+        Hkv, hd, H = c.n_kv_heads, c.head_dim, c.n_heads
+        a = rmsnorm(st.x0[C], dw["ln1"], c.rms_eps)
+        qkv = linear(a, dw["wqkv"])
+        kk = qkv[:, H * hd:(H + Hkv) * hd].reshape(-1, Hkv, hd)
+        vv = qkv[:, (H + Hkv) * hd:].reshape(-1, Hkv, hd)
+        st.dK, st.dV = rope(kk, C, c.rope_theta), vv
+        M = torch.arange(n) if c.xattn_full_memory else C
+        S = st.taps[st.tap][M]
+        kv = linear(S, dw["xkv"])
+        st.mK = kv[:, :Hkv * hd].reshape(-1, Hkv, hd)
+        st.mV = kv[:, Hkv * hd:].reshape(-1, Hkv, hd)
+        st.new_tokens, st.new_pos = [], []
+        return kept, sc, margin
+
+    # ------------------------------------------------------------------ O6
+    def _draft_rows(self, st, toks, pos):
+        """Draft self-attention q, k, v of tokens at given positions (from embeddings)."""
+        c, dw = self.cfg, self.dw
+        H, Hkv, hd = c.n_heads, c.n_kv_heads, c.head_dim
+        x = self.embed_rows(toks)
+        a = rmsnorm(x, dw["ln1"], c.rms_eps)
+        qkv = linear(a, dw["wqkv"])
+        p = torch.as_tensor(pos, dtype=torch.long)
+        q = rope(qkv[:, :H * hd].reshape(-1, H, hd), p, c.rope_theta)
+        k = rope(qkv[:, H * hd:(H + Hkv) * hd].reshape(-1, Hkv, hd), p, c.rope_theta)
+        v = qkv[:, (H + Hkv) * hd:].reshape(-1, Hkv, hd)
+        return x, q, k, v
+
+    def draft_tree(self, st):
+        """Expand the draft token tree from the pending token (Section 3.1, tree drafting).
+
+        Returns a dict with tokens, parent, depth, mask (list of ancestor-or-self sets),
+        cum (cumulative log-probability), and the decision margins met on the way.
+        """
+        c, dw = self.cfg, self.dw
+        H, Hkv, hd, D, K = c.n_heads, c.n_kv_heads, c.head_dim, c.tree_depth, c.tree_topk
+        # tokens verified by the last accept get their permanent draft self-attention rows
+        if st.new_tokens:
+            _, _, k, v = self._draft_rows(st, st.new_tokens, st.new_pos)
+            st.dK, st.dV = torch.cat([st.dK, k], 0), torch.cat([st.dV, v], 0)
+            st.new_tokens, st.new_pos = [], []
+        P = st.P
+        nK, nM = st.dK.shape[0], st.mK.shape[0]
+        # input nodes of the draft: each has a row in the tree regions of both caches
+        in_tok, in_depth, in_anc, in_cum, in_cand = [st.pending], [0], [[0]], [0.0], [-1]
+        tK = torch.empty(0, Hkv, hd, dtype=self.dtype)
+        tV, tmK, tmV = tK.clone(), tK.clone(), tK.clone()
+        cands = []            # (token, parent candidate index or -1 for the root, depth, cum)
+        margins = []          # decision margins: top-K cut of a row, adjacent gaps, beam cut
+        feats, logp_rows = [], []
+        beam = [0]            # indices into in_* of the nodes this pass expands
+        cand_to_in = {}       # candidate index -> input-node index, for candidates that were expanded
+        for p in range(1, D + 1):
+            rows = beam
+            toks = [in_tok[r] for r in rows]
+            pos = [P + in_depth[r] for r in rows]
+            x, q, k, v = self._draft_rows(st, toks, pos)
+            tK, tV = torch.cat([tK, k], 0), torch.cat([tV, v], 0)
+            nt = tK.shape[0]
+            # self-attention: all permanent rows, plus own ancestors and self in the tree region
+            mask = torch.zeros(len(rows), nK + nt, dtype=torch.bool)
+            mask[:, :nK] = True
+            for i, r in enumerate(rows):
+                mask[i, [nK + a for a in in_anc[r]]] = True
+            o, _ = attention(q, torch.cat([st.dK, tK], 0), torch.cat([st.dV, tV], 0), mask)
+            h = x + linear(o, dw["wo"])
+            # cross-attention: verified memory rows plus strict ancestors' draft features
+            qx = linear(rmsnorm(h, dw["lnx"], c.rms_eps), dw["xq"]).reshape(-1, H, hd)
+            ntm = tmK.shape[0]
+            mask = torch.zeros(len(rows), nM + ntm, dtype=torch.bool)
+            mask[:, :nM] = True
+            for i, r in enumerate(rows):
+                mask[i, [nM + a for a in in_anc[r] if a != r]] = True
+            o, _ = attention(qx, torch.cat([st.mK, tmK], 0), torch.cat([st.mV, tmV], 0), mask)
+            h = h + linear(o, dw["xo"])
+            h = h + mlp(rmsnorm(h, dw["ln2"], c.rms_eps), dw["wgu"], dw["wd"], c.d_ff)
+            # e^M: the draft's final feature joins the memory (raw, unnormalised)
+            kv = linear(h, dw["xkv"])
+            tmK = torch.cat([tmK, kv[:, :Hkv * hd].reshape(-1, Hkv, hd)], 0)
+            tmV = torch.cat([tmV, kv[:, Hkv * hd:].reshape(-1, Hkv, hd)], 0)
+            logp = torch.log_softmax(self._logits(h), dim=-1)
+            new = []
+            for i, r in enumerate(rows):
+                feats.append(h[i].clone())
+                logp_rows.append(logp[i].clone())
+                sv, si = torch.sort(logp[i], descending=True, stable=True)
+                margins.append(float(sv[K - 1] - sv[K]))
+                margins.extend(float(sv[j] - sv[j + 1]) for j in range(K - 1))
+                for j in range(K):
+                    cands.append((int(si[j]), in_cand[r], in_depth[r] + 1, in_cum[r] + float(sv[j])))
+                    new.append(len(cands) - 1)
+            if p == D:
+                break
+            # next beam: the `beam` best new candidates by cumulative score
+            cs = torch.tensor([cands[i][3] for i in new], dtype=torch.float64)
+            nb = min(c.tree_beam, len(new))
+            sv, si = torch.sort(cs, descending=True, stable=True)
+            if nb < len(new):
+                margins.append(float(sv[nb - 1] - sv[nb]))
+            margins.extend(float(sv[j] - sv[j + 1]) for j in range(nb - 1))
+            beam = []
+            for j in range(nb):
+                ci = new[int(si[j])]
+                tok, par, dep, cum = cands[ci]
+                par_in = 0 if par < 0 else cand_to_in[par]
+                in_tok.append(tok); in_depth.append(dep); in_cum.append(cum); in_cand.append(ci)
+                in_anc.append(in_anc[par_in] + [len(in_tok) - 1])
+                beam.append(len(in_tok) - 1)
+                cand_to_in[ci] = len(in_tok) - 1
+        # global re-rank: the N best candidates, kept in creation order, root first
+        N = min(c.tree_max_nodes, len(cands))
+        cs = torch.tensor([cd[3] for cd in cands], dtype=torch.float64)
+        sv, si = torch.sort(cs, descending=True, stable=True)
+        if N < len(cands):
+            margins.append(float(sv[N - 1] - sv[N]))
+        chosen = sorted(int(i) for i in si[:N])
+        node_of = {ci: j + 1 for j, ci in enumerate(chosen)}
+        tokens, parent, depth, cum = [st.pending], [-1], [0], [0.0]
+        for ci in chosen:
+            tok, par, dep, cm = cands[ci]
+            tokens.append(tok); depth.append(dep); cum.append(cm)
+            parent.append(0 if par < 0 else node_of[par])
+        mask = [{0}]
+        for i in range(1, len(tokens)):
+            mask.append(mask[parent[i]] | {i})
+        return dict(tokens=tokens, parent=parent, depth=depth, mask=mask, cum=cum,
+                    margins=margins, min_margin=min(margins) if margins else float("inf"),
+                    cands=cands, feats=feats, logp_rows=logp_rows, in_tok=in_tok, in_depth=in_depth)
+
+    # ------------------------------------------------------------------ O7
+    def verify_tree(self, st, tree):
+        """Run the T tree tokens through the target with the tree mask (Section 3.1).
+
+        Node i sits at position P + depth_i, sees the verified prefix and the tail rows
+        of its ancestors and itself.  Returns logits, argmax, margins, per-layer tail
+        K/V and the tapped features of the tail.
+        """
+        c = self.cfg
+        T, P = len(tree["tokens"]), st.P
+        x = self.embed_rows(tree["tokens"])
+        pos = torch.tensor([P + dd for dd in tree["depth"]])
+        mask = torch.zeros(T, P + T, dtype=torch.bool)
+        mask[:, :P] = True
+        for i in range(T):
+            mask[i, [P + j for j in tree["mask"][i]]] = True
+        tailK, tailV, tap_rows = [], [], None
+        for l in range(c.n_layers):
+            x, k, v, _ = self._block(x, l, pos, st.K[l][:P], st.V[l][:P], mask)
+            tailK.append(k); tailV.append(v)
+            if l + 1 == st.tap:
+                tap_rows = x.clone()
+        logits = self._logits(x)
+        am, mg = zip(*(argmax_low(logits[i]) for i in range(T)))
+        return dict(logits=logits, argmax=list(am), margin=list(mg), tailK=tailK, tailV=tailV,
+                    tap_rows=tap_rows, hidden=x)
+
+    # ------------------------------------------------------------------ O8
+    @staticmethod
+    def accept(tree, argmax):
+        """Greedy acceptance: follow the child whose token equals the parent's argmax.
+
+        Returns (A, out_tokens [A+1], path [A+1]) where path[0] = 0 is the root and the
+        last emitted token is the target's own (bonus) token.
+        """
+        T = len(tree["tokens"])
+        cur, path, out = 0, [0], []
+        while True:
+            g = argmax[cur]
+            nxt = [i for i in range(T) if tree["parent"][i] == cur and tree["tokens"][i] == g]
+            if not nxt:
+                out.append(g)
+                return len(path) - 1, out, path
+            cur = nxt[0]
+            path.append(cur)
+            out.append(tree["tokens"][cur])
+
+    # ------------------------------------------------------------------ O9
+    def commit(self, st, tree, ver, path, out_tokens):
+        """Compact the target KV to the accepted path and extend the draft's caches."""
+        c, dw = self.cfg, self.dw
+        Hkv, hd = c.n_kv_heads, c.head_dim
+        P, A1 = st.P, len(path)
+        idx = torch.tensor(path)
+        for l in range(c.n_layers):
+            st.K[l] = torch.cat([st.K[l][:P], ver["tailK"][l][idx]], 0)
+            st.V[l] = torch.cat([st.V[l][:P], ver["tailV"][l][idx]], 0)
+        kv = linear(ver["tap_rows"][idx], dw["xkv"])
+        st.mK = torch.cat([st.mK, kv[:, :Hkv * hd].reshape(-1, Hkv, hd)], 0)
+        st.mV = torch.cat([st.mV, kv[:, Hkv * hd:].reshape(-1, Hkv, hd)], 0)
+        st.new_tokens = [tree["tokens"][i] for i in path]
+        st.new_pos = [P + j for j in range(A1)]
+        st.P = P + A1
+        st.pending = out_tokens[-1]
+        return path
+
+    def step(self, st, tree=None):
+        """One draft + verify + accept + commit round; `tree` overrides the draft's tree."""
+        drafted = self.draft_tree(st)
+        tree = drafted if tree is None else tree
+        ver = self.verify_tree(st, tree)
+        A, out, path = self.accept(tree, ver["argmax"])
+        self.commit(st, tree, ver, path, out)
+        return dict(tree=tree, drafted=drafted, ver=ver, A=A, out=out, path=path)
+
+    # ------------------------------------------------------------------ O10
+    def ar_decode(self, visual, vis_start, ids, n_new):
+        """Plain greedy autoregressive decoding of the target with its own KV cache."""
+        c = self.cfg
+        st, tok, _ = self.prefill(visual, vis_start, ids)
+        out, margins = [tok], []
+        Ks, Vs = [k.clone() for k in st.K], [v.clone() for v in st.V]
+        P = st.P
+        while len(out) < n_new:
+            x = self.embed_rows([out[-1]])
+            pos = torch.tensor([P])
+            for l in range(c.n_layers):
+                mask = torch.ones(1, P + 1, dtype=torch.bool)
+                x, k, v, _ = self._block(x, l, pos, Ks[l], Vs[l], mask)
+                Ks[l], Vs[l] = torch.cat([Ks[l], k], 0), torch.cat([Vs[l], v], 0)
+            P += 1
+            t, m = argmax_low(self._logits(x)[0])
+            out.append(t); margins.append(m)
+        return out, margins
+
+
+def make_tree(tokens, parent):
+    """Build a tree dict (depth, ancestor sets) from tokens and parent indices; node 0 is the root."""
+    depth, mask = [0], [{0}]
+    for i in range(1, len(tokens)):
+        depth.append(depth[parent[i]] + 1)
+        mask.append(mask[parent[i]] | {i})
+    return dict(tokens=list(tokens), parent=list(parent), depth=depth, mask=mask,
+                cum=[0.0] * len(tokens))
