@@ -1,0 +1,209 @@
+/*
+ * dream.h — C ABI of the DREAM draft-and-verify hot path for NVIDIA B200 (sm_100a).
+ *
+ * One library, one GPU, one CUDA stream per context.  The calls follow the paper's
+ * statement of the problem (DREAM, arXiv 2505.19201): a target VLM decoder M_ta with L
+ * blocks processes q text tokens and v visual tokens (Section 3); a one-layer draft
+ * model M_da cross-attends to cached target features over a compressed set of visual
+ * tokens (Section 3.1, Eq. 1; Section 3.3) and expands a token tree (Section 3.1, tree
+ * drafting); the target verifies the tree in one masked pass and the longest matching
+ * path is accepted (Section 2.1; Section 4, evaluation setup).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global-memory addresses valid on the context's device;
+ *     "host" pointers are ordinary process memory.  Every pointer says which it is.
+ *   - Every matrix is row-major [out_features, in_features] ("weight-stationary" layout:
+ *     one output feature is one contiguous row), element type = config.dtype.
+ *   - The library allocates nothing on the device: the caller passes one arena of
+ *     dream_arena_bytes() bytes to dream_init and owns it; weights and in/out buffers are
+ *     the caller's too and are only borrowed (weights for the context's lifetime).
+ *   - Calls enqueue work on the context's stream and return; outputs are device buffers
+ *     and are ready when the stream reaches that point.  Only dream_step_host and
+ *     dream_poll synchronise.
+ *   - Errors: argument and state checks happen on the host before anything is enqueued
+ *     and leave the context untouched; the code is returned and a message is kept for
+ *     dream_last_error.  Device-side anomalies (a bounded wait that expired, an index out
+ *     of range) never trap: they set a status word that dream_poll reports.
+ *   - Not thread-safe: one thread drives one context.
+ *   - Call order: dream_init -> per sequence { dream_prefill -> dream_compress_visual }
+ *     -> loop { dream_draft_tree -> dream_verify_tree -> dream_accept }.
+ */
+#ifndef DREAM_H_
+#define DREAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dream_ctx dream_ctx;
+typedef int32_t dream_status;
+
+enum {
+  DREAM_OK = 0,
+  DREAM_E_ARG = -1,            /* bad argument (null, out of range, misaligned) */
+  DREAM_E_STATE = -2,          /* call out of order for this sequence */
+  DREAM_E_NOMEM = -3,          /* arena too small */
+  DREAM_E_CAPACITY = -4,       /* sequence would outgrow max_seq / max_prompt / page pool */
+  DREAM_E_CUDA = -5,           /* a CUDA runtime or driver call failed */
+  DREAM_E_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired */
+  DREAM_E_UNSUPPORTED = -7     /* shape or dtype outside what the kernels handle */
+};
+enum { DREAM_F32 = 0, DREAM_BF16 = 1 };
+enum { DREAM_TAP_FIXED = 0, DREAM_TAP_ENTROPY_MIN = 1, DREAM_TAP_ENTROPY_MAX = 2 };
+
+/* Shapes and hyper-parameters; plain data, copied by dream_init. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ff, vocab;
+  int32_t dtype;                 /* DREAM_F32 or DREAM_BF16: weights, KV caches, GEMM inputs */
+  float rms_eps, rope_theta;
+  int32_t max_batch;             /* sequences resident at once */
+  int32_t max_seq;               /* verified tokens per sequence, upper bound */
+  int32_t max_prompt;            /* q + v upper bound for dream_prefill */
+  int32_t max_visual;            /* v upper bound */
+  int32_t page_tokens;           /* tokens per target-KV page (power of two, 16..256) */
+  int32_t tree_depth, tree_topk, tree_beam, tree_max_nodes;   /* D, K, beam width, N */
+  int32_t tap_mode, tap_layer, tap_lo, tap_hi;   /* 1-based layers; [lo,hi] = entropy search range */
+  int32_t score_include_self;    /* 1: a token's attention to itself counts in its importance */
+  int32_t xattn_full_memory;     /* 1: cross-attention memory keeps all n prompt positions */
+} dream_config;
+
+/* Target weights (device, borrowed).  Arrays of n_layers device pointers live on the HOST. */
+typedef struct {
+  const void *embed;             /* [vocab, d_model] */
+  const void *const *ln1;        /* each [d_model] */
+  const void *const *wqkv;       /* each [(n_heads + 2 n_kv_heads) head_dim, d_model]: Q rows, K rows, V rows */
+  const void *const *wo;         /* each [d_model, n_heads head_dim] */
+  const void *const *ln2;        /* each [d_model] */
+  const void *const *wgu;        /* each [2 d_ff, d_model]: gate rows then up rows */
+  const void *const *wd;         /* each [d_model, d_ff] */
+  const void *ln_f;              /* [d_model] */
+  const void *lm_head;           /* [vocab, d_model] */
+} dream_target_weights;
+
+/* Draft weights (device, borrowed): one layer = self-attention, cross-attention, MLP.
+ * The draft shares the target's embedding, final norm and LM head. */
+typedef struct {
+  const void *ln1, *wqkv, *wo;           /* self-attention, shapes as in the target */
+  const void *lnx, *xq, *xkv, *xo;       /* cross-attention (Eq. 1): xq [H hd, d], xkv [2 H_kv hd, d] (K rows then V rows), xo [d, H hd] */
+  const void *ln2, *wgu, *wd;            /* fusion MLP */
+} dream_draft_weights;
+
+/* A token tree, caller-allocated DEVICE buffers of capacity tree_nodes = dream_tree_nodes().
+ * Node 0 is the root (the pending token); parents precede children. */
+typedef struct {
+  int32_t *tokens;               /* [T] */
+  int32_t *parent;               /* [T], parent[0] = -1 */
+  int32_t *depth;                /* [T], depth[0] = 0 */
+  uint32_t *mask;                /* [T][4] ancestor-or-self bit set, bit j of word j/32 */
+  float *cum_logp;               /* [T] cumulative draft log-probability; may be NULL on input */
+} dream_tree;
+
+/* Number of tree nodes T = 1 + min(N, candidates) for this configuration (Section 4:
+ * depth, children per node, maximum draft length).  Host-only arithmetic. */
+dream_status dream_tree_nodes(const dream_config *cfg, int32_t *T);
+
+/* Bytes of device memory dream_init needs for this configuration.  Host-only. */
+dream_status dream_arena_bytes(const dream_config *cfg, size_t *bytes);
+
+/* Create a context.  arena: device, >= dream_arena_bytes, 256-byte aligned, zeroed by the
+ * library.  cuda_stream: a cudaStream_t (NULL = legacy default stream).  Weights are
+ * borrowed until dream_free.  The problem set-up of Section 3: one M_ta, one M_da. */
+dream_status dream_init(const dream_config *cfg, const dream_target_weights *tw,
+                        const dream_draft_weights *dw, void *arena, size_t arena_bytes,
+                        void *cuda_stream, dream_ctx **out);
+
+/* Target prefill over the n = q + v prompt (Section 3: M_ta processes all q + v inputs and
+ * emits t_{n+1}).  The sequence holds visual_embeds (device, [v, d_model], dtype) at
+ * positions [vis_start, vis_start + v) and embed[prompt_ids] (device int32 [q]) elsewhere.
+ * Also computes the average attention entropy of every layer (Eq. 2) and selects the
+ * feature-tap layer l* per config.tap_mode (Section 3.2).  Outputs (device, may be NULL):
+ * first_token int32[1], first_margin float[1] (top-1 minus top-2 logit),
+ * layer_entropy float[n_layers], tap_layer int32[1] (1-based). */
+dream_status dream_prefill(dream_ctx *ctx, int32_t seq, const void *visual_embeds, int32_t v,
+                           int32_t vis_start, const int32_t *prompt_ids, int32_t q,
+                           int32_t *first_token, float *first_margin, float *layer_entropy,
+                           int32_t *tap_layer);
+
+/* Override l* of a prefilled sequence (1-based) before dream_compress_visual. */
+dream_status dream_set_tap(dream_ctx *ctx, int32_t seq, int32_t tap_layer);
+
+/* Visual-token compression (Section 3.3): importance of visual token j = attention it
+ * receives at layer l* summed over query rows and heads; the k highest are kept.  Builds
+ * the draft's compressed context (self-attention K/V from input embeddings, cross-attention
+ * memory from the tapped features S^{l*}, Eq. 1).  forced_idx (device int32[k], ascending,
+ * or NULL) replaces the selection.  Outputs (device, may be NULL): kept_idx int32[k]
+ * ascending, scores float[v]. */
+dream_status dream_compress_visual(dream_ctx *ctx, int32_t seq, int32_t k,
+                                   const int32_t *forced_idx, int32_t *kept_idx, float *scores);
+
+/* Draft a token tree for each listed sequence (Section 3.1): D passes of the draft layer
+ * (self-attention over the draft cache, cross-attention over target features plus the
+ * draft's own earlier features, fusion MLP), top-K expansion per pass, beam selection, and
+ * a final re-rank to T nodes.  seqs: HOST int32[n_seqs], distinct.  trees: HOST array of
+ * n_seqs dream_tree structs whose members are DEVICE buffers that receive the trees. */
+dream_status dream_draft_tree(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
+                              const dream_tree *trees);
+
+/* Tree-masked verification by the target (Section 3.1: the same tree mask is used during
+ * verification): the T tree tokens of each sequence run through all L blocks, node i at
+ * position P + depth[i], attending to the verified prefix and to its ancestors' rows.
+ * Outputs (device): node_argmax int32[n_seqs][T]; node_margin float[n_seqs][T] or NULL;
+ * logits float[n_seqs][T][vocab] or NULL. */
+dream_status dream_verify_tree(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
+                               const dream_tree *trees, int32_t *node_argmax,
+                               float *node_margin, float *logits);
+
+/* Greedy acceptance and state update (Section 2.1; Section 4: one extra target token per
+ * round): follows from the root the child whose token equals its parent's argmax; emits
+ * the A accepted tokens plus the target's own next token; compacts the target KV cache so
+ * the accepted path occupies positions P..P+A; appends the accepted rows' tapped features
+ * to the cross-attention memory; P += A + 1.  Outputs (device): accept_len int32[n_seqs];
+ * out_tokens int32[n_seqs][D+1] (first A+1 valid); compaction_src int32[n_seqs][D+1] (tree
+ * node whose KV row moved to P+j; first A+1 valid). */
+dream_status dream_accept(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
+                          const dream_tree *trees, const int32_t *node_argmax,
+                          int32_t *accept_len, int32_t *out_tokens, int32_t *compaction_src);
+
+/* One whole round (draft, verify, accept) with HOST result buffers: runs the three calls
+ * above on the context's internal tree buffers, copies accept_len [n_seqs] and out_tokens
+ * [n_seqs][D+1] to host memory and waits for them.  This is the call a serving loop makes. */
+dream_status dream_step_host(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
+                             int32_t *accept_len_host, int32_t *out_tokens_host);
+
+/* Read back per-sequence state (host outputs; synchronises the stream). */
+dream_status dream_seq_state(dream_ctx *ctx, int32_t seq, int32_t *verified_len,
+                             int32_t *pending_token, int32_t *tap_layer);
+
+/* Debug read-back of internal device buffers for parity tests (synchronises).  what:
+ * 0 = target K row [n_kv_heads*head_dim] of (layer, position) as float,
+ * 1 = target V row, 2 = cross-memory K row (index = memory row), 3 = cross-memory V row,
+ * 4 = draft self-attention K row, 5 = draft self-attention V row,
+ * 6 = tapped features of tree node `index` from the last verify [d_model],
+ * 7 = final hidden state of tree node `index` from the last verify [d_model].
+ * dst: HOST float buffer. */
+dream_status dream_debug_read(dream_ctx *ctx, int32_t seq, int32_t what, int32_t layer,
+                              int32_t index, float *dst);
+
+/* Forget a sequence (its pages return to the pool). */
+dream_status dream_seq_reset(dream_ctx *ctx, int32_t seq);
+
+/* Wait for the stream and report the device status word (DREAM_OK or an error). */
+dream_status dream_poll(dream_ctx *ctx);
+
+/* Number of kernels this context has launched since dream_init. */
+int64_t dream_launch_count(const dream_ctx *ctx);
+
+/* Message of the last failed call on this context (or of the last failed dream_init when
+ * ctx is NULL).  The string is owned by the library. */
+const char *dream_last_error(const dream_ctx *ctx);
+
+/* Destroy the context.  The arena and the weights stay the caller's. */
+void dream_free(dream_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DREAM_H_ */

@@ -1,0 +1,230 @@
+// Attention kernels of the DREAM hot path, one warp per (query row, head):
+//   - causal prefill attention with the entropy accumulators of Eq. 2 fused in,
+//   - visual-token importance (column sums of the attention matrix, Section 3.3),
+//   - tree-masked verification attention over the paged prefix plus the tree tail,
+//   - the draft's self- and cross-attention (Eq. 1) over flat caches plus tree rows.
+// Every lane holds HD/32 consecutive elements of q, k and v; a key costs one coalesced
+// row load, HD/32 FMAs and a butterfly reduction.  Softmax runs online in fp32.
+#pragma once
+#include "common.cuh"
+#include "rows.cuh"
+
+template <int EPL, typename T> struct RowLoad;
+template <int EPL> struct RowLoad<EPL, float> {
+  static __device__ __forceinline__ void ld(const float *p, int lane, float (&o)[EPL]) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) o[e] = p[lane * EPL + e];
+  }
+};
+template <int EPL> struct RowLoad<EPL, bf16> {
+  static __device__ __forceinline__ void ld(const bf16 *p, int lane, float (&o)[EPL]) {
+    const __nv_bfloat162 *p2 = reinterpret_cast<const __nv_bfloat162 *>(p + lane * EPL);
+#pragma unroll
+    for (int e = 0; e < EPL / 2; ++e) {
+      float2 f = __bfloat1622float2(p2[e]);
+      o[2 * e] = f.x; o[2 * e + 1] = f.y;
+    }
+  }
+};
+
+// Online-softmax state of one (row, head): running max m, Z = sum e^{s-m}, the weighted
+// value sum, and U = sum e^{s-m}(s-m) for the entropy  H = ln Z - U/Z  (Eq. 2, inner sum).
+template <int EPL> struct Soft {
+  float m, z, u, acc[EPL];
+  __device__ __forceinline__ void init() {
+    m = -INFINITY; z = 0.f; u = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  }
+  template <bool ENT>
+  __device__ __forceinline__ void push(float s, const float (&v)[EPL]) {
+    if (s > m) {
+      float delta = s - m;                    // may be +inf on the first key
+      float sc = __expf(-delta);              // 0 when m was -inf
+      if (ENT) u = z > 0.f ? sc * (u - delta * z) : 0.f;
+      z *= sc;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[e] *= sc;
+      m = s;
+    }
+    float p = __expf(s - m);
+    z += p;
+    if (ENT) u += p * (s - m);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] += p * v[e];
+  }
+};
+
+template <int EPL>
+__device__ __forceinline__ float dot_lane(const float (&a)[EPL], const float (&b)[EPL]) {
+  float s = 0.f;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) s += a[e] * b[e];
+  return warp_sum(s);
+}
+
+#define ATT_WARPS 8
+
+// ---------------------------------------------------------------------------------------
+// Causal self-attention of the n prompt rows at one layer.  grid (ceil(n/8), H).
+// Outputs: attn_out [n][H*hd] (element type, input of the O projection), lse [H][n] (row
+// log-sum-exp of the scaled scores, for the importance pass), ent [H][n] row entropies.
+template <typename T, int HD>
+__global__ void __launch_bounds__(ATT_WARPS * 32)
+k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
+               T *attn_out, float *lse, float *ent) {
+  constexpr int EPL = HD / 32;
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int i = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
+  if (i >= n) return;
+  int kvh = h / (H / kv.hkv);
+  const T *Kp = (const T *)kv.base, *Vp = (const T *)kv.base + kv.kv_stride;
+  float q[EPL], k[EPL], v[EPL];
+  RowLoad<EPL, float>::ld(qbuf + ((long long)i * H + h) * HD, lane, q);
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) q[e] *= scale;
+  Soft<EPL> st;
+  st.init();
+  for (int j = 0; j <= i; ++j) {
+    long long o = kv.off(seq, j, kvh);
+    RowLoad<EPL, T>::ld(Kp + o, lane, k);
+    RowLoad<EPL, T>::ld(Vp + o, lane, v);
+    st.template push<true>(dot_lane<EPL>(q, k), v);
+  }
+  float inv = 1.f / st.z;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e)
+    attn_out[(long long)i * H * HD + h * HD + lane * EPL + e] = from_f<T>(st.acc[e] * inv);
+  if (lane == 0) {
+    lse[(long long)h * n + i] = st.m + logf(st.z);
+    ent[(long long)h * n + i] = logf(st.z) - st.u / st.z;
+  }
+}
+
+// AE(l) = mean over rows and heads of the row entropies (Eq. 2).  One block, fixed order.
+__global__ void k_entropy_mean(const float *__restrict__ ent, int count, float *out) {
+  __shared__ float sh[33];
+  float s = 0.f;
+  for (int i = threadIdx.x; i < count; i += blockDim.x) s += ent[i];
+  float t = block_sum(s, sh);
+  if (threadIdx.x == 0) *out = t / (float)count;
+}
+
+// Importance of visual token j at this layer (Section 3.3): the attention weight it receives,
+// summed over the later query rows (and its own row when include_self) and over heads.
+// One warp per visual column; heads outer, rows inner, both ascending: a fixed order.
+template <typename T, int HD>
+__global__ void __launch_bounds__(ATT_WARPS * 32)
+k_colsum(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
+         const float *__restrict__ lse, int vis_start, int v, int include_self, float *score) {
+  constexpr int EPL = HD / 32;
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int jv = blockIdx.x * ATT_WARPS + w;
+  if (jv >= v) return;
+  int j = vis_start + jv;
+  const T *Kp = (const T *)kv.base;
+  float tot = 0.f;
+  for (int h = 0; h < H; ++h) {
+    int kvh = h / (H / kv.hkv);
+    float k[EPL], q[EPL];
+    RowLoad<EPL, T>::ld(Kp + kv.off(seq, j, kvh), lane, k);
+    float hs = 0.f;
+    for (int i = include_self ? j : j + 1; i < n; ++i) {
+      RowLoad<EPL, float>::ld(qbuf + ((long long)i * H + h) * HD, lane, q);
+      float s = dot_lane<EPL>(q, k) * scale;
+      hs += __expf(s - lse[(long long)h * n + i]);
+    }
+    tot += hs;
+  }
+  if (lane == 0) score[jv] = tot;
+}
+
+// ---------------------------------------------------------------------------------------
+// Tree-masked verification attention (Section 3.1).  Row r = tree node of sequence
+// row_seq[r]; it sees prefix slots [0, P) and tail slots P + j for every j in its
+// ancestor-or-self bit set.  grid (ceil(R/8), H).
+template <typename T, int HD>
+__global__ void __launch_bounds__(ATT_WARPS * 32)
+k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ row_seq,
+            const int *__restrict__ row_node, const int *__restrict__ P_state,
+            const uint32_t *__restrict__ mask, int R, int T_nodes, int H, float scale, T *attn_out) {
+  constexpr int EPL = HD / 32;
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
+  if (r >= R) return;
+  int seq = row_seq[r], P = P_state[seq];
+  int kvh = h / (H / kv.hkv);
+  const T *Kp = (const T *)kv.base, *Vp = (const T *)kv.base + kv.kv_stride;
+  float q[EPL], k[EPL], v[EPL];
+  RowLoad<EPL, float>::ld(qbuf + ((long long)r * H + h) * HD, lane, q);
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) q[e] *= scale;
+  Soft<EPL> st;
+  st.init();
+  for (int j = 0; j < P; ++j) {
+    long long o = kv.off(seq, j, kvh);
+    RowLoad<EPL, T>::ld(Kp + o, lane, k);
+    RowLoad<EPL, T>::ld(Vp + o, lane, v);
+    st.template push<false>(dot_lane<EPL>(q, k), v);
+  }
+  const uint32_t *mr = mask + (long long)r * 4;
+  for (int j = 0; j < T_nodes; ++j) {
+    if (!((mr[j >> 5] >> (j & 31)) & 1u)) continue;
+    long long o = kv.off(seq, P + j, kvh);
+    RowLoad<EPL, T>::ld(Kp + o, lane, k);
+    RowLoad<EPL, T>::ld(Vp + o, lane, v);
+    st.template push<false>(dot_lane<EPL>(q, k), v);
+  }
+  (void)row_node;
+  float inv = 1.f / st.z;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e)
+    attn_out[(long long)r * H * HD + h * HD + lane * EPL + e] = from_f<T>(st.acc[e] * inv);
+}
+
+// ---------------------------------------------------------------------------------------
+// Draft attention over a flat cache: permanent rows [0, nperm[seq]) are all visible, then
+// tree-region rows nperm + j for each j in the row's ancestor set (self excluded when
+// strict: cross-attention reads the draft features of strict ancestors only, Section 3.1).
+// Rows with row_in < 0 are idle.  grid (ceil(R/8), H).
+template <typename T, int HD>
+__global__ void __launch_bounds__(ATT_WARPS * 32)
+k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ row_seq,
+             const int *__restrict__ row_in, const int *__restrict__ nperm,
+             const unsigned long long *__restrict__ anc, int anc_stride, int strict, int R, int H,
+             float scale, T *attn_out) {
+  constexpr int EPL = HD / 32;
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
+  if (r >= R) return;
+  int in = row_in[r];
+  if (in < 0) return;
+  int seq = row_seq[r], np = nperm[seq];
+  int kvh = h / (H / kv.hkv);
+  const T *base = (const T *)kv.base;
+  long long ok = kv.off(seq, 0, kvh, 0), ov = kv.off(seq, 1, kvh, 0);
+  float q[EPL], k[EPL], v[EPL];
+  RowLoad<EPL, float>::ld(qbuf + ((long long)r * H + h) * HD, lane, q);
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) q[e] *= scale;
+  Soft<EPL> st;
+  st.init();
+  for (int j = 0; j < np; ++j) {
+    RowLoad<EPL, T>::ld(base + ok + (long long)j * HD, lane, k);
+    RowLoad<EPL, T>::ld(base + ov + (long long)j * HD, lane, v);
+    st.template push<false>(dot_lane<EPL>(q, k), v);
+  }
+  unsigned long long bits = anc[(long long)seq * anc_stride + in];
+  if (strict) bits &= ~(1ull << in);
+  while (bits) {
+    int j = __ffsll((long long)bits) - 1;
+    bits &= bits - 1;
+    RowLoad<EPL, T>::ld(base + ok + (long long)(np + j) * HD, lane, k);
+    RowLoad<EPL, T>::ld(base + ov + (long long)(np + j) * HD, lane, v);
+    st.template push<false>(dot_lane<EPL>(q, k), v);
+  }
+  float inv = 1.f / st.z;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e)
+    attn_out[(long long)r * H * HD + h * HD + lane * EPL + e] = from_f<T>(st.acc[e] * inv);
+}

@@ -1,0 +1,72 @@
+// Shared device helpers of the DREAM hot path: element conversion, deterministic block
+// reductions, the split-output descriptor every GEMM consumer reads through.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+#define DREAM_DEV_OK 0
+#define DREAM_DEV_TIMEOUT 1
+#define DREAM_DEV_BAD_INDEX 2
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// Output of a GEMM launch: `count(tile)` partial sums per 128-column tile, stacked in slots
+// of slot_stride floats.  The stream-K tensor-core kernel leaves up to three partials per
+// tile; the SIMT kernel leaves one (upc == 0).
+struct GemmOut {
+  const float *base;
+  long long slot_stride;   // floats between consecutive slots
+  int ld;                  // floats between consecutive rows (tokens)
+  int kb;                  // k-blocks per tile
+  int upc;                 // work units (tile, k-block) per CTA; 0 = single slot
+};
+
+__device__ __forceinline__ float gemm_val(const GemmOut &g, int r, int c) {
+  const float *p = g.base + (long long)r * g.ld + c;
+  if (g.upc == 0) return *p;
+  long long u0 = (long long)(c >> 7) * g.kb;
+  int first = (int)(u0 / g.upc), last = (int)((u0 + g.kb - 1) / g.upc);
+  float s = *p;
+  for (int i = 1; i <= last - first; ++i) s += p[(long long)i * g.slot_stride];
+  return s;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Sum over a block of up to 1024 threads, same value returned to every thread; the order
+// of additions is fixed, so results are reproducible run to run.
+__device__ __forceinline__ float block_sum(float v, float *sh /* >= 33 floats */) {
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  if (w == 0) {
+    float t = lane < nw ? sh[lane] : 0.f;
+    t = warp_sum(t);
+    if (lane == 0) sh[32] = t;
+  }
+  __syncthreads();
+  return sh[32];
+}
+
+// (value, index) ordering used by every top-k / argmax: larger value first, then lower index.
+__device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {
+  return va > vb || (va == vb && ia < ib);
+}

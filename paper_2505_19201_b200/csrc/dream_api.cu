@@ -1,0 +1,827 @@
+// C ABI of the DREAM draft-and-verify hot path: context, arena layout, and the host-side
+// sequences of kernel launches behind each entry point.  Everything the entry points
+// compute runs in the kernels of this library; the host only validates and enqueues.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <vector>
+
+#include "../../include/dream.h"
+#include "attn.cuh"
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "rows.cuh"
+#include "tree.cuh"
+
+#define ROW_CHUNK 256          // rows per GEMM launch (tensor-core tile: up to 256 tokens)
+
+enum { PH_EMPTY = 0, PH_PREFILLED, PH_READY, PH_DRAFTED, PH_VERIFIED };
+
+static char g_init_error[256];
+
+struct dream_ctx {
+  dream_config cfg;
+  cudaStream_t stream;
+  TreeShape ts;
+  int T, esz, qkvN, Hhd, kvN, n_cand, tap_lo_eff, cap_rows, pps, n_pages, RM, XR, gemm_rows_lm;
+  int use_tc;
+  std::vector<const void *> ln1, wqkv, wo, ln2, wgu, wd;
+  const void *embed, *ln_f, *lm_head;
+  dream_draft_weights dw;
+  // arena
+  char *arena;
+  size_t arena_bytes;
+  void *kv_pool;
+  long long kv_stride, layer_stride;
+  int *page_table, *status;
+  SeqDev sd;
+  void *dself, *dmem;
+  DraftTreeDev dt;
+  TreePtrs itree[DREAM_MAX_BATCH];
+  RowMeta rm[2];
+  int *gather_idx, *ctx_pos, *flags;
+  uint32_t *vmask;
+  float *x, *x0, *qbuf, *gout, *lse_pre, *ent_pre, *ae, *scores_all, *taps_store, *tapbuf;
+  void *xn, *raw, *act, *attn_out;
+  float *top_val, *lse_rows, *margin_i;
+  int *top_id, *argmax_i, *accept_len_i, *out_tokens_i, *comp_src_i;
+  size_t gout_floats;
+  // host side
+  int phase[DREAM_MAX_BATCH], n_prompt[DREAM_MAX_BATCH], p_ub[DREAM_MAX_BATCH];
+  int prefill_seq;                     // sequence whose prefill scratch is live (-1 none)
+  int pf_v, pf_vis_start, pf_q;
+  std::vector<int> free_pages;
+  std::vector<int> seq_pages[DREAM_MAX_BATCH];
+  int *h_stage;                        // pinned: page-table staging + step_host results
+  long long launches;
+  GemmTcPlan tc;
+  char err[256];
+};
+
+static dream_status fail(dream_ctx *c, dream_status code, const char *fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(c ? c->err : g_init_error, 256, fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+#define CUDA_OK(c, call)                                                              \
+  do {                                                                                \
+    cudaError_t e_ = (call);                                                          \
+    if (e_ != cudaSuccess) return fail(c, DREAM_E_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+#define LAUNCH(c, kernel, grid, block, smem, ...)          \
+  do {                                                     \
+    kernel<<<grid, block, smem, (c)->stream>>>(__VA_ARGS__); \
+    (c)->launches++;                                       \
+  } while (0)
+
+// ------------------------------------------------------------------------------------- shapes
+
+static int tree_shape(const dream_config *cfg, TreeShape *ts) {
+  int D = cfg->tree_depth, K = cfg->tree_topk, bw = cfg->tree_beam, N = cfg->tree_max_nodes;
+  if (D < 1 || D > DREAM_MAX_DEPTH || K < 1 || K > TOPK_MAX || bw < 1 || N < 1) return -1;
+  memset(ts, 0, sizeof(*ts));
+  ts->D = D; ts->K = K; ts->N = N;
+  ts->beam[0] = 1; ts->in_off[0] = 0; ts->cand_off[0] = 0;
+  int ni = 1, nc = 0;
+  for (int p = 1; p <= D; ++p) {
+    int created = ts->beam[p - 1] * K;
+    if (created > 256) return -1;
+    nc += created;
+    ts->cand_off[p] = nc;
+    ts->beam[p] = created < bw ? created : bw;
+    ts->in_off[p] = ni;
+    if (p < D) ni += ts->beam[p];
+  }
+  ts->NI = ni; ts->NC = nc;
+  ts->T = 1 + (N < nc ? N : nc);
+  if (ni > 64 || ts->T > 128) return -1;
+  return 0;
+}
+
+extern "C" dream_status dream_tree_nodes(const dream_config *cfg, int32_t *T) {
+  TreeShape ts;
+  if (!cfg || !T) return fail(nullptr, DREAM_E_ARG, "null argument");
+  if (tree_shape(cfg, &ts)) return fail(nullptr, DREAM_E_UNSUPPORTED, "tree shape out of range");
+  *T = ts.T;
+  return DREAM_OK;
+}
+
+static int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
+static int imax(int a, int b) { return a > b ? a : b; }
+static int imin(int a, int b) { return a < b ? a : b; }
+
+static dream_status check_config(const dream_config *c, TreeShape *ts) {
+  if (!c) return fail(nullptr, DREAM_E_ARG, "null config");
+  if (c->dtype != DREAM_F32 && c->dtype != DREAM_BF16) return fail(nullptr, DREAM_E_ARG, "dtype");
+  if (c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256)
+    return fail(nullptr, DREAM_E_UNSUPPORTED, "head_dim must be 64, 128 or 256");
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->n_kv_heads < 1 ||
+      c->n_heads % c->n_kv_heads || c->d_ff < 8 || c->vocab < 2)
+    return fail(nullptr, DREAM_E_ARG, "model shape");
+  if (c->d_model % 8 || c->d_ff % 8) return fail(nullptr, DREAM_E_UNSUPPORTED, "d_model, d_ff must be multiples of 8");
+  if (c->max_batch < 1 || c->max_batch > DREAM_MAX_BATCH) return fail(nullptr, DREAM_E_ARG, "max_batch in 1..8");
+  if (c->page_tokens < 16 || c->page_tokens > 256 || (c->page_tokens & (c->page_tokens - 1)))
+    return fail(nullptr, DREAM_E_ARG, "page_tokens must be a power of two in 16..256");
+  if (c->max_prompt < 1 || c->max_visual < 0 || c->max_visual > c->max_prompt || c->max_seq < c->max_prompt)
+    return fail(nullptr, DREAM_E_ARG, "max_seq >= max_prompt >= max_visual required");
+  if (tree_shape(c, ts)) return fail(nullptr, DREAM_E_UNSUPPORTED, "tree: depth<=15, topk<=16, beam*topk<=256, input nodes<=64, nodes<=128");
+  if (c->max_batch * ts->T > ROW_CHUNK) return fail(nullptr, DREAM_E_UNSUPPORTED, "max_batch * tree nodes must be <= 256");
+  if (c->tap_mode == DREAM_TAP_FIXED) {
+    if (c->tap_layer < 1 || c->tap_layer > c->n_layers) return fail(nullptr, DREAM_E_ARG, "tap_layer");
+  } else if (c->tap_mode == DREAM_TAP_ENTROPY_MIN || c->tap_mode == DREAM_TAP_ENTROPY_MAX) {
+    if (c->tap_lo < 1 || c->tap_hi > c->n_layers || c->tap_lo > c->tap_hi) return fail(nullptr, DREAM_E_ARG, "tap range");
+  } else return fail(nullptr, DREAM_E_ARG, "tap_mode");
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- arena
+
+struct Carver {
+  char *base;
+  size_t off;
+  template <typename U> U *take(size_t count) {
+    off = (off + 255) & ~(size_t)255;
+    U *p = base ? reinterpret_cast<U *>(base + off) : nullptr;
+    off += count * sizeof(U);
+    return p;
+  }
+  void *take_bytes(size_t bytes) { return take<char>(bytes); }
+};
+
+static void derive(dream_ctx *c) {
+  const dream_config &f = c->cfg;
+  c->T = c->ts.T;
+  c->esz = f.dtype == DREAM_BF16 ? 2 : 4;
+  c->Hhd = f.n_heads * f.head_dim;
+  c->kvN = 2 * f.n_kv_heads * f.head_dim;
+  c->qkvN = c->Hhd + c->kvN;
+  c->n_cand = f.tap_mode == DREAM_TAP_FIXED ? 1 : f.tap_hi - f.tap_lo + 1;
+  c->tap_lo_eff = f.tap_mode == DREAM_TAP_FIXED ? f.tap_layer : f.tap_lo;
+  c->cap_rows = f.max_seq + c->ts.NI;
+  c->pps = (f.max_seq + f.page_tokens - 1) / f.page_tokens;
+  c->n_pages = c->pps * f.max_batch;
+  c->RM = imax(ROW_CHUNK, f.max_prompt);
+  c->XR = c->RM;
+}
+
+static size_t carve(dream_ctx *c, char *base) {
+  const dream_config &f = c->cfg;
+  Carver a{base, 0};
+  size_t e = c->esz;
+  int MB = f.max_batch, NI = c->ts.NI, NC = c->ts.NC, T = c->T, d = f.d_model;
+  c->kv_stride = (long long)c->n_pages * f.n_kv_heads * f.page_tokens * f.head_dim;
+  c->layer_stride = 2 * c->kv_stride;
+  c->kv_pool = a.take_bytes((size_t)f.n_layers * c->layer_stride * e);
+  c->page_table = a.take<int>((size_t)MB * c->pps);
+  c->status = a.take<int>(64);
+  int *st = a.take<int>((size_t)MB * (9 + 3 * (DREAM_MAX_DEPTH + 1)));
+  if (base) {
+    c->sd.P = st; c->sd.pending = st + MB; c->sd.tap = st + 2 * MB; c->sd.nperm_d = st + 3 * MB;
+    c->sd.nperm_m = st + 4 * MB; c->sd.n_new = st + 5 * MB; c->sd.last_P = st + 6 * MB;
+    c->sd.last_A = st + 7 * MB;
+    c->sd.new_tok = st + 9 * MB; c->sd.new_pos = c->sd.new_tok + MB * (DREAM_MAX_DEPTH + 1);
+    c->sd.path = c->sd.new_pos + MB * (DREAM_MAX_DEPTH + 1);
+  }
+  size_t flat = (size_t)MB * 2 * f.n_kv_heads * c->cap_rows * f.head_dim * e;
+  c->dself = a.take_bytes(flat);
+  c->dmem = a.take_bytes(flat);
+  c->dt.in_tok = a.take<int>((size_t)MB * NI); c->dt.in_depth = a.take<int>((size_t)MB * NI);
+  c->dt.in_cand = a.take<int>((size_t)MB * NI); c->dt.in_cum = a.take<float>((size_t)MB * NI);
+  c->dt.in_anc = a.take<unsigned long long>((size_t)MB * NI);
+  c->dt.cand_tok = a.take<int>((size_t)MB * NC); c->dt.cand_par = a.take<int>((size_t)MB * NC);
+  c->dt.cand_depth = a.take<int>((size_t)MB * NC); c->dt.cand_cum = a.take<float>((size_t)MB * NC);
+  for (int b = 0; b < DREAM_MAX_BATCH; ++b) {
+    if (b < MB) {
+      c->itree[b].tokens = a.take<int>(T); c->itree[b].parent = a.take<int>(T);
+      c->itree[b].depth = a.take<int>(T); c->itree[b].mask = a.take<uint32_t>(4 * T);
+      c->itree[b].cum = a.take<float>(T);
+    } else memset(&c->itree[b], 0, sizeof(TreePtrs));
+  }
+  for (int i = 0; i < 2; ++i) {
+    c->rm[i].seq = a.take<int>(c->RM); c->rm[i].tok = a.take<int>(c->RM); c->rm[i].pos = a.take<int>(c->RM);
+    c->rm[i].slot = a.take<int>(c->RM); c->rm[i].dst = a.take<int>(c->RM); c->rm[i].in = a.take<int>(c->RM);
+  }
+  c->gather_idx = a.take<int>(c->RM);
+  c->ctx_pos = a.take<int>(f.max_prompt);
+  c->flags = a.take<int>(f.max_prompt);
+  c->vmask = a.take<uint32_t>((size_t)ROW_CHUNK * 4);
+  c->x = a.take<float>((size_t)c->XR * d);
+  c->x0 = a.take<float>((size_t)f.max_prompt * d);
+  c->qbuf = a.take<float>((size_t)c->XR * c->Hhd);
+  c->attn_out = a.take_bytes((size_t)c->XR * c->Hhd * e);
+  c->xn = a.take_bytes((size_t)ROW_CHUNK * d * e);
+  c->raw = a.take_bytes((size_t)ROW_CHUNK * d * e);
+  c->act = a.take_bytes((size_t)ROW_CHUNK * f.d_ff * e);
+  int widest = imax(imax(c->qkvN, 2 * f.d_ff), imax(d, c->Hhd));
+  int lm_rows = ((imax(MB * T, MB * imax(c->ts.D + 2, f.tree_beam)) + 15) / 16) * 16;
+  c->gemm_rows_lm = lm_rows;
+  size_t per_slot = (size_t)imax(ROW_CHUNK * widest, 1) ;
+  size_t lm_slot = (size_t)lm_rows * f.vocab;
+  if (lm_slot > per_slot) per_slot = lm_slot;
+  c->gout_floats = per_slot;
+  c->gout = a.take<float>(per_slot * GEMM_TC_MAX_SLOTS);
+  c->lse_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
+  c->ent_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
+  c->ae = a.take<float>(f.n_layers);
+  c->scores_all = a.take<float>((size_t)c->n_cand * imax(f.max_visual, 1));
+  c->taps_store = a.take<float>((size_t)c->n_cand * f.max_prompt * d);
+  c->tapbuf = a.take<float>((size_t)ROW_CHUNK * d);
+  c->top_val = a.take<float>((size_t)ROW_CHUNK * TOPK_MAX);
+  c->top_id = a.take<int>((size_t)ROW_CHUNK * TOPK_MAX);
+  c->lse_rows = a.take<float>(ROW_CHUNK);
+  c->argmax_i = a.take<int>(ROW_CHUNK);
+  c->margin_i = a.take<float>(ROW_CHUNK);
+  c->accept_len_i = a.take<int>(MB);
+  c->out_tokens_i = a.take<int>((size_t)MB * (DREAM_MAX_DEPTH + 1));
+  c->comp_src_i = a.take<int>((size_t)MB * (DREAM_MAX_DEPTH + 1));
+  return (a.off + 255) & ~(size_t)255;
+}
+
+extern "C" dream_status dream_arena_bytes(const dream_config *cfg, size_t *bytes) {
+  if (!cfg || !bytes) return fail(nullptr, DREAM_E_ARG, "null argument");
+  dream_ctx tmp;
+  dream_status s = check_config(cfg, &tmp.ts);
+  if (s) return s;
+  tmp.cfg = *cfg;
+  derive(&tmp);
+  *bytes = carve(&tmp, nullptr);
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- GEMM dispatch
+
+// out[r][c] = sum_k X[r][k] W[c][k] for r < rows, c < N.  Returns the descriptor consumers
+// read the result through.
+template <typename T>
+static GemmOut gemm(dream_ctx *c, const void *W, const void *X, int rows, int N, int K) {
+  GemmOut g;
+  if (c->use_tc && sizeof(T) == 2 && gemm_tc_supported(rows, N, K)) {
+    gemm_tc_launch(&c->tc, c->stream, W, X, rows, N, K, c->gout, (long long)c->gout_floats, &g);
+    c->launches++;
+    return g;
+  }
+  dim3 grid((N + SG_BN - 1) / SG_BN, (rows + SG_BM - 1) / SG_BM);
+  k_gemm_simt<T><<<grid, 256, 0, c->stream>>>((const T *)X, (const T *)W, c->gout, rows, N, K, N);
+  c->launches++;
+  g.base = c->gout; g.slot_stride = 0; g.ld = N; g.kb = 0; g.upc = 0;
+  return g;
+}
+
+static PagedKV paged(dream_ctx *c, int layer) {
+  PagedKV kv;
+  kv.base = (char *)c->kv_pool + (size_t)layer * c->layer_stride * c->esz;
+  kv.kv_stride = c->kv_stride;
+  kv.page_table = c->page_table;
+  kv.pages_per_seq = c->pps;
+  kv.page_tokens = c->cfg.page_tokens;
+  kv.page_shift = ilog2(c->cfg.page_tokens);
+  kv.hkv = c->cfg.n_kv_heads;
+  kv.hd = c->cfg.head_dim;
+  return kv;
+}
+static FlatKV flat(dream_ctx *c, void *base) {
+  FlatKV kv;
+  kv.base = base; kv.cap = c->cap_rows; kv.hkv = c->cfg.n_kv_heads; kv.hd = c->cfg.head_dim;
+  return kv;
+}
+static const GemmOut NO_GEMM = {nullptr, 0, 0, 0, 0};
+
+// ------------------------------------------------------------------------------------- init / free
+
+extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_weights *tw,
+                                   const dream_draft_weights *dw, void *arena, size_t arena_bytes,
+                                   void *cuda_stream, dream_ctx **out) {
+  if (!cfg || !tw || !dw || !arena || !out) return fail(nullptr, DREAM_E_ARG, "null argument");
+  TreeShape ts;
+  dream_status s = check_config(cfg, &ts);
+  if (s) return s;
+  if ((uintptr_t)arena & 255) return fail(nullptr, DREAM_E_ARG, "arena must be 256-byte aligned");
+  dream_ctx *c = new dream_ctx();
+  c->cfg = *cfg; c->ts = ts;
+  derive(c);
+  size_t need = carve(c, nullptr);
+  if (arena_bytes < need) { delete c; return fail(nullptr, DREAM_E_NOMEM, "arena needs %zu bytes, got %zu", need, arena_bytes); }
+  c->arena = (char *)arena; c->arena_bytes = need;
+  carve(c, c->arena);
+  c->stream = (cudaStream_t)cuda_stream;
+  c->embed = tw->embed; c->ln_f = tw->ln_f; c->lm_head = tw->lm_head; c->dw = *dw;
+  const void *dptr[] = {dw->ln1, dw->wqkv, dw->wo, dw->lnx, dw->xq, dw->xkv, dw->xo, dw->ln2, dw->wgu, dw->wd,
+                        tw->embed, tw->ln_f, tw->lm_head};
+  for (const void *p : dptr) if (!p) { delete c; return fail(nullptr, DREAM_E_ARG, "null weight pointer"); }
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    if (!tw->ln1[l] || !tw->wqkv[l] || !tw->wo[l] || !tw->ln2[l] || !tw->wgu[l] || !tw->wd[l]) {
+      delete c; return fail(nullptr, DREAM_E_ARG, "null weight pointer in layer %d", l);
+    }
+    c->ln1.push_back(tw->ln1[l]); c->wqkv.push_back(tw->wqkv[l]); c->wo.push_back(tw->wo[l]);
+    c->ln2.push_back(tw->ln2[l]); c->wgu.push_back(tw->wgu[l]); c->wd.push_back(tw->wd[l]);
+  }
+  cudaError_t e = cudaMemsetAsync(c->arena, 0, need, c->stream);
+  if (e != cudaSuccess) { delete c; return fail(nullptr, DREAM_E_CUDA, "memset arena: %s", cudaGetErrorString(e)); }
+  e = cudaHostAlloc((void **)&c->h_stage, sizeof(int) * ((size_t)cfg->max_batch * c->pps + 64 + cfg->max_batch * (DREAM_MAX_DEPTH + 2)), cudaHostAllocDefault);
+  if (e != cudaSuccess) { delete c; return fail(nullptr, DREAM_E_CUDA, "pinned staging: %s", cudaGetErrorString(e)); }
+  for (int p = c->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
+  for (int b = 0; b < DREAM_MAX_BATCH; ++b) c->phase[b] = PH_EMPTY;
+  c->prefill_seq = -1;
+  c->launches = 0;
+  c->err[0] = 0;
+  const char *mode = getenv("DREAM_GEMM");
+  c->use_tc = cfg->dtype == DREAM_BF16 && !(mode && !strcmp(mode, "simt"));
+  if (c->use_tc) {
+    const char *why = gemm_tc_plan_init(&c->tc);
+    if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
+  }
+  *out = c;
+  return DREAM_OK;
+}
+
+extern "C" void dream_free(dream_ctx *c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->stream);
+  cudaFreeHost(c->h_stage);
+  delete c;
+}
+
+extern "C" const char *dream_last_error(const dream_ctx *c) { return c ? c->err : g_init_error; }
+extern "C" int64_t dream_launch_count(const dream_ctx *c) { return c ? c->launches : 0; }
+
+extern "C" dream_status dream_poll(dream_ctx *c) {
+  if (!c) return DREAM_E_ARG;
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  int st = 0;
+  CUDA_OK(c, cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st == DREAM_DEV_TIMEOUT) return fail(c, DREAM_E_DEVICE_TIMEOUT, "a bounded device-side wait expired");
+  if (st == DREAM_DEV_BAD_INDEX) return fail(c, DREAM_E_STATE, "a kernel met an index or capacity out of range");
+  return DREAM_OK;
+}
+
+static dream_status check_seq(dream_ctx *c, int seq) {
+  if (!c) return DREAM_E_ARG;
+  if (seq < 0 || seq >= c->cfg.max_batch) return fail(c, DREAM_E_ARG, "sequence id %d out of range", seq);
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_seq_reset(dream_ctx *c, int32_t seq) {
+  dream_status s = check_seq(c, seq);
+  if (s) return s;
+  for (int p : c->seq_pages[seq]) c->free_pages.push_back(p);
+  c->seq_pages[seq].clear();
+  c->phase[seq] = PH_EMPTY;
+  if (c->prefill_seq == seq) c->prefill_seq = -1;
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- small kernels
+
+__global__ void k_iota_rows(RowMeta rm, int seq, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  rm.seq[i] = seq; rm.pos[i] = i; rm.slot[i] = i; rm.dst[i] = i; rm.in[i] = -1;
+}
+__global__ void k_set_seq(SeqDev s, int seq, int P, const int *pending_src, int nd, int nm) {
+  if (threadIdx.x) return;
+  if (P >= 0) s.P[seq] = P;
+  if (pending_src) s.pending[seq] = *pending_src;
+  if (nd >= 0) { s.nperm_d[seq] = nd; s.nperm_m[seq] = nm; s.n_new[seq] = 0; }
+}
+__global__ void k_set_int(int *p, int v) { if (!threadIdx.x) *p = v; }
+__global__ void k_first_token(const int *top_id, const float *top_val, int *tok, float *margin) {
+  if (threadIdx.x) return;
+  if (tok) *tok = top_id[0];
+  if (margin) *margin = top_val[0] - top_val[1];
+}
+__global__ void k_argmax_out(const int *top_id, const float *top_val, int R, int *am, float *mg, int *am2) {
+  int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= R) return;
+  am[r] = top_id[2 * r];
+  if (am2) am2[r] = top_id[2 * r];
+  if (mg) mg[r] = top_val[2 * r] - top_val[2 * r + 1];
+}
+__global__ void k_copy_f32(const float *src, float *dst, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[i];
+}
+template <typename T>
+__global__ void k_read_row(const T *src, float *dst, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = to_f(src[i]);
+}
+
+template <typename T, int HD> struct AttnLaunch {
+  static void prefill(dream_ctx *c, int layer, int seq, int n) {
+    dim3 grid((n + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
+    LAUNCH(c, (k_attn_prefill<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n, c->cfg.n_heads,
+           1.f / sqrtf((float)HD), (T *)c->attn_out, c->lse_pre, c->ent_pre);
+  }
+  static void colsum(dream_ctx *c, int layer, int seq, int n, int vis_start, int v, float *score) {
+    if (v == 0) return;
+    LAUNCH(c, (k_colsum<T, HD>), (v + ATT_WARPS - 1) / ATT_WARPS, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n,
+           c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, score);
+  }
+  static void tree(dream_ctx *c, int layer, int R) {
+    dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
+    LAUNCH(c, (k_attn_tree<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
+           c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out);
+  }
+  static void draft(dream_ctx *c, const RowMeta &rm, void *cache, const int *nperm, int strict, int R) {
+    dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
+    LAUNCH(c, (k_attn_draft<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, flat(c, cache), rm.seq, rm.in, nperm,
+           c->dt.in_anc, c->ts.NI, strict, R, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out);
+  }
+};
+
+#define HD_DISPATCH(c, T, call)                                   \
+  do {                                                            \
+    if ((c)->cfg.head_dim == 64) AttnLaunch<T, 64>::call;         \
+    else if ((c)->cfg.head_dim == 128) AttnLaunch<T, 128>::call;  \
+    else AttnLaunch<T, 256>::call;                                \
+  } while (0)
+
+// ------------------------------------------------------------------------------------- prefill
+
+template <typename T>
+static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int v, int vis_start,
+                                 const int *ids, int q, int *first_token, float *first_margin,
+                                 float *layer_entropy, int *tap_layer) {
+  const dream_config &f = c->cfg;
+  int n = q + v, d = f.d_model, L = f.n_layers;
+  LAUNCH(c, k_iota_rows, (n + 255) / 256, 256, 0, c->rm[0], seq, n);
+  LAUNCH(c, (k_build_prompt<T>), n, 256, 0, (const T *)c->embed, (const T *)visual, ids, vis_start, v, c->x, c->x0,
+         d, f.vocab, c->status);
+  for (int l = 0; l < L; ++l) {
+    for (int r0 = 0; r0 < n; r0 += ROW_CHUNK) {
+      int rows = imin(ROW_CHUNK, n - r0);
+      LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, c->x + (size_t)r0 * d, NO_GEMM, 0, (const T *)c->ln1[l], f.rms_eps, d,
+             (T *)c->xn, (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+      GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, rows, c->qkvN, d);
+      LAUNCH(c, (k_qkv_post_target<T>), rows, 128, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
+             paged(c, l), f.n_heads, f.rope_theta);
+    }
+    HD_DISPATCH(c, T, prefill(c, l, seq, n));
+    LAUNCH(c, k_entropy_mean, 1, 1024, 0, c->ent_pre, f.n_heads * n, c->ae + l);
+    int cand = l + 1 - c->tap_lo_eff;
+    bool is_cand = cand >= 0 && cand < c->n_cand;
+    if (is_cand) HD_DISPATCH(c, T, colsum(c, l, seq, n, vis_start, v, c->scores_all + (size_t)cand * imax(f.max_visual, 1)));
+    for (int r0 = 0; r0 < n; r0 += ROW_CHUNK) {
+      int rows = imin(ROW_CHUNK, n - r0);
+      float *xr = c->x + (size_t)r0 * d;
+      GemmOut g = gemm<T>(c, c->wo[l], (const T *)c->attn_out + (size_t)r0 * c->Hhd, rows, d, c->Hhd);
+      LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, xr, g, 1, (const T *)c->ln2[l], f.rms_eps, d, (T *)c->xn,
+             (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+      g = gemm<T>(c, c->wgu[l], c->xn, rows, 2 * f.d_ff, d);
+      LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, rows), 256, 0, g, (T *)c->act, f.d_ff);
+      g = gemm<T>(c, c->wd[l], c->act, rows, d, f.d_ff);
+      float *copy = is_cand ? c->taps_store + ((size_t)cand * f.max_prompt + r0) * d : nullptr;
+      LAUNCH(c, k_resid_add, rows, 256, 0, xr, g, d, copy);
+    }
+  }
+  // first token: LM head on the last prompt row
+  LAUNCH(c, (k_resid_norm<T>), 1, 256, 0, c->x + (size_t)(n - 1) * d, NO_GEMM, 0, (const T *)c->ln_f, f.rms_eps, d,
+         (T *)c->xn, (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+  GemmOut g = gemm<T>(c, c->lm_head, c->xn, 1, f.vocab, d);
+  LAUNCH(c, k_topk_lse, 1, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
+  LAUNCH(c, k_first_token, 1, 32, 0, c->top_id, c->top_val, first_token, first_margin);
+  LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, n, c->top_id, -1, -1);
+  LAUNCH(c, k_select_tap, 1, 32, 0, c->ae, f.tap_mode, f.tap_layer, f.tap_lo, f.tap_hi, c->sd.tap + seq, tap_layer);
+  if (layer_entropy) LAUNCH(c, k_copy_f32, (L + 255) / 256, 256, 0, c->ae, layer_entropy, L);
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_prefill(dream_ctx *c, int32_t seq, const void *visual, int32_t v,
+                                      int32_t vis_start, const int32_t *ids, int32_t q,
+                                      int32_t *first_token, float *first_margin, float *layer_entropy,
+                                      int32_t *tap_layer) {
+  dream_status s = check_seq(c, seq);
+  if (s) return s;
+  const dream_config &f = c->cfg;
+  if (v < 0 || q < 0 || v + q < 1 || (v && !visual) || (q && !ids)) return fail(c, DREAM_E_ARG, "prompt: need v + q >= 1 and buffers");
+  if (vis_start < 0 || vis_start > q) return fail(c, DREAM_E_ARG, "vis_start must lie in [0, q]");
+  if (v > f.max_visual || v + q > f.max_prompt) return fail(c, DREAM_E_CAPACITY, "prompt of %d (+%d visual) exceeds max_prompt/max_visual", v + q, v);
+  if (c->phase[seq] != PH_EMPTY) return fail(c, DREAM_E_STATE, "sequence %d is live; dream_seq_reset it first", seq);
+  if ((int)c->free_pages.size() < c->pps) return fail(c, DREAM_E_CAPACITY, "page pool exhausted");
+  int *stage = c->h_stage + (size_t)seq * c->pps;
+  for (int i = 0; i < c->pps; ++i) {
+    int p = c->free_pages.back();
+    c->free_pages.pop_back();
+    c->seq_pages[seq].push_back(p);
+    stage[i] = p;
+  }
+  CUDA_OK(c, cudaMemcpyAsync(c->page_table + (size_t)seq * c->pps, stage, sizeof(int) * c->pps, cudaMemcpyHostToDevice, c->stream));
+  if (f.dtype == DREAM_BF16) s = prefill_impl<bf16>(c, seq, visual, v, vis_start, ids, q, first_token, first_margin, layer_entropy, tap_layer);
+  else s = prefill_impl<float>(c, seq, visual, v, vis_start, ids, q, first_token, first_margin, layer_entropy, tap_layer);
+  if (s) return s;
+  CUDA_OK(c, cudaGetLastError());
+  c->phase[seq] = PH_PREFILLED;
+  c->n_prompt[seq] = v + q; c->p_ub[seq] = v + q;
+  c->prefill_seq = seq; c->pf_v = v; c->pf_vis_start = vis_start; c->pf_q = q;
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_set_tap(dream_ctx *c, int32_t seq, int32_t tap_layer) {
+  dream_status s = check_seq(c, seq);
+  if (s) return s;
+  if (c->phase[seq] != PH_PREFILLED || c->prefill_seq != seq) return fail(c, DREAM_E_STATE, "dream_set_tap follows dream_prefill of the same sequence");
+  if (tap_layer < c->tap_lo_eff || tap_layer >= c->tap_lo_eff + c->n_cand)
+    return fail(c, DREAM_E_ARG, "tap layer %d outside the stored range [%d, %d]", tap_layer, c->tap_lo_eff, c->tap_lo_eff + c->n_cand - 1);
+  LAUNCH(c, k_set_int, 1, 32, 0, c->sd.tap + seq, tap_layer);
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- compression
+
+template <typename T>
+static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *forced, int *kept, float *scores) {
+  const dream_config &f = c->cfg;
+  int v = c->pf_v, q = c->pf_q, n = v + q, d = f.d_model, nc = q + k;
+  LAUNCH(c, k_select_visual, 1, 1024, 0, c->scores_all, (long long)imax(f.max_visual, 1), c->sd.tap + seq, c->tap_lo_eff,
+         v, k, c->pf_vis_start, n, forced, kept, scores, c->ctx_pos, c->flags);
+  // draft self-attention K/V of the compressed context, from the input embeddings
+  const char *wkv = (const char *)c->dw.wqkv + (size_t)c->Hhd * d * c->esz;
+  for (int r0 = 0; r0 < nc; r0 += ROW_CHUNK) {
+    int rows = imin(ROW_CHUNK, nc - r0);
+    LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, 0, seq, c->rm[0], c->gather_idx, r0);
+    LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL);
+    LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, c->x, NO_GEMM, 0, (const T *)c->dw.ln1, f.rms_eps, d, (T *)c->xn,
+           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+    GemmOut g = gemm<T>(c, wkv, c->xn, rows, c->kvN, d);
+    LAUNCH(c, (k_qkv_post_draft<T>), rows, 128, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
+           flat(c, c->dself), f.n_heads, f.rope_theta);
+  }
+  // cross-attention memory: tapped features at the context positions, projected (Eq. 1)
+  int nm = f.xattn_full_memory ? n : nc;
+  for (int r0 = 0; r0 < nm; r0 += ROW_CHUNK) {
+    int rows = imin(ROW_CHUNK, nm - r0);
+    LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, f.xattn_full_memory, seq, c->rm[0], c->gather_idx, r0);
+    LAUNCH(c, (k_gather_rows<T>), rows, 256, 0, c->taps_store, c->gather_idx, (T *)c->raw, d, c->sd.tap + seq, c->tap_lo_eff,
+           (long long)f.max_prompt * d);
+    GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, rows, c->kvN, d);
+    LAUNCH(c, (k_mem_append<T>), rows, 256, 0, g, c->rm[0].seq, c->rm[0].dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
+  }
+  LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, -1, (const int *)nullptr, nc, nm);
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_compress_visual(dream_ctx *c, int32_t seq, int32_t k, const int32_t *forced,
+                                              int32_t *kept, float *scores) {
+  dream_status s = check_seq(c, seq);
+  if (s) return s;
+  if (c->phase[seq] != PH_PREFILLED || c->prefill_seq != seq)
+    return fail(c, DREAM_E_STATE, "dream_compress_visual follows dream_prefill of the same sequence");
+  if (k < 0 || k > c->pf_v) return fail(c, DREAM_E_ARG, "k = %d outside [0, v = %d]", k, c->pf_v);
+  s = c->cfg.dtype == DREAM_BF16 ? compress_impl<bf16>(c, seq, k, forced, kept, scores)
+                                 : compress_impl<float>(c, seq, k, forced, kept, scores);
+  if (s) return s;
+  CUDA_OK(c, cudaGetLastError());
+  c->phase[seq] = PH_READY;
+  c->prefill_seq = -1;
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- batch helpers
+
+static dream_status make_batch(dream_ctx *c, const int *seqs, int n_seqs, const dream_tree *trees, bool need_cum,
+                               TreeBatch *tb) {
+  if (!c) return DREAM_E_ARG;
+  if (!seqs || n_seqs < 1 || n_seqs > c->cfg.max_batch) return fail(c, DREAM_E_ARG, "n_seqs outside 1..max_batch");
+  memset(tb, 0, sizeof(*tb));
+  for (int b = 0; b < n_seqs; ++b) {
+    dream_status s = check_seq(c, seqs[b]);
+    if (s) return s;
+    for (int a = 0; a < b; ++a) if (seqs[a] == seqs[b]) return fail(c, DREAM_E_ARG, "sequence %d listed twice", seqs[b]);
+    tb->seq[b] = seqs[b];
+    if (trees) {
+      const dream_tree &t = trees[b];
+      if (!t.tokens || !t.parent || !t.depth || !t.mask) return fail(c, DREAM_E_ARG, "tree %d has a null buffer", b);
+      tb->t[b].tokens = t.tokens; tb->t[b].parent = t.parent; tb->t[b].depth = t.depth;
+      tb->t[b].mask = t.mask; tb->t[b].cum = t.cum_logp;
+    } else tb->t[b] = c->itree[seqs[b]];
+    (void)need_cum;
+  }
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- draft
+
+template <typename T>
+static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
+  const dream_config &f = c->cfg;
+  const TreeShape &ts = c->ts;
+  int d = f.d_model, cur = 0;
+  for (int p = 1; p <= ts.D; ++p) {
+    int m = p == 1 ? ts.D + 2 : ts.beam[p - 1];
+    int R = B * m;
+    RowMeta &rm = c->rm[cur], &rn = c->rm[cur ^ 1];
+    if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
+    LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
+    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, NO_GEMM, 0, (const T *)c->dw.ln1, f.rms_eps, d, (T *)c->xn,
+           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+    GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, R, c->qkvN, d);
+    LAUNCH(c, (k_qkv_post_draft<T>), R, 128, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, f.rope_theta);
+    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R));
+    g = gemm<T>(c, c->dw.wo, c->attn_out, R, d, c->Hhd);
+    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->dw.lnx, f.rms_eps, d, (T *)c->xn,
+           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+    g = gemm<T>(c, c->dw.xq, c->xn, R, c->Hhd, d);
+    LAUNCH(c, k_gemm_to_f32, R, 256, 0, g, c->qbuf, c->Hhd);
+    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R));
+    g = gemm<T>(c, c->dw.xo, c->attn_out, R, d, c->Hhd);
+    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->dw.ln2, f.rms_eps, d, (T *)c->xn,
+           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+    g = gemm<T>(c, c->dw.wgu, c->xn, R, 2 * f.d_ff, d);
+    LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, R), 256, 0, g, (T *)c->act, f.d_ff);
+    g = gemm<T>(c, c->dw.wd, c->act, R, d, f.d_ff);
+    // e^M = x: raw copy feeds the memory projection, normalised copy feeds the LM head
+    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->ln_f, f.rms_eps, d, (T *)c->xn,
+           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)c->raw);
+    g = gemm<T>(c, c->dw.xkv, c->raw, R, c->kvN, d);
+    LAUNCH(c, (k_mem_append<T>), R, 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
+    g = gemm<T>(c, c->lm_head, c->xn, R, f.vocab, d);
+    LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, ts.K, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
+    int next_m = p < ts.D ? ts.beam[p] : 1;
+    LAUNCH(c, k_tree_expand, B, 128, 0, tb, c->sd, c->dt, ts, p, m, c->top_val, c->top_id, c->lse_rows, rn, next_m);
+    cur ^= 1;
+  }
+  LAUNCH(c, k_tree_finalize, B, 256, 2 * ts.NC * sizeof(int), tb, c->sd, c->dt, ts);
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_draft_tree(dream_ctx *c, const int32_t *seqs, int32_t n_seqs, const dream_tree *trees) {
+  TreeBatch tb;
+  dream_status s = make_batch(c, seqs, n_seqs, trees, true, &tb);
+  if (s) return s;
+  for (int b = 0; b < n_seqs; ++b)
+    if (c->phase[seqs[b]] != PH_READY) return fail(c, DREAM_E_STATE, "sequence %d: dream_draft_tree follows dream_compress_visual or dream_accept", seqs[b]);
+  s = c->cfg.dtype == DREAM_BF16 ? draft_impl<bf16>(c, tb, n_seqs) : draft_impl<float>(c, tb, n_seqs);
+  if (s) return s;
+  CUDA_OK(c, cudaGetLastError());
+  for (int b = 0; b < n_seqs; ++b) c->phase[seqs[b]] = PH_DRAFTED;
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- verify
+
+template <typename T>
+static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *argmax, float *margin, float *logits) {
+  const dream_config &f = c->cfg;
+  int d = f.d_model, L = f.n_layers, R = B * c->T;
+  RowMeta &rm = c->rm[0];
+  LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
+  LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
+  GemmOut gd = NO_GEMM;
+  for (int l = 0; l < L; ++l) {
+    // completes S^l (for l >= 1) and captures it where a sequence taps layer l
+    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, gd, l > 0, (const T *)c->ln1[l], f.rms_eps, d, (T *)c->xn,
+           l > 0 ? c->tapbuf : (float *)nullptr, rm.seq, c->sd.tap, l, (T *)nullptr);
+    GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, R, c->qkvN, d);
+    LAUNCH(c, (k_qkv_post_target<T>), R, 128, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, f.rope_theta);
+    HD_DISPATCH(c, T, tree(c, l, R));
+    g = gemm<T>(c, c->wo[l], c->attn_out, R, d, c->Hhd);
+    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->ln2[l], f.rms_eps, d, (T *)c->xn,
+           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
+    g = gemm<T>(c, c->wgu[l], c->xn, R, 2 * f.d_ff, d);
+    LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, R), 256, 0, g, (T *)c->act, f.d_ff);
+    gd = gemm<T>(c, c->wd[l], c->act, R, d, f.d_ff);
+  }
+  LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, gd, 1, (const T *)c->ln_f, f.rms_eps, d, (T *)c->xn, c->tapbuf, rm.seq,
+         c->sd.tap, L, (T *)nullptr);
+  GemmOut g = gemm<T>(c, c->lm_head, c->xn, R, f.vocab, d);
+  LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, logits);
+  LAUNCH(c, k_argmax_out, (R + 127) / 128, 128, 0, c->top_id, c->top_val, R, argmax, margin,
+         argmax == c->argmax_i ? (int *)nullptr : c->argmax_i);
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_verify_tree(dream_ctx *c, const int32_t *seqs, int32_t n_seqs, const dream_tree *trees,
+                                          int32_t *node_argmax, float *node_margin, float *logits) {
+  TreeBatch tb;
+  dream_status s = make_batch(c, seqs, n_seqs, trees, false, &tb);
+  if (s) return s;
+  if (!node_argmax) return fail(c, DREAM_E_ARG, "node_argmax is required");
+  for (int b = 0; b < n_seqs; ++b) {
+    if (c->phase[seqs[b]] != PH_DRAFTED) return fail(c, DREAM_E_STATE, "sequence %d: dream_verify_tree follows dream_draft_tree", seqs[b]);
+    if (c->p_ub[seqs[b]] + c->T > c->cfg.max_seq) return fail(c, DREAM_E_CAPACITY, "sequence %d may outgrow max_seq", seqs[b]);
+  }
+  s = c->cfg.dtype == DREAM_BF16 ? verify_impl<bf16>(c, tb, n_seqs, node_argmax, node_margin, logits)
+                                 : verify_impl<float>(c, tb, n_seqs, node_argmax, node_margin, logits);
+  if (s) return s;
+  CUDA_OK(c, cudaGetLastError());
+  for (int b = 0; b < n_seqs; ++b) c->phase[seqs[b]] = PH_VERIFIED;
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- accept
+
+template <typename T>
+static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const int *argmax, int *accept_len,
+                                int *out_tokens, int *comp_src) {
+  const dream_config &f = c->cfg;
+  int D = c->ts.D, d = f.d_model, R = B * (D + 1);
+  RowMeta &rm = c->rm[0];
+  LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
+  LAUNCH(c, (k_compact_kv<T>), dim3(f.n_layers * 2, B), 256, 0, tb, c->sd, c->kv_pool, c->layer_stride, c->kv_stride, paged(c, 0));
+  LAUNCH(c, k_accept_rows, 1, 32, 0, tb, B, c->T, D, c->sd, c->gather_idx, rm, c->cap_rows - c->ts.NI, c->status);
+  LAUNCH(c, (k_gather_rows<T>), R, 256, 0, c->tapbuf, c->gather_idx, (T *)c->raw, d, (const int *)nullptr, 0, 0LL);
+  GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, R, c->kvN, d);
+  LAUNCH(c, (k_mem_append<T>), R, 256, 0, g, rm.seq, rm.dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_accept(dream_ctx *c, const int32_t *seqs, int32_t n_seqs, const dream_tree *trees,
+                                     const int32_t *node_argmax, int32_t *accept_len, int32_t *out_tokens,
+                                     int32_t *comp_src) {
+  TreeBatch tb;
+  dream_status s = make_batch(c, seqs, n_seqs, trees, false, &tb);
+  if (s) return s;
+  if (!node_argmax || !accept_len || !out_tokens) return fail(c, DREAM_E_ARG, "node_argmax, accept_len, out_tokens are required");
+  for (int b = 0; b < n_seqs; ++b)
+    if (c->phase[seqs[b]] != PH_VERIFIED) return fail(c, DREAM_E_STATE, "sequence %d: dream_accept follows dream_verify_tree", seqs[b]);
+  s = c->cfg.dtype == DREAM_BF16 ? accept_impl<bf16>(c, tb, n_seqs, node_argmax, accept_len, out_tokens, comp_src)
+                                 : accept_impl<float>(c, tb, n_seqs, node_argmax, accept_len, out_tokens, comp_src);
+  if (s) return s;
+  CUDA_OK(c, cudaGetLastError());
+  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; }
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- whole step, host results
+
+extern "C" dream_status dream_step_host(dream_ctx *c, const int32_t *seqs, int32_t n_seqs, int32_t *accept_len_host,
+                                        int32_t *out_tokens_host) {
+  if (!c || !accept_len_host || !out_tokens_host) return fail(c, DREAM_E_ARG, "null argument");
+  dream_status s = dream_draft_tree(c, seqs, n_seqs, nullptr);
+  if (s) return s;
+  s = dream_verify_tree(c, seqs, n_seqs, nullptr, c->argmax_i, c->margin_i, nullptr);
+  if (s) return s;
+  s = dream_accept(c, seqs, n_seqs, nullptr, c->argmax_i, c->accept_len_i, c->out_tokens_i, c->comp_src_i);
+  if (s) return s;
+  int D1 = c->ts.D + 1;
+  int *stage = c->h_stage + (size_t)c->cfg.max_batch * c->pps;
+  CUDA_OK(c, cudaMemcpyAsync(stage, c->accept_len_i, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(c, cudaMemcpyAsync(stage + DREAM_MAX_BATCH, c->out_tokens_i, sizeof(int) * n_seqs * D1, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  memcpy(accept_len_host, stage, sizeof(int) * n_seqs);
+  memcpy(out_tokens_host, stage + DREAM_MAX_BATCH, sizeof(int) * n_seqs * D1);
+  return DREAM_OK;
+}
+
+// ------------------------------------------------------------------------------------- read-back
+
+extern "C" dream_status dream_seq_state(dream_ctx *c, int32_t seq, int32_t *verified_len, int32_t *pending, int32_t *tap) {
+  dream_status s = check_seq(c, seq);
+  if (s) return s;
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  if (verified_len) CUDA_OK(c, cudaMemcpy(verified_len, c->sd.P + seq, sizeof(int), cudaMemcpyDeviceToHost));
+  if (pending) CUDA_OK(c, cudaMemcpy(pending, c->sd.pending + seq, sizeof(int), cudaMemcpyDeviceToHost));
+  if (tap) CUDA_OK(c, cudaMemcpy(tap, c->sd.tap + seq, sizeof(int), cudaMemcpyDeviceToHost));
+  return DREAM_OK;
+}
+
+template <typename T>
+static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, int index, float *dst) {
+  const dream_config &f = c->cfg;
+  int w = f.n_kv_heads * f.head_dim, d = f.d_model;
+  float *tmp = c->gout;     // scratch: idle between calls
+  int count = what <= 5 ? w : d;
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  if (what == 0 || what == 1) {
+    if (layer < 0 || layer >= f.n_layers || index < 0 || index >= f.max_seq) return fail(c, DREAM_E_ARG, "layer/position out of range");
+    if (c->seq_pages[seq].empty()) return fail(c, DREAM_E_STATE, "sequence has no pages");
+    int pg = c->seq_pages[seq][index / f.page_tokens], in = index % f.page_tokens;
+    const T *base = (const T *)c->kv_pool + (size_t)layer * c->layer_stride + (size_t)what * c->kv_stride;
+    for (int h = 0; h < f.n_kv_heads; ++h) {
+      const T *src = base + (((size_t)pg * f.n_kv_heads + h) * f.page_tokens + in) * f.head_dim;
+      k_read_row<T><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
+    }
+  } else if (what >= 2 && what <= 5) {
+    if (index < 0 || index >= c->cap_rows) return fail(c, DREAM_E_ARG, "row out of range");
+    const T *base = (const T *)(what <= 3 ? c->dmem : c->dself);
+    int kvsel = (what - 2) & 1;
+    for (int h = 0; h < f.n_kv_heads; ++h) {
+      const T *src = base + ((((size_t)seq * 2 + kvsel) * f.n_kv_heads + h) * c->cap_rows + index) * f.head_dim;
+      k_read_row<T><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
+    }
+  } else if (what == 6 || what == 7) {
+    if (index < 0 || index >= ROW_CHUNK) return fail(c, DREAM_E_ARG, "row out of range");
+    const float *src = (what == 6 ? c->tapbuf : c->x) + (size_t)index * d;
+    k_read_row<float><<<(d + 255) / 256, 256, 0, c->stream>>>(src, tmp, d);
+  } else return fail(c, DREAM_E_ARG, "unknown buffer id %d", what);
+  CUDA_OK(c, cudaMemcpyAsync(dst, tmp, sizeof(float) * count, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_debug_read(dream_ctx *c, int32_t seq, int32_t what, int32_t layer, int32_t index, float *dst) {
+  dream_status s = check_seq(c, seq);
+  if (s) return s;
+  if (!dst) return fail(c, DREAM_E_ARG, "null destination");
+  return c->cfg.dtype == DREAM_BF16 ? debug_read_impl<bf16>(c, seq, what, layer, index, dst)
+                                    : debug_read_impl<float>(c, seq, what, layer, index, dst);
+}

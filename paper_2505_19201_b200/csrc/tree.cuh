@@ -1,0 +1,338 @@
+// Integer side of the loop: per-sequence state, tree expansion and re-ranking
+// (Section 3.1, tree drafting; Section 4: depth, children per node, maximum draft length),
+// verification row set-up, greedy acceptance (Section 2.1) and KV-cache compaction.
+#pragma once
+#include "common.cuh"
+#include "rows.cuh"
+
+#define DREAM_MAX_BATCH 8
+#define DREAM_MAX_DEPTH 15
+
+// Per-sequence device state (arrays indexed by sequence id).
+struct SeqDev {
+  int *P;            // verified length: target KV slots [0, P) are final
+  int *pending;      // token at position P (known, not yet run through the target)
+  int *tap;          // selected feature layer l* (1-based)
+  int *nperm_d;      // permanent rows of the draft self-attention cache
+  int *nperm_m;      // permanent rows of the cross-attention memory
+  int *n_new;        // tokens verified by the last accept, still without draft K/V rows
+  int *new_tok;      // [seq][DREAM_MAX_DEPTH+1]
+  int *new_pos;      // [seq][DREAM_MAX_DEPTH+1]
+  int *last_P;       // P before the last accept
+  int *last_A;       // accepted draft tokens of the last accept
+  int *path;         // [seq][DREAM_MAX_DEPTH+1] tree nodes on the accepted path
+};
+
+// Static shape of the draft tree for one configuration (host-computed).
+struct TreeShape {
+  int D, K, N, T;                       // depth, children per node, node cap, nodes incl. root
+  int beam[DREAM_MAX_DEPTH + 1];        // beam[p] = nodes expanded in pass p+1 (beam[0] = 1)
+  int in_off[DREAM_MAX_DEPTH + 1];      // first input-node index of pass p+1
+  int cand_off[DREAM_MAX_DEPTH + 1];    // first candidate index created by pass p+1
+  int NI, NC;                           // input nodes and candidates in total
+};
+
+// Draft-side tree storage of all sequences (device).
+struct DraftTreeDev {
+  int *in_tok, *in_depth, *in_cand;     // [seq][NI]
+  float *in_cum;                        // [seq][NI]
+  unsigned long long *in_anc;           // [seq][NI] ancestor-or-self bits over input nodes
+  int *cand_tok, *cand_par, *cand_depth;  // [seq][NC]; cand_par = candidate index or -1 (root)
+  float *cand_cum;                      // [seq][NC]
+};
+
+// Row metadata of the current launch set.
+struct RowMeta {
+  int *seq, *tok, *pos, *slot, *dst, *in;
+};
+
+struct TreePtrs {                       // device buffers of one caller-visible tree
+  int *tokens, *parent, *depth;
+  uint32_t *mask;
+  float *cum;
+};
+struct TreeBatch { TreePtrs t[DREAM_MAX_BATCH]; int seq[DREAM_MAX_BATCH]; };
+
+// ---------------------------------------------------------------------------------------
+// Start of a draft call: row set of pass 1 = [root, catch-up rows...] per sequence.
+// The catch-up rows are the tokens verified by the last accept; they receive permanent
+// draft self-attention K/V rows.  One thread per sequence slot b.
+__global__ void k_draft_begin(TreeBatch tb, int B, SeqDev s, DraftTreeDev dt, TreeShape ts,
+                              RowMeta rm, int rows_per_seq, int cap_rows, int *status) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  int seq = tb.seq[b];
+  int P = s.P[seq], nn = s.n_new[seq], np = s.nperm_d[seq];
+  if (np + nn + ts.NI > cap_rows || s.nperm_m[seq] + ts.NI > cap_rows) {
+    atomicMax(status, DREAM_DEV_BAD_INDEX);
+    nn = 0;
+  }
+  int base = b * rows_per_seq;
+  for (int j = 0; j < rows_per_seq; ++j) {
+    int r = base + j;
+    rm.seq[r] = seq;
+    if (j == 0) {
+      rm.tok[r] = s.pending[seq]; rm.pos[r] = P; rm.dst[r] = np + nn; rm.in[r] = 0;
+    } else if (j - 1 < nn) {
+      rm.tok[r] = s.new_tok[seq * (DREAM_MAX_DEPTH + 1) + j - 1];
+      rm.pos[r] = s.new_pos[seq * (DREAM_MAX_DEPTH + 1) + j - 1];
+      rm.dst[r] = np + j - 1; rm.in[r] = -1;
+    } else {
+      rm.tok[r] = -1; rm.pos[r] = 0; rm.dst[r] = -1; rm.in[r] = -1;
+    }
+  }
+  s.nperm_d[seq] = np + nn;
+  s.n_new[seq] = 0;
+  long long o = (long long)seq * ts.NI;
+  dt.in_tok[o] = s.pending[seq]; dt.in_depth[o] = 0; dt.in_cand[o] = -1;
+  dt.in_cum[o] = 0.f; dt.in_anc[o] = 1ull;
+}
+
+// After pass `p` (1-based): turn the per-row top-K into candidates, pick the next beam.
+// One block per sequence slot.  Rows of this pass: row b*rows_per_seq + i expands input
+// node in_off[p-1] + i, i < beam[p-1].
+__global__ void k_tree_expand(TreeBatch tb, SeqDev s, DraftTreeDev dt, TreeShape ts, int p,
+                              int rows_per_seq, const float *__restrict__ top_val,
+                              const int *__restrict__ top_id, const float *__restrict__ lse,
+                              RowMeta rm_next, int next_rows_per_seq) {
+  __shared__ float cum[256];
+  int b = blockIdx.x, seq = tb.seq[b];
+  int K = ts.K, m = ts.beam[p - 1], nnew = m * K;
+  long long io = (long long)seq * ts.NI, co = (long long)seq * ts.NC;
+  int c0 = ts.cand_off[p - 1];
+  for (int t = threadIdx.x; t < nnew; t += blockDim.x) {
+    int i = t / K, j = t - i * K;
+    int node = ts.in_off[p - 1] + i, r = b * rows_per_seq + i;
+    float cm = dt.in_cum[io + node] + (top_val[r * K + j] - lse[r]);
+    dt.cand_tok[co + c0 + t] = top_id[r * K + j];
+    dt.cand_par[co + c0 + t] = dt.in_cand[io + node];
+    dt.cand_depth[co + c0 + t] = dt.in_depth[io + node] + 1;
+    dt.cand_cum[co + c0 + t] = cm;
+    cum[t] = cm;
+  }
+  __syncthreads();
+  if (p >= ts.D) return;
+  int nb = ts.beam[p], P = s.P[seq], np = s.nperm_d[seq];
+  for (int t = threadIdx.x; t < nnew; t += blockDim.x) {
+    int rank = 0;
+    for (int u = 0; u < nnew; ++u) rank += better(cum[u], u, cum[t], t) ? 1 : 0;
+    if (rank >= nb) continue;
+    int i = t / K, par_in = ts.in_off[p - 1] + i, me = ts.in_off[p] + rank;
+    dt.in_tok[io + me] = dt.cand_tok[co + c0 + t];
+    dt.in_depth[io + me] = p;
+    dt.in_cand[io + me] = c0 + t;
+    dt.in_cum[io + me] = cum[t];
+    dt.in_anc[io + me] = dt.in_anc[io + par_in] | (1ull << me);
+    int r = b * next_rows_per_seq + rank;
+    rm_next.seq[r] = seq; rm_next.tok[r] = dt.cand_tok[co + c0 + t]; rm_next.pos[r] = P + p;
+    rm_next.dst[r] = np + me; rm_next.in[r] = me;
+  }
+  for (int t = nb + threadIdx.x; t < next_rows_per_seq; t += blockDim.x) {   // idle tail rows
+    int r = b * next_rows_per_seq + t;
+    rm_next.seq[r] = seq; rm_next.tok[r] = -1; rm_next.pos[r] = 0; rm_next.dst[r] = -1; rm_next.in[r] = -1;
+  }
+}
+
+// After the last pass: keep the N best candidates by cumulative log-probability (ties ->
+// earlier candidate), order them by creation index behind the root, remap parents, build
+// the ancestor-or-self masks.  One block per sequence slot.
+__global__ void k_tree_finalize(TreeBatch tb, SeqDev s, DraftTreeDev dt, TreeShape ts) {
+  extern __shared__ int sm[];
+  int NC = ts.NC, Nsel = ts.T - 1;
+  int *sel = sm, *node_of = sm + NC;       // [NC] each
+  int b = blockIdx.x, seq = tb.seq[b];
+  long long co = (long long)seq * ts.NC;
+  TreePtrs tp = tb.t[b];
+  for (int t = threadIdx.x; t < NC; t += blockDim.x) {
+    float ct = dt.cand_cum[co + t];
+    int rank = 0;
+    for (int u = 0; u < NC; ++u) rank += better(dt.cand_cum[co + u], u, ct, t) ? 1 : 0;
+    sel[t] = rank < Nsel ? 1 : 0;
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < NC; t += blockDim.x) {
+    int before = 0;
+    for (int u = 0; u < t; ++u) before += sel[u];
+    node_of[t] = sel[t] ? before + 1 : -1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    tp.tokens[0] = s.pending[seq]; tp.parent[0] = -1; tp.depth[0] = 0;
+    if (tp.cum) tp.cum[0] = 0.f;
+    tp.mask[0] = 1u; tp.mask[1] = 0u; tp.mask[2] = 0u; tp.mask[3] = 0u;
+  }
+  for (int t = threadIdx.x; t < NC; t += blockDim.x) {
+    int me = node_of[t];
+    if (me < 0) continue;
+    int par = dt.cand_par[co + t];
+    tp.tokens[me] = dt.cand_tok[co + t];
+    tp.parent[me] = par < 0 ? 0 : node_of[par];
+    tp.depth[me] = dt.cand_depth[co + t];
+    if (tp.cum) tp.cum[me] = dt.cand_cum[co + t];
+    uint32_t mk[4] = {1u, 0u, 0u, 0u};               // the root is everyone's ancestor
+    int a = t;
+    while (a >= 0) { int na = node_of[a]; mk[na >> 5] |= 1u << (na & 31); a = dt.cand_par[co + a]; }
+    for (int wd = 0; wd < 4; ++wd) tp.mask[me * 4 + wd] = mk[wd];
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Verification rows: node i of slot b is row b*T + i at position P + depth[i], KV slot P + i.
+__global__ void k_verify_setup(TreeBatch tb, int B, int T, SeqDev s, RowMeta rm, uint32_t *mask,
+                               int max_seq, int *status) {
+  int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= B * T) return;
+  int b = r / T, i = r - b * T, seq = tb.seq[b];
+  TreePtrs tp = tb.t[b];
+  int P = s.P[seq], dep = tp.depth[i], par = tp.parent[i];
+  bool bad = (i == 0 ? par != -1 || dep != 0 : par < 0 || par >= i || dep != tp.depth[par < 0 ? 0 : par] + 1);
+  if (P + T > max_seq) bad = true;
+  if (bad) atomicMax(status, DREAM_DEV_BAD_INDEX);
+  rm.seq[r] = seq; rm.tok[r] = tp.tokens[i]; rm.pos[r] = P + (bad ? 0 : dep);
+  rm.slot[r] = bad ? 0 : P + i; rm.in[r] = i;
+  for (int wd = 0; wd < 4; ++wd) mask[r * 4 + wd] = tp.mask[i * 4 + wd];
+}
+
+// Greedy acceptance (Section 2.1): from the root, move to the child whose token equals the
+// current node's target argmax; stop when there is none.  Emits the accepted tokens plus
+// the target's own token, records the path, and advances the sequence state.
+// One warp per sequence slot.
+__global__ void k_accept(TreeBatch tb, int B, int T, int D, SeqDev s, const int *__restrict__ argmax,
+                         int *accept_len, int *out_tokens, int *comp_src) {
+  int b = blockIdx.x, lane = threadIdx.x, seq = tb.seq[b];
+  TreePtrs tp = tb.t[b];
+  const int *am = argmax + b * T;
+  int cur = 0, A = 0;
+  int *path = s.path + seq * (DREAM_MAX_DEPTH + 1);
+  if (lane == 0) path[0] = 0;
+  while (A < D) {
+    int g = am[cur], found = 0x7fffffff;
+    for (int i = 1 + lane; i < T; i += 32)
+      if (tp.parent[i] == cur && tp.tokens[i] == g) found = min(found, i);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
+    if (found == 0x7fffffff) break;
+    cur = found; ++A;
+    if (lane == 0) { path[A] = cur; out_tokens[b * (D + 1) + A - 1] = tp.tokens[cur]; }
+  }
+  if (lane == 0) {
+    int g = am[cur], P = s.P[seq];
+    out_tokens[b * (D + 1) + A] = g;
+    for (int j = A + 1; j <= D; ++j) out_tokens[b * (D + 1) + j] = -1;
+    accept_len[b] = A;
+    for (int j = 0; j <= D; ++j) {
+      if (comp_src) comp_src[b * (D + 1) + j] = j <= A ? path[j] : -1;
+      if (j <= A) {
+        s.new_tok[seq * (DREAM_MAX_DEPTH + 1) + j] = tp.tokens[path[j]];
+        s.new_pos[seq * (DREAM_MAX_DEPTH + 1) + j] = P + j;
+      }
+    }
+    s.n_new[seq] = A + 1;
+    s.last_P[seq] = P; s.last_A[seq] = A;
+    s.P[seq] = P + A + 1;
+    s.pending[seq] = g;
+  }
+}
+
+// KV compaction: the rows of path node j move from tail slot P + path[j] to P + j, for every
+// layer and both K and V.  path[j] >= j and strictly increasing, and each thread owns one
+// element offset across all rows, so the ascending in-place copy is race-free.
+// grid (L*2, B); also fills the row map for the memory-append GEMM that follows.
+template <typename T>
+__global__ void k_compact_kv(TreeBatch tb, SeqDev s, void *pool, long long layer_stride,
+                             long long kv_stride, PagedKV kv) {
+  int b = blockIdx.y, seq = tb.seq[b];
+  int layer = blockIdx.x >> 1, which = blockIdx.x & 1;
+  T *base = (T *)pool + (long long)layer * layer_stride + (long long)which * kv_stride;
+  int P = s.last_P[seq], A = s.last_A[seq];
+  const int *path = s.path + seq * (DREAM_MAX_DEPTH + 1);
+  int w = kv.hkv * kv.hd;
+  for (int e = threadIdx.x; e < w; e += blockDim.x) {
+    int h = e / kv.hd, x = e - h * kv.hd;
+    for (int j = 1; j <= A; ++j) {
+      int src = path[j];
+      if (src == j) continue;
+      base[kv.off(seq, P + j, h) + x] = base[kv.off(seq, P + src, h) + x];
+    }
+  }
+}
+
+// Row map for the cross-memory append after an accept: row b*(D+1)+j takes the tapped
+// features of path node j (tap-buffer row b*T + path[j]) and lands in memory row
+// nperm_m + j.  Then nperm_m advances.  One thread per sequence slot.
+__global__ void k_accept_rows(TreeBatch tb, int B, int T, int D, SeqDev s, int *gather_idx,
+                              RowMeta rm, int cap_rows, int *status) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  int seq = tb.seq[b], A = s.last_A[seq], nm = s.nperm_m[seq];
+  if (nm + A + 1 > cap_rows) { atomicMax(status, DREAM_DEV_BAD_INDEX); A = -1; }
+  for (int j = 0; j <= D; ++j) {
+    int r = b * (D + 1) + j;
+    rm.seq[r] = seq;
+    gather_idx[r] = j <= A ? b * T + s.path[seq * (DREAM_MAX_DEPTH + 1) + j] : -1;
+    rm.dst[r] = j <= A ? nm + j : -1;
+  }
+  s.nperm_m[seq] = nm + A + 1;
+}
+
+// ---------------------------------------------------------------------------------------
+// Tap-layer selection (Section 3.2): argmin (or argmax) of AE over [lo, hi], ties -> lower layer.
+__global__ void k_select_tap(const float *__restrict__ ae, int mode, int fixed, int lo, int hi,
+                             int *tap_out, int *tap_user) {
+  if (threadIdx.x || blockIdx.x) return;
+  int best = fixed;
+  if (mode != 0) {
+    best = lo;
+    for (int l = lo + 1; l <= hi; ++l) {
+      float a = ae[l - 1], bb = ae[best - 1];
+      if (mode == 1 ? a < bb : a > bb) best = l;
+    }
+  }
+  *tap_out = best;
+  if (tap_user) *tap_user = best;
+}
+
+// Visual-token selection (Section 3.3): the k visual tokens with the largest importance (ties
+// -> lower index), returned ascending; then the compressed context C = kept visual
+// positions plus all text positions, ascending.  One block.
+__global__ void k_select_visual(const float *__restrict__ scores_all, long long layer_stride,
+                                const int *__restrict__ tap, int tap_lo, int v, int k, int vis_start,
+                                int n, const int *__restrict__ forced, int *kept, float *scores_out,
+                                int *ctx_pos, int *flags /* [n] scratch */) {
+  const float *sc = scores_all + (long long)(*tap - tap_lo) * layer_stride;
+  for (int j = threadIdx.x; j < n; j += blockDim.x) flags[j] = (j < vis_start || j >= vis_start + v) ? 1 : 0;
+  __syncthreads();
+  if (forced) {
+    for (int j = threadIdx.x; j < k; j += blockDim.x) flags[vis_start + forced[j]] = 1;
+  } else {
+    for (int j = threadIdx.x; j < v; j += blockDim.x) {
+      float sj = sc[j];
+      int rank = 0;
+      for (int u = 0; u < v; ++u) rank += better(sc[u], u, sj, j) ? 1 : 0;
+      if (rank < k) flags[vis_start + j] = 1;
+    }
+  }
+  for (int j = threadIdx.x; j < v; j += blockDim.x) if (scores_out) scores_out[j] = sc[j];
+  __syncthreads();
+  for (int j = threadIdx.x; j < n; j += blockDim.x) {
+    if (!flags[j]) continue;
+    int before = 0;
+    for (int u = 0; u < j; ++u) before += flags[u];
+    ctx_pos[before] = j;
+    if (j >= vis_start && j < vis_start + v && kept) {
+      int bv = 0;
+      for (int u = vis_start; u < j; ++u) bv += flags[u];
+      kept[bv] = j - vis_start;
+    }
+  }
+}
+
+// Row maps of the context-building GEMMs after compression: row i <-> context position
+// ctx_pos[i] (or position i when the memory keeps every prompt position).
+__global__ void k_ctx_rows(const int *__restrict__ ctx_pos, int count, int identity, int seq,
+                           RowMeta rm, int *gather_idx, int row0) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  int p = identity ? row0 + i : ctx_pos[i];
+  rm.seq[i] = seq; rm.pos[i] = p; rm.dst[i] = row0 + i; gather_idx[i] = p;
+}

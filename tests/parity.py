@@ -1,0 +1,211 @@
+"""GPU-vs-oracle parity harness (used by the -m gpu tests, the smoke check and nothing else).
+
+Runs the CUDA path through the C ABI and the CPU oracle on the same seeded inputs, step by
+step, and compares them.  Integer decisions (token ids, tap layer, kept indices, tree
+arrays, accept lengths, compaction maps) must be bit-exact wherever the oracle's decision
+margin exceeds `dec_tol`; inside the margin either choice is accepted, the oracle adopts
+the GPU's choice so that later steps stay comparable, and the exemption is counted.
+Floating-point outputs must agree within (max_abs, rel_l2).
+"""
+import torch
+
+from oracle.dream_oracle import DreamOracle, OracleConfig, make_tree
+from paper_2505_19201_b200 import api, configs, synth
+
+
+class Tol:
+    def __init__(self, dtype):
+        bf = dtype == "bf16"
+        self.max_abs = 3e-2 if bf else 1e-4       # logits, hidden states (stated for bf16; derived for fp32)
+        self.rel_l2 = 1e-2 if bf else 1e-5
+        self.dec = 1e-2                           # decision margin below which either choice is accepted
+        self.ae_abs = 1e-3 if bf else 1e-5        # average attention entropy
+        self.score_rel = 1e-3 if bf else 1e-5     # visual-token importance, relative to the largest score
+
+
+def close(a, b, tol, what, report):
+    a, b = a.double().flatten(), b.double().flatten()
+    ma = float((a - b).abs().max()) if a.numel() else 0.0
+    rl = float((a - b).norm() / (b.norm() + 1e-30))
+    report.setdefault("float", []).append((what, ma, rl))
+    assert ma <= tol.max_abs, f"{what}: max-abs {ma:.3e} > {tol.max_abs} (rel-L2 {rl:.3e})"
+    assert rl <= tol.rel_l2, f"{what}: rel-L2 {rl:.3e} > {tol.rel_l2} (max-abs {ma:.3e})"
+
+
+def valid_tree(t, T):
+    assert len(t["tokens"]) == T and t["parent"][0] == -1 and t["depth"][0] == 0
+    for i in range(1, T):
+        p = t["parent"][i]
+        assert 0 <= p < i and t["depth"][i] == t["depth"][p] + 1
+        assert t["mask"][i] == t["mask"][p] | {i}
+    for i in range(T):
+        kids = [t["tokens"][j] for j in range(1, T) if t["parent"][j] == i]
+        assert len(kids) == len(set(kids))
+
+
+class Pair:
+    """One model on both sides: the oracle on the CPU and a library context on the GPU."""
+
+    def __init__(self, preset, oracle_dtype=None, device="cuda:0", seed=0, max_batch=None, **over):
+        self.p = p = configs.scaled(preset, **over) if isinstance(preset, str) else dict(preset, **over)
+        self.tol = Tol(p["dtype"])
+        self.device = device
+        odt = oracle_dtype or (torch.float32 if p["dtype"] == "bf16" else torch.float64)
+        self.twg = synth.target_weights(p, seed, device)
+        self.dwg = synth.draft_weights(p, seed, device)
+        cpu = lambda w: [t.cpu() for t in w] if isinstance(w, list) else w.cpu()
+        self.orc = DreamOracle(OracleConfig.from_preset(p), {k: cpu(v) for k, v in self.twg.items()},
+                               {k: cpu(v) for k, v in self.dwg.items()}, odt)
+        self.odt = odt
+        self.cfg = api.make_config(p, max_batch=max_batch)
+        self.ctx = api.Context(self.cfg, self.twg, self.dwg, device)
+        self.T = self.ctx.T
+        self.report = dict(exempt=0, decisions=0)
+        self.st = {}
+
+    def _decide(self, same, margin, what):
+        self.report["decisions"] += 1
+        if same:
+            return True
+        assert margin <= self.tol.dec, f"{what}: mismatch with oracle margin {margin:.3e} > {self.tol.dec}"
+        self.report["exempt"] += 1
+        return False
+
+    # ------------------------------------------------------------------ prefill + compression
+    def prefill(self, seq=0, seq_seed=0, vis_start=0, k=None):
+        p, dev, tol = self.p, self.device, self.tol
+        vis, ids = synth.request_inputs(p, seq_seed, dev)
+        tok = torch.zeros(1, dtype=torch.int32, device=dev)
+        mg = torch.zeros(1, dtype=torch.float32, device=dev)
+        ae = torch.zeros(p["n_layers"], dtype=torch.float32, device=dev)
+        tap = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.ctx.dream_prefill(seq, vis, vis_start, ids, tok, mg, ae, tap)
+        st, otok, omargin = self.orc.prefill(vis.cpu().to(self.odt), vis_start, ids.cpu().tolist())
+        self.ctx.dream_poll()
+        assert float((ae.cpu().double() - st.entropy).abs().max()) <= tol.ae_abs, "layer entropy"
+        if not self._decide(int(tok) == otok, omargin, "first token"):
+            st.pending = int(tok)
+        if not self._decide(int(tap) == st.tap, getattr(st, "tap_margin", float("inf")), "tap layer"):
+            st.tap = int(tap)
+        k = p["k_visual"] if k is None else k
+        kept = torch.zeros(max(k, 1), dtype=torch.int32, device=dev)
+        sc = torch.zeros(max(p["n_visual"], 1), dtype=torch.float32, device=dev)
+        self.ctx.dream_compress_visual(seq, k, None, kept, sc)
+        okept, osc, omargin = self.orc.compress_visual(st, k)
+        self.ctx.dream_poll()
+        scale = float(osc.abs().max()) if osc.numel() else 1.0
+        assert float((sc.cpu().double()[:p["n_visual"]] - osc.double()).abs().max()) <= tol.score_rel * scale, "importance"
+        gk = kept.cpu().tolist()[:k]
+        if not self._decide(gk == okept.tolist(), omargin / max(scale, 1e-30) * (tol.dec / tol.score_rel), "kept visual tokens"):
+            assert gk == sorted(set(gk)) and all(0 <= j < p["n_visual"] for j in gk)
+            self.orc.compress_visual(st, k, forced_idx=gk)
+        self.st[seq] = st
+        self.report["first_token"] = int(tok)
+        self.report["entropy_gap"] = float((ae.cpu().double() - st.entropy).abs().max())
+        return st
+
+    # ------------------------------------------------------------------ one round
+    def step(self, seqs=(0,), inject=None, check_cache_rows=2):
+        """Draft, verify, accept on both sides; `inject` maps seq -> oracle-format tree to verify instead."""
+        p, dev, tol, T, ctx, orc = self.p, self.device, self.tol, self.T, self.ctx, self.orc
+        B, D, V = len(seqs), p["tree_depth"], p["vocab"]
+        trees = [ctx.new_tree() for _ in seqs]
+        ctx.dream_draft_tree(list(seqs), trees)
+        use = []
+        for b, s in enumerate(seqs):
+            st = self.st[s]
+            od = orc.draft_tree(st)
+            gd = trees[b].to_host()
+            valid_tree(gd, T)
+            same = all(gd[k] == od[k] for k in ("tokens", "parent", "depth", "mask"))
+            self._decide(same, od["min_margin"], "draft tree")
+            if same:
+                close(torch.tensor(gd["cum"]), torch.tensor(od["cum"]), tol, "draft cum_logp", self.report)
+            else:       # near-tie: compare scores of the nodes both sides kept
+                key = lambda t, i: self._path(t, i)
+                om = {key(od, i): od["cum"][i] for i in range(len(od["tokens"]))}
+                common = [(gd["cum"][i], om[key(gd, i)]) for i in range(T) if key(gd, i) in om]
+                self.report.setdefault("tree_overlap", []).append(len(common) / T)
+                if common:
+                    a, bb = zip(*common)
+                    assert max(abs(x - y) for x, y in zip(a, bb)) <= max(tol.max_abs, 3 * tol.dec), "draft cum_logp (common nodes)"
+            chosen = od if inject is None or s not in inject else inject[s]
+            if inject is not None and s in inject:
+                chosen = make_tree(inject[s]["tokens"], inject[s]["parent"])
+                assert len(chosen["tokens"]) == T
+            if not same and (inject is None or s not in inject):
+                chosen = gd                       # the oracle adopts the GPU's (valid) tree on a near-tie
+            trees[b].load(chosen["tokens"], chosen["parent"])
+            use.append(chosen)
+        am = torch.zeros(B * T, dtype=torch.int32, device=dev)
+        mg = torch.zeros(B * T, dtype=torch.float32, device=dev)
+        lg = torch.zeros(B * T, V, dtype=torch.float32, device=dev)
+        ctx.dream_verify_tree(list(seqs), trees, am, mg, lg)
+        alen = torch.zeros(B, dtype=torch.int32, device=dev)
+        outt = torch.zeros(B * (D + 1), dtype=torch.int32, device=dev)
+        csrc = torch.zeros(B * (D + 1), dtype=torch.int32, device=dev)
+        ctx.dream_poll()
+        gam, glg = am.cpu().tolist(), lg.cpu()
+        hid = {(b, i): ctx.dream_debug_read(seqs[b], 7, 0, b * T + i) for b in range(B) for i in (0, T - 1)}
+        tapr = {(b, i): ctx.dream_debug_read(seqs[b], 6, 0, b * T + i) for b in range(B) for i in (0, T - 1)}
+        ctx.dream_accept(list(seqs), trees, am, alen, outt, csrc)
+        ctx.dream_poll()
+        results = []
+        for b, s in enumerate(seqs):
+            st, tree = self.st[s], use[b]
+            ver = orc.verify_tree(st, tree)
+            close(glg[b * T:(b + 1) * T], ver["logits"], tol, "verify logits", self.report)
+            for i in (0, T - 1):
+                close(hid[(b, i)], ver["hidden"][i], tol, "final hidden", self.report)
+                close(tapr[(b, i)], ver["tap_rows"][i], tol, "tapped features", self.report)
+            for i in range(T):
+                if not self._decide(gam[b * T + i] == ver["argmax"][i], ver["margin"][i], f"argmax of node {i}"):
+                    ver["argmax"][i] = gam[b * T + i]
+            A, out, path = orc.accept(tree, ver["argmax"])
+            P0 = st.P
+            orc.commit(st, tree, ver, path, out)
+            assert int(alen[b]) == A, f"accept length {int(alen[b])} != {A}"
+            assert outt.cpu().tolist()[b * (D + 1):b * (D + 1) + A + 1] == out, "emitted tokens"
+            assert csrc.cpu().tolist()[b * (D + 1):b * (D + 1) + A + 1] == path, "compaction map"
+            gP, gpend, _ = ctx.dream_seq_state(s)
+            assert (gP, gpend) == (st.P, st.pending), "sequence state"
+            # cache rows after compaction: the accepted path, a prefix row, the newest memory rows
+            L = p["n_layers"]
+            for l in sorted({0, L - 1}):
+                for pos in sorted({0, P0 - 1, P0, st.P - 1})[:2 + check_cache_rows]:
+                    close(ctx.dream_debug_read(s, 0, l, pos), st.K[l][pos].flatten(), tol, "target K row", self.report)
+                    close(ctx.dream_debug_read(s, 1, l, pos), st.V[l][pos].flatten(), tol, "target V row", self.report)
+            nm = st.mK.shape[0]
+            for row in sorted({0, nm - A - 1, nm - 1}):
+                close(ctx.dream_debug_read(s, 2, 0, row), st.mK[row].flatten(), tol, "memory K row", self.report)
+                close(ctx.dream_debug_read(s, 3, 0, row), st.mV[row].flatten(), tol, "memory V row", self.report)
+            results.append(dict(A=A, out=out, path=path))
+        return results
+
+    def check_draft_cache(self, seq=0):
+        """Draft self-attention rows (context + caught-up tokens) against the oracle's."""
+        st = self.st[seq]
+        n = st.dK.shape[0]
+        for row in sorted({0, n // 2, n - 1}):
+            close(self.ctx.dream_debug_read(seq, 4, 0, row), st.dK[row].flatten(), self.tol, "draft K row", self.report)
+            close(self.ctx.dream_debug_read(seq, 5, 0, row), st.dV[row].flatten(), self.tol, "draft V row", self.report)
+
+    @staticmethod
+    def _path(t, i):
+        out = []
+        while i > 0:
+            out.append(t["tokens"][i])
+            i = t["parent"][i]
+        return tuple(reversed(out))
+
+    def summary(self):
+        r = self.report
+        worst = {}
+        for what, ma, rl in r.get("float", []):
+            w = worst.setdefault(what, [0.0, 0.0])
+            w[0], w[1] = max(w[0], ma), max(w[1], rl)
+        return dict(decisions=r["decisions"], exempt=r["exempt"], worst=worst,
+                    tree_overlap=r.get("tree_overlap", []))
+
+    def close(self):
+        self.ctx.close()
