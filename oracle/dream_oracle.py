@@ -6,9 +6,11 @@ written from the paper's method section with plain PyTorch CPU tensor ops
 It shares no code with the CUDA path and imports nothing from it.  Only the
 tests, the smoke check and the benchmark's CPU-baseline leg may call it.
 
-Precision: `dtype` is the arithmetic and activation/KV storage type.  float64 is
+Precision: `dtype` is the arithmetic and activation storage type.  float64 is
 used for the pins and the toy model; float32 is used for the bf16 model shapes
-(weights are taken as given, i.e. bf16-rounded values, and up-converted).
+(weights are taken as given, i.e. bf16-rounded values, and up-converted).  For
+those shapes the target KV cache is a bf16 store: `kv_dtype=torch.bfloat16` rounds
+each K/V row once on entry to the cache; everything computed from it stays fp32.
 
 Readings taken where the paper is silent (each is listed in the design notes):
 pre-norm decoder blocks with RMSNorm, rotary positions (half-split pairing) on
@@ -167,8 +169,11 @@ class SeqState:
 
 
 class DreamOracle:
-    def __init__(self, cfg, tw, dw, dtype=torch.float64):
-        self.cfg, self.tw, self.dw, self.dtype = cfg, tw, dw, dtype
+    def __init__(self, cfg, tw, dw, dtype=torch.float64, kv_dtype=None):
+        """kv_dtype: storage type of the target KV cache (None = same as dtype).  With
+        torch.bfloat16 every K/V row is rounded once, when it enters the cache, and read
+        back from there by all later arithmetic (which stays in `dtype`)."""
+        self.cfg, self.tw, self.dw, self.dtype, self.kv_dtype = cfg, tw, dw, dtype, kv_dtype
 
     # ------------------------------------------------------------------ target block
     def _block(self, x, l, pos, Kc, Vc, mask, want_probs=False):
@@ -185,6 +190,8 @@ class DreamOracle:
         k = qkv[:, H * hd:(H + Hkv) * hd].reshape(-1, Hkv, hd)
         v = qkv[:, (H + Hkv) * hd:].reshape(-1, Hkv, hd)
         q, k = rope(q, pos, c.rope_theta), rope(k, pos, c.rope_theta)
+        if self.kv_dtype is not None:           # the cache's storage format
+            k, v = k.to(self.kv_dtype).to(self.dtype), v.to(self.kv_dtype).to(self.dtype)
         Kall = torch.cat([Kc, k], 0) if Kc is not None and Kc.shape[0] else k
         Vall = torch.cat([Vc, v], 0) if Vc is not None and Vc.shape[0] else v
         o, probs = attention(q, Kall, Vall, mask)

@@ -72,7 +72,7 @@ __device__ __forceinline__ float dot_lane(const float (&a)[EPL], const float (&b
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
-               T *attn_out, float *lse, float *ent) {
+               T *attn_out, long long lo_delta, float *lse, float *ent) {
   constexpr int EPL = HD / 32;
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int i = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
@@ -94,7 +94,7 @@ k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H
   float inv = 1.f / st.z;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
-    attn_out[(long long)i * H * HD + h * HD + lane * EPL + e] = from_f<T>(st.acc[e] * inv);
+    store_split<T>(attn_out + (long long)i * H * HD + h * HD + lane * EPL + e, lo_delta, st.acc[e] * inv);
   if (lane == 0) {
     lse[(long long)h * n + i] = st.m + logf(st.z);
     ent[(long long)h * n + i] = logf(st.z) - st.u / st.z;
@@ -147,7 +147,8 @@ template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ row_seq,
             const int *__restrict__ row_node, const int *__restrict__ P_state,
-            const uint32_t *__restrict__ mask, int R, int T_nodes, int H, float scale, T *attn_out) {
+            const uint32_t *__restrict__ mask, int R, int T_nodes, int H, float scale, T *attn_out,
+            long long lo_delta) {
   constexpr int EPL = HD / 32;
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
@@ -179,7 +180,7 @@ k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ 
   float inv = 1.f / st.z;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
-    attn_out[(long long)r * H * HD + h * HD + lane * EPL + e] = from_f<T>(st.acc[e] * inv);
+    store_split<T>(attn_out + (long long)r * H * HD + h * HD + lane * EPL + e, lo_delta, st.acc[e] * inv);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -192,7 +193,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ row_seq,
              const int *__restrict__ row_in, const int *__restrict__ nperm,
              const unsigned long long *__restrict__ anc, int anc_stride, int strict, int R, int H,
-             float scale, T *attn_out) {
+             float scale, T *attn_out, long long lo_delta) {
   constexpr int EPL = HD / 32;
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
@@ -201,7 +202,7 @@ k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ 
   if (in < 0) return;
   int seq = row_seq[r], np = nperm[seq];
   int kvh = h / (H / kv.hkv);
-  const T *base = (const T *)kv.base;
+  const float *base = kv.base;
   long long ok = kv.off(seq, 0, kvh, 0), ov = kv.off(seq, 1, kvh, 0);
   float q[EPL], k[EPL], v[EPL];
   RowLoad<EPL, float>::ld(qbuf + ((long long)r * H + h) * HD, lane, q);
@@ -210,8 +211,8 @@ k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ 
   Soft<EPL> st;
   st.init();
   for (int j = 0; j < np; ++j) {
-    RowLoad<EPL, T>::ld(base + ok + (long long)j * HD, lane, k);
-    RowLoad<EPL, T>::ld(base + ov + (long long)j * HD, lane, v);
+    RowLoad<EPL, float>::ld(base + ok + (long long)j * HD, lane, k);
+    RowLoad<EPL, float>::ld(base + ov + (long long)j * HD, lane, v);
     st.template push<false>(dot_lane<EPL>(q, k), v);
   }
   unsigned long long bits = anc[(long long)seq * anc_stride + in];
@@ -219,12 +220,12 @@ k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ 
   while (bits) {
     int j = __ffsll((long long)bits) - 1;
     bits &= bits - 1;
-    RowLoad<EPL, T>::ld(base + ok + (long long)(np + j) * HD, lane, k);
-    RowLoad<EPL, T>::ld(base + ov + (long long)(np + j) * HD, lane, v);
+    RowLoad<EPL, float>::ld(base + ok + (long long)(np + j) * HD, lane, k);
+    RowLoad<EPL, float>::ld(base + ov + (long long)(np + j) * HD, lane, v);
     st.template push<false>(dot_lane<EPL>(q, k), v);
   }
   float inv = 1.f / st.z;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
-    attn_out[(long long)r * H * HD + h * HD + lane * EPL + e] = from_f<T>(st.acc[e] * inv);
+    store_split<T>(attn_out + (long long)r * H * HD + h * HD + lane * EPL + e, lo_delta, st.acc[e] * inv);
 }

@@ -17,24 +17,45 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
 
+// A bf16 GEMM input row is stored as two bf16 rows, hi = bf16(v) and lo = bf16(v - hi), so the
+// tensor cores see the activation to ~16 mantissa bits while the weights stream once; the two
+// partial products are added by whoever reads the GEMM output.  fp32 inputs have no lo part.
+template <typename T> __device__ __forceinline__ void store_split(T *p, long long lo_delta, float v);
+template <> __device__ __forceinline__ void store_split<float>(float *p, long long, float v) { *p = v; }
+template <> __device__ __forceinline__ void store_split<bf16>(bf16 *p, long long lo_delta, float v) {
+  bf16 hi = __float2bfloat16_rn(v);
+  *p = hi;
+  if (lo_delta) p[lo_delta] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
 // Output of a GEMM launch: `count(tile)` partial sums per 128-column tile, stacked in slots
 // of slot_stride floats.  The stream-K tensor-core kernel leaves up to three partials per
-// tile; the SIMT kernel leaves one (upc == 0).
+// tile; the SIMT kernel leaves one (upc == 0).  When the input was split into hi and lo rows
+// the products of the lo rows sit lo_off rows further down.
 struct GemmOut {
   const float *base;
   long long slot_stride;   // floats between consecutive slots
   int ld;                  // floats between consecutive rows (tokens)
   int kb;                  // k-blocks per tile
   int upc;                 // work units (tile, k-block) per CTA; 0 = single slot
+  int lo_off;              // rows between a token's hi and lo products; 0 = unsplit
 };
 
 __device__ __forceinline__ float gemm_val(const GemmOut &g, int r, int c) {
   const float *p = g.base + (long long)r * g.ld + c;
-  if (g.upc == 0) return *p;
-  long long u0 = (long long)(c >> 7) * g.kb;
-  int first = (int)(u0 / g.upc), last = (int)((u0 + g.kb - 1) / g.upc);
   float s = *p;
-  for (int i = 1; i <= last - first; ++i) s += p[(long long)i * g.slot_stride];
+  int extra = 0;
+  if (g.upc) {
+    long long u0 = (long long)(c >> 7) * g.kb;
+    extra = (int)((u0 + g.kb - 1) / g.upc) - (int)(u0 / g.upc);
+    for (int i = 1; i <= extra; ++i) s += p[(long long)i * g.slot_stride];
+  }
+  if (g.lo_off) {
+    const float *q = p + (long long)g.lo_off * g.ld;
+    float t = *q;
+    for (int i = 1; i <= extra; ++i) t += q[(long long)i * g.slot_stride];
+    s += t;
+  }
   return s;
 }
 

@@ -18,7 +18,7 @@
 #include "rows.cuh"
 #include "tree.cuh"
 
-#define ROW_CHUNK 256          // rows per GEMM launch (tensor-core tile: up to 256 tokens)
+#define ROW_CHUNK 256          // GEMM rows per launch, hi and lo rows together (tensor-core N <= 256)
 
 enum { PH_EMPTY = 0, PH_PREFILLED, PH_READY, PH_DRAFTED, PH_VERIFIED };
 
@@ -30,6 +30,8 @@ struct dream_ctx {
   TreeShape ts;
   int T, esz, qkvN, Hhd, kvN, n_cand, tap_lo_eff, cap_rows, pps, n_pages, RM, XR, gemm_rows_lm;
   int use_tc;
+  int chunk;                           // token rows per GEMM launch (128 when inputs are split)
+  long long lo_xn, lo_act, lo_att;     // element offsets of the lo planes (0 = fp32, unsplit)
   std::vector<const void *> ln1, wqkv, wo, ln2, wgu, wd;
   const void *embed, *ln_f, *lm_head;
   dream_draft_weights dw;
@@ -40,7 +42,7 @@ struct dream_ctx {
   long long kv_stride, layer_stride;
   int *page_table, *status;
   SeqDev sd;
-  void *dself, *dmem;
+  float *dself, *dmem;
   DraftTreeDev dt;
   TreePtrs itree[DREAM_MAX_BATCH];
   RowMeta rm[2];
@@ -169,6 +171,7 @@ static void derive(dream_ctx *c) {
   c->cap_rows = f.max_seq + c->ts.NI;
   c->pps = (f.max_seq + f.page_tokens - 1) / f.page_tokens;
   c->n_pages = c->pps * f.max_batch;
+  c->chunk = f.dtype == DREAM_BF16 ? ROW_CHUNK / 2 : ROW_CHUNK;
   c->RM = imax(ROW_CHUNK, f.max_prompt);
   c->XR = c->RM;
 }
@@ -191,9 +194,9 @@ static size_t carve(dream_ctx *c, char *base) {
     c->sd.new_tok = st + 9 * MB; c->sd.new_pos = c->sd.new_tok + MB * (DREAM_MAX_DEPTH + 1);
     c->sd.path = c->sd.new_pos + MB * (DREAM_MAX_DEPTH + 1);
   }
-  size_t flat = (size_t)MB * 2 * f.n_kv_heads * c->cap_rows * f.head_dim * e;
-  c->dself = a.take_bytes(flat);
-  c->dmem = a.take_bytes(flat);
+  size_t flat = (size_t)MB * 2 * f.n_kv_heads * c->cap_rows * f.head_dim;
+  c->dself = a.take<float>(flat);
+  c->dmem = a.take<float>(flat);
   c->dt.in_tok = a.take<int>((size_t)MB * NI); c->dt.in_depth = a.take<int>((size_t)MB * NI);
   c->dt.in_cand = a.take<int>((size_t)MB * NI); c->dt.in_cum = a.take<float>((size_t)MB * NI);
   c->dt.in_anc = a.take<unsigned long long>((size_t)MB * NI);
@@ -217,15 +220,19 @@ static size_t carve(dream_ctx *c, char *base) {
   c->x = a.take<float>((size_t)c->XR * d);
   c->x0 = a.take<float>((size_t)f.max_prompt * d);
   c->qbuf = a.take<float>((size_t)c->XR * c->Hhd);
-  c->attn_out = a.take_bytes((size_t)c->XR * c->Hhd * e);
-  c->xn = a.take_bytes((size_t)ROW_CHUNK * d * e);
-  c->raw = a.take_bytes((size_t)ROW_CHUNK * d * e);
-  c->act = a.take_bytes((size_t)ROW_CHUNK * f.d_ff * e);
+  int planes = f.dtype == DREAM_BF16 ? 2 : 1;
+  c->lo_xn = planes == 2 ? (long long)ROW_CHUNK * d : 0;
+  c->lo_act = planes == 2 ? (long long)ROW_CHUNK * f.d_ff : 0;
+  c->lo_att = planes == 2 ? (long long)c->XR * c->Hhd : 0;
+  c->attn_out = a.take_bytes((size_t)planes * c->XR * c->Hhd * e);
+  c->xn = a.take_bytes((size_t)planes * ROW_CHUNK * d * e);
+  c->raw = a.take_bytes((size_t)planes * ROW_CHUNK * d * e);
+  c->act = a.take_bytes((size_t)planes * ROW_CHUNK * f.d_ff * e);
   int widest = imax(imax(c->qkvN, 2 * f.d_ff), imax(d, c->Hhd));
   int lm_rows = ((imax(MB * T, MB * imax(c->ts.D + 2, f.tree_beam)) + 15) / 16) * 16;
   c->gemm_rows_lm = lm_rows;
   size_t per_slot = (size_t)imax(ROW_CHUNK * widest, 1) ;
-  size_t lm_slot = (size_t)lm_rows * f.vocab;
+  size_t lm_slot = (size_t)imin(2 * lm_rows, ROW_CHUNK) * f.vocab;
   if (lm_slot > per_slot) per_slot = lm_slot;
   c->gout_floats = per_slot;
   c->gout = a.take<float>(per_slot * GEMM_TC_MAX_SLOTS);
@@ -259,20 +266,23 @@ extern "C" dream_status dream_arena_bytes(const dream_config *cfg, size_t *bytes
 
 // ------------------------------------------------------------------------------------- GEMM dispatch
 
-// out[r][c] = sum_k X[r][k] W[c][k] for r < rows, c < N.  Returns the descriptor consumers
-// read the result through.
+// out[r][c] = sum_k X[r][k] W[c][k] for r < rows, c < N.  lo_delta != 0: X carries a second
+// plane of low-order parts lo_delta elements further on, multiplied in the same launch.
+// Returns the descriptor consumers read the result through.
 template <typename T>
-static GemmOut gemm(dream_ctx *c, const void *W, const void *X, int rows, int N, int K) {
+static GemmOut gemm(dream_ctx *c, const void *W, const void *X, long long lo_delta, int rows, int N, int K) {
   GemmOut g;
-  if (c->use_tc && sizeof(T) == 2 && gemm_tc_supported(rows, N, K)) {
-    gemm_tc_launch(&c->tc, c->stream, W, X, rows, N, K, c->gout, (long long)c->gout_floats, &g);
+  int rows_pad = (rows + 15) & ~15;
+  if (c->use_tc && sizeof(T) == 2 && gemm_tc_supported(rows_pad * (lo_delta ? 2 : 1), N, K)) {
+    gemm_tc_launch(&c->tc, c->stream, W, X, lo_delta, rows, N, K, c->gout, (long long)c->gout_floats, &g);
     c->launches++;
     return g;
   }
-  dim3 grid((N + SG_BN - 1) / SG_BN, (rows + SG_BM - 1) / SG_BM);
-  k_gemm_simt<T><<<grid, 256, 0, c->stream>>>((const T *)X, (const T *)W, c->gout, rows, N, K, N);
+  int tiles = (rows + SG_BM - 1) / SG_BM;
+  dim3 grid((N + SG_BN - 1) / SG_BN, tiles * (lo_delta ? 2 : 1));
+  k_gemm_simt<T><<<grid, 256, 0, c->stream>>>((const T *)X, (const T *)W, c->gout, rows, N, K, N, tiles, lo_delta, rows_pad);
   c->launches++;
-  g.base = c->gout; g.slot_stride = 0; g.ld = N; g.kb = 0; g.upc = 0;
+  g.base = c->gout; g.slot_stride = 0; g.ld = N; g.kb = 0; g.upc = 0; g.lo_off = lo_delta ? rows_pad : 0;
   return g;
 }
 
@@ -288,12 +298,12 @@ static PagedKV paged(dream_ctx *c, int layer) {
   kv.hd = c->cfg.head_dim;
   return kv;
 }
-static FlatKV flat(dream_ctx *c, void *base) {
+static FlatKV flat(dream_ctx *c, float *base) {
   FlatKV kv;
   kv.base = base; kv.cap = c->cap_rows; kv.hkv = c->cfg.n_kv_heads; kv.hd = c->cfg.head_dim;
   return kv;
 }
-static const GemmOut NO_GEMM = {nullptr, 0, 0, 0, 0};
+static const GemmOut NO_GEMM = {nullptr, 0, 0, 0, 0, 0};
 
 // ------------------------------------------------------------------------------------- init / free
 
@@ -415,26 +425,29 @@ __global__ void k_read_row(const T *src, float *dst, int n) {
   if (i < n) dst[i] = to_f(src[i]);
 }
 
+// Split GEMM inputs into hi and lo rows when both fit one launch (see store_split).
+static bool lo_on(const dream_ctx *c, int rows) { return c->cfg.dtype == DREAM_BF16 && ((rows + 15) & ~15) * 2 <= ROW_CHUNK; }
+
 template <typename T, int HD> struct AttnLaunch {
   static void prefill(dream_ctx *c, int layer, int seq, int n) {
     dim3 grid((n + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_prefill<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n, c->cfg.n_heads,
-           1.f / sqrtf((float)HD), (T *)c->attn_out, c->lse_pre, c->ent_pre);
+           1.f / sqrtf((float)HD), (T *)c->attn_out, c->lo_att, c->lse_pre, c->ent_pre);
   }
   static void colsum(dream_ctx *c, int layer, int seq, int n, int vis_start, int v, float *score) {
     if (v == 0) return;
     LAUNCH(c, (k_colsum<T, HD>), (v + ATT_WARPS - 1) / ATT_WARPS, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n,
            c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, score);
   }
-  static void tree(dream_ctx *c, int layer, int R) {
+  static void tree(dream_ctx *c, int layer, int R, bool lo) {
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_tree<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
-           c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out);
+           c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, lo ? c->lo_att : 0LL);
   }
-  static void draft(dream_ctx *c, const RowMeta &rm, void *cache, const int *nperm, int strict, int R) {
+  static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, bool lo) {
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_draft<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, flat(c, cache), rm.seq, rm.in, nperm,
-           c->dt.in_anc, c->ts.NI, strict, R, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out);
+           c->dt.in_anc, c->ts.NI, strict, R, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, lo ? c->lo_att : 0LL);
   }
 };
 
@@ -445,6 +458,22 @@ template <typename T, int HD> struct AttnLaunch {
     else AttnLaunch<T, 256>::call;                                \
   } while (0)
 
+// x (+= GEMM output) -> RMSNorm -> GEMM input rows in c->xn; see k_resid_norm for the side outputs.
+template <typename T>
+static void norm_rows(dream_ctx *c, float *x, const GemmOut &gin, bool has_in, const void *gain, int rows, bool lo,
+                      float *copy = nullptr, const int *row_seq = nullptr, const int *tap = nullptr, int layer = 0,
+                      bool want_raw = false) {
+  LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, lo ? c->lo_xn : 0LL);
+}
+template <typename T>
+static GemmOut mlp_rows(dream_ctx *c, const void *wgu, const void *wd, int rows, bool lo) {
+  const dream_config &f = c->cfg;
+  GemmOut g = gemm<T>(c, wgu, c->xn, lo ? c->lo_xn : 0, rows, 2 * f.d_ff, f.d_model);
+  LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, rows), 256, 0, g, (T *)c->act, f.d_ff, lo ? c->lo_act : 0LL);
+  return gemm<T>(c, wd, c->act, lo ? c->lo_act : 0, rows, f.d_model, f.d_ff);
+}
+
 // ------------------------------------------------------------------------------------- prefill
 
 template <typename T>
@@ -452,16 +481,16 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
                                  const int *ids, int q, int *first_token, float *first_margin,
                                  float *layer_entropy, int *tap_layer) {
   const dream_config &f = c->cfg;
-  int n = q + v, d = f.d_model, L = f.n_layers;
+  int n = q + v, d = f.d_model, L = f.n_layers, CH = c->chunk;
   LAUNCH(c, k_iota_rows, (n + 255) / 256, 256, 0, c->rm[0], seq, n);
   LAUNCH(c, (k_build_prompt<T>), n, 256, 0, (const T *)c->embed, (const T *)visual, ids, vis_start, v, c->x, c->x0,
          d, f.vocab, c->status);
   for (int l = 0; l < L; ++l) {
-    for (int r0 = 0; r0 < n; r0 += ROW_CHUNK) {
-      int rows = imin(ROW_CHUNK, n - r0);
-      LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, c->x + (size_t)r0 * d, NO_GEMM, 0, (const T *)c->ln1[l], f.rms_eps, d,
-             (T *)c->xn, (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-      GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, rows, c->qkvN, d);
+    for (int r0 = 0; r0 < n; r0 += CH) {
+      int rows = imin(CH, n - r0);
+      bool lo = lo_on(c, rows);
+      norm_rows<T>(c, c->x + (size_t)r0 * d, NO_GEMM, false, c->ln1[l], rows, lo);
+      GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, lo ? c->lo_xn : 0, rows, c->qkvN, d);
       LAUNCH(c, (k_qkv_post_target<T>), rows, 128, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
              paged(c, l), f.n_heads, f.rope_theta);
     }
@@ -470,23 +499,20 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
     int cand = l + 1 - c->tap_lo_eff;
     bool is_cand = cand >= 0 && cand < c->n_cand;
     if (is_cand) HD_DISPATCH(c, T, colsum(c, l, seq, n, vis_start, v, c->scores_all + (size_t)cand * imax(f.max_visual, 1)));
-    for (int r0 = 0; r0 < n; r0 += ROW_CHUNK) {
-      int rows = imin(ROW_CHUNK, n - r0);
+    for (int r0 = 0; r0 < n; r0 += CH) {
+      int rows = imin(CH, n - r0);
+      bool lo = lo_on(c, rows);
       float *xr = c->x + (size_t)r0 * d;
-      GemmOut g = gemm<T>(c, c->wo[l], (const T *)c->attn_out + (size_t)r0 * c->Hhd, rows, d, c->Hhd);
-      LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, xr, g, 1, (const T *)c->ln2[l], f.rms_eps, d, (T *)c->xn,
-             (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-      g = gemm<T>(c, c->wgu[l], c->xn, rows, 2 * f.d_ff, d);
-      LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, rows), 256, 0, g, (T *)c->act, f.d_ff);
-      g = gemm<T>(c, c->wd[l], c->act, rows, d, f.d_ff);
+      GemmOut g = gemm<T>(c, c->wo[l], (const T *)c->attn_out + (size_t)r0 * c->Hhd, c->lo_att, rows, d, c->Hhd);
+      norm_rows<T>(c, xr, g, true, c->ln2[l], rows, lo);
+      g = mlp_rows<T>(c, c->wgu[l], c->wd[l], rows, lo);
       float *copy = is_cand ? c->taps_store + ((size_t)cand * f.max_prompt + r0) * d : nullptr;
       LAUNCH(c, k_resid_add, rows, 256, 0, xr, g, d, copy);
     }
   }
   // first token: LM head on the last prompt row
-  LAUNCH(c, (k_resid_norm<T>), 1, 256, 0, c->x + (size_t)(n - 1) * d, NO_GEMM, 0, (const T *)c->ln_f, f.rms_eps, d,
-         (T *)c->xn, (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-  GemmOut g = gemm<T>(c, c->lm_head, c->xn, 1, f.vocab, d);
+  norm_rows<T>(c, c->x + (size_t)(n - 1) * d, NO_GEMM, false, c->ln_f, 1, lo_on(c, 1));
+  GemmOut g = gemm<T>(c, c->lm_head, c->xn, lo_on(c, 1) ? c->lo_xn : 0, 1, f.vocab, d);
   LAUNCH(c, k_topk_lse, 1, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
   LAUNCH(c, k_first_token, 1, 32, 0, c->top_id, c->top_val, first_token, first_margin);
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, n, c->top_id, -1, -1);
@@ -540,30 +566,31 @@ extern "C" dream_status dream_set_tap(dream_ctx *c, int32_t seq, int32_t tap_lay
 template <typename T>
 static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *forced, int *kept, float *scores) {
   const dream_config &f = c->cfg;
-  int v = c->pf_v, q = c->pf_q, n = v + q, d = f.d_model, nc = q + k;
+  int v = c->pf_v, q = c->pf_q, n = v + q, d = f.d_model, nc = q + k, CH = c->chunk;
   LAUNCH(c, k_select_visual, 1, 1024, 0, c->scores_all, (long long)imax(f.max_visual, 1), c->sd.tap + seq, c->tap_lo_eff,
          v, k, c->pf_vis_start, n, forced, kept, scores, c->ctx_pos, c->flags);
   // draft self-attention K/V of the compressed context, from the input embeddings
   const char *wkv = (const char *)c->dw.wqkv + (size_t)c->Hhd * d * c->esz;
-  for (int r0 = 0; r0 < nc; r0 += ROW_CHUNK) {
-    int rows = imin(ROW_CHUNK, nc - r0);
+  for (int r0 = 0; r0 < nc; r0 += CH) {
+    int rows = imin(CH, nc - r0);
+    bool lo = lo_on(c, rows);
     LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, 0, seq, c->rm[0], c->gather_idx, r0);
-    LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL);
-    LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, c->x, NO_GEMM, 0, (const T *)c->dw.ln1, f.rms_eps, d, (T *)c->xn,
-           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-    GemmOut g = gemm<T>(c, wkv, c->xn, rows, c->kvN, d);
-    LAUNCH(c, (k_qkv_post_draft<T>), rows, 128, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
+    LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL, 0LL);
+    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, rows, lo);
+    GemmOut g = gemm<T>(c, wkv, c->xn, lo ? c->lo_xn : 0, rows, c->kvN, d);
+    LAUNCH(c, k_qkv_post_draft, rows, 128, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
            flat(c, c->dself), f.n_heads, f.rope_theta);
   }
   // cross-attention memory: tapped features at the context positions, projected (Eq. 1)
   int nm = f.xattn_full_memory ? n : nc;
-  for (int r0 = 0; r0 < nm; r0 += ROW_CHUNK) {
-    int rows = imin(ROW_CHUNK, nm - r0);
+  for (int r0 = 0; r0 < nm; r0 += CH) {
+    int rows = imin(CH, nm - r0);
+    bool lo = lo_on(c, rows);
     LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, f.xattn_full_memory, seq, c->rm[0], c->gather_idx, r0);
     LAUNCH(c, (k_gather_rows<T>), rows, 256, 0, c->taps_store, c->gather_idx, (T *)c->raw, d, c->sd.tap + seq, c->tap_lo_eff,
-           (long long)f.max_prompt * d);
-    GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, rows, c->kvN, d);
-    LAUNCH(c, (k_mem_append<T>), rows, 256, 0, g, c->rm[0].seq, c->rm[0].dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
+           (long long)f.max_prompt * d, lo ? c->lo_xn : 0LL);
+    GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, lo ? c->lo_xn : 0, rows, c->kvN, d);
+    LAUNCH(c, k_mem_append, rows, 256, 0, g, c->rm[0].seq, c->rm[0].dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
   }
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, -1, (const int *)nullptr, nc, nm);
   return DREAM_OK;
@@ -618,32 +645,28 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
   for (int p = 1; p <= ts.D; ++p) {
     int m = p == 1 ? ts.D + 2 : ts.beam[p - 1];
     int R = B * m;
+    bool lo = lo_on(c, R);
+    long long lx = lo ? c->lo_xn : 0, la = lo ? c->lo_att : 0;
     RowMeta &rm = c->rm[cur], &rn = c->rm[cur ^ 1];
     if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
     LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
-    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, NO_GEMM, 0, (const T *)c->dw.ln1, f.rms_eps, d, (T *)c->xn,
-           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-    GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, R, c->qkvN, d);
-    LAUNCH(c, (k_qkv_post_draft<T>), R, 128, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, f.rope_theta);
-    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R));
-    g = gemm<T>(c, c->dw.wo, c->attn_out, R, d, c->Hhd);
-    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->dw.lnx, f.rms_eps, d, (T *)c->xn,
-           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-    g = gemm<T>(c, c->dw.xq, c->xn, R, c->Hhd, d);
+    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, lo);
+    GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, lx, R, c->qkvN, d);
+    LAUNCH(c, k_qkv_post_draft, R, 128, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, f.rope_theta);
+    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, lo));
+    g = gemm<T>(c, c->dw.wo, c->attn_out, la, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, lo);
+    g = gemm<T>(c, c->dw.xq, c->xn, lx, R, c->Hhd, d);
     LAUNCH(c, k_gemm_to_f32, R, 256, 0, g, c->qbuf, c->Hhd);
-    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R));
-    g = gemm<T>(c, c->dw.xo, c->attn_out, R, d, c->Hhd);
-    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->dw.ln2, f.rms_eps, d, (T *)c->xn,
-           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-    g = gemm<T>(c, c->dw.wgu, c->xn, R, 2 * f.d_ff, d);
-    LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, R), 256, 0, g, (T *)c->act, f.d_ff);
-    g = gemm<T>(c, c->dw.wd, c->act, R, d, f.d_ff);
-    // e^M = x: raw copy feeds the memory projection, normalised copy feeds the LM head
-    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->ln_f, f.rms_eps, d, (T *)c->xn,
-           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)c->raw);
-    g = gemm<T>(c, c->dw.xkv, c->raw, R, c->kvN, d);
-    LAUNCH(c, (k_mem_append<T>), R, 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
-    g = gemm<T>(c, c->lm_head, c->xn, R, f.vocab, d);
+    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, lo));
+    g = gemm<T>(c, c->dw.xo, c->attn_out, la, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, lo);
+    g = mlp_rows<T>(c, c->dw.wgu, c->dw.wd, R, lo);
+    // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
+    norm_rows<T>(c, c->x, g, true, c->ln_f, R, lo, nullptr, nullptr, nullptr, 0, true);
+    g = gemm<T>(c, c->dw.xkv, c->raw, lx, R, c->kvN, d);
+    LAUNCH(c, k_mem_append, R, 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
+    g = gemm<T>(c, c->lm_head, c->xn, lx, R, f.vocab, d);
     LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, ts.K, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
     int next_m = p < ts.D ? ts.beam[p] : 1;
     LAUNCH(c, k_tree_expand, B, 128, 0, tb, c->sd, c->dt, ts, p, m, c->top_val, c->top_id, c->lse_rows, rn, next_m);
@@ -672,27 +695,24 @@ template <typename T>
 static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *argmax, float *margin, float *logits) {
   const dream_config &f = c->cfg;
   int d = f.d_model, L = f.n_layers, R = B * c->T;
+  bool lo = lo_on(c, R);
+  long long lx = lo ? c->lo_xn : 0, la = lo ? c->lo_att : 0;
   RowMeta &rm = c->rm[0];
   LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
   LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
   GemmOut gd = NO_GEMM;
   for (int l = 0; l < L; ++l) {
     // completes S^l (for l >= 1) and captures it where a sequence taps layer l
-    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, gd, l > 0, (const T *)c->ln1[l], f.rms_eps, d, (T *)c->xn,
-           l > 0 ? c->tapbuf : (float *)nullptr, rm.seq, c->sd.tap, l, (T *)nullptr);
-    GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, R, c->qkvN, d);
+    norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, lo, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
+    GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, lx, R, c->qkvN, d);
     LAUNCH(c, (k_qkv_post_target<T>), R, 128, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, f.rope_theta);
-    HD_DISPATCH(c, T, tree(c, l, R));
-    g = gemm<T>(c, c->wo[l], c->attn_out, R, d, c->Hhd);
-    LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, g, 1, (const T *)c->ln2[l], f.rms_eps, d, (T *)c->xn,
-           (float *)nullptr, (const int *)nullptr, (const int *)nullptr, 0, (T *)nullptr);
-    g = gemm<T>(c, c->wgu[l], c->xn, R, 2 * f.d_ff, d);
-    LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, R), 256, 0, g, (T *)c->act, f.d_ff);
-    gd = gemm<T>(c, c->wd[l], c->act, R, d, f.d_ff);
+    HD_DISPATCH(c, T, tree(c, l, R, lo));
+    g = gemm<T>(c, c->wo[l], c->attn_out, la, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->ln2[l], R, lo);
+    gd = mlp_rows<T>(c, c->wgu[l], c->wd[l], R, lo);
   }
-  LAUNCH(c, (k_resid_norm<T>), R, 256, 0, c->x, gd, 1, (const T *)c->ln_f, f.rms_eps, d, (T *)c->xn, c->tapbuf, rm.seq,
-         c->sd.tap, L, (T *)nullptr);
-  GemmOut g = gemm<T>(c, c->lm_head, c->xn, R, f.vocab, d);
+  norm_rows<T>(c, c->x, gd, true, c->ln_f, R, lo, c->tapbuf, rm.seq, c->sd.tap, L);
+  GemmOut g = gemm<T>(c, c->lm_head, c->xn, lx, R, f.vocab, d);
   LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, logits);
   LAUNCH(c, k_argmax_out, (R + 127) / 128, 128, 0, c->top_id, c->top_val, R, argmax, margin,
          argmax == c->argmax_i ? (int *)nullptr : c->argmax_i);
@@ -728,9 +748,10 @@ static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const 
   LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
   LAUNCH(c, (k_compact_kv<T>), dim3(f.n_layers * 2, B), 256, 0, tb, c->sd, c->kv_pool, c->layer_stride, c->kv_stride, paged(c, 0));
   LAUNCH(c, k_accept_rows, 1, 32, 0, tb, B, c->T, D, c->sd, c->gather_idx, rm, c->cap_rows - c->ts.NI, c->status);
-  LAUNCH(c, (k_gather_rows<T>), R, 256, 0, c->tapbuf, c->gather_idx, (T *)c->raw, d, (const int *)nullptr, 0, 0LL);
-  GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, R, c->kvN, d);
-  LAUNCH(c, (k_mem_append<T>), R, 256, 0, g, rm.seq, rm.dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
+  bool lo = lo_on(c, R);
+  LAUNCH(c, (k_gather_rows<T>), R, 256, 0, c->tapbuf, c->gather_idx, (T *)c->raw, d, (const int *)nullptr, 0, 0LL, lo ? c->lo_xn : 0LL);
+  GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, lo ? c->lo_xn : 0, R, c->kvN, d);
+  LAUNCH(c, k_mem_append, R, 256, 0, g, rm.seq, rm.dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
   return DREAM_OK;
 }
 
@@ -802,11 +823,11 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
     }
   } else if (what >= 2 && what <= 5) {
     if (index < 0 || index >= c->cap_rows) return fail(c, DREAM_E_ARG, "row out of range");
-    const T *base = (const T *)(what <= 3 ? c->dmem : c->dself);
+    const float *base = what <= 3 ? c->dmem : c->dself;
     int kvsel = (what - 2) & 1;
     for (int h = 0; h < f.n_kv_heads; ++h) {
-      const T *src = base + ((((size_t)seq * 2 + kvsel) * f.n_kv_heads + h) * c->cap_rows + index) * f.head_dim;
-      k_read_row<T><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
+      const float *src = base + ((((size_t)seq * 2 + kvsel) * f.n_kv_heads + h) * c->cap_rows + index) * f.head_dim;
+      k_read_row<float><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
     }
   } else if (what == 6 || what == 7) {
     if (index < 0 || index >= ROW_CHUNK) return fail(c, DREAM_E_ARG, "row out of range");

@@ -5,4 +5,4 @@
 struct GemmTcPlan { int dummy; };
 static inline const char *gemm_tc_plan_init(GemmTcPlan *) { return nullptr; }
 static inline bool gemm_tc_supported(int, int, int) { return false; }
-static inline void gemm_tc_launch(GemmTcPlan *, cudaStream_t, const void *, const void *, int, int, int, float *, long long, GemmOut *) {}
+static inline void gemm_tc_launch(GemmTcPlan *, cudaStream_t, const void *, const void *, long long, int, int, int, float *, long long, GemmOut *) {}

@@ -45,7 +45,7 @@ __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict_
 template <typename T>
 __global__ void k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
                              float eps, int d, T *xn, float *copy, const int *row_seq,
-                             const int *tap_state, int layer, T *raw) {
+                             const int *tap_state, int layer, T *raw, long long lo_delta) {
   __shared__ float sh[33];
   int r = blockIdx.x;
   float *xr = x + (long long)r * d;
@@ -61,8 +61,8 @@ __global__ void k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restr
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     float v = xr[i];
     if (do_copy) copy[(long long)r * d + i] = v;
-    if (raw) raw[(long long)r * d + i] = from_f<T>(v);
-    if (xn) xn[(long long)r * d + i] = from_f<T>(v * inv * to_f(gain[i]));
+    if (raw) store_split<T>(raw + (long long)r * d + i, lo_delta, v);
+    if (xn) store_split<T>(xn + (long long)r * d + i, lo_delta, v * inv * to_f(gain[i]));
   }
 }
 
@@ -119,9 +119,9 @@ __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
   }
 }
 
-// Draft caches are flat per sequence: [seq][2][H_kv][cap][hd].
+// Draft caches are flat per sequence, always fp32 (they are small): [seq][2][H_kv][cap][hd].
 struct FlatKV {
-  void *base;
+  float *base;
   int cap, hkv, hd;
   __device__ __forceinline__ long long off(int seq, int kv, int kvh, int row) const {
     return ((((long long)seq * 2 + kv) * hkv + kvh) * cap + row) * hd;
@@ -131,7 +131,6 @@ struct FlatKV {
 // After a draft QKV GEMM (col0 = first column of the K block inside the GEMM output, or
 // H*hd when the GEMM produced q too): rotary, q -> qbuf (when has_q), k/v -> draft
 // self-attention cache row row_dst[r] (skipped when < 0).
-template <typename T>
 __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
                                  const int *__restrict__ row_pos, const int *__restrict__ row_dst,
                                  int row0, int has_q, float *qbuf, FlatKV kv, int H, float theta) {
@@ -140,7 +139,7 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
   int hd = kv.hd, half = hd >> 1, Hkv = kv.hkv;
   int seq = row_seq[r], pos = row_pos[r];
   int kcol = has_q ? H * hd : 0;
-  T *base = (T *)kv.base;
+  float *base = kv.base;
   for (int i = threadIdx.x; i < half; i += blockDim.x) {
     float c, s;
     rope_cs(pos, i, hd, theta, &c, &s);
@@ -155,10 +154,10 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
       for (int h = 0; h < Hkv; ++h) {
         float a = gemm_val(g, lr, kcol + h * hd + i), b = gemm_val(g, lr, kcol + h * hd + i + half);
         long long ok = kv.off(seq, 0, h, dst), ov = kv.off(seq, 1, h, dst);
-        base[ok + i] = from_f<T>(a * c - b * s);
-        base[ok + i + half] = from_f<T>(b * c + a * s);
-        base[ov + i] = from_f<T>(gemm_val(g, lr, kcol + (Hkv + h) * hd + i));
-        base[ov + i + half] = from_f<T>(gemm_val(g, lr, kcol + (Hkv + h) * hd + i + half));
+        base[ok + i] = a * c - b * s;
+        base[ok + i + half] = b * c + a * s;
+        base[ov + i] = gemm_val(g, lr, kcol + (Hkv + h) * hd + i);
+        base[ov + i + half] = gemm_val(g, lr, kcol + (Hkv + h) * hd + i + half);
       }
   }
 }
@@ -172,7 +171,6 @@ __global__ void k_gemm_to_f32(GemmOut g, float *dst, int width) {
 // Cross-attention memory rows (Eq. 1: K = S W_K, V = S W_V): GEMM output [rows][2 H_kv hd]
 // -> memory cache row of sequence row_seq[r]: row_dst[r] when nperm is null, else the
 // tree-region row nperm[seq] + row_in[r].  Negative indices skip the row.
-template <typename T>
 __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
                              const int *__restrict__ row_dst, const int *__restrict__ row_in,
                              const int *__restrict__ nperm, int row0, FlatKV kv) {
@@ -181,22 +179,22 @@ __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
   int dst = nperm ? (row_in[r] < 0 ? -1 : nperm[seq] + row_in[r]) : row_dst[r];
   if (dst < 0) return;
   int w = kv.hkv * kv.hd;
-  T *base = (T *)kv.base;
+  float *base = kv.base;
   for (int i = threadIdx.x; i < w; i += blockDim.x) {
     int h = i / kv.hd, e = i - h * kv.hd;
-    base[kv.off(seq, 0, h, dst) + e] = from_f<T>(gemm_val(g, lr, i));
-    base[kv.off(seq, 1, h, dst) + e] = from_f<T>(gemm_val(g, lr, w + i));
+    base[kv.off(seq, 0, h, dst) + e] = gemm_val(g, lr, i);
+    base[kv.off(seq, 1, h, dst) + e] = gemm_val(g, lr, w + i);
   }
 }
 
 // act = silu(gate) * up, from a GEMM output whose columns are [gate(ff) | up(ff)].
 template <typename T>
-__global__ void k_silu_mul(GemmOut g, T *act, int ff) {
+__global__ void k_silu_mul(GemmOut g, T *act, int ff, long long lo_delta) {
   int r = blockIdx.y;
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= ff) return;
   float a = gemm_val(g, r, i), b = gemm_val(g, r, ff + i);
-  act[(long long)r * ff + i] = from_f<T>(a / (1.f + __expf(-a)) * b);
+  store_split<T>(act + (long long)r * ff + i, lo_delta, a / (1.f + __expf(-a)) * b);
 }
 
 // x += GEMM output; optional fp32 copy into a per-layer store (prefill tap candidates).
@@ -212,11 +210,12 @@ __global__ void k_resid_add(float *x, GemmOut g, int d, float *copy) {
 // Gather fp32 rows into element-type GEMM input rows: dst[r] = src[idx[r]] (idx < 0 -> zeros).
 template <typename T>
 __global__ void k_gather_rows(const float *__restrict__ src, const int *__restrict__ idx, T *dst,
-                              int d, const int *layer_ptr, int layer_lo, long long layer_stride) {
+                              int d, const int *layer_ptr, int layer_lo, long long layer_stride,
+                              long long lo_delta) {
   int r = blockIdx.x, s = idx[r];
   if (layer_ptr) src += (long long)(*layer_ptr - layer_lo) * layer_stride;
   for (int i = threadIdx.x; i < d; i += blockDim.x)
-    dst[(long long)r * d + i] = from_f<T>(s >= 0 ? src[(long long)s * d + i] : 0.f);
+    store_split<T>(dst + (long long)r * d + i, lo_delta, s >= 0 ? src[(long long)s * d + i] : 0.f);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -20,7 +20,9 @@ class Tol:
         self.rel_l2 = 1e-2 if bf else 1e-5
         self.dec = 1e-2                           # decision margin below which either choice is accepted
         self.ae_abs = 1e-3 if bf else 1e-5        # average attention entropy
-        self.score_rel = 1e-3 if bf else 1e-5     # visual-token importance, relative to the largest score
+        # visual-token importance, per element and relative: bf16 rounds both the GEMM input
+        # and the cached K row (2^-9 each), which shifts every logit of a column alike
+        self.score_rel = 5e-3 if bf else 1e-5
 
 
 def close(a, b, tol, what, report):
@@ -30,6 +32,23 @@ def close(a, b, tol, what, report):
     report.setdefault("float", []).append((what, ma, rl))
     assert ma <= tol.max_abs, f"{what}: max-abs {ma:.3e} > {tol.max_abs} (rel-L2 {rl:.3e})"
     assert rl <= tol.rel_l2, f"{what}: rel-L2 {rl:.3e} > {tol.rel_l2} (max-abs {ma:.3e})"
+
+
+def close_stored(a, b, tol, what, report, bf16_store, where=""):
+    """Rows read back from a bf16 store may differ from the oracle's by one bf16 unit in the
+    last place where the two sides rounded values a few 1e-6 apart to different neighbours."""
+    if not bf16_store:
+        return close(a, b, tol, what, report)
+    a, b = a.double().flatten(), b.double().flatten()
+    gap = (a - b).abs()
+    rl = float(gap.norm() / (b.norm() + 1e-30))
+    report.setdefault("float", []).append((what, float(gap.max()), rl))
+    bad = gap > b.abs() * 2.0 ** -7 + tol.max_abs
+    if bool(bad.any()):
+        i = int(torch.argmax(gap - b.abs() * 2.0 ** -7))
+        raise AssertionError(f"{what} {where}: more than one bf16 ulp apart at element {i}: {float(a[i])} vs {float(b[i])}; "
+                             f"{int(bad.sum())} of {bad.numel()} elements, rel-L2 {rl:.3e}")
+    assert rl <= tol.rel_l2, f"{what}: rel-L2 {rl:.3e} > {tol.rel_l2}"
 
 
 def valid_tree(t, T):
@@ -55,7 +74,8 @@ class Pair:
         self.dwg = synth.draft_weights(p, seed, device)
         cpu = lambda w: [t.cpu() for t in w] if isinstance(w, list) else w.cpu()
         self.orc = DreamOracle(OracleConfig.from_preset(p), {k: cpu(v) for k, v in self.twg.items()},
-                               {k: cpu(v) for k, v in self.dwg.items()}, odt)
+                               {k: cpu(v) for k, v in self.dwg.items()}, odt,
+                               kv_dtype=torch.bfloat16 if p["dtype"] == "bf16" else None)
         self.odt = odt
         self.cfg = api.make_config(p, max_batch=max_batch)
         self.ctx = api.Context(self.cfg, self.twg, self.dwg, device)
@@ -82,7 +102,8 @@ class Pair:
         self.ctx.dream_prefill(seq, vis, vis_start, ids, tok, mg, ae, tap)
         st, otok, omargin = self.orc.prefill(vis.cpu().to(self.odt), vis_start, ids.cpu().tolist())
         self.ctx.dream_poll()
-        assert float((ae.cpu().double() - st.entropy).abs().max()) <= tol.ae_abs, "layer entropy"
+        egap = float((ae.cpu().double() - st.entropy).abs().max())
+        assert egap <= tol.ae_abs, f"layer entropy: gap {egap:.3e}"
         if not self._decide(int(tok) == otok, omargin, "first token"):
             st.pending = int(tok)
         if not self._decide(int(tap) == st.tap, getattr(st, "tap_margin", float("inf")), "tap layer"):
@@ -94,9 +115,14 @@ class Pair:
         okept, osc, omargin = self.orc.compress_visual(st, k)
         self.ctx.dream_poll()
         scale = float(osc.abs().max()) if osc.numel() else 1.0
-        assert float((sc.cpu().double()[:p["n_visual"]] - osc.double()).abs().max()) <= tol.score_rel * scale, "importance"
+        g64, o64 = sc.cpu().double()[:p["n_visual"]], osc.double()
+        rel = float(((g64 - o64).abs() / o64.abs().clamp_min(1e-3 * scale)).max()) if osc.numel() else 0.0
+        self.report["score_gap_rel"] = rel
+        assert rel <= tol.score_rel, f"importance: per-element relative gap {rel:.3e} > {tol.score_rel}"
         gk = kept.cpu().tolist()[:k]
-        if not self._decide(gk == okept.tolist(), omargin / max(scale, 1e-30) * (tol.dec / tol.score_rel), "kept visual tokens"):
+        cut = float(torch.sort(o64, descending=True).values[k - 1]) if 0 < k < p["n_visual"] else 1.0
+        exempt_below = 2 * tol.score_rel * max(cut, 1e-3 * scale)
+        if not self._decide(gk == okept.tolist(), omargin * (tol.dec / exempt_below), "kept visual tokens"):
             assert gk == sorted(set(gk)) and all(0 <= j < p["n_visual"] for j in gk)
             self.orc.compress_visual(st, k, forced_idx=gk)
         self.st[seq] = st
@@ -119,16 +145,20 @@ class Pair:
             valid_tree(gd, T)
             same = all(gd[k] == od[k] for k in ("tokens", "parent", "depth", "mask"))
             self._decide(same, od["min_margin"], "draft tree")
+            # a cumulative score is a sum of `depth` log-probabilities, each held to max_abs
+            cum_ok = lambda g, o, dep: abs(g - o) <= tol.max_abs * max(dep, 1)
             if same:
-                close(torch.tensor(gd["cum"]), torch.tensor(od["cum"]), tol, "draft cum_logp", self.report)
+                gap = max(abs(g - o) / max(dd, 1) for g, o, dd in zip(gd["cum"], od["cum"], od["depth"]))
+                self.report.setdefault("float", []).append(("draft logp (per level)", gap, gap))
+                assert gap <= tol.max_abs, f"draft cum_logp: {gap:.3e} per level > {tol.max_abs}"
             else:       # near-tie: compare scores of the nodes both sides kept
                 key = lambda t, i: self._path(t, i)
                 om = {key(od, i): od["cum"][i] for i in range(len(od["tokens"]))}
-                common = [(gd["cum"][i], om[key(gd, i)]) for i in range(T) if key(gd, i) in om]
+                common = [(gd["cum"][i], om[key(gd, i)], gd["depth"][i]) for i in range(T) if key(gd, i) in om]
                 self.report.setdefault("tree_overlap", []).append(len(common) / T)
-                if common:
-                    a, bb = zip(*common)
-                    assert max(abs(x - y) for x, y in zip(a, bb)) <= max(tol.max_abs, 3 * tol.dec), "draft cum_logp (common nodes)"
+                gap = max(abs(g - o) / max(dd, 1) for g, o, dd in common)
+                self.report.setdefault("float", []).append(("draft logp (per level)", gap, gap))
+                assert gap <= tol.max_abs, f"draft cum_logp (common nodes): {gap:.3e} per level > {tol.max_abs}"
             chosen = od if inject is None or s not in inject else inject[s]
             if inject is not None and s in inject:
                 chosen = make_tree(inject[s]["tokens"], inject[s]["parent"])
@@ -173,8 +203,9 @@ class Pair:
             L = p["n_layers"]
             for l in sorted({0, L - 1}):
                 for pos in sorted({0, P0 - 1, P0, st.P - 1})[:2 + check_cache_rows]:
-                    close(ctx.dream_debug_read(s, 0, l, pos), st.K[l][pos].flatten(), tol, "target K row", self.report)
-                    close(ctx.dream_debug_read(s, 1, l, pos), st.V[l][pos].flatten(), tol, "target V row", self.report)
+                    bf = p["dtype"] == "bf16"
+                    close_stored(ctx.dream_debug_read(s, 0, l, pos), st.K[l][pos].flatten(), tol, "target K row", self.report, bf, f"(layer {l}, pos {pos}, P0 {P0}, A {A})")
+                    close_stored(ctx.dream_debug_read(s, 1, l, pos), st.V[l][pos].flatten(), tol, "target V row", self.report, bf, f"(layer {l}, pos {pos}, P0 {P0}, A {A})")
             nm = st.mK.shape[0]
             for row in sorted({0, nm - A - 1, nm - 1}):
                 close(ctx.dream_debug_read(s, 2, 0, row), st.mK[row].flatten(), tol, "memory K row", self.report)

@@ -32,3 +32,13 @@ def test_toy_fp32_full_decode():
     """Config 1: toy VLM in fp32, complete binary tree of depth 3, 16 decode steps."""
     pr, s = _run("toy", 16)
     assert s["exempt"] <= 2
+
+
+def test_llava_shape_4_layers_bf16():
+    """LLaVA-7B-shaped widths (d 4096, 32 heads of 128, MLP 11008, vocab 32000), 4 layers."""
+    pr, s = _run("llava7b", 3, n_layers=4, decode_steps=8)
+
+
+def test_smolvlm_shape_full_bf16():
+    """Config 2: SmolVLM-2B-shaped target, all 24 layers, 4 decode steps."""
+    pr, s = _run("smolvlm2b", 4)
