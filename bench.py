@@ -1,0 +1,289 @@
+#!/usr/bin/env python
+"""Benchmark of the DREAM draft+verify(+accept) step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one whole round of the hot path (draft tree, tree-masked verification, greedy
+acceptance with KV compaction) for one batch of sequences on seeded synthetic inputs and
+random-init weights.  The metric is verified tree-tokens per second: B*T tree tokens pass
+the target per step.  With N > 1 every rank runs an independent replica (the path has no
+exchange step); the timed region is bracketed by a barrier and the slowest rank counts.
+
+One JSON line is printed by rank 0.  `--impl reference` times the CPU oracle instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_19201_b200 import configs, synth  # noqa: E402
+
+METRIC = "verified_tree_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def step_bytes(p, T, P0):
+    """Algorithmic bytes of one step (weights + KV read), bf16 storage, one-layer draft."""
+    e = 2 if p["dtype"] == "bf16" else 4
+    d, H, Hkv, hd, ff, V, L = (p[k] for k in ("d_model", "n_heads", "n_kv_heads", "head_dim", "d_ff", "vocab", "n_layers"))
+    Hhd, kvw = H * hd, 2 * Hkv * hd
+    layer = (Hhd + kvw) * d + d * Hhd + 3 * d * ff
+    head = V * d
+    draft_layer = layer + Hhd * d + kvw * d + d * Hhd      # + cross-attention q, kv, o
+    kv_tok = L * kvw
+    B = p["batch"]
+    verify = (L * layer + head) * e + B * P0 * kv_tok * e
+    n_ctx = p["n_prompt"] + p["k_visual"]
+    draft_pass = (draft_layer + head) * e + B * 2 * n_ctx * kvw * 4   # draft caches are fp32
+    draft = p["tree_depth"] * draft_pass
+    accept = kvw * d * e
+    return dict(verify=verify, draft=draft, accept=accept, total=verify + draft + accept,
+                gemm_weights=(L * layer + head + p["tree_depth"] * (draft_layer + head) + kvw * d) * e)
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.rows, self.stop_flag = index, [], False
+
+    def run(self):
+        while not self.stop_flag:
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                parts = [x.strip() for x in out.strip().split(",")]
+                if len(parts) >= 7:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            time.sleep(0.05)
+
+    def summary(self):
+        if not self.rows:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unsampled"])
+        mhz = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in self.rows)]
+        return dict(sm_mhz=statistics.median(mhz) if mhz else None, sm_max_mhz=float(self.rows[0][1]),
+                    samples=len(self.rows), reasons=reasons)
+
+
+def peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return dict(hbm_gbs=6650.0, bf16_tflops=1590.0), "fallback"
+
+
+def oracle_sample(p, twg, dwg, T):
+    """Time one full draft+verify+accept step of the CPU oracle, as it stands, on this
+    workload's shapes at the initial prefix length.  The sequence state is filled with
+    random values instead of a CPU prefill (timing does not depend on values)."""
+    from oracle.dream_oracle import DreamOracle, OracleConfig, SeqState
+    dt = torch.float32 if p["dtype"] == "bf16" else torch.float64
+    cpu = lambda w: [t.cpu() for t in w] if isinstance(w, list) else w.cpu()
+    orc = DreamOracle(OracleConfig.from_preset(p), {k: cpu(v) for k, v in twg.items()},
+                      {k: cpu(v) for k, v in dwg.items()}, dt,
+                      kv_dtype=torch.bfloat16 if p["dtype"] == "bf16" else None)
+    n = p["n_visual"] + p["n_prompt"]
+    nc = p["n_prompt"] + p["k_visual"]
+    Hkv, hd = p["n_kv_heads"], p["head_dim"]
+    g = torch.Generator().manual_seed(0)
+    rnd = lambda rows: torch.randn(rows, Hkv, hd, dtype=dt, generator=g)
+    st = SeqState(P=n, pending=1, n_prompt_total=n, vis_start=0, n_visual=p["n_visual"], tap=max(1, p["n_layers"] // 2))
+    st.K = [rnd(n) for _ in range(p["n_layers"])]
+    st.V = [rnd(n) for _ in range(p["n_layers"])]
+    st.dK, st.dV, st.mK, st.mV = rnd(nc), rnd(nc), rnd(nc), rnd(nc)
+    t0 = time.perf_counter()
+    orc.step(st)
+    dt_s = time.perf_counter() - t0
+    return dict(value=T / dt_s, unit=UNIT, cores=torch.get_num_threads(), kind="oracle",
+                sample=f"1 full draft+verify+accept step of 1 sequence, {p['name']} shapes, prefix {n}, "
+                       f"state filled with random values (no CPU prefill); {dt_s:.1f} s", seconds=dt_s)
+
+
+def run_reference(args, p):
+    """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    twg, dwg = synth.target_weights(p, 0, dev), synth.draft_weights(p, 0, dev)
+    from paper_2505_19201_b200 import api
+    T = 1 + min(p["tree_max_nodes"], p["tree_topk"] + (p["tree_depth"] - 1) * min(p["tree_beam"], p["tree_topk"]) * p["tree_topk"])
+    times = []
+    for i in range(args.warmup + args.steps):
+        r = oracle_sample(p, twg, dwg, T)
+        if i >= args.warmup:
+            times.append(r["seconds"])
+        if sum(times) > 150:
+            break
+    ms = 1e3 * sum(times) / len(times)
+    val = T / (ms / 1e3)
+    line = dict(metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=len(times), warmup=args.warmup,
+                ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f32" if p["dtype"] == "bf16" else "f64", data="synthetic", impl="reference",
+                config=dict(workload=p["name"], batch=1, tree_nodes=T, note="CPU oracle, one sequence per step"),
+                cpu_baseline=dict(value=val, unit=UNIT, cores=torch.get_num_threads(), kind="oracle", sample=r["sample"]),
+                e2e=dict(value=val, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--workload", default="llava7b")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-gemm", type=int, default=1)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    p = dict(configs.PRESETS[args.workload])
+    if args.impl == "reference":
+        return run_reference(args, p)
+
+    from paper_2505_19201_b200 import api
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = f"cuda:{local}"
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    B = p["batch"]
+    p["decode_steps"] = args.steps + args.warmup + 8 + 2 * args.steps   # room for every timed pass
+    twg, dwg = synth.target_weights(p, 0, dev), synth.draft_weights(p, 0, dev)
+    cfg = api.make_config(p)
+    ctx = api.Context(cfg, twg, dwg, dev)
+    T = ctx.T
+    seqs = list(range(B))
+    for s in seqs:
+        vis, ids = synth.request_inputs(p, s + 100 * rank, dev)
+        ctx.dream_prefill(s, vis, 0, ids)
+        ctx.dream_compress_visual(s, p["k_visual"])
+    ctx.dream_poll()
+    P0 = p["n_visual"] + p["n_prompt"]
+
+    trees = None                              # the context's own tree buffers
+    am = torch.zeros(B * T, dtype=torch.int32, device=dev)
+    alen = torch.zeros(B, dtype=torch.int32, device=dev)
+    outt = torch.zeros(B * (p["tree_depth"] + 1), dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def one_step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        ctx.dream_draft_tree(seqs, trees)
+        if ev:
+            ev[1].record(stream)
+        ctx.dream_verify_tree(seqs, trees, am)
+        if ev:
+            ev[2].record(stream)
+        ctx.dream_accept(seqs, trees, am, alen, outt)
+        if ev:
+            ev[3].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    # ---- timed region: device-resident inputs, CUDA events on the launching stream
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = ctx.dream_launch_count()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for i in range(args.steps):
+        one_step(evs[i])
+    t_end.record(stream)
+    barrier()
+    sampler.stop_flag = True
+    launches = ctx.dream_launch_count() - l0
+    total_ms = t_start.elapsed_time(t_end)
+    draft_us = statistics.median(e[0].elapsed_time(e[1]) for e in evs) * 1e3
+    verify_us = statistics.median(e[1].elapsed_time(e[2]) for e in evs) * 1e3
+    accept_us = statistics.median(e[2].elapsed_time(e[3]) for e in evs) * 1e3
+    ctx.dream_poll()
+    # ---- end to end: the serving call with host result buffers, synchronising every step
+    alen_h = torch.zeros(B, dtype=torch.int32).pin_memory()
+    outt_h = torch.zeros(B * (p["tree_depth"] + 1), dtype=torch.int32).pin_memory()
+    for _ in range(2):
+        ctx.dream_step_host(seqs, alen_h, outt_h)
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        ctx.dream_step_host(seqs, alen_h, outt_h)
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
+    # ---- dominant kernel: the weight-streaming GEMM, timed per launch with CUDA events
+    gemm = None
+    if args.profile_gemm and hasattr(ctx, "dream_profile_gemm"):
+        gemm = ctx.dream_profile_gemm(one_step, args.steps)
+    ms = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(ms[0]), float(ms[1])
+    if rank != 0:
+        return
+    pk, pk_src = peaks()
+    sb = step_bytes(p, T, P0)
+    ms_step = total_ms / args.steps
+    value = world * B * T / (ms_step / 1e3)
+    step_gbs = sb["total"] / (ms_step / 1e3) / 1e9
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16" if p["dtype"] == "bf16" else "f32", data="synthetic",
+                config=dict(workload=p["name"], batch=B, tree_nodes=T, prefix=P0, parallelism=f"replicas{world}",
+                            l2="step working set (weights, %.1f GB) exceeds the 126 MB L2" % (sb["gemm_weights"] / 1e9)),
+                draft_us=draft_us, verify_us=verify_us, accept_us=accept_us,
+                step_bytes=sb["total"], step_gbs=step_gbs,
+                step_roofline_frac=step_gbs / pk["hbm_gbs"], step_roofline_frac_nominal_8tbs=step_gbs / 8000.0,
+                clocks=sampler.summary(), gpu_launches=int(launches),
+                e2e=dict(value=world * B * T / (e2e_ms / args.steps / 1e3), unit=UNIT,
+                         h2d_bytes_per_step=4 * B, d2h_bytes_per_step=4 * B * (p["tree_depth"] + 2)))
+    if gemm:
+        line["roofline"] = dict(bound="hbm", achieved=gemm["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
+                                frac=gemm["gbs"] / pk["hbm_gbs"], traffic=None, peak_source=pk_src,
+                                kernel=gemm["kernel"], launches_per_step=gemm["launches_per_step"],
+                                bytes_per_step=gemm["bytes_per_step"], ms_per_step=gemm["ms_per_step"])
+    else:
+        line["roofline"] = dict(bound="hbm", achieved=step_gbs, peak=pk["hbm_gbs"], unit="GB/s",
+                                frac=step_gbs / pk["hbm_gbs"], traffic=None, peak_source=pk_src, kernel="whole step")
+    if not args.no_cpu_baseline and world == 1:
+        cb = oracle_sample(p, twg, dwg, T)
+        cb.pop("seconds")
+        line["cpu_baseline"] = cb
+    print(json.dumps(line))
+    ctx.close()
+
+
+if __name__ == "__main__":
+    main()
