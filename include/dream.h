@@ -187,6 +187,16 @@ dream_status dream_seq_state(dream_ctx *ctx, int32_t seq, int32_t *verified_len,
 dream_status dream_debug_read(dream_ctx *ctx, int32_t seq, int32_t what, int32_t layer,
                               int32_t index, float *dst);
 
+/* Test hook: out[r][c] = sum_k X[r][k] W[c][k] through the context's GEMM path (the same
+ * kernels every projection of the model uses).  W: device [N][K] in config.dtype; X: device
+ * float [rows][K]; out: device float [rows][N]; rows <= 128 (256 when split == 0 or dtype is
+ * fp32); K <= max(d_model, d_ff).  split != 0 feeds bf16 inputs as hi + lo parts. */
+dream_status dream_debug_gemm(dream_ctx *ctx, const void *W, const float *X, int32_t rows,
+                              int32_t N, int32_t K, int32_t split, float *out);
+
+/* How many GEMM launches so far went to the tensor-core kernel and to the CUDA-core kernel. */
+dream_status dream_gemm_counts(const dream_ctx *ctx, int64_t *tensor_core, int64_t *cuda_core);
+
 /* Forget a sequence (its pages return to the pool). */
 dream_status dream_seq_reset(dream_ctx *ctx, int32_t seq);
 

@@ -75,6 +75,8 @@ def lib():
             "dream_seq_state": [vp, i32, i32p, i32p, i32p],
             "dream_debug_read": [vp, i32, i32, i32, i32, vp],
             "dream_seq_reset": [vp, i32],
+            "dream_debug_gemm": [vp, vp, vp, i32, i32, i32, i32, vp],
+            "dream_gemm_counts": [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
             "dream_poll": [vp],
         }
         for name, args in sig.items():
@@ -255,6 +257,18 @@ class Context:
         out = torch.empty(n, dtype=torch.float32)
         _check(self.h, lib().dream_debug_read(self.h, seq, what, layer, index, C.c_void_p(out.data_ptr())))
         return out
+
+    def dream_debug_gemm(self, W, X, split=1):
+        rows, K = X.shape
+        N = W.shape[0]
+        out = torch.empty(rows, N, dtype=torch.float32, device=self.device)
+        _check(self.h, lib().dream_debug_gemm(self.h, _ptr(W), _ptr(X), rows, N, K, split, _ptr(out)))
+        return out
+
+    def dream_gemm_counts(self):
+        a, b = C.c_int64(), C.c_int64()
+        _check(self.h, lib().dream_gemm_counts(self.h, C.byref(a), C.byref(b)))
+        return a.value, b.value
 
     def dream_seq_reset(self, seq):
         _check(self.h, lib().dream_seq_reset(self.h, seq))

@@ -15,7 +15,8 @@ TAP_FIXED, TAP_ENTROPY_MIN, TAP_ENTROPY_MAX = 0, 1, 2
 
 def _mid(L):
     """Middle-layer range used by the entropy tap modes: [ceil(L/4), floor(3L/4)], 1-based."""
-    return (L + 3) // 4, (3 * L) // 4
+    lo = (L + 3) // 4
+    return lo, max(lo, (3 * L) // 4)
 
 
 def _preset(name, dtype, L, d, H, Hkv, hd, ff, V, v, k, q, D, K, N, steps, batch,

@@ -60,7 +60,7 @@ struct dream_ctx {
   std::vector<int> free_pages;
   std::vector<int> seq_pages[DREAM_MAX_BATCH];
   int *h_stage;                        // pinned: page-table staging + step_host results
-  long long launches;
+  long long launches, tc_launches, simt_launches;
   GemmTcPlan tc;
   char err[256];
 };
@@ -172,7 +172,7 @@ static void derive(dream_ctx *c) {
   c->pps = (f.max_seq + f.page_tokens - 1) / f.page_tokens;
   c->n_pages = c->pps * f.max_batch;
   c->chunk = f.dtype == DREAM_BF16 ? ROW_CHUNK / 2 : ROW_CHUNK;
-  c->RM = imax(ROW_CHUNK, f.max_prompt);
+  c->RM = (imax(ROW_CHUNK, f.max_prompt) + 15) & ~15;
   c->XR = c->RM;
 }
 
@@ -231,11 +231,12 @@ static size_t carve(dream_ctx *c, char *base) {
   int widest = imax(imax(c->qkvN, 2 * f.d_ff), imax(d, c->Hhd));
   int lm_rows = ((imax(MB * T, MB * imax(c->ts.D + 2, f.tree_beam)) + 15) / 16) * 16;
   c->gemm_rows_lm = lm_rows;
-  size_t per_slot = (size_t)imax(ROW_CHUNK * widest, 1) ;
-  size_t lm_slot = (size_t)imin(2 * lm_rows, ROW_CHUNK) * f.vocab;
-  if (lm_slot > per_slot) per_slot = lm_slot;
-  c->gout_floats = per_slot;
-  c->gout = a.take<float>(per_slot * GEMM_TC_MAX_SLOTS);
+  // room for the stream-K partial slots: a tile is shared by at most ceil(KB/upc) + 1 CTAs and
+  // upc >= tiles*KB/148, so slots * N <= (148/tiles + 2) * N <= 148*128 + 2N (+ slack)
+  size_t wide = (size_t)ROW_CHUNK * (2 * (size_t)widest + 19200);
+  size_t lm = (size_t)imin(2 * lm_rows, ROW_CHUNK) * (2 * (size_t)f.vocab + 19200);
+  c->gout_floats = wide > lm ? wide : lm;
+  c->gout = a.take<float>(c->gout_floats);
   c->lse_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
   c->ent_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
   c->ae = a.take<float>(f.n_layers);
@@ -273,11 +274,13 @@ template <typename T>
 static GemmOut gemm(dream_ctx *c, const void *W, const void *X, long long lo_delta, int rows, int N, int K) {
   GemmOut g;
   int rows_pad = (rows + 15) & ~15;
-  if (c->use_tc && sizeof(T) == 2 && gemm_tc_supported(rows_pad * (lo_delta ? 2 : 1), N, K)) {
-    gemm_tc_launch(&c->tc, c->stream, W, X, lo_delta, rows, N, K, c->gout, (long long)c->gout_floats, &g);
+  if (c->use_tc && sizeof(T) == 2 && gemm_tc_supported(rows_pad * (lo_delta ? 2 : 1), N, K) &&
+      gemm_tc_launch(&c->tc, c->stream, W, X, lo_delta, rows, N, K, c->gout, (long long)c->gout_floats, &g)) {
     c->launches++;
+    c->tc_launches++;
     return g;
   }
+  c->simt_launches++;
   int tiles = (rows + SG_BM - 1) / SG_BM;
   dim3 grid((N + SG_BN - 1) / SG_BN, tiles * (lo_delta ? 2 : 1));
   k_gemm_simt<T><<<grid, 256, 0, c->stream>>>((const T *)X, (const T *)W, c->gout, rows, N, K, N, tiles, lo_delta, rows_pad);
@@ -341,12 +344,12 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   for (int p = c->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
   for (int b = 0; b < DREAM_MAX_BATCH; ++b) c->phase[b] = PH_EMPTY;
   c->prefill_seq = -1;
-  c->launches = 0;
+  c->launches = 0; c->tc_launches = 0; c->simt_launches = 0;
   c->err[0] = 0;
   const char *mode = getenv("DREAM_GEMM");
   c->use_tc = cfg->dtype == DREAM_BF16 && !(mode && !strcmp(mode, "simt"));
   if (c->use_tc) {
-    const char *why = gemm_tc_plan_init(&c->tc);
+    const char *why = gemm_tc_plan_init(&c->tc, c->status);
     if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
   }
   *out = c;
@@ -836,6 +839,48 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
   } else return fail(c, DREAM_E_ARG, "unknown buffer id %d", what);
   CUDA_OK(c, cudaMemcpyAsync(dst, tmp, sizeof(float) * count, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  return DREAM_OK;
+}
+
+// out[r][c] = sum_k X[r][k] W[c][k] through the context's GEMM path (test hook).
+__global__ void k_split_rows(const float *src, void *dst, int K, long long lo_delta, int is_bf16) {
+  int r = blockIdx.x;
+  for (int i = threadIdx.x; i < K; i += blockDim.x) {
+    float v = src[(long long)r * K + i];
+    if (is_bf16) store_split<bf16>((bf16 *)dst + (long long)r * K + i, lo_delta, v);
+    else ((float *)dst)[(long long)r * K + i] = v;
+  }
+}
+__global__ void k_gemm_collect(GemmOut g, float *dst, int N) {
+  int r = blockIdx.y, c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < N) dst[(long long)r * N + c] = gemm_val(g, r, c);
+}
+
+extern "C" dream_status dream_debug_gemm(dream_ctx *c, const void *W, const float *X, int32_t rows, int32_t N,
+                                         int32_t K, int32_t split, float *out) {
+  if (!c || !W || !X || !out) return fail(c, DREAM_E_ARG, "null argument");
+  const dream_config &f = c->cfg;
+  bool bf = f.dtype == DREAM_BF16;
+  bool lo = bf && split && lo_on(c, rows);
+  void *buf; long long lod;
+  if (K <= f.d_model) { buf = c->xn; lod = (long long)ROW_CHUNK * K; if (lod > c->lo_xn) lod = c->lo_xn; }
+  else if (K <= f.d_ff) { buf = c->act; lod = (long long)ROW_CHUNK * K; if (lod > c->lo_act) lod = c->lo_act; }
+  else return fail(c, DREAM_E_ARG, "K exceeds the context's widest GEMM input");
+  if (rows < 1 || rows > (lo ? ROW_CHUNK / 2 : ROW_CHUNK)) return fail(c, DREAM_E_ARG, "rows out of range");
+  if (bf && K % 8) return fail(c, DREAM_E_ARG, "K must be a multiple of 8");
+  long long ld = lo ? (long long)ROW_CHUNK * K : 0;
+  (void)lod;
+  LAUNCH(c, k_split_rows, rows, 256, 0, X, buf, K, ld, bf ? 1 : 0);
+  GemmOut g = bf ? gemm<bf16>(c, W, buf, ld, rows, N, K) : gemm<float>(c, W, buf, 0, rows, N, K);
+  LAUNCH(c, k_gemm_collect, dim3((N + 255) / 256, rows), 256, 0, g, out, N);
+  CUDA_OK(c, cudaGetLastError());
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_gemm_counts(const dream_ctx *c, int64_t *tensor_core, int64_t *cuda_core) {
+  if (!c) return DREAM_E_ARG;
+  if (tensor_core) *tensor_core = c->tc_launches;
+  if (cuda_core) *cuda_core = c->simt_launches;
   return DREAM_OK;
 }
 
