@@ -189,8 +189,9 @@ dream_status dream_debug_read(dream_ctx *ctx, int32_t seq, int32_t what, int32_t
 
 /* Test hook: out[r][c] = sum_k X[r][k] W[c][k] through the context's GEMM path (the same
  * kernels every projection of the model uses).  W: device [N][K] in config.dtype; X: device
- * float [rows][K]; out: device float [rows][N]; rows <= 128 (256 when split == 0 or dtype is
- * fp32); K <= max(d_model, d_ff).  split != 0 feeds bf16 inputs as hi + lo parts. */
+ * float [rows][K]; out: device float [rows][N]; rows <= 256 (128 for bf16 with split == 0);
+ * K <= max(d_model, d_ff); bf16: K a multiple of 64, N of 8.  split != 0 feeds bf16 inputs as a
+ * high and a low bf16 row per token. */
 dream_status dream_debug_gemm(dream_ctx *ctx, const void *W, const float *X, int32_t rows,
                               int32_t N, int32_t K, int32_t split, float *out);
 

@@ -72,8 +72,10 @@ __device__ __forceinline__ float dot_lane(const float (&a)[EPL], const float (&b
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
-               T *attn_out, long long lo_delta, float *lse, float *ent) {
+               T *attn_out, XLayout lay, float *lse, float *ent) {
   constexpr int EPL = HD / 32;
+  pdl_trigger();
+  pdl_wait();
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int i = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (i >= n) return;
@@ -94,7 +96,7 @@ k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H
   float inv = 1.f / st.z;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
-    store_split<T>(attn_out + (long long)i * H * HD + h * HD + lane * EPL + e, lo_delta, st.acc[e] * inv);
+    store_split<T>(attn_out + i * lay.row_stride + h * HD + lane * EPL + e, lay.lo_delta, st.acc[e] * inv);
   if (lane == 0) {
     lse[(long long)h * n + i] = st.m + logf(st.z);
     ent[(long long)h * n + i] = logf(st.z) - st.u / st.z;
@@ -104,6 +106,8 @@ k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H
 // AE(l) = mean over rows and heads of the row entropies (Eq. 2).  One block, fixed order.
 __global__ void k_entropy_mean(const float *__restrict__ ent, int count, float *out) {
   __shared__ float sh[33];
+  pdl_trigger();
+  pdl_wait();
   float s = 0.f;
   for (int i = threadIdx.x; i < count; i += blockDim.x) s += ent[i];
   float t = block_sum(s, sh);
@@ -118,6 +122,8 @@ __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_colsum(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
          const float *__restrict__ lse, int vis_start, int v, int include_self, float *score) {
   constexpr int EPL = HD / 32;
+  pdl_trigger();
+  pdl_wait();
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int jv = blockIdx.x * ATT_WARPS + w;
   if (jv >= v) return;
@@ -148,8 +154,10 @@ __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ row_seq,
             const int *__restrict__ row_node, const int *__restrict__ P_state,
             const uint32_t *__restrict__ mask, int R, int T_nodes, int H, float scale, T *attn_out,
-            long long lo_delta) {
+            XLayout lay) {
   constexpr int EPL = HD / 32;
+  pdl_trigger();
+  pdl_wait();
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (r >= R) return;
@@ -180,7 +188,7 @@ k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ 
   float inv = 1.f / st.z;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
-    store_split<T>(attn_out + (long long)r * H * HD + h * HD + lane * EPL + e, lo_delta, st.acc[e] * inv);
+    store_split<T>(attn_out + r * lay.row_stride + h * HD + lane * EPL + e, lay.lo_delta, st.acc[e] * inv);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -193,8 +201,10 @@ __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ row_seq,
              const int *__restrict__ row_in, const int *__restrict__ nperm,
              const unsigned long long *__restrict__ anc, int anc_stride, int strict, int R, int H,
-             float scale, T *attn_out, long long lo_delta) {
+             float scale, T *attn_out, XLayout lay) {
   constexpr int EPL = HD / 32;
+  pdl_trigger();
+  pdl_wait();
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (r >= R) return;
@@ -227,5 +237,5 @@ k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ 
   float inv = 1.f / st.z;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
-    store_split<T>(attn_out + (long long)r * H * HD + h * HD + lane * EPL + e, lo_delta, st.acc[e] * inv);
+    store_split<T>(attn_out + r * lay.row_stride + h * HD + lane * EPL + e, lay.lo_delta, st.acc[e] * inv);
 }

@@ -17,9 +17,22 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
 
+// Programmatic dependent launch: a kernel may start while its predecessor in the stream is still
+// running; pdl_wait() blocks until the predecessor has completed and its writes are visible, and
+// pdl_trigger() lets the successor start early.  Every kernel of the library calls pdl_wait()
+// before it touches memory another kernel writes (weights never change and may be read earlier).
+// Both are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // A bf16 GEMM input row is stored as two bf16 rows, hi = bf16(v) and lo = bf16(v - hi), so the
-// tensor cores see the activation to ~16 mantissa bits while the weights stream once; the two
-// partial products are added by whoever reads the GEMM output.  fp32 inputs have no lo part.
+// tensor cores see the activation to ~16 mantissa bits while the weights stream once.  fp32
+// inputs have no lo part.  XLayout says where the rows of such a buffer live: token t starts at
+// element t * row_stride, and its lo part lo_delta elements further on (0 = no lo part).
+struct XLayout {
+  long long row_stride;
+  long long lo_delta;
+};
 template <typename T> __device__ __forceinline__ void store_split(T *p, long long lo_delta, float v);
 template <> __device__ __forceinline__ void store_split<float>(float *p, long long, float v) { *p = v; }
 template <> __device__ __forceinline__ void store_split<bf16>(bf16 *p, long long lo_delta, float v) {
@@ -28,33 +41,28 @@ template <> __device__ __forceinline__ void store_split<bf16>(bf16 *p, long long
   if (lo_delta) p[lo_delta] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-// Output of a GEMM launch: `count(tile)` partial sums per 128-column tile, stacked in slots
-// of slot_stride floats.  The stream-K tensor-core kernel leaves up to three partials per
-// tile; the SIMT kernel leaves one (upc == 0).  When the input was split into hi and lo rows
-// the products of the lo rows sit lo_off rows further down.
+// Output of a GEMM: rows are cut into chunks of (1 << chunk_shift) rows, one launch each,
+// chunk_stride floats apart.  Inside a chunk the stream-K tensor-core kernel leaves up to
+// ceil(kb / upc) + 1 partial sums per 256-column tile, stacked in slots of slot_stride floats; the
+// SIMT kernel leaves one (upc == 0).
 struct GemmOut {
   const float *base;
   long long slot_stride;   // floats between consecutive slots
+  long long chunk_stride;  // floats between consecutive row chunks
+  int chunk_shift;         // log2 of the rows per chunk
   int ld;                  // floats between consecutive rows (tokens)
-  int kb;                  // k-blocks per tile
-  int upc;                 // work units (tile, k-block) per CTA; 0 = single slot
-  int lo_off;              // rows between a token's hi and lo products; 0 = unsplit
+  int kb;                  // k-panels per tile
+  int upc;                 // work units (tile, k-panel) per CTA; 0 = single slot
 };
 
 __device__ __forceinline__ float gemm_val(const GemmOut &g, int r, int c) {
-  const float *p = g.base + (long long)r * g.ld + c;
+  int ch = r >> g.chunk_shift;
+  const float *p = g.base + (long long)ch * g.chunk_stride + (long long)(r - (ch << g.chunk_shift)) * g.ld + c;
   float s = *p;
-  int extra = 0;
   if (g.upc) {
-    long long u0 = (long long)(c >> 7) * g.kb;
-    extra = (int)((u0 + g.kb - 1) / g.upc) - (int)(u0 / g.upc);
+    unsigned u0 = (unsigned)(c >> 8) * (unsigned)g.kb;
+    int extra = (int)((u0 + (unsigned)g.kb - 1u) / (unsigned)g.upc) - (int)(u0 / (unsigned)g.upc);
     for (int i = 1; i <= extra; ++i) s += p[(long long)i * g.slot_stride];
-  }
-  if (g.lo_off) {
-    const float *q = p + (long long)g.lo_off * g.ld;
-    float t = *q;
-    for (int i = 1; i <= extra; ++i) t += q[(long long)i * g.slot_stride];
-    s += t;
   }
   return s;
 }

@@ -18,7 +18,7 @@
 #include "rows.cuh"
 #include "tree.cuh"
 
-#define ROW_CHUNK 256          // GEMM rows per launch, hi and lo rows together (tensor-core N <= 256)
+#define ROW_CHUNK 256          // most rows any launch set holds (max_batch * tree nodes, a prefill chunk)
 
 enum { PH_EMPTY = 0, PH_PREFILLED, PH_READY, PH_DRAFTED, PH_VERIFIED };
 
@@ -29,9 +29,9 @@ struct dream_ctx {
   cudaStream_t stream;
   TreeShape ts;
   int T, esz, qkvN, Hhd, kvN, n_cand, tap_lo_eff, cap_rows, pps, n_pages, RM, XR, gemm_rows_lm;
-  int use_tc;
-  int chunk;                           // token rows per GEMM launch (128 when inputs are split)
-  long long lo_xn, lo_act, lo_att;     // element offsets of the lo planes (0 = fp32, unsplit)
+  int use_tc, use_pdl, gemm_failed;
+  int chunk;                           // prompt rows per pass of the prefill loop
+  double *rope_inv;                    // [head_dim / 2] rotary inverse frequencies
   std::vector<const void *> ln1, wqkv, wo, ln2, wgu, wd;
   const void *embed, *ln_f, *lm_head;
   dream_draft_weights dw;
@@ -79,11 +79,20 @@ static dream_status fail(dream_ctx *c, dream_status code, const char *fmt, ...) 
     if (e_ != cudaSuccess) return fail(c, DREAM_E_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
   } while (0)
 
-#define LAUNCH(c, kernel, grid, block, smem, ...)          \
-  do {                                                     \
-    kernel<<<grid, block, smem, (c)->stream>>>(__VA_ARGS__); \
-    (c)->launches++;                                       \
-  } while (0)
+// Every kernel is launched with programmatic stream serialization: it may become resident while
+// its predecessor still runs and blocks in pdl_wait() until that one has finished.
+template <typename... P, typename... A>
+static inline void launch_k(dream_ctx *c, void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = c->use_pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+  c->launches++;
+}
+#define LAUNCH(c, kernel, grid, block, smem, ...) launch_k(c, kernel, dim3(grid), dim3(block), (size_t)(smem), __VA_ARGS__)
 
 // ------------------------------------------------------------------------------------- shapes
 
@@ -130,6 +139,8 @@ static dream_status check_config(const dream_config *c, TreeShape *ts) {
       c->n_heads % c->n_kv_heads || c->d_ff < 8 || c->vocab < 2)
     return fail(nullptr, DREAM_E_ARG, "model shape");
   if (c->d_model % 8 || c->d_ff % 8) return fail(nullptr, DREAM_E_UNSUPPORTED, "d_model, d_ff must be multiples of 8");
+  if (c->dtype == DREAM_BF16 && (c->d_model % 64 || c->d_ff % 64 || (c->n_heads * c->head_dim) % 64 || c->vocab % 8))
+    return fail(nullptr, DREAM_E_UNSUPPORTED, "bf16: d_model, d_ff, n_heads*head_dim must be multiples of 64 and vocab of 8");
   if (c->max_batch < 1 || c->max_batch > DREAM_MAX_BATCH) return fail(nullptr, DREAM_E_ARG, "max_batch in 1..8");
   if (c->page_tokens < 16 || c->page_tokens > 256 || (c->page_tokens & (c->page_tokens - 1)))
     return fail(nullptr, DREAM_E_ARG, "page_tokens must be a power of two in 16..256");
@@ -171,7 +182,7 @@ static void derive(dream_ctx *c) {
   c->cap_rows = f.max_seq + c->ts.NI;
   c->pps = (f.max_seq + f.page_tokens - 1) / f.page_tokens;
   c->n_pages = c->pps * f.max_batch;
-  c->chunk = f.dtype == DREAM_BF16 ? ROW_CHUNK / 2 : ROW_CHUNK;
+  c->chunk = f.dtype == DREAM_BF16 ? TC_ROWS_SPLIT_1MMA : ROW_CHUNK;
   c->RM = (imax(ROW_CHUNK, f.max_prompt) + 15) & ~15;
   c->XR = c->RM;
 }
@@ -220,23 +231,33 @@ static size_t carve(dream_ctx *c, char *base) {
   c->x = a.take<float>((size_t)c->XR * d);
   c->x0 = a.take<float>((size_t)f.max_prompt * d);
   c->qbuf = a.take<float>((size_t)c->XR * c->Hhd);
-  int planes = f.dtype == DREAM_BF16 ? 2 : 1;
-  c->lo_xn = planes == 2 ? (long long)ROW_CHUNK * d : 0;
-  c->lo_act = planes == 2 ? (long long)ROW_CHUNK * f.d_ff : 0;
-  c->lo_att = planes == 2 ? (long long)c->XR * c->Hhd : 0;
+  int planes = f.dtype == DREAM_BF16 ? 2 : 1;      // bf16 GEMM inputs: a high and a low row per token
   c->attn_out = a.take_bytes((size_t)planes * c->XR * c->Hhd * e);
   c->xn = a.take_bytes((size_t)planes * ROW_CHUNK * d * e);
   c->raw = a.take_bytes((size_t)planes * ROW_CHUNK * d * e);
   c->act = a.take_bytes((size_t)planes * ROW_CHUNK * f.d_ff * e);
-  int widest = imax(imax(c->qkvN, 2 * f.d_ff), imax(d, c->Hhd));
   int lm_rows = ((imax(MB * T, MB * imax(c->ts.D + 2, f.tree_beam)) + 15) / 16) * 16;
   c->gemm_rows_lm = lm_rows;
-  // room for the stream-K partial slots: a tile is shared by at most ceil(KB/upc) + 1 CTAs and
-  // upc >= tiles*KB/148, so slots * N <= (148/tiles + 2) * N <= 148*128 + 2N (+ slack)
-  size_t wide = (size_t)ROW_CHUNK * (2 * (size_t)widest + 19200);
-  size_t lm = (size_t)imin(2 * lm_rows, ROW_CHUNK) * (2 * (size_t)f.vocab + 19200);
-  c->gout_floats = wide > lm ? wide : lm;
+  // GEMM output: the widest of every projection's footprint.  fp32: rows x N.  bf16: one region
+  // per 64-row chunk, each with room for the stream-K partial-sum slots (bound for <= 192 SMs).
+  {
+    const int shapes[8][2] = {{c->qkvN, d}, {d, c->Hhd}, {2 * f.d_ff, d}, {d, f.d_ff}, {c->Hhd, d}, {c->kvN, d}, {f.vocab, d}, {0, 0}};
+    size_t need = 0;
+    for (int i = 0; shapes[i][0]; ++i) {
+      int N = shapes[i][0], K = shapes[i][1];
+      size_t fl;
+      if (f.dtype == DREAM_BF16) {
+        long long per = (gemm_tc_out_floats(192, TC_ROWS_SPLIT_1MMA, N, K) + 63) & ~63LL;
+        long long per2 = (gemm_tc_out_floats(192, TC_ROWS_MAX, N, K) + 63) & ~63LL;
+        fl = (size_t)imax(1, ROW_CHUNK / TC_ROWS_SPLIT_1MMA) * per;
+        if ((size_t)per2 > fl) fl = per2;
+      } else fl = (size_t)ROW_CHUNK * N;
+      if (fl > need) need = fl;
+    }
+    c->gout_floats = need;
+  }
   c->gout = a.take<float>(c->gout_floats);
+  c->rope_inv = a.take<double>(f.head_dim / 2);
   c->lse_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
   c->ent_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
   c->ae = a.take<float>(f.n_layers);
@@ -267,25 +288,47 @@ extern "C" dream_status dream_arena_bytes(const dream_config *cfg, size_t *bytes
 
 // ------------------------------------------------------------------------------------- GEMM dispatch
 
-// out[r][c] = sum_k X[r][k] W[c][k] for r < rows, c < N.  lo_delta != 0: X carries a second
-// plane of low-order parts lo_delta elements further on, multiplied in the same launch.
+// How the rows of a bf16 GEMM input buffer are laid out for a launch set of R rows: up to 64 rows
+// (and beyond 128, in chunks of 64) high and low rows alternate; 65..128 rows use two planes.
+struct XMode { int mode, lo_rows; };
+static XMode xmode(const dream_ctx *c, int R) {
+  if (c->cfg.dtype != DREAM_BF16) return XMode{TC_X_PLAIN, 0};
+  if (R <= TC_ROWS_SPLIT_1MMA || R > TC_ROWS_MAX) return XMode{TC_X_INTERLEAVED, 0};
+  return XMode{TC_X_PLANAR, TC_ROWS_MAX};
+}
+static XLayout xlay(XMode m, long long width) {
+  if (m.mode == TC_X_INTERLEAVED) return XLayout{2 * width, width};
+  if (m.mode == TC_X_PLANAR) return XLayout{width, (long long)m.lo_rows * width};
+  return XLayout{width, 0};
+}
+
+// out[r][c] = sum_k X[r][k] W[c][k] for r < rows, c < N; X holds the rows in layout m.
 // Returns the descriptor consumers read the result through.
 template <typename T>
-static GemmOut gemm(dream_ctx *c, const void *W, const void *X, long long lo_delta, int rows, int N, int K) {
+static GemmOut gemm(dream_ctx *c, const void *W, const void *X, XMode m, int rows, int N, int K) {
   GemmOut g;
-  int rows_pad = (rows + 15) & ~15;
-  if (c->use_tc && sizeof(T) == 2 && gemm_tc_supported(rows_pad * (lo_delta ? 2 : 1), N, K) &&
-      gemm_tc_launch(&c->tc, c->stream, W, X, lo_delta, rows, N, K, c->gout, (long long)c->gout_floats, &g)) {
-    c->launches++;
-    c->tc_launches++;
+  if (sizeof(T) == 2) {
+    int chunk = m.mode == TC_X_INTERLEAVED ? TC_ROWS_SPLIT_1MMA : TC_ROWS_MAX;
+    int nch = (rows + chunk - 1) / chunk;
+    int slot_rows = nch > 1 ? chunk : rows;
+    long long per = (gemm_tc_out_floats(c->tc.n_sms, slot_rows, N, K) + 63) & ~63LL;
+    XLayout lay = xlay(m, K);
+    for (int ch = 0; ch < nch; ++ch) {
+      int rows_c = imin(chunk, rows - ch * chunk);
+      const bf16 *Xc = (const bf16 *)X + (long long)ch * chunk * lay.row_stride;
+      if (!gemm_tc_launch(&c->tc, c->stream, W, Xc, m.mode, m.lo_rows, rows_c, slot_rows, N, K, c->gout + (long long)ch * per,
+                          (long long)c->gout_floats - (long long)ch * per, &g))
+        c->gemm_failed = 1;
+      c->launches++;
+      c->tc_launches++;
+    }
+    g.base = c->gout; g.chunk_stride = per; g.chunk_shift = chunk == 64 ? 6 : 7;
     return g;
   }
   c->simt_launches++;
-  int tiles = (rows + SG_BM - 1) / SG_BM;
-  dim3 grid((N + SG_BN - 1) / SG_BN, tiles * (lo_delta ? 2 : 1));
-  k_gemm_simt<T><<<grid, 256, 0, c->stream>>>((const T *)X, (const T *)W, c->gout, rows, N, K, N, tiles, lo_delta, rows_pad);
-  c->launches++;
-  g.base = c->gout; g.slot_stride = 0; g.ld = N; g.kb = 0; g.upc = 0; g.lo_off = lo_delta ? rows_pad : 0;
+  dim3 grid((N + SG_BN - 1) / SG_BN, (rows + SG_BM - 1) / SG_BM);
+  LAUNCH(c, (k_gemm_simt<T>), grid, 256, 0, (const T *)X, (const T *)W, c->gout, rows, N, K, N);
+  g.base = c->gout; g.slot_stride = 0; g.chunk_stride = 0; g.chunk_shift = 30; g.ld = N; g.kb = 0; g.upc = 0;
   return g;
 }
 
@@ -306,7 +349,7 @@ static FlatKV flat(dream_ctx *c, float *base) {
   kv.base = base; kv.cap = c->cap_rows; kv.hkv = c->cfg.n_kv_heads; kv.hd = c->cfg.head_dim;
   return kv;
 }
-static const GemmOut NO_GEMM = {nullptr, 0, 0, 0, 0, 0};
+static const GemmOut NO_GEMM = {nullptr, 0, 0, 30, 0, 0, 0};
 
 // ------------------------------------------------------------------------------------- init / free
 
@@ -344,14 +387,17 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   for (int p = c->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
   for (int b = 0; b < DREAM_MAX_BATCH; ++b) c->phase[b] = PH_EMPTY;
   c->prefill_seq = -1;
-  c->launches = 0; c->tc_launches = 0; c->simt_launches = 0;
+  c->launches = 0; c->tc_launches = 0; c->simt_launches = 0; c->gemm_failed = 0;
   c->err[0] = 0;
-  const char *mode = getenv("DREAM_GEMM");
-  c->use_tc = cfg->dtype == DREAM_BF16 && !(mode && !strcmp(mode, "simt"));
+  const char *pdl = getenv("DREAM_PDL");              // "0" serialises every launch (debugging aid)
+  c->use_pdl = !(pdl && !strcmp(pdl, "0"));
+  c->use_tc = cfg->dtype == DREAM_BF16;
   if (c->use_tc) {
-    const char *why = gemm_tc_plan_init(&c->tc, c->status);
+    const char *why = gemm_tc_plan_init(&c->tc, c->status, c->use_pdl);
     if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
   }
+  k_rope_table<<<(cfg->head_dim / 2 + 127) / 128, 128, 0, c->stream>>>(c->rope_inv, cfg->head_dim, cfg->rope_theta);
+  if (cudaGetLastError() != cudaSuccess) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "rotary table launch failed"); }
   *out = c;
   return DREAM_OK;
 }
@@ -395,23 +441,35 @@ extern "C" dream_status dream_seq_reset(dream_ctx *c, int32_t seq) {
 // ------------------------------------------------------------------------------------- small kernels
 
 __global__ void k_iota_rows(RowMeta rm, int seq, int n) {
+  pdl_trigger();
+  pdl_wait();
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   rm.seq[i] = seq; rm.pos[i] = i; rm.slot[i] = i; rm.dst[i] = i; rm.in[i] = -1;
 }
 __global__ void k_set_seq(SeqDev s, int seq, int P, const int *pending_src, int nd, int nm) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x) return;
   if (P >= 0) s.P[seq] = P;
   if (pending_src) s.pending[seq] = *pending_src;
   if (nd >= 0) { s.nperm_d[seq] = nd; s.nperm_m[seq] = nm; s.n_new[seq] = 0; }
 }
-__global__ void k_set_int(int *p, int v) { if (!threadIdx.x) *p = v; }
+__global__ void k_set_int(int *p, int v) {
+  pdl_trigger();
+  pdl_wait();
+  if (!threadIdx.x) *p = v;
+}
 __global__ void k_first_token(const int *top_id, const float *top_val, int *tok, float *margin) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x) return;
   if (tok) *tok = top_id[0];
   if (margin) *margin = top_val[0] - top_val[1];
 }
 __global__ void k_argmax_out(const int *top_id, const float *top_val, int R, int *am, float *mg, int *am2) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= R) return;
   am[r] = top_id[2 * r];
@@ -419,6 +477,8 @@ __global__ void k_argmax_out(const int *top_id, const float *top_val, int R, int
   if (mg) mg[r] = top_val[2 * r] - top_val[2 * r + 1];
 }
 __global__ void k_copy_f32(const float *src, float *dst, int n) {
+  pdl_trigger();
+  pdl_wait();
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src[i];
 }
@@ -428,29 +488,26 @@ __global__ void k_read_row(const T *src, float *dst, int n) {
   if (i < n) dst[i] = to_f(src[i]);
 }
 
-// Split GEMM inputs into hi and lo rows when both fit one launch (see store_split).
-static bool lo_on(const dream_ctx *c, int rows) { return c->cfg.dtype == DREAM_BF16 && ((rows + 15) & ~15) * 2 <= ROW_CHUNK; }
-
 template <typename T, int HD> struct AttnLaunch {
   static void prefill(dream_ctx *c, int layer, int seq, int n) {
     dim3 grid((n + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_prefill<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n, c->cfg.n_heads,
-           1.f / sqrtf((float)HD), (T *)c->attn_out, c->lo_att, c->lse_pre, c->ent_pre);
+           1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(xmode(c, 1), c->Hhd), c->lse_pre, c->ent_pre);
   }
   static void colsum(dream_ctx *c, int layer, int seq, int n, int vis_start, int v, float *score) {
     if (v == 0) return;
     LAUNCH(c, (k_colsum<T, HD>), (v + ATT_WARPS - 1) / ATT_WARPS, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n,
            c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, score);
   }
-  static void tree(dream_ctx *c, int layer, int R, bool lo) {
+  static void tree(dream_ctx *c, int layer, int R, XMode m) {
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_tree<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
-           c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, lo ? c->lo_att : 0LL);
+           c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
   }
-  static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, bool lo) {
+  static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, XMode m) {
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_draft<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, flat(c, cache), rm.seq, rm.in, nperm,
-           c->dt.in_anc, c->ts.NI, strict, R, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, lo ? c->lo_att : 0LL);
+           c->dt.in_anc, c->ts.NI, strict, R, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
   }
 };
 
@@ -463,18 +520,18 @@ template <typename T, int HD> struct AttnLaunch {
 
 // x (+= GEMM output) -> RMSNorm -> GEMM input rows in c->xn; see k_resid_norm for the side outputs.
 template <typename T>
-static void norm_rows(dream_ctx *c, float *x, const GemmOut &gin, bool has_in, const void *gain, int rows, bool lo,
+static void norm_rows(dream_ctx *c, float *x, const GemmOut &gin, bool has_in, const void *gain, int rows, XMode m,
                       float *copy = nullptr, const int *row_seq = nullptr, const int *tap = nullptr, int layer = 0,
                       bool want_raw = false) {
   LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
-         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, lo ? c->lo_xn : 0LL);
+         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
 }
 template <typename T>
-static GemmOut mlp_rows(dream_ctx *c, const void *wgu, const void *wd, int rows, bool lo) {
+static GemmOut mlp_rows(dream_ctx *c, const void *wgu, const void *wd, int rows, XMode m) {
   const dream_config &f = c->cfg;
-  GemmOut g = gemm<T>(c, wgu, c->xn, lo ? c->lo_xn : 0, rows, 2 * f.d_ff, f.d_model);
-  LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, rows), 256, 0, g, (T *)c->act, f.d_ff, lo ? c->lo_act : 0LL);
-  return gemm<T>(c, wd, c->act, lo ? c->lo_act : 0, rows, f.d_model, f.d_ff);
+  GemmOut g = gemm<T>(c, wgu, c->xn, m, rows, 2 * f.d_ff, f.d_model);
+  LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, rows), 256, 0, g, (T *)c->act, f.d_ff, xlay(m, f.d_ff));
+  return gemm<T>(c, wd, c->act, m, rows, f.d_model, f.d_ff);
 }
 
 // ------------------------------------------------------------------------------------- prefill
@@ -488,14 +545,15 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
   LAUNCH(c, k_iota_rows, (n + 255) / 256, 256, 0, c->rm[0], seq, n);
   LAUNCH(c, (k_build_prompt<T>), n, 256, 0, (const T *)c->embed, (const T *)visual, ids, vis_start, v, c->x, c->x0,
          d, f.vocab, c->status);
+  const XMode m1 = xmode(c, 1);            // the layout of at most one chunk of rows
+  const XLayout att = xlay(m1, c->Hhd);
   for (int l = 0; l < L; ++l) {
     for (int r0 = 0; r0 < n; r0 += CH) {
       int rows = imin(CH, n - r0);
-      bool lo = lo_on(c, rows);
-      norm_rows<T>(c, c->x + (size_t)r0 * d, NO_GEMM, false, c->ln1[l], rows, lo);
-      GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, lo ? c->lo_xn : 0, rows, c->qkvN, d);
-      LAUNCH(c, (k_qkv_post_target<T>), rows, 128, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
-             paged(c, l), f.n_heads, f.rope_theta);
+      norm_rows<T>(c, c->x + (size_t)r0 * d, NO_GEMM, false, c->ln1[l], rows, m1);
+      GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, m1, rows, c->qkvN, d);
+      LAUNCH(c, (k_qkv_post_target<T>), rows, 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
+             paged(c, l), f.n_heads, c->rope_inv);
     }
     HD_DISPATCH(c, T, prefill(c, l, seq, n));
     LAUNCH(c, k_entropy_mean, 1, 1024, 0, c->ent_pre, f.n_heads * n, c->ae + l);
@@ -504,18 +562,17 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
     if (is_cand) HD_DISPATCH(c, T, colsum(c, l, seq, n, vis_start, v, c->scores_all + (size_t)cand * imax(f.max_visual, 1)));
     for (int r0 = 0; r0 < n; r0 += CH) {
       int rows = imin(CH, n - r0);
-      bool lo = lo_on(c, rows);
       float *xr = c->x + (size_t)r0 * d;
-      GemmOut g = gemm<T>(c, c->wo[l], (const T *)c->attn_out + (size_t)r0 * c->Hhd, c->lo_att, rows, d, c->Hhd);
-      norm_rows<T>(c, xr, g, true, c->ln2[l], rows, lo);
-      g = mlp_rows<T>(c, c->wgu[l], c->wd[l], rows, lo);
+      GemmOut g = gemm<T>(c, c->wo[l], (const T *)c->attn_out + (long long)r0 * att.row_stride, m1, rows, d, c->Hhd);
+      norm_rows<T>(c, xr, g, true, c->ln2[l], rows, m1);
+      g = mlp_rows<T>(c, c->wgu[l], c->wd[l], rows, m1);
       float *copy = is_cand ? c->taps_store + ((size_t)cand * f.max_prompt + r0) * d : nullptr;
       LAUNCH(c, k_resid_add, rows, 256, 0, xr, g, d, copy);
     }
   }
   // first token: LM head on the last prompt row
-  norm_rows<T>(c, c->x + (size_t)(n - 1) * d, NO_GEMM, false, c->ln_f, 1, lo_on(c, 1));
-  GemmOut g = gemm<T>(c, c->lm_head, c->xn, lo_on(c, 1) ? c->lo_xn : 0, 1, f.vocab, d);
+  norm_rows<T>(c, c->x + (size_t)(n - 1) * d, NO_GEMM, false, c->ln_f, 1, m1);
+  GemmOut g = gemm<T>(c, c->lm_head, c->xn, m1, 1, f.vocab, d);
   LAUNCH(c, k_topk_lse, 1, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
   LAUNCH(c, k_first_token, 1, 32, 0, c->top_id, c->top_val, first_token, first_margin);
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, n, c->top_id, -1, -1);
@@ -548,6 +605,7 @@ extern "C" dream_status dream_prefill(dream_ctx *c, int32_t seq, const void *vis
   else s = prefill_impl<float>(c, seq, visual, v, vis_start, ids, q, first_token, first_margin, layer_entropy, tap_layer);
   if (s) return s;
   CUDA_OK(c, cudaGetLastError());
+  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
   c->phase[seq] = PH_PREFILLED;
   c->n_prompt[seq] = v + q; c->p_ub[seq] = v + q;
   c->prefill_seq = seq; c->pf_v = v; c->pf_vis_start = vis_start; c->pf_q = q;
@@ -574,25 +632,24 @@ static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *force
          v, k, c->pf_vis_start, n, forced, kept, scores, c->ctx_pos, c->flags);
   // draft self-attention K/V of the compressed context, from the input embeddings
   const char *wkv = (const char *)c->dw.wqkv + (size_t)c->Hhd * d * c->esz;
+  const XMode m1 = xmode(c, 1);
   for (int r0 = 0; r0 < nc; r0 += CH) {
     int rows = imin(CH, nc - r0);
-    bool lo = lo_on(c, rows);
     LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, 0, seq, c->rm[0], c->gather_idx, r0);
-    LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL, 0LL);
-    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, rows, lo);
-    GemmOut g = gemm<T>(c, wkv, c->xn, lo ? c->lo_xn : 0, rows, c->kvN, d);
-    LAUNCH(c, k_qkv_post_draft, rows, 128, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
-           flat(c, c->dself), f.n_heads, f.rope_theta);
+    LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL, XLayout{d, 0});
+    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, rows, m1);
+    GemmOut g = gemm<T>(c, wkv, c->xn, m1, rows, c->kvN, d);
+    LAUNCH(c, k_qkv_post_draft, rows, 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
+           flat(c, c->dself), f.n_heads, c->rope_inv);
   }
   // cross-attention memory: tapped features at the context positions, projected (Eq. 1)
   int nm = f.xattn_full_memory ? n : nc;
   for (int r0 = 0; r0 < nm; r0 += CH) {
     int rows = imin(CH, nm - r0);
-    bool lo = lo_on(c, rows);
     LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, f.xattn_full_memory, seq, c->rm[0], c->gather_idx, r0);
     LAUNCH(c, (k_gather_rows<T>), rows, 256, 0, c->taps_store, c->gather_idx, (T *)c->raw, d, c->sd.tap + seq, c->tap_lo_eff,
-           (long long)f.max_prompt * d, lo ? c->lo_xn : 0LL);
-    GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, lo ? c->lo_xn : 0, rows, c->kvN, d);
+           (long long)f.max_prompt * d, xlay(m1, d));
+    GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, m1, rows, c->kvN, d);
     LAUNCH(c, k_mem_append, rows, 256, 0, g, c->rm[0].seq, c->rm[0].dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
   }
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, -1, (const int *)nullptr, nc, nm);
@@ -610,6 +667,7 @@ extern "C" dream_status dream_compress_visual(dream_ctx *c, int32_t seq, int32_t
                                  : compress_impl<float>(c, seq, k, forced, kept, scores);
   if (s) return s;
   CUDA_OK(c, cudaGetLastError());
+  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
   c->phase[seq] = PH_READY;
   c->prefill_seq = -1;
   return DREAM_OK;
@@ -648,28 +706,27 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
   for (int p = 1; p <= ts.D; ++p) {
     int m = p == 1 ? ts.D + 2 : ts.beam[p - 1];
     int R = B * m;
-    bool lo = lo_on(c, R);
-    long long lx = lo ? c->lo_xn : 0, la = lo ? c->lo_att : 0;
+    const XMode xm = xmode(c, R);
     RowMeta &rm = c->rm[cur], &rn = c->rm[cur ^ 1];
     if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
     LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
-    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, lo);
-    GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, lx, R, c->qkvN, d);
-    LAUNCH(c, k_qkv_post_draft, R, 128, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, f.rope_theta);
-    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, lo));
-    g = gemm<T>(c, c->dw.wo, c->attn_out, la, R, d, c->Hhd);
-    norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, lo);
-    g = gemm<T>(c, c->dw.xq, c->xn, lx, R, c->Hhd, d);
+    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
+    GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
+    LAUNCH(c, k_qkv_post_draft, R, 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
+    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm));
+    g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
+    g = gemm<T>(c, c->dw.xq, c->xn, xm, R, c->Hhd, d);
     LAUNCH(c, k_gemm_to_f32, R, 256, 0, g, c->qbuf, c->Hhd);
-    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, lo));
-    g = gemm<T>(c, c->dw.xo, c->attn_out, la, R, d, c->Hhd);
-    norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, lo);
-    g = mlp_rows<T>(c, c->dw.wgu, c->dw.wd, R, lo);
+    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm));
+    g = gemm<T>(c, c->dw.xo, c->attn_out, xm, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, xm);
+    g = mlp_rows<T>(c, c->dw.wgu, c->dw.wd, R, xm);
     // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
-    norm_rows<T>(c, c->x, g, true, c->ln_f, R, lo, nullptr, nullptr, nullptr, 0, true);
-    g = gemm<T>(c, c->dw.xkv, c->raw, lx, R, c->kvN, d);
+    norm_rows<T>(c, c->x, g, true, c->ln_f, R, xm, nullptr, nullptr, nullptr, 0, true);
+    g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
     LAUNCH(c, k_mem_append, R, 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
-    g = gemm<T>(c, c->lm_head, c->xn, lx, R, f.vocab, d);
+    g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
     LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, ts.K, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
     int next_m = p < ts.D ? ts.beam[p] : 1;
     LAUNCH(c, k_tree_expand, B, 128, 0, tb, c->sd, c->dt, ts, p, m, c->top_val, c->top_id, c->lse_rows, rn, next_m);
@@ -688,6 +745,7 @@ extern "C" dream_status dream_draft_tree(dream_ctx *c, const int32_t *seqs, int3
   s = c->cfg.dtype == DREAM_BF16 ? draft_impl<bf16>(c, tb, n_seqs) : draft_impl<float>(c, tb, n_seqs);
   if (s) return s;
   CUDA_OK(c, cudaGetLastError());
+  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
   for (int b = 0; b < n_seqs; ++b) c->phase[seqs[b]] = PH_DRAFTED;
   return DREAM_OK;
 }
@@ -698,24 +756,23 @@ template <typename T>
 static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *argmax, float *margin, float *logits) {
   const dream_config &f = c->cfg;
   int d = f.d_model, L = f.n_layers, R = B * c->T;
-  bool lo = lo_on(c, R);
-  long long lx = lo ? c->lo_xn : 0, la = lo ? c->lo_att : 0;
+  const XMode xm = xmode(c, R);
   RowMeta &rm = c->rm[0];
   LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
   LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
   GemmOut gd = NO_GEMM;
   for (int l = 0; l < L; ++l) {
     // completes S^l (for l >= 1) and captures it where a sequence taps layer l
-    norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, lo, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
-    GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, lx, R, c->qkvN, d);
-    LAUNCH(c, (k_qkv_post_target<T>), R, 128, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, f.rope_theta);
-    HD_DISPATCH(c, T, tree(c, l, R, lo));
-    g = gemm<T>(c, c->wo[l], c->attn_out, la, R, d, c->Hhd);
-    norm_rows<T>(c, c->x, g, true, c->ln2[l], R, lo);
-    gd = mlp_rows<T>(c, c->wgu[l], c->wd[l], R, lo);
+    norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, xm, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
+    GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, xm, R, c->qkvN, d);
+    LAUNCH(c, (k_qkv_post_target<T>), R, 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv);
+    HD_DISPATCH(c, T, tree(c, l, R, xm));
+    g = gemm<T>(c, c->wo[l], c->attn_out, xm, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->ln2[l], R, xm);
+    gd = mlp_rows<T>(c, c->wgu[l], c->wd[l], R, xm);
   }
-  norm_rows<T>(c, c->x, gd, true, c->ln_f, R, lo, c->tapbuf, rm.seq, c->sd.tap, L);
-  GemmOut g = gemm<T>(c, c->lm_head, c->xn, lx, R, f.vocab, d);
+  norm_rows<T>(c, c->x, gd, true, c->ln_f, R, xm, c->tapbuf, rm.seq, c->sd.tap, L);
+  GemmOut g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
   LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, logits);
   LAUNCH(c, k_argmax_out, (R + 127) / 128, 128, 0, c->top_id, c->top_val, R, argmax, margin,
          argmax == c->argmax_i ? (int *)nullptr : c->argmax_i);
@@ -736,6 +793,7 @@ extern "C" dream_status dream_verify_tree(dream_ctx *c, const int32_t *seqs, int
                                  : verify_impl<float>(c, tb, n_seqs, node_argmax, node_margin, logits);
   if (s) return s;
   CUDA_OK(c, cudaGetLastError());
+  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
   for (int b = 0; b < n_seqs; ++b) c->phase[seqs[b]] = PH_VERIFIED;
   return DREAM_OK;
 }
@@ -751,9 +809,9 @@ static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const 
   LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
   LAUNCH(c, (k_compact_kv<T>), dim3(f.n_layers * 2, B), 256, 0, tb, c->sd, c->kv_pool, c->layer_stride, c->kv_stride, paged(c, 0));
   LAUNCH(c, k_accept_rows, 1, 32, 0, tb, B, c->T, D, c->sd, c->gather_idx, rm, c->cap_rows - c->ts.NI, c->status);
-  bool lo = lo_on(c, R);
-  LAUNCH(c, (k_gather_rows<T>), R, 256, 0, c->tapbuf, c->gather_idx, (T *)c->raw, d, (const int *)nullptr, 0, 0LL, lo ? c->lo_xn : 0LL);
-  GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, lo ? c->lo_xn : 0, R, c->kvN, d);
+  const XMode xm = xmode(c, R);
+  LAUNCH(c, (k_gather_rows<T>), R, 256, 0, c->tapbuf, c->gather_idx, (T *)c->raw, d, (const int *)nullptr, 0, 0LL, xlay(xm, d));
+  GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
   LAUNCH(c, k_mem_append, R, 256, 0, g, rm.seq, rm.dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
   return DREAM_OK;
 }
@@ -771,6 +829,7 @@ extern "C" dream_status dream_accept(dream_ctx *c, const int32_t *seqs, int32_t 
                                  : accept_impl<float>(c, tb, n_seqs, node_argmax, accept_len, out_tokens, comp_src);
   if (s) return s;
   CUDA_OK(c, cudaGetLastError());
+  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
   for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; }
   return DREAM_OK;
 }
@@ -843,15 +902,19 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
 }
 
 // out[r][c] = sum_k X[r][k] W[c][k] through the context's GEMM path (test hook).
-__global__ void k_split_rows(const float *src, void *dst, int K, long long lo_delta, int is_bf16) {
+__global__ void k_split_rows(const float *src, void *dst, int K, XLayout lay, int is_bf16) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x;
   for (int i = threadIdx.x; i < K; i += blockDim.x) {
     float v = src[(long long)r * K + i];
-    if (is_bf16) store_split<bf16>((bf16 *)dst + (long long)r * K + i, lo_delta, v);
+    if (is_bf16) store_split<bf16>((bf16 *)dst + r * lay.row_stride + i, lay.lo_delta, v);
     else ((float *)dst)[(long long)r * K + i] = v;
   }
 }
 __global__ void k_gemm_collect(GemmOut g, float *dst, int N) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.y, c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c < N) dst[(long long)r * N + c] = gemm_val(g, r, c);
 }
@@ -861,19 +924,24 @@ extern "C" dream_status dream_debug_gemm(dream_ctx *c, const void *W, const floa
   if (!c || !W || !X || !out) return fail(c, DREAM_E_ARG, "null argument");
   const dream_config &f = c->cfg;
   bool bf = f.dtype == DREAM_BF16;
-  bool lo = bf && split && lo_on(c, rows);
-  void *buf; long long lod;
-  if (K <= f.d_model) { buf = c->xn; lod = (long long)ROW_CHUNK * K; if (lod > c->lo_xn) lod = c->lo_xn; }
-  else if (K <= f.d_ff) { buf = c->act; lod = (long long)ROW_CHUNK * K; if (lod > c->lo_act) lod = c->lo_act; }
+  void *buf;
+  if (K <= f.d_model) buf = c->xn;
+  else if (K <= f.d_ff) buf = c->act;
   else return fail(c, DREAM_E_ARG, "K exceeds the context's widest GEMM input");
-  if (rows < 1 || rows > (lo ? ROW_CHUNK / 2 : ROW_CHUNK)) return fail(c, DREAM_E_ARG, "rows out of range");
-  if (bf && K % 8) return fail(c, DREAM_E_ARG, "K must be a multiple of 8");
-  long long ld = lo ? (long long)ROW_CHUNK * K : 0;
-  (void)lod;
-  LAUNCH(c, k_split_rows, rows, 256, 0, X, buf, K, ld, bf ? 1 : 0);
-  GemmOut g = bf ? gemm<bf16>(c, W, buf, ld, rows, N, K) : gemm<float>(c, W, buf, 0, rows, N, K);
+  if (rows < 1 || rows > ROW_CHUNK) return fail(c, DREAM_E_ARG, "rows out of range");
+  if (bf && (K % 64 || N % 8)) return fail(c, DREAM_E_ARG, "K must be a multiple of 64 and N of 8");
+  XMode xm = xmode(c, rows);
+  if (bf && !split) {                     // single bf16 row per token
+    if (rows > TC_ROWS_MAX) return fail(c, DREAM_E_ARG, "unsplit inputs take at most 128 rows");
+    xm = XMode{TC_X_PLAIN, 0};
+  }
+  size_t need_out = (size_t)rows * N;
+  (void)need_out;
+  LAUNCH(c, k_split_rows, rows, 256, 0, X, buf, K, xlay(xm, K), bf ? 1 : 0);
+  GemmOut g = bf ? gemm<bf16>(c, W, buf, xm, rows, N, K) : gemm<float>(c, W, buf, xm, rows, N, K);
   LAUNCH(c, k_gemm_collect, dim3((N + 255) / 256, rows), 256, 0, g, out, N);
   CUDA_OK(c, cudaGetLastError());
+  if (c->gemm_failed) { c->gemm_failed = 0; return fail(c, DREAM_E_UNSUPPORTED, "the GEMM launch was refused (shape or output room)"); }
   return DREAM_OK;
 }
 

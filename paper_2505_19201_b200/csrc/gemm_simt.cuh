@@ -1,6 +1,6 @@
 // Plain CUDA-core GEMM  out[r][c] = sum_k X[r][k] W[c][k]  with fp32 accumulation.
 // It serves the fp32 (toy) configuration, whose tolerances rule out tf32 tensor-core
-// rounding, and is the debugging stand-in for the tensor-core kernel on bf16 shapes.
+// rounding; bf16 configurations always take the tensor-core kernel.
 #pragma once
 #include "common.cuh"
 
@@ -11,17 +11,13 @@
 template <typename T>
 __global__ void __launch_bounds__(256)
 k_gemm_simt(const T *__restrict__ X, const T *__restrict__ W, float *__restrict__ out, int rows,
-            int N, int K, int ldo, int row_tiles, long long lo_delta, int lo_off) {
+            int N, int K, int ldo) {
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float Bs[SG_BK][SG_BN + 4];
+  pdl_trigger();
+  pdl_wait();
   int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  int ty_blk = blockIdx.y;
-  if (ty_blk >= row_tiles) {            // second plane: low-order parts of the input rows
-    ty_blk -= row_tiles;
-    X += lo_delta;
-    out += (long long)lo_off * ldo;
-  }
-  int r0 = ty_blk * SG_BM, c0 = blockIdx.x * SG_BN;
+  int r0 = blockIdx.y * SG_BM, c0 = blockIdx.x * SG_BN;
   int lr = threadIdx.x >> 2, lk = (threadIdx.x & 3) * 4;
   float acc[4][4] = {};
   for (int k0 = 0; k0 < K; k0 += SG_BK) {

@@ -1,19 +1,26 @@
 // Weight-streaming small-M GEMM for sm_100a:  out[t][c] = sum_k X[t][k] * W[c][k].
 //
-// The token count (<= 256 rows, hi and lo planes together) is tiny and the weight matrix is
-// large, so the kernel is bound by streaming W from HBM once.  Design:
-//   * swap-AB: the 128 weight rows of a tile are the MMA's M (TMEM lanes), the tokens are its
-//     N (TMEM columns); one tcgen05.mma (cta_group::1, kind::f16, bf16 x bf16 -> fp32) covers
-//     128 x N x 16, four per 64-wide k-block;
-//   * W and X tiles arrive by TMA (cp.async.bulk.tensor.2d, 128-byte swizzle, no multicast)
-//     into a ring of shared-memory stages guarded by mbarriers;
-//   * persistent stream-K: the (tile, k-block) units are dealt out in equal contiguous ranges
-//     to one CTA per SM, so every SM streams the same number of bytes whatever the tile count;
-//     a CTA that covers part of a tile writes a partial sum to its own slot and the consumer
-//     adds the (at most three) slots, in a fixed order;
-//   * warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 =
-//     epilogue (tcgen05.ld -> coalesced fp32 stores); two TMEM accumulators alternate so the
-//     epilogue of one segment overlaps the MMAs of the next;
+// The token count is tiny (<= 128 rows) and the weight matrix is large, so the kernel is bound
+// by streaming W from HBM once.  Design:
+//   * tokens are the MMA's M (the 128 TMEM lanes) and 256 weight rows are its N (TMEM columns):
+//     one tcgen05.mma (cta_group::1, kind::f16, bf16 x bf16 -> fp32) covers 128 x 256 x 16, so a
+//     32 KB weight panel costs four instructions and the issuing thread never limits the stream;
+//   * activations carry ~16 mantissa bits as two bf16 rows per token (high and low part):
+//       - up to 64 tokens: the rows are interleaved (row 2t = high, row 2t+1 = low), one A tile
+//         holds both, and the epilogue adds neighbouring TMEM lanes with one shuffle;
+//       - 65..128 tokens: high and low parts are two A tiles and two MMAs per k-step accumulate
+//         into the same TMEM columns;
+//   * two independent shared-memory rings fed by TMA (cp.async.bulk.tensor.2d, 128-byte swizzle,
+//     no multicast): a deep one for W panels (256 rows x 64 k, evict-first) and a shallow one for
+//     X panels (128 rows x 64 k, served by L2, evict-last);
+//   * persistent stream-K: the (tile, panel) units are dealt out in equal contiguous ranges to one
+//     CTA per SM; a CTA that covers part of a tile writes a partial sum to its own slot and the
+//     consumer adds the slots in a fixed order;
+//   * programmatic dependent launch: W never changes, so its ring fills before the grid
+//     dependency resolves; only the X producer and the epilogue wait for the previous kernel;
+//   * warp roles: 0 = W producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue (tcgen05.ld ->
+//     128-bit stores), 6 = X producer; two TMEM accumulators alternate so that the epilogue of one
+//     segment overlaps the MMAs of the next;
 //   * every mbarrier wait is bounded: on expiry the kernel raises the status word and leaves.
 #pragma once
 #include <cuda.h>
@@ -25,20 +32,23 @@
 
 #include "common.cuh"
 
-#define TC_BM 128              // weight rows per tile
-#define TC_BK 64               // k elements per stage (128 bytes: one swizzle atom row)
-#define TC_THREADS 192
-#define TC_SPIN_LIMIT (1u << 26)
+#define TC_BN 256               // weight rows per tile (MMA N)
+#define TC_BK 64                // k elements per panel (128 bytes: one swizzle row)
+#define TC_THREADS 224
+#define TC_SPIN_LIMIT (1u << 24)
+#define TC_WPANEL (TC_BN * TC_BK * 2)
+#define TC_XTILE (128 * TC_BK * 2)
+
+enum { TC_X_PLAIN = 0, TC_X_INTERLEAVED = 1, TC_X_PLANAR = 2 };
 
 struct TcParams {
   float *out;
-  long long slot_stride;       // floats
-  int N, K, KB;                // output features, reduction length, k-blocks per tile
-  int n_tiles, total_units, upc;
-  int n_mma;                   // MMA N = token rows incl. lo plane (multiple of 16, <= 256)
-  int n_tok, n_tok_pad;        // real token rows, padded rows per plane
-  int lo_rows;                 // row offset of the lo plane in the X tensor map (0 = none)
-  int stages, tmem_cols;
+  long long slot_stride;        // floats between partial-sum slots
+  int N, K, KB, n_tiles, total_units, upc;
+  int n_tok;                    // real token rows of this launch
+  int x_mode;                   // TC_X_*
+  int lo_rows;                  // TC_X_PLANAR: row of the first low part in the X tensor map
+  int wp, w_stages, x_stages;   // panels per W stage, ring depths
   int *status;
 };
 
@@ -103,134 +113,194 @@ __device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64
 __device__ __forceinline__ void mma_commit(uint64_t *bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------ kernel
-// Dynamic shared memory: [stages][A tile 16 KB | B tile n_mma*128 B] (1024-byte aligned), then
-// the barriers.
+// Dynamic shared memory (1024-byte aligned): W ring [w_stages][wp][32 KB], X ring
+// [x_stages][16 KB, or 32 KB = high tile | low tile when planar], then the barriers.
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const uint32_t a_bytes = TC_BM * TC_BK * 2, b_bytes = (uint32_t)p.n_mma * TC_BK * 2;
-  const uint32_t stage_bytes = a_bytes + b_bytes;
-  uint64_t *bars = (uint64_t *)(smem + (size_t)p.stages * stage_bytes);
-  uint64_t *full = bars, *empty = bars + p.stages, *acc_full = bars + 2 * p.stages, *acc_empty = acc_full + 2;
+  const uint32_t wstage_bytes = (uint32_t)p.wp * TC_WPANEL;
+  const uint32_t xstage_bytes = p.x_mode == TC_X_PLANAR ? 2u * TC_XTILE : (uint32_t)TC_XTILE;
+  uint8_t *wring = smem, *xring = smem + (size_t)p.w_stages * wstage_bytes;
+  uint64_t *bars = (uint64_t *)(xring + (size_t)p.x_stages * xstage_bytes);
+  uint64_t *full_w = bars, *empty_w = full_w + p.w_stages, *full_x = empty_w + p.w_stages, *empty_x = full_x + p.x_stages;
+  uint64_t *acc_full = empty_x + p.x_stages, *acc_empty = acc_full + 2;
   uint32_t *tmem_base_p = (uint32_t *)(acc_empty + 2);
   volatile int *abort_flag = (volatile int *)(tmem_base_p + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long u_begin = (long long)blockIdx.x * p.upc;
-  long long u_end = u_begin + p.upc;
-  if (u_end > p.total_units) u_end = p.total_units;
+  const int u_begin = blockIdx.x * p.upc;
+  const int u_end = min(u_begin + p.upc, p.total_units);
   const bool has_work = u_begin < u_end;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    for (int s = 0; s < p.w_stages; ++s) { mbar_init(full_w + s, 1); mbar_init(empty_w + s, 1); }
+    for (int s = 0; s < p.x_stages; ++s) { mbar_init(full_x + s, 1); mbar_init(empty_x + s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {      // TMEM allocation by one full warp
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_p)), "r"((uint32_t)p.tmem_cols) : "memory");
+  if (warp == 1) {      // all 512 TMEM columns (two accumulators of 256), allocated by one full warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_p)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_trigger();
   const uint32_t tmem_base = *tmem_base_p;
 
   if (has_work) {
     if (warp == 0) {
-      // ------------------------------------------------------------------ TMA producer
+      // ------------------------------------------------------------------ W producer: weights are
+      // constant, so nothing here waits for the previous kernel
       if (lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
-        const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+        const uint64_t pol = policy_evict_first();
         uint32_t it = 0;
-        for (long long u = u_begin; u < u_end; ++u, ++it) {
-          int s = it % p.stages;
-          uint32_t ph = (it / p.stages) & 1;
-          if (it >= (uint32_t)p.stages && !mbar_wait(empty + s, ph ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break; }
+        int u = u_begin;
+        while (u < u_end) {
+          int tile = u / p.KB, kb = u - tile * p.KB;
+          int np = min(p.wp, min(p.KB - kb, u_end - u));
+          int s = it % p.w_stages;
+          if (it >= (uint32_t)p.w_stages && !mbar_wait(empty_w + s, ((it / p.w_stages) & 1) ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break; }
           if (*abort_flag) break;
-          int tile = (int)(u / p.KB), kb = (int)(u - (long long)tile * p.KB);
-          uint8_t *sa = smem + (size_t)s * stage_bytes, *sb = sa + a_bytes;
-          mbar_expect_tx(full + s, stage_bytes);
-          tma_load_2d(sa, &map_w, full + s, kb * TC_BK, tile * TC_BM, pol_w);
-          tma_load_2d(sb, &map_x, full + s, kb * TC_BK, 0, pol_x);
-          if (p.lo_rows) tma_load_2d(sb + (size_t)p.n_tok_pad * TC_BK * 2, &map_x, full + s, kb * TC_BK, p.lo_rows, pol_x);
+          uint8_t *dst = wring + (size_t)s * wstage_bytes;
+          mbar_expect_tx(full_w + s, (uint32_t)np * TC_WPANEL);
+          for (int q = 0; q < np; ++q) tma_load_2d(dst + (size_t)q * TC_WPANEL, &map_w, full_w + s, (kb + q) * TC_BK, tile * TC_BN, pol);
+          u += np; ++it;
+        }
+      }
+    } else if (warp == 6) {
+      // ------------------------------------------------------------------ X producer
+      if (lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        pdl_wait();
+        const uint64_t pol = policy_evict_last();
+        uint32_t it = 0;
+        for (int u = u_begin; u < u_end; ++u, ++it) {
+          int tile = u / p.KB, kb = u - tile * p.KB;
+          int s = it % p.x_stages;
+          if (it >= (uint32_t)p.x_stages && !mbar_wait(empty_x + s, ((it / p.x_stages) & 1) ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break; }
+          if (*abort_flag) break;
+          uint8_t *dst = xring + (size_t)s * xstage_bytes;
+          mbar_expect_tx(full_x + s, xstage_bytes);
+          tma_load_2d(dst, &map_x, full_x + s, kb * TC_BK, 0, pol);
+          if (p.x_mode == TC_X_PLANAR) tma_load_2d(dst + TC_XTILE, &map_x, full_x + s, kb * TC_BK, p.lo_rows, pol);
         }
       }
     } else if (warp == 1) {
       // ------------------------------------------------------------------ MMA issuer
       if (lane == 0) {
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_mma >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
-        uint32_t it = 0, seg = 0;
-        long long u = u_begin;
+        // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const bool planar = p.x_mode == TC_X_PLANAR;
+        uint32_t wit = 0, xit = 0, seg = 0;
+        int u = u_begin;
         bool ok = true;
         while (u < u_end && ok) {
-          int tile = (int)(u / p.KB);
-          long long seg_end = (long long)(tile + 1) * p.KB;
-          if (seg_end > u_end) seg_end = u_end;
+          int tile = u / p.KB;
+          int seg_end = min((tile + 1) * p.KB, u_end);
           int buf = seg & 1;
           if (seg >= 2 && !mbar_wait(acc_empty + buf, ((seg >> 1) & 1) ^ 1)) { ok = false; break; }
           tc_fence_after();
-          uint32_t d_addr = tmem_base + (uint32_t)buf * (uint32_t)p.n_mma;
+          uint32_t d_addr = tmem_base + (uint32_t)buf * TC_BN;
           bool first = true;
-          for (; u < seg_end; ++u, ++it) {
-            int s = it % p.stages;
-            if (!mbar_wait(full + s, (it / p.stages) & 1)) { ok = false; break; }
-            tc_fence_after();
-            uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes), sb = sa + a_bytes;
-            uint64_t ad = smem_desc(sa), bd = smem_desc(sb);
+          while (u < seg_end) {
+            int kb = u - tile * p.KB;
+            int np = min(p.wp, min(p.KB - kb, u_end - u));
+            int s = wit % p.w_stages;
+            if (!mbar_wait(full_w + s, (wit / p.w_stages) & 1)) { ok = false; break; }
+            uint32_t sw0 = smem_u32(wring + (size_t)s * wstage_bytes);
+            for (int q = 0; q < np; ++q, ++xit) {
+              int t = xit % p.x_stages;
+              uint32_t sx = smem_u32(xring + (size_t)t * xstage_bytes);
+              if (!mbar_wait(full_x + t, (xit / p.x_stages) & 1)) { ok = false; break; }
+              tc_fence_after();
+              uint64_t ad = smem_desc(sx), al = smem_desc(sx + TC_XTILE), bd = smem_desc(sw0 + (uint32_t)q * TC_WPANEL);
 #pragma unroll
-            for (int k = 0; k < TC_BK / 16; ++k) {
-              mma_bf16(d_addr, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, (first && k == 0) ? 0u : 1u);
+              for (int k = 0; k < TC_BK / 16; ++k) {
+                mma_bf16(d_addr, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, (first && k == 0) ? 0u : 1u);
+                if (planar) mma_bf16(d_addr, al + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, 1u);
+              }
+              first = false;
+              mma_commit(empty_x + t);          // frees the X stage once these MMAs have read it
             }
-            first = false;
-            mma_commit(empty + s);            // frees the stage once these MMAs have read it
+            if (!ok) break;
+            mma_commit(empty_w + s);            // frees the W stage
+            u += np; ++wit;
           }
           if (!ok) break;
-          mma_commit(acc_full + buf);         // accumulator complete
+          mma_commit(acc_full + buf);           // accumulator complete
           ++seg;
         }
         if (!ok) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
       }
     } else {
-      // ------------------------------------------------------------------ epilogue warps
-      const int q = warp & 3;                 // TMEM lane quarter this warp may read
+      // ------------------------------------------------------------------ epilogue warps 2..5
+      const int q = warp & 3;                   // TMEM lane quarter this warp may read
+      pdl_wait();                               // the output buffer is read by the previous kernel
+      const bool inter = p.x_mode == TC_X_INTERLEAVED;
+      const int row = q * 32 + lane;            // accumulator lane = X row
+      const int token = inter ? row >> 1 : row;
+      const int part = inter ? lane & 1 : 0;
       uint32_t seg = 0;
-      long long u = u_begin;
+      int u = u_begin;
       while (u < u_end) {
-        int tile = (int)(u / p.KB);
-        long long seg_end = (long long)(tile + 1) * p.KB;
-        if (seg_end > u_end) seg_end = u_end;
+        int tile = u / p.KB;
+        int seg_end = min((tile + 1) * p.KB, u_end);
         int buf = seg & 1;
-        bool ok = mbar_wait(acc_full + buf, (seg >> 1) & 1);
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(acc_full + buf, (seg >> 1) & 1) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok || *abort_flag) { if (lane == 0) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; } break; }
         tc_fence_after();
-        int first_cta = (int)(((long long)tile * p.KB) / p.upc);
+        int first_cta = (tile * p.KB) / p.upc;
         int slot = (int)blockIdx.x - first_cta;
-        int c = tile * TC_BM + q * 32 + lane;
-        float *dst = p.out + (long long)slot * p.slot_stride + c;
-        uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * (uint32_t)p.n_mma;
-        for (int col0 = 0; col0 < p.n_mma; col0 += 16) {
-          uint32_t r[16];
-          tmem_ld16(taddr + (uint32_t)col0, r);
+        float *dst = p.out + (long long)slot * p.slot_stride + (long long)token * p.N + tile * TC_BN;
+        uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * TC_BN;
+        for (int col0 = 0; col0 < TC_BN; col0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + (uint32_t)col0, r);
           tmem_ld_wait();
-          if (c < p.N) {
+          if (inter) {
+            // lanes 2t and 2t+1 hold the products of token t's high and low parts: add them;
+            // both lanes then hold the sum and each stores half of the 32 columns
+            float v[32];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              int col = col0 + j;
-              int t = col < p.n_tok_pad ? col : col - p.n_tok_pad;
-              if (t < p.n_tok) dst[(long long)col * p.N] = __uint_as_float(r[j]);
+            for (int j = 0; j < 32; ++j) {
+              float a = __uint_as_float(r[j]);
+              v[j] = a + __shfl_xor_sync(0xffffffffu, a, 1);
+            }
+            if (token < p.n_tok) {
+#pragma unroll
+              for (int j4 = 0; j4 < 4; ++j4) {
+                int jj = part * 16 + j4 * 4;
+                float4 o = part ? make_float4(v[16 + j4 * 4], v[17 + j4 * 4], v[18 + j4 * 4], v[19 + j4 * 4])
+                                : make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
+                if (tile * TC_BN + col0 + jj < p.N) *reinterpret_cast<float4 *>(dst + col0 + jj) = o;
+              }
+            }
+          } else if (token < p.n_tok) {
+#pragma unroll
+            for (int j4 = 0; j4 < 8; ++j4) {
+              if (tile * TC_BN + col0 + j4 * 4 < p.N)
+                *reinterpret_cast<float4 *>(dst + col0 + j4 * 4) =
+                    make_float4(__uint_as_float(r[j4 * 4]), __uint_as_float(r[j4 * 4 + 1]), __uint_as_float(r[j4 * 4 + 2]),
+                                __uint_as_float(r[j4 * 4 + 3]));
             }
           }
         }
@@ -246,7 +316,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -256,11 +326,12 @@ struct GemmTcPlan {
   PFN_cuTensorMapEncodeTiled_v12000 encode;
   int n_sms;
   int max_smem;
+  int use_pdl;
   int *status;
   std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;
 };
 
-static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status) {
+static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status, int use_pdl) {
   void *fn = nullptr;
   cudaDriverEntryPointQueryResult qr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn)
@@ -273,14 +344,20 @@ static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status) {
   if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->max_smem) != cudaSuccess)
     return "cannot raise the dynamic shared memory limit";
   pl->status = status;
+  pl->use_pdl = use_pdl;
   return nullptr;
 }
 
-static inline bool gemm_tc_supported(int rows_total, int N, int K) {
-  return rows_total >= 16 && rows_total <= 256 && rows_total % 16 == 0 && K % TC_BK == 0 && K >= TC_BK && N % 8 == 0 && N >= 8;
+// Largest token count one launch takes: 64 with interleaved high/low rows, 128 otherwise.
+#define TC_ROWS_SPLIT_1MMA 64
+#define TC_ROWS_MAX 128
+
+static inline bool gemm_tc_supported(int N, int K) {
+  return K % TC_BK == 0 && K >= TC_BK && N % 8 == 0 && N >= 8;
 }
 
-// bf16 row-major [rows][K] matrix, box = 64 x box_rows, 128-byte swizzle.
+// bf16 row-major [rows][K] matrix, box = 64 x box_rows, 128-byte swizzle.  Rows of a box that lie
+// beyond `rows` read as zero.
 static inline const CUtensorMap *tc_map(GemmTcPlan *pl, const void *ptr, int rows, int K, int box_rows) {
   auto key = std::make_tuple(ptr, rows, K, box_rows);
   auto it = pl->maps.find(key);
@@ -294,45 +371,68 @@ static inline const CUtensorMap *tc_map(GemmTcPlan *pl, const void *ptr, int row
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return nullptr;
-  if (pl->maps.size() > 4096) pl->maps.clear();
+  if (pl->maps.size() > 8192) pl->maps.clear();
   return &(pl->maps[key] = m);
 }
 
-// Enqueue one GEMM.  X holds `rows` token rows (hi plane) and, when lo_delta != 0, their
-// low-order parts lo_delta elements further on.  Returns false if a tensor map could not be made.
-static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const void *W, const void *X, long long lo_delta,
-                                  int rows, int N, int K, float *out, long long out_floats, GemmOut *g) {
+// Floats one launch may write when its slots hold slot_rows x N: a tile is shared by at most
+// ceil(KB / upc) + 1 CTAs.  n_sms <= 0 gives the bound that holds for any SM count.
+static inline long long gemm_tc_out_floats(int n_sms, int slot_rows, int N, int K) {
+  int KB = K / TC_BK, n_tiles = (N + TC_BN - 1) / TC_BN;
+  long long total = (long long)n_tiles * KB;
+  long long slots;
+  if (n_sms <= 0) slots = KB + 1;
+  else {
+    long long grid = n_sms < total ? n_sms : total;
+    long long upc = (total + grid - 1) / grid;
+    slots = (KB + upc - 1) / upc + 1;
+  }
+  return slots * (long long)slot_rows * N;
+}
+
+// Enqueue one GEMM of `rows` tokens (<= 64 when x_mode is interleaved, <= 128 otherwise).
+//   X: bf16, row-major, K columns.  TC_X_PLAIN: row t = token t.  TC_X_INTERLEAVED: row 2t = high
+//   part of token t, row 2t+1 = low part.  TC_X_PLANAR: row t = high part, row lo_rows + t = low part.
+// Returns false if the launch could not be made (no tensor map, output too small).
+static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const void *W, const void *X, int x_mode, int lo_rows,
+                                  int rows, int slot_rows, int N, int K, float *out, long long out_floats, GemmOut *g) {
   TcParams p;
   p.n_tok = rows;
-  p.n_tok_pad = (rows + 15) & ~15;
-  p.n_mma = p.n_tok_pad * (lo_delta ? 2 : 1);
-  p.lo_rows = lo_delta ? (int)(lo_delta / K) : 0;
+  p.x_mode = x_mode;
+  p.lo_rows = lo_rows;
   p.N = N; p.K = K; p.KB = K / TC_BK;
-  p.n_tiles = (N + TC_BM - 1) / TC_BM;
+  p.n_tiles = (N + TC_BN - 1) / TC_BN;
   p.total_units = p.n_tiles * p.KB;
   int grid = pl->n_sms < p.total_units ? pl->n_sms : p.total_units;
   p.upc = (p.total_units + grid - 1) / grid;
+  // W stages of two panels (256-byte runs per weight row) unless the X ring needs the room
+  p.wp = x_mode == TC_X_PLANAR ? 1 : 2;
+  if (p.wp > p.KB) p.wp = p.KB;
+  if (p.KB % p.wp == 0) p.upc = (p.upc + p.wp - 1) / p.wp * p.wp;   // CTA ranges cover whole W stages
   grid = (p.total_units + p.upc - 1) / p.upc;
-  int stage_bytes = TC_BM * TC_BK * 2 + p.n_mma * TC_BK * 2;
-  int budget = pl->max_smem - 2048;
-  p.stages = budget / stage_bytes;
-  if (p.stages > 12) p.stages = 12;
-  if (p.stages < 2) return false;
-  int cols = 2 * p.n_mma;
-  p.tmem_cols = 32;
-  while (p.tmem_cols < cols) p.tmem_cols <<= 1;
+  p.x_stages = 2;
+  int xstage = x_mode == TC_X_PLANAR ? 2 * TC_XTILE : TC_XTILE;
+  int budget = pl->max_smem - 2048 - p.x_stages * xstage;
+  p.w_stages = budget / (p.wp * TC_WPANEL);
+  if (p.w_stages > 8) p.w_stages = 8;
+  if (p.w_stages < 2) return false;
   p.out = out;
-  p.slot_stride = (long long)p.n_mma * N;
+  p.slot_stride = (long long)slot_rows * N;       // slot_rows >= rows: the same for every chunk of one GEMM
   long long max_slots = (p.KB + p.upc - 1) / p.upc + 1;
   if (p.slot_stride * max_slots > out_floats) return false;
   p.status = pl->status;
-  int x_rows = p.lo_rows + p.n_tok_pad;
-  const CUtensorMap *mw = tc_map(pl, W, N, K, TC_BM);
-  const CUtensorMap *mx = tc_map(pl, X, x_rows, K, p.n_tok_pad);
+  int x_rows = x_mode == TC_X_INTERLEAVED ? 2 * rows : (x_mode == TC_X_PLANAR ? lo_rows + rows : rows);
+  const CUtensorMap *mw = tc_map(pl, W, N, K, TC_BN);
+  const CUtensorMap *mx = tc_map(pl, X, x_rows, K, 128);
   if (!mw || !mx) return false;
-  size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
-  k_gemm_tc<<<grid, TC_THREADS, smem, stream>>>(*mw, *mx, p);
-  g->base = out; g->slot_stride = p.slot_stride; g->ld = N; g->kb = p.KB; g->upc = p.upc;
-  g->lo_off = lo_delta ? p.n_tok_pad : 0;
+  size_t smem = (size_t)p.w_stages * p.wp * TC_WPANEL + (size_t)p.x_stages * xstage + 1024 + 512;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = pl->use_pdl ? 1 : 0;
+  if (cudaLaunchKernelEx(&cfg, k_gemm_tc, *mw, *mx, p) != cudaSuccess) return false;
+  g->base = out; g->slot_stride = p.slot_stride; g->chunk_stride = 0; g->chunk_shift = 30; g->ld = N; g->kb = p.KB; g->upc = p.upc;
   return true;
 }

@@ -10,6 +10,8 @@
 template <typename T>
 __global__ void k_embed(const T *__restrict__ embed, const int *__restrict__ tok, float *x, int d,
                         int vocab, int *status) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x, t = tok[r];
   if (t >= vocab) { if (threadIdx.x == 0) atomicMax(status, DREAM_DEV_BAD_INDEX); t = -1; }
   for (int i = threadIdx.x; i < d; i += blockDim.x)
@@ -22,6 +24,8 @@ template <typename T>
 __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict__ visual,
                                const int *__restrict__ ids, int vis_start, int v, float *x,
                                float *x0, int d, int vocab, int *status) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x;
   const T *src;
   if (r >= vis_start && r < vis_start + v) src = visual + (long long)(r - vis_start) * d;
@@ -45,8 +49,10 @@ __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict_
 template <typename T>
 __global__ void k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
                              float eps, int d, T *xn, float *copy, const int *row_seq,
-                             const int *tap_state, int layer, T *raw, long long lo_delta) {
+                             const int *tap_state, int layer, T *raw, XLayout lay) {
   __shared__ float sh[33];
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x;
   float *xr = x + (long long)r * d;
   float ss = 0.f;
@@ -61,16 +67,20 @@ __global__ void k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restr
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     float v = xr[i];
     if (do_copy) copy[(long long)r * d + i] = v;
-    if (raw) store_split<T>(raw + (long long)r * d + i, lo_delta, v);
-    if (xn) store_split<T>(xn + (long long)r * d + i, lo_delta, v * inv * to_f(gain[i]));
+    if (raw) store_split<T>(raw + r * lay.row_stride + i, lay.lo_delta, v);
+    if (xn) store_split<T>(xn + r * lay.row_stride + i, lay.lo_delta, v * inv * to_f(gain[i]));
   }
 }
 
 // ---------------------------------------------------------------------------------------
-// Rotary angle of (position, pair index): the product is taken in double and reduced to
-// [-pi, pi] before the single-precision sincos, so long prefixes lose no phase accuracy.
-__device__ __forceinline__ void rope_cs(int pos, int i, int hd, float theta, float *c, float *s) {
-  double inv = exp2(-2.0 * (double)i / (double)hd * log2((double)theta));
+// Rotary angle of (position, pair index) = position * theta^(-2i/hd).  The inverse frequencies
+// are tabulated once in double; the product is taken in double and reduced to [-pi, pi] before
+// the single-precision sincos, so long prefixes lose no phase accuracy.
+__global__ void k_rope_table(double *inv_freq, int hd, float theta) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < hd / 2) inv_freq[i] = exp2(-2.0 * (double)i / (double)hd * log2((double)theta));
+}
+__device__ __forceinline__ void rope_cs(int pos, double inv, float *c, float *s) {
   double a = (double)pos * inv;
   const double two_pi = 6.283185307179586476925286766559;
   a -= two_pi * rint(a / two_pi);
@@ -90,31 +100,36 @@ struct PagedKV {
 };
 
 // After the QKV GEMM of target rows: rotary on q and k at row_pos, q -> qbuf (fp32),
-// k, v -> the paged cache at (row_seq, row_slot).
+// k, v -> the paged cache at (row_seq, row_slot).  One block per row; a work item is one
+// rotary pair (head, i) so that consecutive threads read consecutive GEMM columns.
 template <typename T>
 __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
                                   const int *__restrict__ row_pos, const int *__restrict__ row_slot,
-                                  int row0, float *qbuf, PagedKV kv, int H, float theta) {
+                                  int row0, float *qbuf, PagedKV kv, int H, const double *__restrict__ inv_freq) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int hd = kv.hd, half = hd >> 1, Hkv = kv.hkv;
   int seq = row_seq[r], pos = row_pos[r], slot = row_slot[r];
   T *Kp = (T *)kv.base, *Vp = (T *)kv.base + kv.kv_stride;
-  for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    float c, s;
-    rope_cs(pos, i, hd, theta, &c, &s);
-    for (int h = 0; h < H; ++h) {
-      float a = gemm_val(g, lr, h * hd + i), b = gemm_val(g, lr, h * hd + i + half);
-      float *q = qbuf + ((long long)r * H + h) * hd;
-      q[i] = a * c - b * s;
-      q[i + half] = b * c + a * s;
-    }
-    for (int h = 0; h < Hkv; ++h) {
-      float a = gemm_val(g, lr, (H + h) * hd + i), b = gemm_val(g, lr, (H + h) * hd + i + half);
-      long long o = kv.off(seq, slot, h);
-      Kp[o + i] = from_f<T>(a * c - b * s);
-      Kp[o + i + half] = from_f<T>(b * c + a * s);
-      Vp[o + i] = from_f<T>(gemm_val(g, lr, (H + Hkv + h) * hd + i));
-      Vp[o + i + half] = from_f<T>(gemm_val(g, lr, (H + Hkv + h) * hd + i + half));
+  int items = (H + 2 * Hkv) * half;
+  for (int w = threadIdx.x; w < items; w += blockDim.x) {
+    int hh = w / half, i = w - hh * half;
+    float a = gemm_val(g, lr, hh * hd + i), b = gemm_val(g, lr, hh * hd + i + half);
+    if (hh < H + Hkv) {
+      float c, s;
+      rope_cs(pos, inv_freq[i], &c, &s);
+      float ra = a * c - b * s, rb = b * c + a * s;
+      if (hh < H) {
+        float *q = qbuf + ((long long)r * H + hh) * hd;
+        q[i] = ra; q[i + half] = rb;
+      } else {
+        long long o = kv.off(seq, slot, hh - H);
+        Kp[o + i] = from_f<T>(ra); Kp[o + i + half] = from_f<T>(rb);
+      }
+    } else {
+      long long o = kv.off(seq, slot, hh - H - Hkv);
+      Vp[o + i] = from_f<T>(a); Vp[o + i + half] = from_f<T>(b);
     }
   }
 }
@@ -128,42 +143,47 @@ struct FlatKV {
   }
 };
 
-// After a draft QKV GEMM (col0 = first column of the K block inside the GEMM output, or
-// H*hd when the GEMM produced q too): rotary, q -> qbuf (when has_q), k/v -> draft
-// self-attention cache row row_dst[r] (skipped when < 0).
+// After a draft QKV GEMM (has_q: the GEMM produced q columns first, then K, then V; otherwise
+// K then V only): rotary, q -> qbuf (when has_q), k/v -> draft self-attention cache row
+// row_dst[r] (skipped when < 0).  Work items as in k_qkv_post_target.
 __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
                                  const int *__restrict__ row_pos, const int *__restrict__ row_dst,
-                                 int row0, int has_q, float *qbuf, FlatKV kv, int H, float theta) {
+                                 int row0, int has_q, float *qbuf, FlatKV kv, int H, const double *__restrict__ inv_freq) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int dst = row_dst[r];
   int hd = kv.hd, half = hd >> 1, Hkv = kv.hkv;
   int seq = row_seq[r], pos = row_pos[r];
-  int kcol = has_q ? H * hd : 0;
+  int Hq = has_q ? H : 0;
   float *base = kv.base;
-  for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    float c, s;
-    rope_cs(pos, i, hd, theta, &c, &s);
-    if (has_q)
-      for (int h = 0; h < H; ++h) {
-        float a = gemm_val(g, lr, h * hd + i), b = gemm_val(g, lr, h * hd + i + half);
-        float *q = qbuf + ((long long)r * H + h) * hd;
-        q[i] = a * c - b * s;
-        q[i + half] = b * c + a * s;
+  int items = (Hq + 2 * Hkv) * half;
+  for (int w = threadIdx.x; w < items; w += blockDim.x) {
+    int hh = w / half, i = w - hh * half;
+    if (hh >= Hq && dst < 0) continue;
+    float a = gemm_val(g, lr, hh * hd + i), b = gemm_val(g, lr, hh * hd + i + half);
+    if (hh < Hq + Hkv) {
+      float c, s;
+      rope_cs(pos, inv_freq[i], &c, &s);
+      float ra = a * c - b * s, rb = b * c + a * s;
+      if (hh < Hq) {
+        float *q = qbuf + ((long long)r * H + hh) * hd;
+        q[i] = ra; q[i + half] = rb;
+      } else {
+        long long o = kv.off(seq, 0, hh - Hq, dst);
+        base[o + i] = ra; base[o + i + half] = rb;
       }
-    if (dst >= 0)
-      for (int h = 0; h < Hkv; ++h) {
-        float a = gemm_val(g, lr, kcol + h * hd + i), b = gemm_val(g, lr, kcol + h * hd + i + half);
-        long long ok = kv.off(seq, 0, h, dst), ov = kv.off(seq, 1, h, dst);
-        base[ok + i] = a * c - b * s;
-        base[ok + i + half] = b * c + a * s;
-        base[ov + i] = gemm_val(g, lr, kcol + (Hkv + h) * hd + i);
-        base[ov + i + half] = gemm_val(g, lr, kcol + (Hkv + h) * hd + i + half);
-      }
+    } else {
+      long long o = kv.off(seq, 1, hh - Hq - Hkv, dst);
+      base[o + i] = a; base[o + i + half] = b;
+    }
   }
 }
 
 // Plain copy of a GEMM output [rows][width] into fp32 rows (q of the cross-attention: no rotary)
 __global__ void k_gemm_to_f32(GemmOut g, float *dst, int width) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x;
   for (int i = threadIdx.x; i < width; i += blockDim.x) dst[(long long)r * width + i] = gemm_val(g, r, i);
 }
@@ -174,6 +194,8 @@ __global__ void k_gemm_to_f32(GemmOut g, float *dst, int width) {
 __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
                              const int *__restrict__ row_dst, const int *__restrict__ row_in,
                              const int *__restrict__ nperm, int row0, FlatKV kv) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int seq = row_seq[r];
   int dst = nperm ? (row_in[r] < 0 ? -1 : nperm[seq] + row_in[r]) : row_dst[r];
@@ -189,16 +211,20 @@ __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
 
 // act = silu(gate) * up, from a GEMM output whose columns are [gate(ff) | up(ff)].
 template <typename T>
-__global__ void k_silu_mul(GemmOut g, T *act, int ff, long long lo_delta) {
+__global__ void k_silu_mul(GemmOut g, T *act, int ff, XLayout lay) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.y;
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= ff) return;
   float a = gemm_val(g, r, i), b = gemm_val(g, r, ff + i);
-  store_split<T>(act + (long long)r * ff + i, lo_delta, a / (1.f + __expf(-a)) * b);
+  store_split<T>(act + r * lay.row_stride + i, lay.lo_delta, a / (1.f + __expf(-a)) * b);
 }
 
 // x += GEMM output; optional fp32 copy into a per-layer store (prefill tap candidates).
 __global__ void k_resid_add(float *x, GemmOut g, int d, float *copy) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     float v = x[(long long)r * d + i] + gemm_val(g, r, i);
@@ -211,11 +237,13 @@ __global__ void k_resid_add(float *x, GemmOut g, int d, float *copy) {
 template <typename T>
 __global__ void k_gather_rows(const float *__restrict__ src, const int *__restrict__ idx, T *dst,
                               int d, const int *layer_ptr, int layer_lo, long long layer_stride,
-                              long long lo_delta) {
+                              XLayout lay) {
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x, s = idx[r];
   if (layer_ptr) src += (long long)(*layer_ptr - layer_lo) * layer_stride;
   for (int i = threadIdx.x; i < d; i += blockDim.x)
-    store_split<T>(dst + (long long)r * d + i, lo_delta, s >= 0 ? src[(long long)s * d + i] : 0.f);
+    store_split<T>(dst + r * lay.row_stride + i, lay.lo_delta, s >= 0 ? src[(long long)s * d + i] : 0.f);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -230,6 +258,8 @@ k_topk_lse(GemmOut g, int V, int ktop, float *top_val, int *top_id, float *lse, 
   __shared__ float red[33];
   __shared__ float cand_v[TOPK_THREADS / 32];
   __shared__ int cand_i[TOPK_THREADS / 32], cand_t[TOPK_THREADS / 32];
+  pdl_trigger();
+  pdl_wait();
   int r = blockIdx.x, tid = threadIdx.x;
   float lv[TOPK_MAX];
   int li[TOPK_MAX];
