@@ -67,6 +67,46 @@ __device__ __forceinline__ float gemm_val(const GemmOut &g, int r, int c) {
   return s;
 }
 
+// Four consecutive columns c..c+3 (c a multiple of 4: they share a tile, hence a slot count).
+__device__ __forceinline__ float4 gemm_val4(const GemmOut &g, int r, int c) {
+  int ch = r >> g.chunk_shift;
+  const float4 *p = reinterpret_cast<const float4 *>(g.base + (long long)ch * g.chunk_stride +
+                                                     (long long)(r - (ch << g.chunk_shift)) * g.ld + c);
+  float4 s = *p;
+  if (g.upc) {
+    unsigned u0 = (unsigned)(c >> 8) * (unsigned)g.kb;
+    int extra = (int)((u0 + (unsigned)g.kb - 1u) / (unsigned)g.upc) - (int)(u0 / (unsigned)g.upc);
+    long long st4 = g.slot_stride >> 2;
+    for (int i = 1; i <= extra; ++i) {
+      float4 t = p[(long long)i * st4];
+      s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+    }
+  }
+  return s;
+}
+
+// Four consecutive elements of a GEMM input row, high (and low) parts, as 8-byte stores.
+template <typename T> __device__ __forceinline__ void store_split4(T *p, long long lo_delta, float4 v);
+template <> __device__ __forceinline__ void store_split4<float>(float *p, long long, float4 v) {
+  *reinterpret_cast<float4 *>(p) = v;
+}
+template <> __device__ __forceinline__ void store_split4<bf16>(bf16 *p, long long lo_delta, float4 v) {
+  __nv_bfloat162 h0 = __floats2bfloat162_rn(v.x, v.y), h1 = __floats2bfloat162_rn(v.z, v.w);
+  uint2 hv = make_uint2(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1));
+  *reinterpret_cast<uint2 *>(p) = hv;
+  if (lo_delta) {
+    float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+    __nv_bfloat162 l0 = __floats2bfloat162_rn(v.x - f0.x, v.y - f0.y), l1 = __floats2bfloat162_rn(v.z - f1.x, v.w - f1.y);
+    *reinterpret_cast<uint2 *>(p + lo_delta) = make_uint2(*reinterpret_cast<uint32_t *>(&l0), *reinterpret_cast<uint32_t *>(&l1));
+  }
+}
+__device__ __forceinline__ float4 ld_f4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 ld_f4(const bf16 *p) {
+  uint2 u = *reinterpret_cast<const uint2 *>(p);
+  float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162 *>(&u.x)), b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162 *>(&u.y));
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

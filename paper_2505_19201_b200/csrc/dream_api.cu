@@ -51,6 +51,8 @@ struct dream_ctx {
   float *x, *x0, *qbuf, *gout, *lse_pre, *ent_pre, *ae, *scores_all, *taps_store, *tapbuf;
   void *xn, *raw, *act, *attn_out;
   float *top_val, *lse_rows, *margin_i;
+  TopkScratch tks;
+  int tk_nsplit;
   int *top_id, *argmax_i, *accept_len_i, *out_tokens_i, *comp_src_i;
   size_t gout_floats;
   // host side
@@ -139,6 +141,7 @@ static dream_status check_config(const dream_config *c, TreeShape *ts) {
       c->n_heads % c->n_kv_heads || c->d_ff < 8 || c->vocab < 2)
     return fail(nullptr, DREAM_E_ARG, "model shape");
   if (c->d_model % 8 || c->d_ff % 8) return fail(nullptr, DREAM_E_UNSUPPORTED, "d_model, d_ff must be multiples of 8");
+  if (c->vocab > TOPK_THREADS * TOPK_COLS) return fail(nullptr, DREAM_E_UNSUPPORTED, "vocab above 1048576");
   if (c->dtype == DREAM_BF16 && (c->d_model % 64 || c->d_ff % 64 || (c->n_heads * c->head_dim) % 64 || c->vocab % 8))
     return fail(nullptr, DREAM_E_UNSUPPORTED, "bf16: d_model, d_ff, n_heads*head_dim must be multiples of 64 and vocab of 8");
   if (c->max_batch < 1 || c->max_batch > DREAM_MAX_BATCH) return fail(nullptr, DREAM_E_ARG, "max_batch in 1..8");
@@ -267,6 +270,12 @@ static size_t carve(dream_ctx *c, char *base) {
   c->top_val = a.take<float>((size_t)ROW_CHUNK * TOPK_MAX);
   c->top_id = a.take<int>((size_t)ROW_CHUNK * TOPK_MAX);
   c->lse_rows = a.take<float>(ROW_CHUNK);
+  c->tk_nsplit = (f.vocab + TOPK_COLS - 1) / TOPK_COLS;
+  c->tks.pv = a.take<float>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
+  c->tks.pi = a.take<int>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
+  c->tks.pm = a.take<float>((size_t)ROW_CHUNK * c->tk_nsplit);
+  c->tks.pz = a.take<float>((size_t)ROW_CHUNK * c->tk_nsplit);
+  c->tks.counter = a.take<int>(ROW_CHUNK);
   c->argmax_i = a.take<int>(ROW_CHUNK);
   c->margin_i = a.take<float>(ROW_CHUNK);
   c->accept_len_i = a.take<int>(MB);
@@ -523,14 +532,14 @@ template <typename T>
 static void norm_rows(dream_ctx *c, float *x, const GemmOut &gin, bool has_in, const void *gain, int rows, XMode m,
                       float *copy = nullptr, const int *row_seq = nullptr, const int *tap = nullptr, int layer = 0,
                       bool want_raw = false) {
-  LAUNCH(c, (k_resid_norm<T>), rows, 256, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+  LAUNCH(c, (k_resid_norm<T>), rows, NORM_THREADS, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
          (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
 }
 template <typename T>
 static GemmOut mlp_rows(dream_ctx *c, const void *wgu, const void *wd, int rows, XMode m) {
   const dream_config &f = c->cfg;
   GemmOut g = gemm<T>(c, wgu, c->xn, m, rows, 2 * f.d_ff, f.d_model);
-  LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 255) / 256, rows), 256, 0, g, (T *)c->act, f.d_ff, xlay(m, f.d_ff));
+  LAUNCH(c, (k_silu_mul<T>), dim3((f.d_ff + 1023) / 1024, rows), 256, 0, g, (T *)c->act, f.d_ff, xlay(m, f.d_ff));
   return gemm<T>(c, wd, c->act, m, rows, f.d_model, f.d_ff);
 }
 
@@ -552,7 +561,7 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
       int rows = imin(CH, n - r0);
       norm_rows<T>(c, c->x + (size_t)r0 * d, NO_GEMM, false, c->ln1[l], rows, m1);
       GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, m1, rows, c->qkvN, d);
-      LAUNCH(c, (k_qkv_post_target<T>), rows, 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
+      LAUNCH(c, (k_qkv_post_target<T>), dim3(rows, (c->qkvN / 8 + 255) / 256), 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
              paged(c, l), f.n_heads, c->rope_inv);
     }
     HD_DISPATCH(c, T, prefill(c, l, seq, n));
@@ -567,13 +576,13 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
       norm_rows<T>(c, xr, g, true, c->ln2[l], rows, m1);
       g = mlp_rows<T>(c, c->wgu[l], c->wd[l], rows, m1);
       float *copy = is_cand ? c->taps_store + ((size_t)cand * f.max_prompt + r0) * d : nullptr;
-      LAUNCH(c, k_resid_add, rows, 256, 0, xr, g, d, copy);
+      LAUNCH(c, k_resid_add, dim3(rows, (d + 1023) / 1024), 256, 0, xr, g, d, copy);
     }
   }
   // first token: LM head on the last prompt row
   norm_rows<T>(c, c->x + (size_t)(n - 1) * d, NO_GEMM, false, c->ln_f, 1, m1);
   GemmOut g = gemm<T>(c, c->lm_head, c->xn, m1, 1, f.vocab, d);
-  LAUNCH(c, k_topk_lse, 1, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
+  LAUNCH(c, k_topk_lse, dim3(1, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, 2, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
   LAUNCH(c, k_first_token, 1, 32, 0, c->top_id, c->top_val, first_token, first_margin);
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, n, c->top_id, -1, -1);
   LAUNCH(c, k_select_tap, 1, 32, 0, c->ae, f.tap_mode, f.tap_layer, f.tap_lo, f.tap_hi, c->sd.tap + seq, tap_layer);
@@ -639,7 +648,7 @@ static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *force
     LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL, XLayout{d, 0});
     norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, rows, m1);
     GemmOut g = gemm<T>(c, wkv, c->xn, m1, rows, c->kvN, d);
-    LAUNCH(c, k_qkv_post_draft, rows, 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
+    LAUNCH(c, k_qkv_post_draft, dim3(rows, (c->kvN / 8 + 255) / 256), 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
            flat(c, c->dself), f.n_heads, c->rope_inv);
   }
   // cross-attention memory: tapped features at the context positions, projected (Eq. 1)
@@ -650,7 +659,7 @@ static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *force
     LAUNCH(c, (k_gather_rows<T>), rows, 256, 0, c->taps_store, c->gather_idx, (T *)c->raw, d, c->sd.tap + seq, c->tap_lo_eff,
            (long long)f.max_prompt * d, xlay(m1, d));
     GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, m1, rows, c->kvN, d);
-    LAUNCH(c, k_mem_append, rows, 256, 0, g, c->rm[0].seq, c->rm[0].dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
+    LAUNCH(c, k_mem_append, dim3(rows, (c->kvN + 1023) / 1024), 256, 0, g, c->rm[0].seq, c->rm[0].dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
   }
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, -1, (const int *)nullptr, nc, nm);
   return DREAM_OK;
@@ -712,12 +721,12 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
     norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
     GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
-    LAUNCH(c, k_qkv_post_draft, R, 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
+    LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
     HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm));
     g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
     g = gemm<T>(c, c->dw.xq, c->xn, xm, R, c->Hhd, d);
-    LAUNCH(c, k_gemm_to_f32, R, 256, 0, g, c->qbuf, c->Hhd);
+    LAUNCH(c, k_gemm_to_f32, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, c->Hhd);
     HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm));
     g = gemm<T>(c, c->dw.xo, c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, xm);
@@ -725,9 +734,9 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
     norm_rows<T>(c, c->x, g, true, c->ln_f, R, xm, nullptr, nullptr, nullptr, 0, true);
     g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
-    LAUNCH(c, k_mem_append, R, 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
+    LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
     g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
-    LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, ts.K, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
+    LAUNCH(c, k_topk_lse, dim3(R, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, ts.K, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
     int next_m = p < ts.D ? ts.beam[p] : 1;
     LAUNCH(c, k_tree_expand, B, 128, 0, tb, c->sd, c->dt, ts, p, m, c->top_val, c->top_id, c->lse_rows, rn, next_m);
     cur ^= 1;
@@ -765,7 +774,7 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
     // completes S^l (for l >= 1) and captures it where a sequence taps layer l
     norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, xm, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
     GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, xm, R, c->qkvN, d);
-    LAUNCH(c, (k_qkv_post_target<T>), R, 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv);
+    LAUNCH(c, (k_qkv_post_target<T>), dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv);
     HD_DISPATCH(c, T, tree(c, l, R, xm));
     g = gemm<T>(c, c->wo[l], c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->ln2[l], R, xm);
@@ -773,7 +782,7 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
   }
   norm_rows<T>(c, c->x, gd, true, c->ln_f, R, xm, c->tapbuf, rm.seq, c->sd.tap, L);
   GemmOut g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
-  LAUNCH(c, k_topk_lse, R, TOPK_THREADS, 0, g, f.vocab, 2, c->top_val, c->top_id, c->lse_rows, logits);
+  LAUNCH(c, k_topk_lse, dim3(R, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, 2, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, logits);
   LAUNCH(c, k_argmax_out, (R + 127) / 128, 128, 0, c->top_id, c->top_val, R, argmax, margin,
          argmax == c->argmax_i ? (int *)nullptr : c->argmax_i);
   return DREAM_OK;
@@ -812,7 +821,7 @@ static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const 
   const XMode xm = xmode(c, R);
   LAUNCH(c, (k_gather_rows<T>), R, 256, 0, c->tapbuf, c->gather_idx, (T *)c->raw, d, (const int *)nullptr, 0, 0LL, xlay(xm, d));
   GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
-  LAUNCH(c, k_mem_append, R, 256, 0, g, rm.seq, rm.dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
+  LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
   return DREAM_OK;
 }
 

@@ -46,30 +46,69 @@ __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict_
 // Optional side outputs of the updated residual: `copy` (fp32; when tap_state is given the
 // row is copied only if its sequence's tap layer equals `layer`) and `raw` (element type,
 // unnormalised: the memory side of Eq. 1 takes features without a norm).
+#define NORM_THREADS 512
+#define NORM_NV 4                // float4 groups a thread keeps in registers (rows up to 8192 wide)
 template <typename T>
-__global__ void k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
-                             float eps, int d, T *xn, float *copy, const int *row_seq,
-                             const int *tap_state, int layer, T *raw, XLayout lay) {
+__global__ void __launch_bounds__(NORM_THREADS)
+k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
+             float eps, int d, T *xn, float *copy, const int *row_seq,
+             const int *tap_state, int layer, T *raw, XLayout lay) {
   __shared__ float sh[33];
   pdl_trigger();
   pdl_wait();
-  int r = blockIdx.x;
+  int r = blockIdx.x, d4 = d >> 2;
   float *xr = x + (long long)r * d;
+  float4 v[NORM_NV];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = xr[i];
-    if (has_in) { v += gemm_val(gin, r, i); xr[i] = v; }
-    ss += v * v;
+  // every load of the row is issued before the first use
+#pragma unroll
+  for (int j = 0; j < NORM_NV; ++j) {
+    int i = threadIdx.x + j * NORM_THREADS;
+    v[j] = i < d4 ? ld_f4(xr + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (has_in) {
+    float4 gv[NORM_NV];
+#pragma unroll
+    for (int j = 0; j < NORM_NV; ++j) {
+      int i = threadIdx.x + j * NORM_THREADS;
+      gv[j] = i < d4 ? gemm_val4(gin, r, 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < NORM_NV; ++j) {
+      int i = threadIdx.x + j * NORM_THREADS;
+      v[j].x += gv[j].x; v[j].y += gv[j].y; v[j].z += gv[j].z; v[j].w += gv[j].w;
+      if (i < d4) *reinterpret_cast<float4 *>(xr + 4 * i) = v[j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < NORM_NV; ++j) ss += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
+  for (int i = threadIdx.x + NORM_NV * NORM_THREADS; i < d4; i += NORM_THREADS) {      // rows wider than 8192
+    float4 t = ld_f4(xr + 4 * i);
+    if (has_in) {
+      float4 gq = gemm_val4(gin, r, 4 * i);
+      t.x += gq.x; t.y += gq.y; t.z += gq.z; t.w += gq.w;
+      *reinterpret_cast<float4 *>(xr + 4 * i) = t;
+    }
+    ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
   }
   float tot = block_sum(ss, sh);
   float inv = rsqrtf(tot / (float)d + eps);
   bool do_copy = copy != nullptr && (tap_state == nullptr || tap_state[row_seq[r]] == layer);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = xr[i];
-    if (do_copy) copy[(long long)r * d + i] = v;
-    if (raw) store_split<T>(raw + r * lay.row_stride + i, lay.lo_delta, v);
-    if (xn) store_split<T>(xn + r * lay.row_stride + i, lay.lo_delta, v * inv * to_f(gain[i]));
+  auto emit = [&](int i, float4 t) {
+    if (do_copy) *reinterpret_cast<float4 *>(copy + (long long)r * d + 4 * i) = t;
+    if (raw) store_split4<T>(raw + r * lay.row_stride + 4 * i, lay.lo_delta, t);
+    if (xn) {
+      float4 gq = ld_f4(gain + 4 * i);
+      store_split4<T>(xn + r * lay.row_stride + 4 * i, lay.lo_delta,
+                      make_float4(t.x * inv * gq.x, t.y * inv * gq.y, t.z * inv * gq.z, t.w * inv * gq.w));
+    }
+  };
+#pragma unroll
+  for (int j = 0; j < NORM_NV; ++j) {
+    int i = threadIdx.x + j * NORM_THREADS;
+    if (i < d4) emit(i, v[j]);
   }
+  for (int i = threadIdx.x + NORM_NV * NORM_THREADS; i < d4; i += NORM_THREADS) emit(i, ld_f4(xr + 4 * i));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -100,8 +139,8 @@ struct PagedKV {
 };
 
 // After the QKV GEMM of target rows: rotary on q and k at row_pos, q -> qbuf (fp32),
-// k, v -> the paged cache at (row_seq, row_slot).  One block per row; a work item is one
-// rotary pair (head, i) so that consecutive threads read consecutive GEMM columns.
+// k, v -> the paged cache at (row_seq, row_slot).  grid (rows, ceil(items / 256)); a work item
+// is four neighbouring rotary pairs of one head, read and written as 128-bit words.
 template <typename T>
 __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
                                   const int *__restrict__ row_pos, const int *__restrict__ row_slot,
@@ -109,28 +148,32 @@ __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
   pdl_trigger();
   pdl_wait();
   int r = blockIdx.x + row0, lr = blockIdx.x;
-  int hd = kv.hd, half = hd >> 1, Hkv = kv.hkv;
+  int hd = kv.hd, half = hd >> 1, q4 = half >> 2, Hkv = kv.hkv;
+  int w = blockIdx.y * blockDim.x + threadIdx.x;
+  if (w >= (H + 2 * Hkv) * q4) return;
+  int hh = w / q4, i = (w - hh * q4) * 4;
   int seq = row_seq[r], pos = row_pos[r], slot = row_slot[r];
   T *Kp = (T *)kv.base, *Vp = (T *)kv.base + kv.kv_stride;
-  int items = (H + 2 * Hkv) * half;
-  for (int w = threadIdx.x; w < items; w += blockDim.x) {
-    int hh = w / half, i = w - hh * half;
-    float a = gemm_val(g, lr, hh * hd + i), b = gemm_val(g, lr, hh * hd + i + half);
-    if (hh < H + Hkv) {
-      float c, s;
-      rope_cs(pos, inv_freq[i], &c, &s);
-      float ra = a * c - b * s, rb = b * c + a * s;
-      if (hh < H) {
-        float *q = qbuf + ((long long)r * H + hh) * hd;
-        q[i] = ra; q[i + half] = rb;
-      } else {
-        long long o = kv.off(seq, slot, hh - H);
-        Kp[o + i] = from_f<T>(ra); Kp[o + i + half] = from_f<T>(rb);
-      }
+  float4 a = gemm_val4(g, lr, hh * hd + i), b = gemm_val4(g, lr, hh * hd + i + half);
+  if (hh < H + Hkv) {
+    float c0, s0, c1, s1, c2, s2, c3, s3;
+    rope_cs(pos, inv_freq[i], &c0, &s0); rope_cs(pos, inv_freq[i + 1], &c1, &s1);
+    rope_cs(pos, inv_freq[i + 2], &c2, &s2); rope_cs(pos, inv_freq[i + 3], &c3, &s3);
+    float4 ra = make_float4(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1, a.z * c2 - b.z * s2, a.w * c3 - b.w * s3);
+    float4 rb = make_float4(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1, b.z * c2 + a.z * s2, b.w * c3 + a.w * s3);
+    if (hh < H) {
+      float *q = qbuf + ((long long)r * H + hh) * hd;
+      *reinterpret_cast<float4 *>(q + i) = ra;
+      *reinterpret_cast<float4 *>(q + i + half) = rb;
     } else {
-      long long o = kv.off(seq, slot, hh - H - Hkv);
-      Vp[o + i] = from_f<T>(a); Vp[o + i + half] = from_f<T>(b);
+      long long o = kv.off(seq, slot, hh - H);
+      store_split4<T>(Kp + o + i, 0, ra);
+      store_split4<T>(Kp + o + i + half, 0, rb);
     }
+  } else {
+    long long o = kv.off(seq, slot, hh - H - Hkv);
+    store_split4<T>(Vp + o + i, 0, a);
+    store_split4<T>(Vp + o + i + half, 0, b);
   }
 }
 
@@ -145,52 +188,51 @@ struct FlatKV {
 
 // After a draft QKV GEMM (has_q: the GEMM produced q columns first, then K, then V; otherwise
 // K then V only): rotary, q -> qbuf (when has_q), k/v -> draft self-attention cache row
-// row_dst[r] (skipped when < 0).  Work items as in k_qkv_post_target.
+// row_dst[r] (skipped when < 0).  Work items and grid as in k_qkv_post_target.
 __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
                                  const int *__restrict__ row_pos, const int *__restrict__ row_dst,
                                  int row0, int has_q, float *qbuf, FlatKV kv, int H, const double *__restrict__ inv_freq) {
   pdl_trigger();
   pdl_wait();
   int r = blockIdx.x + row0, lr = blockIdx.x;
-  int dst = row_dst[r];
-  int hd = kv.hd, half = hd >> 1, Hkv = kv.hkv;
-  int seq = row_seq[r], pos = row_pos[r];
+  int hd = kv.hd, half = hd >> 1, q4 = half >> 2, Hkv = kv.hkv;
   int Hq = has_q ? H : 0;
+  int w = blockIdx.y * blockDim.x + threadIdx.x;
+  if (w >= (Hq + 2 * Hkv) * q4) return;
+  int hh = w / q4, i = (w - hh * q4) * 4;
+  int dst = row_dst[r], seq = row_seq[r], pos = row_pos[r];
+  if (hh >= Hq && dst < 0) return;
   float *base = kv.base;
-  int items = (Hq + 2 * Hkv) * half;
-  for (int w = threadIdx.x; w < items; w += blockDim.x) {
-    int hh = w / half, i = w - hh * half;
-    if (hh >= Hq && dst < 0) continue;
-    float a = gemm_val(g, lr, hh * hd + i), b = gemm_val(g, lr, hh * hd + i + half);
-    if (hh < Hq + Hkv) {
-      float c, s;
-      rope_cs(pos, inv_freq[i], &c, &s);
-      float ra = a * c - b * s, rb = b * c + a * s;
-      if (hh < Hq) {
-        float *q = qbuf + ((long long)r * H + hh) * hd;
-        q[i] = ra; q[i + half] = rb;
-      } else {
-        long long o = kv.off(seq, 0, hh - Hq, dst);
-        base[o + i] = ra; base[o + i + half] = rb;
-      }
-    } else {
-      long long o = kv.off(seq, 1, hh - Hq - Hkv, dst);
-      base[o + i] = a; base[o + i + half] = b;
-    }
+  float4 a = gemm_val4(g, lr, hh * hd + i), b = gemm_val4(g, lr, hh * hd + i + half);
+  if (hh < Hq + Hkv) {
+    float c0, s0, c1, s1, c2, s2, c3, s3;
+    rope_cs(pos, inv_freq[i], &c0, &s0); rope_cs(pos, inv_freq[i + 1], &c1, &s1);
+    rope_cs(pos, inv_freq[i + 2], &c2, &s2); rope_cs(pos, inv_freq[i + 3], &c3, &s3);
+    float4 ra = make_float4(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1, a.z * c2 - b.z * s2, a.w * c3 - b.w * s3);
+    float4 rb = make_float4(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1, b.z * c2 + a.z * s2, b.w * c3 + a.w * s3);
+    float *o = hh < Hq ? qbuf + ((long long)r * H + hh) * hd : base + kv.off(seq, 0, hh - Hq, dst);
+    *reinterpret_cast<float4 *>(o + i) = ra;
+    *reinterpret_cast<float4 *>(o + i + half) = rb;
+  } else {
+    float *o = base + kv.off(seq, 1, hh - Hq - Hkv, dst);
+    *reinterpret_cast<float4 *>(o + i) = a;
+    *reinterpret_cast<float4 *>(o + i + half) = b;
   }
 }
 
-// Plain copy of a GEMM output [rows][width] into fp32 rows (q of the cross-attention: no rotary)
+// Plain copy of a GEMM output [rows][width] into fp32 rows (q of the cross-attention: no rotary).
+// grid (rows, ceil(width / 1024)).
 __global__ void k_gemm_to_f32(GemmOut g, float *dst, int width) {
   pdl_trigger();
   pdl_wait();
-  int r = blockIdx.x;
-  for (int i = threadIdx.x; i < width; i += blockDim.x) dst[(long long)r * width + i] = gemm_val(g, r, i);
+  int r = blockIdx.x, i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+  if (i < width) *reinterpret_cast<float4 *>(dst + (long long)r * width + i) = gemm_val4(g, r, i);
 }
 
 // Cross-attention memory rows (Eq. 1: K = S W_K, V = S W_V): GEMM output [rows][2 H_kv hd]
 // -> memory cache row of sequence row_seq[r]: row_dst[r] when nperm is null, else the
 // tree-region row nperm[seq] + row_in[r].  Negative indices skip the row.
+// grid (rows, ceil(2 H_kv hd / 1024)).
 __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
                              const int *__restrict__ row_dst, const int *__restrict__ row_in,
                              const int *__restrict__ nperm, int row0, FlatKV kv) {
@@ -201,36 +243,39 @@ __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
   int dst = nperm ? (row_in[r] < 0 ? -1 : nperm[seq] + row_in[r]) : row_dst[r];
   if (dst < 0) return;
   int w = kv.hkv * kv.hd;
-  float *base = kv.base;
-  for (int i = threadIdx.x; i < w; i += blockDim.x) {
-    int h = i / kv.hd, e = i - h * kv.hd;
-    base[kv.off(seq, 0, h, dst) + e] = gemm_val(g, lr, i);
-    base[kv.off(seq, 1, h, dst) + e] = gemm_val(g, lr, w + i);
-  }
+  int i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+  if (i >= 2 * w) return;
+  int which = i >= w ? 1 : 0, j = i - which * w;
+  int h = j / kv.hd, e = j - h * kv.hd;
+  *reinterpret_cast<float4 *>(kv.base + kv.off(seq, which, h, dst) + e) = gemm_val4(g, lr, i);
 }
 
 // act = silu(gate) * up, from a GEMM output whose columns are [gate(ff) | up(ff)].
+// grid (ceil(ff / 1024), rows).
 template <typename T>
 __global__ void k_silu_mul(GemmOut g, T *act, int ff, XLayout lay) {
   pdl_trigger();
   pdl_wait();
   int r = blockIdx.y;
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= ff) return;
-  float a = gemm_val(g, r, i), b = gemm_val(g, r, ff + i);
-  store_split<T>(act + r * lay.row_stride + i, lay.lo_delta, a / (1.f + __expf(-a)) * b);
+  float4 a = gemm_val4(g, r, i), b = gemm_val4(g, r, ff + i);
+  float4 o = make_float4(a.x / (1.f + __expf(-a.x)) * b.x, a.y / (1.f + __expf(-a.y)) * b.y,
+                         a.z / (1.f + __expf(-a.z)) * b.z, a.w / (1.f + __expf(-a.w)) * b.w);
+  store_split4<T>(act + r * lay.row_stride + i, lay.lo_delta, o);
 }
 
 // x += GEMM output; optional fp32 copy into a per-layer store (prefill tap candidates).
+// grid (rows, ceil(d / 1024)).
 __global__ void k_resid_add(float *x, GemmOut g, int d, float *copy) {
   pdl_trigger();
   pdl_wait();
-  int r = blockIdx.x;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = x[(long long)r * d + i] + gemm_val(g, r, i);
-    x[(long long)r * d + i] = v;
-    if (copy) copy[(long long)r * d + i] = v;
-  }
+  int r = blockIdx.x, i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+  if (i >= d) return;
+  float4 v = ld_f4(x + (long long)r * d + i), t = gemm_val4(g, r, i);
+  v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+  *reinterpret_cast<float4 *>(x + (long long)r * d + i) = v;
+  if (copy) *reinterpret_cast<float4 *>(copy + (long long)r * d + i) = v;
 }
 
 // Gather fp32 rows into element-type GEMM input rows: dst[r] = src[idx[r]] (idx < 0 -> zeros).
@@ -242,57 +287,36 @@ __global__ void k_gather_rows(const float *__restrict__ src, const int *__restri
   pdl_wait();
   int r = blockIdx.x, s = idx[r];
   if (layer_ptr) src += (long long)(*layer_ptr - layer_lo) * layer_stride;
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    store_split<T>(dst + r * lay.row_stride + i, lay.lo_delta, s >= 0 ? src[(long long)s * d + i] : 0.f);
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4)
+    store_split4<T>(dst + r * lay.row_stride + i, lay.lo_delta,
+                    s >= 0 ? ld_f4(src + (long long)s * d + i) : make_float4(0.f, 0.f, 0.f, 0.f));
 }
 
 // ---------------------------------------------------------------------------------------
 // Per row of a [rows][V] GEMM output: the KTOP largest logits (ties -> lower id), in
-// descending order, and the log-sum-exp of the row.  One block per row.
+// descending order, and the log-sum-exp of the row.  grid (rows, nsplit): block (r, sp) scans
+// columns [sp * TOPK_COLS, (sp + 1) * TOPK_COLS) and leaves a sorted partial list and an (m, z)
+// pair; the block that finishes a row last merges the partials, always in the same order.
 #define TOPK_MAX 16
 #define TOPK_THREADS 256
-__global__ void __launch_bounds__(TOPK_THREADS)
-k_topk_lse(GemmOut g, int V, int ktop, float *top_val, int *top_id, float *lse, float *logits_out) {
-  __shared__ float sv[TOPK_THREADS * TOPK_MAX];
-  __shared__ int si[TOPK_THREADS * TOPK_MAX];
-  __shared__ float red[33];
-  __shared__ float cand_v[TOPK_THREADS / 32];
-  __shared__ int cand_i[TOPK_THREADS / 32], cand_t[TOPK_THREADS / 32];
-  pdl_trigger();
-  pdl_wait();
-  int r = blockIdx.x, tid = threadIdx.x;
-  float lv[TOPK_MAX];
-  int li[TOPK_MAX];
-  for (int j = 0; j < TOPK_MAX; ++j) { lv[j] = -INFINITY; li[j] = 0x7fffffff; }
-  float m = -INFINITY, z = 0.f;
-  for (int c = tid; c < V; c += TOPK_THREADS) {
-    float v = gemm_val(g, r, c);
-    if (logits_out) logits_out[(long long)r * V + c] = v;
-    if (v > m) { z = z * __expf(m - v) + 1.f; m = v; } else z += __expf(v - m);
-    if (better(v, c, lv[ktop - 1], li[ktop - 1])) {
-      int j = ktop - 1;
-      while (j > 0 && better(v, c, lv[j - 1], li[j - 1])) { lv[j] = lv[j - 1]; li[j] = li[j - 1]; --j; }
-      lv[j] = v; li[j] = c;
-    }
-  }
-  // log-sum-exp: combine (m, z) pairs in a fixed order
-  float bm = m;
-  bm = warp_max(bm);
-  __syncthreads();
-  if ((tid & 31) == 0) red[tid >> 5] = bm;
-  __syncthreads();
-  if (tid < 32) { float t = tid < TOPK_THREADS / 32 ? red[tid] : -INFINITY; t = warp_max(t); if (tid == 0) red[32] = t; }
-  __syncthreads();
-  float gm = red[32];
-  float tot = block_sum(m == -INFINITY ? 0.f : z * __expf(m - gm), red);
-  if (tid == 0) lse[r] = gm + logf(tot);
-  // merge the per-thread sorted lists: ktop rounds of a block-wide "best head" selection
-  for (int j = 0; j < ktop; ++j) { sv[tid * TOPK_MAX + j] = lv[j]; si[tid * TOPK_MAX + j] = li[j]; }
-  int head = 0;
-  __syncthreads();
+#define TOPK_COLS 4096
+struct TopkScratch {
+  float *pv;       // [rows][nsplit][TOPK_MAX] partial values
+  int *pi;         // [rows][nsplit][TOPK_MAX] partial ids
+  float *pm, *pz;  // [rows][nsplit] running max and sum of exp
+  int *counter;    // [rows] blocks done; zero between launches
+};
+
+// Block-wide selection of the `ktop` best heads of per-thread sorted lists kept in shared memory
+// (list t = sv/si[t * TOPK_MAX ..], `len` valid entries for t < nlists).  Round j's winner goes
+// to out_v/out_i[j].
+__device__ __forceinline__ void topk_merge_lists(const float *sv, const int *si, int nlists, int len, int ktop,
+                                                 float *out_v, int *out_i, float *cand_v, int *cand_i, int *cand_t) {
+  int tid = threadIdx.x, head = 0;
   for (int round = 0; round < ktop; ++round) {
-    float v = head < ktop ? sv[tid * TOPK_MAX + head] : -INFINITY;
-    int id = head < ktop ? si[tid * TOPK_MAX + head] : 0x7fffffff;
+    bool live = tid < nlists && head < len;
+    float v = live ? sv[tid * TOPK_MAX + head] : -INFINITY;
+    int id = live ? si[tid * TOPK_MAX + head] : 0x7fffffff;
     int t = tid;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -306,7 +330,87 @@ k_topk_lse(GemmOut g, int V, int ktop, float *top_val, int *top_id, float *lse, 
     for (int w = 1; w < TOPK_THREADS / 32; ++w)
       if (better(cand_v[w], cand_i[w], bv, bi)) { bv = cand_v[w]; bi = cand_i[w]; bt = cand_t[w]; }
     if (tid == bt) ++head;
-    if (tid == 0) { top_val[r * ktop + round] = bv; top_id[r * ktop + round] = bi; }
+    if (tid == 0) { out_v[round] = bv; out_i[round] = bi; }
     __syncthreads();
   }
+}
+
+__global__ void __launch_bounds__(TOPK_THREADS)
+k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_val, int *top_id, float *lse,
+           float *logits_out) {
+  __shared__ float sv[TOPK_THREADS * TOPK_MAX];
+  __shared__ int si[TOPK_THREADS * TOPK_MAX];
+  __shared__ float red[33];
+  __shared__ float cand_v[TOPK_THREADS / 32];
+  __shared__ int cand_i[TOPK_THREADS / 32], cand_t[TOPK_THREADS / 32];
+  __shared__ int is_last;
+  pdl_trigger();
+  pdl_wait();
+  int r = blockIdx.x, sp = blockIdx.y, tid = threadIdx.x;
+  int c0 = sp * TOPK_COLS, c1 = min(V, c0 + TOPK_COLS);
+  float lv[TOPK_MAX];
+  int li[TOPK_MAX];
+  for (int j = 0; j < TOPK_MAX; ++j) { lv[j] = -INFINITY; li[j] = 0x7fffffff; }
+  float m = -INFINITY, z = 0.f;
+  auto consider = [&](float v, int c) {
+    if (v > m) { z = z * __expf(m - v) + 1.f; m = v; } else z += __expf(v - m);
+    if (better(v, c, lv[ktop - 1], li[ktop - 1])) {
+      int j = ktop - 1;
+      while (j > 0 && better(v, c, lv[j - 1], li[j - 1])) { lv[j] = lv[j - 1]; li[j] = li[j - 1]; --j; }
+      lv[j] = v; li[j] = c;
+    }
+  };
+  if ((V & 3) == 0) {
+    for (int c = c0 + tid * 4; c < c1; c += TOPK_THREADS * 4) {
+      float4 v = gemm_val4(g, r, c);
+      if (logits_out) *reinterpret_cast<float4 *>(logits_out + (long long)r * V + c) = v;
+      consider(v.x, c); consider(v.y, c + 1); consider(v.z, c + 2); consider(v.w, c + 3);
+    }
+  } else {
+    for (int c = c0 + tid; c < c1; c += TOPK_THREADS) {
+      float v = gemm_val(g, r, c);
+      if (logits_out) logits_out[(long long)r * V + c] = v;
+      consider(v, c);
+    }
+  }
+  // (m, z) of this block's columns, combined in a fixed order
+  float bm = warp_max(m);
+  __syncthreads();
+  if ((tid & 31) == 0) red[tid >> 5] = bm;
+  __syncthreads();
+  if (tid < 32) { float t = tid < TOPK_THREADS / 32 ? red[tid] : -INFINITY; t = warp_max(t); if (tid == 0) red[32] = t; }
+  __syncthreads();
+  float gm = red[32];
+  float tot = block_sum(m == -INFINITY ? 0.f : z * __expf(m - gm), red);
+  long long po = (long long)r * nsplit + sp;
+  if (tid == 0) { ts.pm[po] = gm; ts.pz[po] = tot; }
+  // this block's sorted top-ktop
+  for (int j = 0; j < ktop; ++j) { sv[tid * TOPK_MAX + j] = lv[j]; si[tid * TOPK_MAX + j] = li[j]; }
+  __syncthreads();
+  topk_merge_lists(sv, si, TOPK_THREADS, ktop, ktop, ts.pv + po * TOPK_MAX, ts.pi + po * TOPK_MAX, cand_v, cand_i, cand_t);
+  // the last block of the row merges
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    int old = atomicAdd(ts.counter + r, 1);
+    is_last = old == nsplit - 1;
+    if (is_last) ts.counter[r] = 0;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  if (tid < nsplit) {
+    for (int j = 0; j < ktop; ++j) {
+      sv[tid * TOPK_MAX + j] = __ldcg(ts.pv + ((long long)r * nsplit + tid) * TOPK_MAX + j);
+      si[tid * TOPK_MAX + j] = __ldcg(ts.pi + ((long long)r * nsplit + tid) * TOPK_MAX + j);
+    }
+  }
+  if (tid == 0) {
+    float mm = -INFINITY, zz = 0.f;
+    for (int q = 0; q < nsplit; ++q) mm = fmaxf(mm, __ldcg(ts.pm + (long long)r * nsplit + q));
+    for (int q = 0; q < nsplit; ++q) zz += __ldcg(ts.pz + (long long)r * nsplit + q) * __expf(__ldcg(ts.pm + (long long)r * nsplit + q) - mm);
+    lse[r] = mm + logf(zz);
+  }
+  __syncthreads();
+  topk_merge_lists(sv, si, nsplit, ktop, ktop, top_val + (long long)r * ktop, top_id + (long long)r * ktop, cand_v, cand_i, cand_t);
 }
