@@ -212,7 +212,7 @@ k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ 
   if (in < 0) return;
   int seq = row_seq[r], np = nperm[seq];
   int kvh = h / (H / kv.hkv);
-  const float *base = kv.base;
+  const float *base = (const float *)kv.base;          // fp32 configurations only
   long long ok = kv.off(seq, 0, kvh, 0), ov = kv.off(seq, 1, kvh, 0);
   float q[EPL], k[EPL], v[EPL];
   RowLoad<EPL, float>::ld(qbuf + ((long long)r * H + h) * HD, lane, q);

@@ -12,12 +12,14 @@
 
 #include "../../include/dream.h"
 #include "attn.cuh"
+#include "attn_mma.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "rows.cuh"
 #include "tree.cuh"
 
+#define AM_MAX_CHUNKS 32        // most key chunks the split-K attention cuts a sequence into
 #define ROW_CHUNK 256          // most rows any launch set holds (max_batch * tree nodes, a prefill chunk)
 
 enum { PH_EMPTY = 0, PH_PREFILLED, PH_READY, PH_DRAFTED, PH_VERIFIED };
@@ -52,6 +54,10 @@ struct dream_ctx {
   void *xn, *raw, *act, *attn_out;
   float *top_val, *lse_rows, *margin_i;
   TopkScratch tks;
+  float *am_part_o, *am_part_ml;       // split-K attention partials
+  int *am_counters;
+  int am_rt_max;
+  int key_ub[DREAM_MAX_BATCH];         // upper bound of the draft caches' permanent rows
   int tk_nsplit;
   int *top_id, *argmax_i, *accept_len_i, *out_tokens_i, *comp_src_i;
   size_t gout_floats;
@@ -270,6 +276,13 @@ static size_t carve(dream_ctx *c, char *base) {
   c->top_val = a.take<float>((size_t)ROW_CHUNK * TOPK_MAX);
   c->top_id = a.take<int>((size_t)ROW_CHUNK * TOPK_MAX);
   c->lse_rows = a.take<float>(ROW_CHUNK);
+  c->am_rt_max = (T * (f.n_heads / f.n_kv_heads) + AM_ROWS - 1) / AM_ROWS;
+  if (f.dtype == DREAM_BF16) {
+    size_t prow = (size_t)MB * AM_MAX_CHUNKS * f.n_kv_heads * c->am_rt_max * AM_ROWS;
+    c->am_part_o = a.take<float>(prow * f.head_dim);
+    c->am_part_ml = a.take<float>(prow * 2);
+    c->am_counters = a.take<int>((size_t)MB * f.n_kv_heads * c->am_rt_max);
+  } else { c->am_part_o = nullptr; c->am_part_ml = nullptr; c->am_counters = nullptr; }
   c->tk_nsplit = (f.vocab + TOPK_COLS - 1) / TOPK_COLS;
   c->tks.pv = a.take<float>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
   c->tks.pi = a.take<int>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
@@ -356,11 +369,20 @@ static PagedKV paged(dream_ctx *c, int layer) {
 static FlatKV flat(dream_ctx *c, float *base) {
   FlatKV kv;
   kv.base = base; kv.cap = c->cap_rows; kv.hkv = c->cfg.n_kv_heads; kv.hd = c->cfg.head_dim;
+  kv.split = c->cfg.dtype == DREAM_BF16 ? 1 : 0;
   return kv;
 }
 static const GemmOut NO_GEMM = {nullptr, 0, 0, 30, 0, 0, 0};
 
 // ------------------------------------------------------------------------------------- init / free
+
+template <int HD>
+static const char *attn_mma_setup() {
+  if (cudaFuncSetAttribute(k_attn_mma<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_mma_smem<HD, true>()) != cudaSuccess ||
+      cudaFuncSetAttribute(k_attn_mma<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_mma_smem<HD, false>()) != cudaSuccess)
+    return "cannot raise the attention kernel's shared memory limit";
+  return nullptr;
+}
 
 extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_weights *tw,
                                    const dream_draft_weights *dw, void *arena, size_t arena_bytes,
@@ -404,6 +426,10 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   if (c->use_tc) {
     const char *why = gemm_tc_plan_init(&c->tc, c->status, c->use_pdl);
     if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
+  }
+  if (c->use_tc) {
+    const char *why = cfg->head_dim == 64 ? attn_mma_setup<64>() : cfg->head_dim == 128 ? attn_mma_setup<128>() : attn_mma_setup<256>();
+    if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "%s", why); }
   }
   k_rope_table<<<(cfg->head_dim / 2 + 127) / 128, 128, 0, c->stream>>>(c->rope_inv, cfg->head_dim, cfg->rope_theta);
   if (cudaGetLastError() != cudaSuccess) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "rotary table launch failed"); }
@@ -491,6 +517,11 @@ __global__ void k_copy_f32(const float *src, float *dst, int n) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src[i];
 }
+// A draft-cache row of a bf16 configuration: hd high parts then hd low parts.
+__global__ void k_read_row_split(const bf16 *src, float *dst, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = to_f(src[i]) + to_f(src[n + i]);
+}
 template <typename T>
 __global__ void k_read_row(const T *src, float *dst, int n) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -508,12 +539,45 @@ template <typename T, int HD> struct AttnLaunch {
     LAUNCH(c, (k_colsum<T, HD>), (v + ATT_WARPS - 1) / ATT_WARPS, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n,
            c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, score);
   }
-  static void tree(dream_ctx *c, int layer, int R, XMode m) {
+  // Split-K plan and launch of the tensor-core attention (bf16 configurations).
+  template <bool PAGED>
+  static void mma(dream_ctx *c, AttnMmaArgs a, int B, int rows_per_seq, int key_ub) {
+    const dream_config &f = c->cfg;
+    constexpr int KBLK = AmShape<HD>::KBLK;
+    a.q = c->qbuf; a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+    a.n_rt = (rows_per_seq * a.G + AM_ROWS - 1) / AM_ROWS;
+    int nb_ub = imax(1, (key_ub + KBLK - 1) / KBLK), ctas = f.n_kv_heads * a.n_rt * B;
+    int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, (2 * c->tc.n_sms + ctas - 1) / ctas));
+    a.blocks_per_chunk = (nb_ub + want - 1) / want;
+    a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
+    a.part_o = c->am_part_o; a.part_ml = c->am_part_ml; a.counters = c->am_counters;
+    a.out = c->attn_out;
+    dim3 grid(a.n_chunks, f.n_kv_heads * a.n_rt, B);
+    LAUNCH(c, (k_attn_mma<HD, PAGED>), grid, AM_THREADS, (attn_mma_smem<HD, PAGED>()), a);
+  }
+  static void tree(dream_ctx *c, int layer, int R, XMode m, int B, int key_ub) {
+    if (sizeof(T) == 2) {
+      AttnMmaArgs a = {};
+      a.row_seq = c->rm[0].seq; a.row_in = nullptr; a.prefix_len = c->sd.P; a.mask = c->vmask; a.anc = nullptr;
+      a.tail_len = c->T; a.lay = xlay(m, c->Hhd); a.paged = paged(c, layer);
+      mma<true>(c, a, B, c->T, key_ub);
+      return;
+    }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_tree<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
            c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
   }
-  static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, XMode m) {
+  static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, XMode m, int B,
+                    int rows_per_seq, int key_ub) {
+    if (sizeof(T) == 2) {
+      AttnMmaArgs a = {};
+      a.row_seq = rm.seq; a.row_in = rm.in; a.prefix_len = nperm; a.mask = nullptr; a.anc = c->dt.in_anc;
+      a.anc_stride = c->ts.NI; a.strict = strict; a.tail_len = c->ts.NI; a.lay = xlay(m, c->Hhd);
+      a.flat.base = (bf16 *)cache; a.flat.cap = c->cap_rows; a.flat.hkv = c->cfg.n_kv_heads; a.flat.hd = HD;
+      mma<false>(c, a, B, rows_per_seq, key_ub);
+      return;
+    }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
     LAUNCH(c, (k_attn_draft<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, flat(c, cache), rm.seq, rm.in, nperm,
            c->dt.in_anc, c->ts.NI, strict, R, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
@@ -678,6 +742,7 @@ extern "C" dream_status dream_compress_visual(dream_ctx *c, int32_t seq, int32_t
   CUDA_OK(c, cudaGetLastError());
   if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
   c->phase[seq] = PH_READY;
+  c->key_ub[seq] = c->pf_q + (c->cfg.xattn_full_memory ? c->pf_v : k);
   c->prefill_seq = -1;
   return DREAM_OK;
 }
@@ -712,6 +777,8 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
   const dream_config &f = c->cfg;
   const TreeShape &ts = c->ts;
   int d = f.d_model, cur = 0;
+  int key_ub = 0;                 // most keys any listed sequence can hold in a draft cache
+  for (int b = 0; b < B; ++b) key_ub = imax(key_ub, c->key_ub[tb.seq[b]] + ts.D + 1 + ts.NI);
   for (int p = 1; p <= ts.D; ++p) {
     int m = p == 1 ? ts.D + 2 : ts.beam[p - 1];
     int R = B * m;
@@ -722,12 +789,12 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
     GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
     LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
-    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm));
+    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub));
     g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
     g = gemm<T>(c, c->dw.xq, c->xn, xm, R, c->Hhd, d);
     LAUNCH(c, k_gemm_to_f32, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, c->Hhd);
-    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm));
+    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm, B, m, key_ub));
     g = gemm<T>(c, c->dw.xo, c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, xm);
     g = mlp_rows<T>(c, c->dw.wgu, c->dw.wd, R, xm);
@@ -767,6 +834,8 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
   int d = f.d_model, L = f.n_layers, R = B * c->T;
   const XMode xm = xmode(c, R);
   RowMeta &rm = c->rm[0];
+  int key_ub = 0;
+  for (int b = 0; b < B; ++b) key_ub = imax(key_ub, c->p_ub[tb.seq[b]] + c->T);
   LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
   LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
   GemmOut gd = NO_GEMM;
@@ -775,7 +844,7 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
     norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, xm, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
     GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, xm, R, c->qkvN, d);
     LAUNCH(c, (k_qkv_post_target<T>), dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv);
-    HD_DISPATCH(c, T, tree(c, l, R, xm));
+    HD_DISPATCH(c, T, tree(c, l, R, xm, B, key_ub));
     g = gemm<T>(c, c->wo[l], c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->ln2[l], R, xm);
     gd = mlp_rows<T>(c, c->wgu[l], c->wd[l], R, xm);
@@ -839,7 +908,7 @@ extern "C" dream_status dream_accept(dream_ctx *c, const int32_t *seqs, int32_t 
   if (s) return s;
   CUDA_OK(c, cudaGetLastError());
   if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
-  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; }
+  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; c->key_ub[seqs[b]] += c->ts.D + 1; }
   return DREAM_OK;
 }
 
@@ -898,7 +967,8 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
     int kvsel = (what - 2) & 1;
     for (int h = 0; h < f.n_kv_heads; ++h) {
       const float *src = base + ((((size_t)seq * 2 + kvsel) * f.n_kv_heads + h) * c->cap_rows + index) * f.head_dim;
-      k_read_row<float><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
+      if (sizeof(T) == 2) k_read_row_split<<<1, 256, 0, c->stream>>>((const bf16 *)src, tmp + h * f.head_dim, f.head_dim);
+      else k_read_row<float><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
     }
   } else if (what == 6 || what == 7) {
     if (index < 0 || index >= ROW_CHUNK) return fail(c, DREAM_E_ARG, "row out of range");

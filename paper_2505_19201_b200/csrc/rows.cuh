@@ -177,12 +177,18 @@ __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
   }
 }
 
-// Draft caches are flat per sequence, always fp32 (they are small): [seq][2][H_kv][cap][hd].
+// Draft caches are flat per sequence and hold 4 bytes per element (they are small):
+// [seq][2][H_kv][cap] rows of hd floats (fp32 configurations), or of 2 * hd bf16 = a high row
+// then a low row (bf16 configurations: what the tensor-core attention reads directly).
 struct FlatKV {
-  float *base;
-  int cap, hkv, hd;
+  void *base;
+  int cap, hkv, hd, split;
   __device__ __forceinline__ long long off(int seq, int kv, int kvh, int row) const {
-    return ((((long long)seq * 2 + kv) * hkv + kvh) * cap + row) * hd;
+    return ((((long long)seq * 2 + kv) * hkv + kvh) * cap + row) * (split ? 2 : 1) * hd;
+  }
+  __device__ __forceinline__ void store4(long long o, int e, float4 v) const {
+    if (split) store_split4<bf16>((bf16 *)base + o + e, hd, v);
+    else *reinterpret_cast<float4 *>((float *)base + o + e) = v;
   }
 };
 
@@ -202,7 +208,6 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
   int hh = w / q4, i = (w - hh * q4) * 4;
   int dst = row_dst[r], seq = row_seq[r], pos = row_pos[r];
   if (hh >= Hq && dst < 0) return;
-  float *base = kv.base;
   float4 a = gemm_val4(g, lr, hh * hd + i), b = gemm_val4(g, lr, hh * hd + i + half);
   if (hh < Hq + Hkv) {
     float c0, s0, c1, s1, c2, s2, c3, s3;
@@ -210,13 +215,19 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
     rope_cs(pos, inv_freq[i + 2], &c2, &s2); rope_cs(pos, inv_freq[i + 3], &c3, &s3);
     float4 ra = make_float4(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1, a.z * c2 - b.z * s2, a.w * c3 - b.w * s3);
     float4 rb = make_float4(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1, b.z * c2 + a.z * s2, b.w * c3 + a.w * s3);
-    float *o = hh < Hq ? qbuf + ((long long)r * H + hh) * hd : base + kv.off(seq, 0, hh - Hq, dst);
-    *reinterpret_cast<float4 *>(o + i) = ra;
-    *reinterpret_cast<float4 *>(o + i + half) = rb;
+    if (hh < Hq) {
+      float *o = qbuf + ((long long)r * H + hh) * hd;
+      *reinterpret_cast<float4 *>(o + i) = ra;
+      *reinterpret_cast<float4 *>(o + i + half) = rb;
+    } else {
+      long long o = kv.off(seq, 0, hh - Hq, dst);
+      kv.store4(o, i, ra);
+      kv.store4(o, i + half, rb);
+    }
   } else {
-    float *o = base + kv.off(seq, 1, hh - Hq - Hkv, dst);
-    *reinterpret_cast<float4 *>(o + i) = a;
-    *reinterpret_cast<float4 *>(o + i + half) = b;
+    long long o = kv.off(seq, 1, hh - Hq - Hkv, dst);
+    kv.store4(o, i, a);
+    kv.store4(o, i + half, b);
   }
 }
 
@@ -247,7 +258,7 @@ __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
   if (i >= 2 * w) return;
   int which = i >= w ? 1 : 0, j = i - which * w;
   int h = j / kv.hd, e = j - h * kv.hd;
-  *reinterpret_cast<float4 *>(kv.base + kv.off(seq, which, h, dst) + e) = gemm_val4(g, lr, i);
+  kv.store4(kv.off(seq, which, h, dst), e, gemm_val4(g, lr, i));
 }
 
 // act = silu(gate) * up, from a GEMM output whose columns are [gate(ff) | up(ff)].
