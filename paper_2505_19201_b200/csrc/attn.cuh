@@ -27,6 +27,23 @@ template <int EPL> struct RowLoad<EPL, bf16> {
   }
 };
 
+// Lane's share of the query of (row, head) rh; bf16 configurations store a high and a low row.
+template <int EPL, typename T> struct QLoad;
+template <int EPL> struct QLoad<EPL, float> {
+  static __device__ __forceinline__ void ld(const void *qbuf, long long rh, int lane, float (&o)[EPL]) {
+    RowLoad<EPL, float>::ld((const float *)qbuf + rh * (EPL * 32), lane, o);
+  }
+};
+template <int EPL> struct QLoad<EPL, bf16> {
+  static __device__ __forceinline__ void ld(const void *qbuf, long long rh, int lane, float (&o)[EPL]) {
+    float lo[EPL];
+    RowLoad<EPL, bf16>::ld((const bf16 *)qbuf + rh * 2 * (EPL * 32), lane, o);
+    RowLoad<EPL, bf16>::ld((const bf16 *)qbuf + rh * 2 * (EPL * 32) + EPL * 32, lane, lo);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) o[e] += lo[e];
+  }
+};
+
 // Online-softmax state of one (row, head): running max m, Z = sum e^{s-m}, the weighted
 // value sum, and U = sum e^{s-m}(s-m) for the entropy  H = ln Z - U/Z  (Eq. 2, inner sum).
 template <int EPL> struct Soft {
@@ -71,7 +88,7 @@ __device__ __forceinline__ float dot_lane(const float (&a)[EPL], const float (&b
 // log-sum-exp of the scaled scores, for the importance pass), ent [H][n] row entropies.
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
-k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
+k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
                T *attn_out, XLayout lay, float *lse, float *ent) {
   constexpr int EPL = HD / 32;
   pdl_trigger();
@@ -82,7 +99,7 @@ k_attn_prefill(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H
   int kvh = h / (H / kv.hkv);
   const T *Kp = (const T *)kv.base, *Vp = (const T *)kv.base + kv.kv_stride;
   float q[EPL], k[EPL], v[EPL];
-  RowLoad<EPL, float>::ld(qbuf + ((long long)i * H + h) * HD, lane, q);
+  QLoad<EPL, T>::ld(qbuf, (long long)i * H + h, lane, q);
 #pragma unroll
   for (int e = 0; e < EPL; ++e) q[e] *= scale;
   Soft<EPL> st;
@@ -119,7 +136,7 @@ __global__ void k_entropy_mean(const float *__restrict__ ent, int count, float *
 // One warp per visual column; heads outer, rows inner, both ascending: a fixed order.
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
-k_colsum(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
+k_colsum(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
          const float *__restrict__ lse, int vis_start, int v, int include_self, float *score) {
   constexpr int EPL = HD / 32;
   pdl_trigger();
@@ -136,7 +153,7 @@ k_colsum(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, floa
     RowLoad<EPL, T>::ld(Kp + kv.off(seq, j, kvh), lane, k);
     float hs = 0.f;
     for (int i = include_self ? j : j + 1; i < n; ++i) {
-      RowLoad<EPL, float>::ld(qbuf + ((long long)i * H + h) * HD, lane, q);
+      QLoad<EPL, T>::ld(qbuf, (long long)i * H + h, lane, q);
       float s = dot_lane<EPL>(q, k) * scale;
       hs += __expf(s - lse[(long long)h * n + i]);
     }
@@ -151,7 +168,7 @@ k_colsum(const float *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, floa
 // ancestor-or-self bit set.  grid (ceil(R/8), H).
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
-k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ row_seq,
+k_attn_tree(const void *__restrict__ qbuf, PagedKV kv, const int *__restrict__ row_seq,
             const int *__restrict__ row_node, const int *__restrict__ P_state,
             const uint32_t *__restrict__ mask, int R, int T_nodes, int H, float scale, T *attn_out,
             XLayout lay) {
@@ -165,7 +182,7 @@ k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ 
   int kvh = h / (H / kv.hkv);
   const T *Kp = (const T *)kv.base, *Vp = (const T *)kv.base + kv.kv_stride;
   float q[EPL], k[EPL], v[EPL];
-  RowLoad<EPL, float>::ld(qbuf + ((long long)r * H + h) * HD, lane, q);
+  QLoad<EPL, T>::ld(qbuf, (long long)r * H + h, lane, q);
 #pragma unroll
   for (int e = 0; e < EPL; ++e) q[e] *= scale;
   Soft<EPL> st;
@@ -198,7 +215,7 @@ k_attn_tree(const float *__restrict__ qbuf, PagedKV kv, const int *__restrict__ 
 // Rows with row_in < 0 are idle.  grid (ceil(R/8), H).
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
-k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ row_seq,
+k_attn_draft(const void *__restrict__ qbuf, FlatKV kv, const int *__restrict__ row_seq,
              const int *__restrict__ row_in, const int *__restrict__ nperm,
              const unsigned long long *__restrict__ anc, int anc_stride, int strict, int R, int H,
              float scale, T *attn_out, XLayout lay) {
@@ -215,7 +232,7 @@ k_attn_draft(const float *__restrict__ qbuf, FlatKV kv, const int *__restrict__ 
   const float *base = (const float *)kv.base;          // fp32 configurations only
   long long ok = kv.off(seq, 0, kvh, 0), ov = kv.off(seq, 1, kvh, 0);
   float q[EPL], k[EPL], v[EPL];
-  RowLoad<EPL, float>::ld(qbuf + ((long long)r * H + h) * HD, lane, q);
+  QLoad<EPL, T>::ld(qbuf, (long long)r * H + h, lane, q);
 #pragma unroll
   for (int e = 0; e < EPL; ++e) q[e] *= scale;
   Soft<EPL> st;

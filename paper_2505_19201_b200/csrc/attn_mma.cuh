@@ -8,10 +8,10 @@
 // cp.async (double buffered, 16-byte segments, padded rows: conflict-free ldmatrix), computes
 // S = Q K^T, an online softmax in the exp2 domain, and O += P V, all in registers.  Queries and
 // probabilities enter the tensor cores as a high and a low bf16 part, so the products keep ~16
-// mantissa bits; K and V are used as stored.  Each chunk leaves (m, l, O) partials; the CTA that
-// finishes a (sequence, KV head, row tile) last merges them in chunk order and writes the rows
-// as GEMM input.  Visible keys of a row: every key below prefix_len[seq], plus tail key j for
-// every bit j of the row's mask.
+// mantissa bits; K and V are used as stored.  Each chunk leaves (m, l, O) partials that
+// k_attn_combine merges in chunk order, one thread per four output values, and writes as GEMM
+// input rows (a single chunk writes them itself).  Visible keys of a row: every key below
+// prefix_len[seq], plus tail key j for every bit j of the row's mask.
 #pragma once
 #include "common.cuh"
 #include "rows.cuh"
@@ -57,7 +57,7 @@ struct FlatKV2 {
 };
 
 struct AttnMmaArgs {
-  const float *q;                   // [R][H][hd] fp32 queries (rotary applied), unscaled
+  const bf16 *q;                    // [R][H][2][hd] queries (rotary applied, unscaled): high row, low row
   const int *row_seq;               // [R] sequence of each row
   const int *row_in;                // [R] or null: rows with a negative entry are idle; index into anc
   const int *prefix_len;            // by sequence: keys [0, prefix) are visible to every row
@@ -68,7 +68,6 @@ struct AttnMmaArgs {
   float scale_log2;                 // softmax scale times log2(e)
   int n_chunks, blocks_per_chunk, n_rt;
   float *part_o, *part_ml;          // [slot][chunk][kvh][rt][64][hd], [..][64][2]
-  int *counters;                    // [slot][kvh][rt], zero between launches
   void *out;                        // [R][H*hd] rows in GEMM-input layout
   XLayout lay;
   PagedKV paged;                    // PAGED kernels
@@ -96,7 +95,6 @@ k_attn_mma(AttnMmaArgs a) {
   bf16 *Qh = reinterpret_cast<bf16 *>(am_smem), *Ql = Qh + AM_ROWS * LD, *KV = Ql + AM_ROWS * LD;
   uint32_t *mwords = reinterpret_cast<uint32_t *>(KV + 2 * BUF_ELEMS);          // [64][4]
   int *row_r = reinterpret_cast<int *>(mwords + AM_ROWS * 4), *row_h = row_r + AM_ROWS;
-  __shared__ int is_last;
   pdl_trigger();
   pdl_wait();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -131,16 +129,13 @@ k_attn_mma(AttnMmaArgs a) {
     for (int wd = 0; wd < 4; ++wd) mwords[tid * 4 + wd] = mw[wd];
   }
   __syncthreads();
-  // ---- queries: fp32 -> high and low bf16 rows in shared memory
-  for (int idx = tid; idx < AM_ROWS * (HD / 4); idx += AM_THREADS) {
-    int lr = idx / (HD / 4), c4 = idx - lr * (HD / 4);
+  // ---- queries: high and low rows copied asynchronously (joins the first K/V block's group)
+  for (int idx = tid; idx < AM_ROWS * (HD / 8); idx += AM_THREADS) {
+    int lr = idx / (HD / 8), sg = idx - lr * (HD / 8);
     int r = row_r[lr];
-    float4 v = r >= 0 ? ld_f4(a.q + ((long long)r * a.H + row_h[lr]) * HD + c4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    uint32_t h0, l0, h1, l1;
-    split_pair(v.x, v.y, h0, l0);
-    split_pair(v.z, v.w, h1, l1);
-    *reinterpret_cast<uint2 *>(Qh + lr * LD + c4 * 4) = make_uint2(h0, h1);
-    *reinterpret_cast<uint2 *>(Ql + lr * LD + c4 * 4) = make_uint2(l0, l1);
+    const bf16 *src = a.q + (r >= 0 ? ((long long)r * a.H + row_h[lr]) * 2 * HD + sg * 8 : 0);
+    cp_async16(smem_addr(Qh + lr * LD + sg * 8), src, r >= 0 ? 16 : 0);
+    cp_async16(smem_addr(Ql + lr * LD + sg * 8), src + (r >= 0 ? HD : 0), r >= 0 ? 16 : 0);
   }
 
   auto load_block = [&](int blk, int buf) {
@@ -180,7 +175,7 @@ k_attn_mma(AttnMmaArgs a) {
   const int k_row = l7 + (mi >> 1) * 8, k_col = (mi & 1) * 8;          // K fragments (non-transposed)
   const int v_row = l7 + (mi & 1) * 8, v_col = (mi >> 1) * 8;          // V fragments (transposed)
 
-  if (b0 < b1) load_block(b0, 0);
+  if (b0 < b1) load_block(b0, 0); else { cp_async_commit(); cp_async_wait<0>(); }
   for (int blk = b0; blk < b1; ++blk) {
     const int buf = (blk - b0) & 1;
     if (blk + 1 < b1) { load_block(blk + 1, buf ^ 1); cp_async_wait<1>(); } else cp_async_wait<0>();
@@ -309,39 +304,40 @@ k_attn_mma(AttnMmaArgs a) {
     for (int n = 0; n < NT_O; ++n) *reinterpret_cast<float2 *>(po + n * 8) = make_float2(o_acc[n][rs * 2], o_acc[n][rs * 2 + 1]);
     if (t == 0) *reinterpret_cast<float2 *>(a.part_ml + (pbase + lr) * 2) = make_float2(m_run[rs], l_run[rs]);
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    int *cnt = a.counters + ((long long)slot * Hkv + kvh) * a.n_rt + rt;
-    int old = atomicAdd(cnt, 1);
-    is_last = old == a.n_chunks - 1;
-    if (is_last) *cnt = 0;
+}
+
+// Merge of the chunk partials: out[r][h] = sum_c w_c O_c / sum_c w_c l_c with w_c = 2^(m_c - max m).
+// One thread per (row, head, four output columns); grid = ceil(R * H * hd / 4 / 256).
+template <int HD>
+__global__ void __launch_bounds__(256)
+k_attn_combine(AttnMmaArgs a, int R) {
+  pdl_trigger();
+  pdl_wait();
+  long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  int c4 = (int)(idx % (HD / 4));
+  long long rh = idx / (HD / 4);
+  int h = (int)(rh % a.H), r = (int)(rh / a.H);
+  if (r >= R) return;
+  if (a.row_in && a.row_in[r] < 0) return;
+  const int Hkv = a.H / a.G;
+  int slot = r / a.rows_per_seq, node = r - slot * a.rows_per_seq;
+  int kvh = h / a.G, rr = node * a.G + (h - kvh * a.G);
+  int rt = rr / AM_ROWS, lr = rr - rt * AM_ROWS;
+  const long long cstride = (long long)Hkv * a.n_rt * AM_ROWS;
+  const long long p0 = (((long long)slot * a.n_chunks * Hkv + kvh) * a.n_rt + rt) * AM_ROWS + lr;
+  float M = -INFINITY;
+  for (int c = 0; c < a.n_chunks; ++c) M = fmaxf(M, __ldcg(a.part_ml + (p0 + c * cstride) * 2));
+  float L = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int c = 0; c < a.n_chunks; ++c) {
+    long long pr = p0 + c * cstride;
+    float2 ml = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + pr * 2));
+    float4 o = __ldcg(reinterpret_cast<const float4 *>(a.part_o + pr * HD + c4 * 4));
+    float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+    L += ml.y * w;
+    acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
   }
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  // ---- merge the chunks of these 64 rows, in chunk order
-  const long long cstride = (long long)Hkv * a.n_rt * AM_ROWS;          // rows between chunks
-  const long long p0 = (((long long)slot * a.n_chunks * Hkv + kvh) * a.n_rt + rt) * AM_ROWS;
-  for (int idx = tid; idx < AM_ROWS * (HD / 4); idx += AM_THREADS) {
-    int lr = idx / (HD / 4), c4 = idx - lr * (HD / 4);
-    int r = row_r[lr];
-    if (r < 0) continue;
-    float M = -INFINITY;
-    for (int c = 0; c < a.n_chunks; ++c) M = fmaxf(M, __ldcg(a.part_ml + (p0 + c * cstride + lr) * 2));
-    float L = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = 0; c < a.n_chunks; ++c) {
-      long long pr = p0 + c * cstride + lr;
-      float2 ml = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + pr * 2));
-      if (ml.x == -INFINITY) continue;
-      float w = exp2f(ml.x - M);
-      float4 o = __ldcg(reinterpret_cast<const float4 *>(a.part_o + pr * HD + c4 * 4));
-      L += ml.y * w;
-      acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
-    }
-    float inv = L > 0.f ? 1.f / L : 0.f;
-    store_split4<bf16>(out + r * a.lay.row_stride + row_h[lr] * HD + c4 * 4, a.lay.lo_delta,
-                       make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
-  }
+  float inv = L > 0.f ? 1.f / L : 0.f;
+  store_split4<bf16>(reinterpret_cast<bf16 *>(a.out) + r * a.lay.row_stride + h * HD + c4 * 4, a.lay.lo_delta,
+                     make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
 }

@@ -107,6 +107,15 @@ __device__ __forceinline__ float4 ld_f4(const bf16 *p) {
   return make_float4(a.x, a.y, b.x, b.y);
 }
 
+// Query rows between the QKV post-processing and the attention kernels: one block of hd
+// values per (row, head): fp32 (fp32 configurations), or hd high parts then hd low parts in bf16
+// (bf16 configurations: what the tensor-core attention copies straight into shared memory).
+// Four bytes per element either way.  rh = row * H + head.
+__device__ __forceinline__ void q_store4(void *qbuf, int split, long long rh, int hd, int i, float4 v) {
+  if (split) store_split4<bf16>((bf16 *)qbuf + rh * 2 * hd + i, hd, v);
+  else *reinterpret_cast<float4 *>((float *)qbuf + rh * hd + i) = v;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -50,12 +50,12 @@ struct dream_ctx {
   RowMeta rm[2];
   int *gather_idx, *ctx_pos, *flags;
   uint32_t *vmask;
-  float *x, *x0, *qbuf, *gout, *lse_pre, *ent_pre, *ae, *scores_all, *taps_store, *tapbuf;
+  void *qbuf;                          // query rows, 4 bytes per element (see q_store4)
+  float *x, *x0, *gout, *lse_pre, *ent_pre, *ae, *scores_all, *taps_store, *tapbuf;
   void *xn, *raw, *act, *attn_out;
   float *top_val, *lse_rows, *margin_i;
   TopkScratch tks;
   float *am_part_o, *am_part_ml;       // split-K attention partials
-  int *am_counters;
   int am_rt_max;
   int key_ub[DREAM_MAX_BATCH];         // upper bound of the draft caches' permanent rows
   int tk_nsplit;
@@ -281,8 +281,7 @@ static size_t carve(dream_ctx *c, char *base) {
     size_t prow = (size_t)MB * AM_MAX_CHUNKS * f.n_kv_heads * c->am_rt_max * AM_ROWS;
     c->am_part_o = a.take<float>(prow * f.head_dim);
     c->am_part_ml = a.take<float>(prow * 2);
-    c->am_counters = a.take<int>((size_t)MB * f.n_kv_heads * c->am_rt_max);
-  } else { c->am_part_o = nullptr; c->am_part_ml = nullptr; c->am_counters = nullptr; }
+  } else { c->am_part_o = nullptr; c->am_part_ml = nullptr; }
   c->tk_nsplit = (f.vocab + TOPK_COLS - 1) / TOPK_COLS;
   c->tks.pv = a.take<float>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
   c->tks.pi = a.take<int>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
@@ -544,17 +543,21 @@ template <typename T, int HD> struct AttnLaunch {
   static void mma(dream_ctx *c, AttnMmaArgs a, int B, int rows_per_seq, int key_ub) {
     const dream_config &f = c->cfg;
     constexpr int KBLK = AmShape<HD>::KBLK;
-    a.q = c->qbuf; a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq;
+    a.q = (const bf16 *)c->qbuf; a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
     a.n_rt = (rows_per_seq * a.G + AM_ROWS - 1) / AM_ROWS;
     int nb_ub = imax(1, (key_ub + KBLK - 1) / KBLK), ctas = f.n_kv_heads * a.n_rt * B;
     int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, (2 * c->tc.n_sms + ctas - 1) / ctas));
     a.blocks_per_chunk = (nb_ub + want - 1) / want;
     a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
-    a.part_o = c->am_part_o; a.part_ml = c->am_part_ml; a.counters = c->am_counters;
+    a.part_o = c->am_part_o; a.part_ml = c->am_part_ml;
     a.out = c->attn_out;
     dim3 grid(a.n_chunks, f.n_kv_heads * a.n_rt, B);
     LAUNCH(c, (k_attn_mma<HD, PAGED>), grid, AM_THREADS, (attn_mma_smem<HD, PAGED>()), a);
+    if (a.n_chunks > 1) {
+      long long items = (long long)B * rows_per_seq * f.n_heads * (HD / 4);
+      LAUNCH(c, (k_attn_combine<HD>), (unsigned)((items + 255) / 256), 256, 0, a, B * rows_per_seq);
+    }
   }
   static void tree(dream_ctx *c, int layer, int R, XMode m, int B, int key_ub) {
     if (sizeof(T) == 2) {
@@ -793,7 +796,7 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
     g = gemm<T>(c, c->dw.xq, c->xn, xm, R, c->Hhd, d);
-    LAUNCH(c, k_gemm_to_f32, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, c->Hhd);
+    LAUNCH(c, k_gemm_to_q, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, f.n_heads, f.head_dim, sizeof(T) == 2 ? 1 : 0);
     HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm, B, m, key_ub));
     g = gemm<T>(c, c->dw.xo, c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, xm);

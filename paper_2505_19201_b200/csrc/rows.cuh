@@ -144,7 +144,7 @@ struct PagedKV {
 template <typename T>
 __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
                                   const int *__restrict__ row_pos, const int *__restrict__ row_slot,
-                                  int row0, float *qbuf, PagedKV kv, int H, const double *__restrict__ inv_freq) {
+                                  int row0, void *qbuf, PagedKV kv, int H, const double *__restrict__ inv_freq) {
   pdl_trigger();
   pdl_wait();
   int r = blockIdx.x + row0, lr = blockIdx.x;
@@ -162,9 +162,8 @@ __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
     float4 ra = make_float4(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1, a.z * c2 - b.z * s2, a.w * c3 - b.w * s3);
     float4 rb = make_float4(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1, b.z * c2 + a.z * s2, b.w * c3 + a.w * s3);
     if (hh < H) {
-      float *q = qbuf + ((long long)r * H + hh) * hd;
-      *reinterpret_cast<float4 *>(q + i) = ra;
-      *reinterpret_cast<float4 *>(q + i + half) = rb;
+      q_store4(qbuf, sizeof(T) == 2, (long long)r * H + hh, hd, i, ra);
+      q_store4(qbuf, sizeof(T) == 2, (long long)r * H + hh, hd, i + half, rb);
     } else {
       long long o = kv.off(seq, slot, hh - H);
       store_split4<T>(Kp + o + i, 0, ra);
@@ -197,7 +196,7 @@ struct FlatKV {
 // row_dst[r] (skipped when < 0).  Work items and grid as in k_qkv_post_target.
 __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
                                  const int *__restrict__ row_pos, const int *__restrict__ row_dst,
-                                 int row0, int has_q, float *qbuf, FlatKV kv, int H, const double *__restrict__ inv_freq) {
+                                 int row0, int has_q, void *qbuf, FlatKV kv, int H, const double *__restrict__ inv_freq) {
   pdl_trigger();
   pdl_wait();
   int r = blockIdx.x + row0, lr = blockIdx.x;
@@ -216,9 +215,8 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
     float4 ra = make_float4(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1, a.z * c2 - b.z * s2, a.w * c3 - b.w * s3);
     float4 rb = make_float4(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1, b.z * c2 + a.z * s2, b.w * c3 + a.w * s3);
     if (hh < Hq) {
-      float *o = qbuf + ((long long)r * H + hh) * hd;
-      *reinterpret_cast<float4 *>(o + i) = ra;
-      *reinterpret_cast<float4 *>(o + i + half) = rb;
+      q_store4(qbuf, kv.split, (long long)r * H + hh, hd, i, ra);
+      q_store4(qbuf, kv.split, (long long)r * H + hh, hd, i + half, rb);
     } else {
       long long o = kv.off(seq, 0, hh - Hq, dst);
       kv.store4(o, i, ra);
@@ -231,13 +229,15 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
   }
 }
 
-// Plain copy of a GEMM output [rows][width] into fp32 rows (q of the cross-attention: no rotary).
-// grid (rows, ceil(width / 1024)).
-__global__ void k_gemm_to_f32(GemmOut g, float *dst, int width) {
+// A GEMM output [rows][H * hd] becomes the query rows of the cross-attention (no rotary).
+// grid (rows, ceil(H * hd / 1024)).
+__global__ void k_gemm_to_q(GemmOut g, void *qbuf, int H, int hd, int split) {
   pdl_trigger();
   pdl_wait();
   int r = blockIdx.x, i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
-  if (i < width) *reinterpret_cast<float4 *>(dst + (long long)r * width + i) = gemm_val4(g, r, i);
+  if (i >= H * hd) return;
+  int h = i / hd;
+  q_store4(qbuf, split, (long long)r * H + h, hd, i - h * hd, gemm_val4(g, r, i));
 }
 
 // Cross-attention memory rows (Eq. 1: K = S W_K, V = S W_V): GEMM output [rows][2 H_kv hd]
