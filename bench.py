@@ -27,6 +27,10 @@ sys.path.insert(0, ROOT)
 
 from paper_2505_19201_b200 import configs, synth  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum per k_gemm_tc launch (mean over the launches of a
+# step) from an ncu capture of the current kernel; None until one has been taken (profiles/).
+TRAFFIC = {}
+
 METRIC = "verified_tree_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -170,7 +174,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
     B = p["batch"]
-    p["decode_steps"] = args.steps + args.warmup + 8 + 2 * args.steps   # room for every timed pass
+    p["decode_steps"] = args.steps + args.warmup + 16 + 2 * args.steps   # room for every timed pass
     twg, dwg = synth.target_weights(p, 0, dev), synth.draft_weights(p, 0, dev)
     cfg = api.make_config(p)
     ctx = api.Context(cfg, twg, dwg, dev)
@@ -243,10 +247,19 @@ def main():
     e1.record(stream)
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
-    # ---- dominant kernel: the weight-streaming GEMM, timed per launch with CUDA events
+    # ---- dominant kernel: the weight-streaming GEMM, each launch bracketed by CUDA events on the
+    # library's stream, in a pass of its own (the brackets keep its neighbours from overlapping it)
     gemm = None
-    if args.profile_gemm and hasattr(ctx, "dream_profile_gemm"):
-        gemm = ctx.dream_profile_gemm(one_step, args.steps)
+    if args.profile_gemm:
+        ctx.dream_gemm_timing(True)
+        nprof = max(1, min(args.steps, 8))
+        for _ in range(nprof):
+            one_step()
+        n_l, g_ms, g_bytes = ctx.dream_gemm_timing(False)
+        if n_l and g_ms > 0:
+            gemm = dict(kernel="k_gemm_tc", launches=n_l, launches_per_step=n_l / nprof, bytes_per_launch=g_bytes / n_l,
+                        us_per_launch=1e3 * g_ms / n_l, gbs=g_bytes / g_ms / 1e6, ms_per_step=g_ms / nprof,
+                        bytes_per_step=g_bytes / nprof)
     ms = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(ms, op=dist.ReduceOp.MAX)
@@ -271,9 +284,11 @@ def main():
                          h2d_bytes_per_step=4 * B, d2h_bytes_per_step=4 * B * (p["tree_depth"] + 2)))
     if gemm:
         line["roofline"] = dict(bound="hbm", achieved=gemm["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
-                                frac=gemm["gbs"] / pk["hbm_gbs"], traffic=None, peak_source=pk_src,
+                                frac=gemm["gbs"] / pk["hbm_gbs"], traffic=TRAFFIC.get(p["name"]), peak_source=pk_src,
                                 kernel=gemm["kernel"], launches_per_step=gemm["launches_per_step"],
-                                bytes_per_step=gemm["bytes_per_step"], ms_per_step=gemm["ms_per_step"])
+                                bytes_per_launch=gemm["bytes_per_launch"], us_per_launch=gemm["us_per_launch"],
+                                bytes_per_step=gemm["bytes_per_step"], ms_per_step=gemm["ms_per_step"],
+                                note="algorithmic bytes = weight bytes of each launch; duration = CUDA events around each launch")
     else:
         line["roofline"] = dict(bound="hbm", achieved=step_gbs, peak=pk["hbm_gbs"], unit="GB/s",
                                 frac=step_gbs / pk["hbm_gbs"], traffic=None, peak_source=pk_src, kernel="whole step")

@@ -198,6 +198,16 @@ dream_status dream_debug_gemm(dream_ctx *ctx, const void *W, const float *X, int
 /* How many GEMM launches so far went to the tensor-core kernel and to the CUDA-core kernel. */
 dream_status dream_gemm_counts(const dream_ctx *ctx, int64_t *tensor_core, int64_t *cuda_core);
 
+/* Per-launch timing of the weight-streaming GEMM, the kernel that moves nearly all of a step's
+ * bytes (Section 4 reports whole-step speed only; this is the measurement hook for the kernel's
+ * bandwidth).  on != 0: from now on every tensor-core GEMM launch is bracketed by two CUDA events
+ * on the context's stream (up to 8192 launches; the brackets keep neighbouring kernels from
+ * overlapping it, so use it in a pass of its own).  on == 0: stop, wait for the stream and
+ * return the number of timed launches, the sum of their durations in milliseconds and the
+ * weight bytes they streamed (HOST outputs, may be NULL). */
+dream_status dream_gemm_timing(dream_ctx *ctx, int32_t on, int64_t *launches, double *total_ms,
+                               double *weight_bytes);
+
 /* Forget a sequence (its pages return to the pool). */
 dream_status dream_seq_reset(dream_ctx *ctx, int32_t seq);
 

@@ -77,6 +77,7 @@ def lib():
             "dream_seq_reset": [vp, i32],
             "dream_debug_gemm": [vp, vp, vp, i32, i32, i32, i32, vp],
             "dream_gemm_counts": [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
+            "dream_gemm_timing": [vp, i32, C.POINTER(C.c_int64), C.POINTER(C.c_double), C.POINTER(C.c_double)],
             "dream_poll": [vp],
         }
         for name, args in sig.items():
@@ -269,6 +270,12 @@ class Context:
         a, b = C.c_int64(), C.c_int64()
         _check(self.h, lib().dream_gemm_counts(self.h, C.byref(a), C.byref(b)))
         return a.value, b.value
+
+    def dream_gemm_timing(self, on):
+        """on=True starts bracketing GEMM launches with events; on=False returns (launches, ms, bytes)."""
+        n, ms, by = C.c_int64(), C.c_double(), C.c_double()
+        _check(self.h, lib().dream_gemm_timing(self.h, 1 if on else 0, C.byref(n), C.byref(ms), C.byref(by)))
+        return n.value, ms.value, by.value
 
     def dream_seq_reset(self, seq):
         _check(self.h, lib().dream_seq_reset(self.h, seq))

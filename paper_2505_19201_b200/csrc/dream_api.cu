@@ -70,6 +70,10 @@ struct dream_ctx {
   int *h_stage;                        // pinned: page-table staging + step_host results
   long long launches, tc_launches, simt_launches;
   GemmTcPlan tc;
+  // per-launch timing of the weight-streaming GEMM (dream_gemm_timing)
+  int prof_on, prof_n;
+  double prof_bytes;
+  std::vector<cudaEvent_t> prof_ev;
   char err[256];
 };
 
@@ -337,9 +341,12 @@ static GemmOut gemm(dream_ctx *c, const void *W, const void *X, XMode m, int row
     for (int ch = 0; ch < nch; ++ch) {
       int rows_c = imin(chunk, rows - ch * chunk);
       const bf16 *Xc = (const bf16 *)X + (long long)ch * chunk * lay.row_stride;
+      bool timed = c->prof_on && 2 * (c->prof_n + 1) <= (int)c->prof_ev.size();
+      if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], c->stream);
       if (!gemm_tc_launch(&c->tc, c->stream, W, Xc, m.mode, m.lo_rows, rows_c, slot_rows, N, K, c->gout + (long long)ch * per,
                           (long long)c->gout_floats - (long long)ch * per, &g))
         c->gemm_failed = 1;
+      if (timed) { cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], c->stream); c->prof_n++; c->prof_bytes += 2.0 * N * K; }
       c->launches++;
       c->tc_launches++;
     }
@@ -418,6 +425,7 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   for (int b = 0; b < DREAM_MAX_BATCH; ++b) c->phase[b] = PH_EMPTY;
   c->prefill_seq = -1;
   c->launches = 0; c->tc_launches = 0; c->simt_launches = 0; c->gemm_failed = 0;
+  c->prof_on = 0; c->prof_n = 0; c->prof_bytes = 0.0;
   c->err[0] = 0;
   const char *pdl = getenv("DREAM_PDL");              // "0" serialises every launch (debugging aid)
   c->use_pdl = !(pdl && !strcmp(pdl, "0"));
@@ -439,6 +447,7 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
 extern "C" void dream_free(dream_ctx *c) {
   if (!c) return;
   cudaStreamSynchronize(c->stream);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   cudaFreeHost(c->h_stage);
   delete c;
 }
@@ -1024,6 +1033,32 @@ extern "C" dream_status dream_debug_gemm(dream_ctx *c, const void *W, const floa
   LAUNCH(c, k_gemm_collect, dim3((N + 255) / 256, rows), 256, 0, g, out, N);
   CUDA_OK(c, cudaGetLastError());
   if (c->gemm_failed) { c->gemm_failed = 0; return fail(c, DREAM_E_UNSUPPORTED, "the GEMM launch was refused (shape or output room)"); }
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_gemm_timing(dream_ctx *c, int32_t on, int64_t *launches, double *total_ms, double *weight_bytes) {
+  if (!c) return DREAM_E_ARG;
+  if (on) {
+    const int cap = 8192;                       // timed launches per measurement window
+    while ((int)c->prof_ev.size() < 2 * cap) {
+      cudaEvent_t e;
+      CUDA_OK(c, cudaEventCreate(&e));
+      c->prof_ev.push_back(e);
+    }
+    c->prof_on = 1; c->prof_n = 0; c->prof_bytes = 0.0;
+    return DREAM_OK;
+  }
+  c->prof_on = 0;
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  double ms = 0.0;
+  for (int i = 0; i < c->prof_n; ++i) {
+    float t = 0.f;
+    CUDA_OK(c, cudaEventElapsedTime(&t, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]));
+    ms += t;
+  }
+  if (launches) *launches = c->prof_n;
+  if (total_ms) *total_ms = ms;
+  if (weight_bytes) *weight_bytes = c->prof_bytes;
   return DREAM_OK;
 }
 
