@@ -208,6 +208,28 @@ dream_status dream_gemm_counts(const dream_ctx *ctx, int64_t *tensor_core, int64
 dream_status dream_gemm_timing(dream_ctx *ctx, int32_t on, int64_t *launches, double *total_ms,
                                double *weight_bytes);
 
+/* Top-k and log-sum-exp of a logits matrix with no arena and no allocation.  The paper has no
+ * counterpart to this call; it exists for callers that are not allowed to allocate device memory:
+ * a serving process that froze its memory pool after start-up, a plug-in that only gets the
+ * buffers its host hands it, or code that must not call cudaMalloc because that call
+ * synchronises the whole device.  It runs the library's k_topk_lse kernel (the one behind the
+ * LM heads of dream_draft_tree and dream_verify_tree) on a caller-owned matrix.
+ *   logits : device float [rows][vocab], row-major, 16-byte aligned
+ *   outputs: device top_val float [rows][ktop] (descending; equal values -> lower id first),
+ *            top_id int32 [rows][ktop], lse float [rows]
+ *   cuda_stream: a cudaStream_t of the current device (NULL = legacy default stream)
+ * The kernel's scratch (partial lists and counters) is a fixed ~1.1 MB array built into the
+ * library, held by every GPU that loads it until the process ends.  Limits: rows <= 128,
+ * vocab <= 262144, ktop <= 16; larger sizes return DREAM_E_CAPACITY and enqueue nothing.  The
+ * first call on each device looks the array's device address up (no allocation); make that call
+ * with the device current and before any stream capture.  All calls share the one array: it
+ * keeps the previous call's contents (the call clears the counters it needs at zero), and two
+ * calls whose kernels can overlap on the GPU (different streams, no ordering between them) race
+ * on it and give wrong results, so order them.  Asynchronous like the other calls; errors are
+ * reported through dream_last_error(NULL). */
+dream_status dream_topk_lse_static(const float *logits, int32_t rows, int32_t vocab, int32_t ktop,
+                                   float *top_val, int32_t *top_id, float *lse, void *cuda_stream);
+
 /* Forget a sequence (its pages return to the pool). */
 dream_status dream_seq_reset(dream_ctx *ctx, int32_t seq);
 

@@ -79,6 +79,7 @@ def lib():
             "dream_gemm_counts": [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
             "dream_gemm_timing": [vp, i32, C.POINTER(C.c_int64), C.POINTER(C.c_double), C.POINTER(C.c_double)],
             "dream_poll": [vp],
+            "dream_topk_lse_static": [vp, i32, i32, i32, vp, vp, vp, vp],
         }
         for name, args in sig.items():
             fn = getattr(L, name)
@@ -126,6 +127,17 @@ def dream_arena_bytes(cfg):
 def _check(ctx, code):
     if code != 0:
         raise DreamError(code, lib().dream_last_error(ctx).decode())
+
+
+def dream_topk_lse_static(logits, ktop, top_val, top_id, lse, stream=None):
+    """Top-k and log-sum-exp of a device float32 matrix [rows][vocab] through the entry point that
+    needs no arena (its scratch is built into the library).  Outputs are caller-allocated device
+    tensors: top_val [rows][ktop] float32, top_id [rows][ktop] int32, lse [rows] float32."""
+    rows, vocab = logits.shape
+    st = stream or torch.cuda.current_stream(logits.device)
+    with torch.cuda.device(logits.device):
+        _check(None, lib().dream_topk_lse_static(_ptr(logits), rows, vocab, ktop, _ptr(top_val), _ptr(top_id), _ptr(lse),
+                                                 C.c_void_p(st.cuda_stream)))
 
 
 class Tree:

@@ -1036,6 +1036,62 @@ extern "C" dream_status dream_debug_gemm(dream_ctx *c, const void *W, const floa
   return DREAM_OK;
 }
 
+// ------------------------------------------------------------------------------------- top-k without an arena
+
+// Scratch of dream_topk_lse_static: partial lists, (m, z) pairs and the per-row block counters of
+// k_topk_lse for up to NA_MAX_ROWS rows and NA_MAX_SPLIT vocabulary blocks.  It lives in the
+// library image, so every GPU that loads the library holds these ~1.1 MB until the process exits.
+#define NA_MAX_ROWS 128
+#define NA_MAX_SPLIT 64
+struct NaScratch {
+  float pv[NA_MAX_ROWS * NA_MAX_SPLIT * TOPK_MAX];
+  int pi[NA_MAX_ROWS * NA_MAX_SPLIT * TOPK_MAX];
+  float pm[NA_MAX_ROWS * NA_MAX_SPLIT];
+  float pz[NA_MAX_ROWS * NA_MAX_SPLIT];
+  int counter[NA_MAX_ROWS];
+};
+static __device__ __align__(256) unsigned char g_na_scratch[sizeof(NaScratch)];
+// In host code g_na_scratch is only a handle; the address a kernel can use comes from
+// cudaGetSymbolAddress, looked up once per device.
+#define NA_MAX_DEVICES 64
+static NaScratch *g_na_dev_ptr[NA_MAX_DEVICES];
+
+extern "C" dream_status dream_topk_lse_static(const float *logits, int32_t rows, int32_t vocab, int32_t ktop,
+                                              float *top_val, int32_t *top_id, float *lse, void *cuda_stream) {
+  if (!logits || !top_val || !top_id || !lse) return fail(nullptr, DREAM_E_ARG, "dream_topk_lse_static: null buffer");
+  if (rows < 1 || rows > NA_MAX_ROWS)
+    return fail(nullptr, DREAM_E_CAPACITY, "dream_topk_lse_static: rows = %d outside 1..%d (the built-in scratch is fixed)", rows, NA_MAX_ROWS);
+  if (vocab < 2 || vocab > NA_MAX_SPLIT * TOPK_COLS)
+    return fail(nullptr, DREAM_E_CAPACITY, "dream_topk_lse_static: vocab = %d outside 2..%d (the built-in scratch is fixed)", vocab, NA_MAX_SPLIT * TOPK_COLS);
+  if (ktop < 1 || ktop > TOPK_MAX || ktop > vocab)
+    return fail(nullptr, DREAM_E_ARG, "dream_topk_lse_static: ktop = %d outside 1..%d", ktop, TOPK_MAX);
+  if ((uintptr_t)logits & 15) return fail(nullptr, DREAM_E_ARG, "dream_topk_lse_static: logits must be 16-byte aligned");
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(nullptr, DREAM_E_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= NA_MAX_DEVICES) return fail(nullptr, DREAM_E_UNSUPPORTED, "device ordinal %d not supported", dev);
+  if (!g_na_dev_ptr[dev]) {                    // first call on this device, with it current
+    void *ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_na_scratch);
+    if (e != cudaSuccess || !ptr) return fail(nullptr, DREAM_E_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+    g_na_dev_ptr[dev] = (NaScratch *)ptr;
+  }
+  NaScratch *sc = g_na_dev_ptr[dev];
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  // the scratch keeps whatever the last call left: only the block counters have to start at zero
+  e = cudaMemsetAsync(sc->counter, 0, sizeof(int) * rows, stream);
+  if (e != cudaSuccess) return fail(nullptr, DREAM_E_CUDA, "clearing the counters: %s", cudaGetErrorString(e));
+  TopkScratch ts;
+  ts.pv = sc->pv; ts.pi = sc->pi; ts.pm = sc->pm; ts.pz = sc->pz; ts.counter = sc->counter;
+  GemmOut g;                                   // a plain [rows][vocab] matrix: one slot, one chunk
+  g.base = logits; g.slot_stride = 0; g.chunk_stride = 0; g.chunk_shift = 30; g.ld = vocab; g.kb = 0; g.upc = 0;
+  int nsplit = (vocab + TOPK_COLS - 1) / TOPK_COLS;
+  k_topk_lse<<<dim3(rows, nsplit), TOPK_THREADS, 0, stream>>>(g, vocab, ktop, nsplit, ts, top_val, top_id, lse, (float *)nullptr);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(nullptr, DREAM_E_CUDA, "k_topk_lse launch: %s", cudaGetErrorString(e));
+  return DREAM_OK;
+}
+
 extern "C" dream_status dream_gemm_timing(dream_ctx *c, int32_t on, int64_t *launches, double *total_ms, double *weight_bytes) {
   if (!c) return DREAM_E_ARG;
   if (on) {
