@@ -230,6 +230,17 @@ dream_status dream_gemm_timing(dream_ctx *ctx, int32_t on, int64_t *launches, do
 dream_status dream_topk_lse_static(const float *logits, int32_t rows, int32_t vocab, int32_t ktop,
                                    float *top_val, int32_t *top_id, float *lse, void *cuda_stream);
 
+/* Timeline of the context's stream (a measurement hook; Section 4 times whole steps only).
+ * buffer: DEVICE array of 2 + 2 * capacity_entries 64-bit words, or NULL to stop tracing.  While
+ * installed, every kernel of the library appends (kernel id, nanosecond timer) at the moment its
+ * predecessor in the stream has completed; word 0 counts the entries.  Differences between
+ * consecutive entries give each kernel's time on the critical path, overlap included.  The
+ * buffer is process-wide (one traced context at a time).  Synchronises the stream. */
+dream_status dream_trace(dream_ctx *ctx, unsigned long long *buffer, int64_t capacity_entries);
+
+/* Name of a kernel id found in a trace buffer.  Host-only. */
+const char *dream_trace_name(int32_t id);
+
 /* Forget a sequence (its pages return to the pool). */
 dream_status dream_seq_reset(dream_ctx *ctx, int32_t seq);
 

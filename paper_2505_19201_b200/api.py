@@ -79,6 +79,7 @@ def lib():
             "dream_gemm_counts": [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)],
             "dream_gemm_timing": [vp, i32, C.POINTER(C.c_int64), C.POINTER(C.c_double), C.POINTER(C.c_double)],
             "dream_poll": [vp],
+            "dream_trace": [vp, vp, C.c_int64],
             "dream_topk_lse_static": [vp, i32, i32, i32, vp, vp, vp, vp],
         }
         for name, args in sig.items():
@@ -87,6 +88,7 @@ def lib():
         L.dream_launch_count.argtypes, L.dream_launch_count.restype = [vp], C.c_int64
         L.dream_last_error.argtypes, L.dream_last_error.restype = [vp], C.c_char_p
         L.dream_free.argtypes, L.dream_free.restype = [vp], None
+        L.dream_trace_name.argtypes, L.dream_trace_name.restype = [i32], C.c_char_p
         _LIB = L
     return _LIB
 
@@ -288,6 +290,17 @@ class Context:
         n, ms, by = C.c_int64(), C.c_double(), C.c_double()
         _check(self.h, lib().dream_gemm_timing(self.h, 1 if on else 0, C.byref(n), C.byref(ms), C.byref(by)))
         return n.value, ms.value, by.value
+
+    def dream_trace(self, capacity=0):
+        """capacity > 0: start a timeline of this context's stream; 0: stop and return [(kernel, ns)]."""
+        if capacity:
+            self._trace = torch.zeros(2 + 2 * capacity, dtype=torch.int64, device=self.device)
+            _check(self.h, lib().dream_trace(self.h, C.c_void_p(self._trace.data_ptr()), capacity))
+            return None
+        _check(self.h, lib().dream_trace(self.h, None, 0))
+        t = self._trace.cpu().tolist()
+        n = min(t[0], t[1])
+        return [(lib().dream_trace_name(int(t[2 + 2 * i])).decode(), t[3 + 2 * i]) for i in range(n)]
 
     def dream_seq_reset(self, seq):
         _check(self.h, lib().dream_seq_reset(self.h, seq))

@@ -91,8 +91,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
                T *attn_out, XLayout lay, float *lse, float *ent) {
   constexpr int EPL = HD / 32;
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_attn_prefill);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int i = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (i >= n) return;
@@ -123,8 +122,7 @@ k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H,
 // AE(l) = mean over rows and heads of the row entropies (Eq. 2).  One block, fixed order.
 __global__ void k_entropy_mean(const float *__restrict__ ent, int count, float *out) {
   __shared__ float sh[33];
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_entropy_mean);
   float s = 0.f;
   for (int i = threadIdx.x; i < count; i += blockDim.x) s += ent[i];
   float t = block_sum(s, sh);
@@ -139,8 +137,7 @@ __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_colsum(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
          const float *__restrict__ lse, int vis_start, int v, int include_self, float *score) {
   constexpr int EPL = HD / 32;
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_colsum);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int jv = blockIdx.x * ATT_WARPS + w;
   if (jv >= v) return;
@@ -173,8 +170,7 @@ k_attn_tree(const void *__restrict__ qbuf, PagedKV kv, const int *__restrict__ r
             const uint32_t *__restrict__ mask, int R, int T_nodes, int H, float scale, T *attn_out,
             XLayout lay) {
   constexpr int EPL = HD / 32;
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_attn_tree);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (r >= R) return;
@@ -220,8 +216,7 @@ k_attn_draft(const void *__restrict__ qbuf, FlatKV kv, const int *__restrict__ r
              const unsigned long long *__restrict__ anc, int anc_stride, int strict, int R, int H,
              float scale, T *attn_out, XLayout lay) {
   constexpr int EPL = HD / 32;
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_attn_draft);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (r >= R) return;

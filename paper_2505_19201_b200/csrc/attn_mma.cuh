@@ -95,8 +95,7 @@ k_attn_mma(AttnMmaArgs a) {
   bf16 *Qh = reinterpret_cast<bf16 *>(am_smem), *Ql = Qh + AM_ROWS * LD, *KV = Ql + AM_ROWS * LD;
   uint32_t *mwords = reinterpret_cast<uint32_t *>(KV + 2 * BUF_ELEMS);          // [64][4]
   int *row_r = reinterpret_cast<int *>(mwords + AM_ROWS * 4), *row_h = row_r + AM_ROWS;
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_attn_mma);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int chunk = blockIdx.x, kvh = blockIdx.y / a.n_rt, rt = blockIdx.y - kvh * a.n_rt, slot = blockIdx.z;
   const int Hkv = a.H / a.G;
@@ -311,8 +310,7 @@ k_attn_mma(AttnMmaArgs a) {
 template <int HD>
 __global__ void __launch_bounds__(256)
 k_attn_combine(AttnMmaArgs a, int R) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_attn_combine);
   long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   int c4 = (int)(idx % (HD / 4));
   long long rh = idx / (HD / 4);

@@ -25,6 +25,71 @@ template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __flo
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Optional timeline of a stream: when a trace buffer is installed (dream_trace), thread 0 of block
+// 0 of every kernel appends (kernel id, %globaltimer) right after its grid dependency resolved,
+// i.e. when its predecessor has completed.  Differences between consecutive entries are the
+// critical-path time of each kernel as it runs in the stream, overlap included.  Layout of the
+// buffer: word 0 = entries written, word 1 = capacity, then pairs (id, nanoseconds).
+__device__ unsigned long long *g_dream_trace;
+enum {
+  TR_none = 0,
+  TR_k_embed,
+  TR_k_build_prompt,
+  TR_k_resid_norm,
+  TR_k_qkv_post_target,
+  TR_k_qkv_post_draft,
+  TR_k_gemm_to_q,
+  TR_k_mem_append,
+  TR_k_silu_mul,
+  TR_k_resid_add,
+  TR_k_gather_rows,
+  TR_k_topk_lse,
+  TR_k_attn_prefill,
+  TR_k_entropy_mean,
+  TR_k_colsum,
+  TR_k_attn_tree,
+  TR_k_attn_draft,
+  TR_k_attn_mma,
+  TR_k_attn_combine,
+  TR_k_draft_begin,
+  TR_k_tree_expand,
+  TR_k_tree_finalize,
+  TR_k_verify_setup,
+  TR_k_accept,
+  TR_k_compact_kv,
+  TR_k_accept_rows,
+  TR_k_select_tap,
+  TR_k_select_visual,
+  TR_k_ctx_rows,
+  TR_k_gemm_simt,
+  TR_k_iota_rows,
+  TR_k_set_seq,
+  TR_k_set_int,
+  TR_k_first_token,
+  TR_k_argmax_out,
+  TR_k_copy_f32,
+  TR_k_split_rows,
+  TR_k_gemm_collect,
+  TR_k_gemm_tc,
+  TR_count
+};
+#define DREAM_TRACE_NAMES {"none", "k_embed", "k_build_prompt", "k_resid_norm", "k_qkv_post_target", "k_qkv_post_draft", "k_gemm_to_q", "k_mem_append", "k_silu_mul", "k_resid_add", "k_gather_rows", "k_topk_lse", "k_attn_prefill", "k_entropy_mean", "k_colsum", "k_attn_tree", "k_attn_draft", "k_attn_mma", "k_attn_combine", "k_draft_begin", "k_tree_expand", "k_tree_finalize", "k_verify_setup", "k_accept", "k_compact_kv", "k_accept_rows", "k_select_tap", "k_select_visual", "k_ctx_rows", "k_gemm_simt", "k_iota_rows", "k_set_seq", "k_set_int", "k_first_token", "k_argmax_out", "k_copy_f32", "k_split_rows", "k_gemm_collect", "k_gemm_tc"}
+__device__ __forceinline__ void trace_stamp(int id) {
+  unsigned long long *tr = g_dream_trace;
+  if (tr) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    unsigned long long i = atomicAdd(tr, 1ull);
+    if (i < tr[1]) { tr[2 + 2 * i] = (unsigned long long)id; tr[3 + 2 * i] = t; }
+  }
+}
+// Entry of every kernel of the library: let the successor start, wait for the predecessor.
+__device__ __forceinline__ void kernel_entry(int id) {
+  pdl_trigger();
+  pdl_wait();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) trace_stamp(id);
+}
+
 // A bf16 GEMM input row is stored as two bf16 rows, hi = bf16(v) and lo = bf16(v - hi), so the
 // tensor cores see the activation to ~16 mantissa bits while the weights stream once.  fp32
 // inputs have no lo part.  XLayout says where the rows of such a buffer live: token t starts at

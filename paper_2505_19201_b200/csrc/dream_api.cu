@@ -484,35 +484,30 @@ extern "C" dream_status dream_seq_reset(dream_ctx *c, int32_t seq) {
 // ------------------------------------------------------------------------------------- small kernels
 
 __global__ void k_iota_rows(RowMeta rm, int seq, int n) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_iota_rows);
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   rm.seq[i] = seq; rm.pos[i] = i; rm.slot[i] = i; rm.dst[i] = i; rm.in[i] = -1;
 }
 __global__ void k_set_seq(SeqDev s, int seq, int P, const int *pending_src, int nd, int nm) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_set_seq);
   if (threadIdx.x) return;
   if (P >= 0) s.P[seq] = P;
   if (pending_src) s.pending[seq] = *pending_src;
   if (nd >= 0) { s.nperm_d[seq] = nd; s.nperm_m[seq] = nm; s.n_new[seq] = 0; }
 }
 __global__ void k_set_int(int *p, int v) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_set_int);
   if (!threadIdx.x) *p = v;
 }
 __global__ void k_first_token(const int *top_id, const float *top_val, int *tok, float *margin) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_first_token);
   if (threadIdx.x) return;
   if (tok) *tok = top_id[0];
   if (margin) *margin = top_val[0] - top_val[1];
 }
 __global__ void k_argmax_out(const int *top_id, const float *top_val, int R, int *am, float *mg, int *am2) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_argmax_out);
   int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= R) return;
   am[r] = top_id[2 * r];
@@ -520,8 +515,7 @@ __global__ void k_argmax_out(const int *top_id, const float *top_val, int R, int
   if (mg) mg[r] = top_val[2 * r] - top_val[2 * r + 1];
 }
 __global__ void k_copy_f32(const float *src, float *dst, int n) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_copy_f32);
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src[i];
 }
@@ -797,7 +791,7 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     const XMode xm = xmode(c, R);
     RowMeta &rm = c->rm[cur], &rn = c->rm[cur ^ 1];
     if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
-    LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
+    LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
     norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
     GemmOut g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
     LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
@@ -849,7 +843,7 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
   int key_ub = 0;
   for (int b = 0; b < B; ++b) key_ub = imax(key_ub, c->p_ub[tb.seq[b]] + c->T);
   LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
-  LAUNCH(c, (k_embed<T>), R, 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
+  LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
   GemmOut gd = NO_GEMM;
   for (int l = 0; l < L; ++l) {
     // completes S^l (for l >= 1) and captures it where a sequence taps layer l
@@ -994,8 +988,7 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
 
 // out[r][c] = sum_k X[r][k] W[c][k] through the context's GEMM path (test hook).
 __global__ void k_split_rows(const float *src, void *dst, int K, XLayout lay, int is_bf16) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_split_rows);
   int r = blockIdx.x;
   for (int i = threadIdx.x; i < K; i += blockDim.x) {
     float v = src[(long long)r * K + i];
@@ -1004,8 +997,7 @@ __global__ void k_split_rows(const float *src, void *dst, int K, XLayout lay, in
   }
 }
 __global__ void k_gemm_collect(GemmOut g, float *dst, int N) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_gemm_collect);
   int r = blockIdx.y, c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c < N) dst[(long long)r * N + c] = gemm_val(g, r, c);
 }
@@ -1090,6 +1082,26 @@ extern "C" dream_status dream_topk_lse_static(const float *logits, int32_t rows,
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(nullptr, DREAM_E_CUDA, "k_topk_lse launch: %s", cudaGetErrorString(e));
   return DREAM_OK;
+}
+
+static const char *const g_trace_names[] = DREAM_TRACE_NAMES;
+
+extern "C" dream_status dream_trace(dream_ctx *c, unsigned long long *buffer, int64_t capacity_entries) {
+  if (!c) return DREAM_E_ARG;
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  unsigned long long *ptr = nullptr;
+  if (buffer) {
+    if (capacity_entries < 1) return fail(c, DREAM_E_ARG, "trace capacity");
+    unsigned long long head[2] = {0ull, (unsigned long long)capacity_entries};
+    CUDA_OK(c, cudaMemcpy(buffer, head, sizeof(head), cudaMemcpyHostToDevice));
+    ptr = buffer;
+  }
+  CUDA_OK(c, cudaMemcpyToSymbol(g_dream_trace, &ptr, sizeof(ptr)));
+  return DREAM_OK;
+}
+
+extern "C" const char *dream_trace_name(int32_t id) {
+  return id >= 0 && id < TR_count ? g_trace_names[id] : "?";
 }
 
 extern "C" dream_status dream_gemm_timing(dream_ctx *c, int32_t on, int64_t *launches, double *total_ms, double *weight_bytes) {

@@ -14,8 +14,7 @@ k_gemm_simt(const T *__restrict__ X, const T *__restrict__ W, float *__restrict_
             int N, int K, int ldo) {
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float Bs[SG_BK][SG_BN + 4];
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_gemm_simt);
   int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   int r0 = blockIdx.y * SG_BM, c0 = blockIdx.x * SG_BN;
   int lr = threadIdx.x >> 2, lk = (threadIdx.x & 3) * 4;

@@ -18,9 +18,10 @@
 //     consumer adds the slots in a fixed order;
 //   * programmatic dependent launch: W never changes, so its ring fills before the grid
 //     dependency resolves; only the X producer and the epilogue wait for the previous kernel;
-//   * warp roles: 0 = W producer, 1 = MMA issuer and TMEM owner, 2..5 = epilogue (tcgen05.ld ->
-//     128-bit stores), 6 = X producer; two TMEM accumulators alternate so that the epilogue of one
-//     segment overlaps the MMAs of the next;
+//   * warp roles: 0 = W producer, 1 = MMA issuer and TMEM owner, 6 = X producer, 2..5 and 7..10 =
+//     epilogue (tcgen05.ld -> 128-bit stores; the first set drains accumulator columns 0..127, the
+//     second 128..255, loads software-pipelined); two TMEM accumulators alternate so that the
+//     epilogue of one segment overlaps the MMAs of the next;
 //   * every mbarrier wait is bounded: on expiry the kernel raises the status word and leaves.
 #pragma once
 #include <cuda.h>
@@ -34,7 +35,7 @@
 
 #define TC_BN 256               // weight rows per tile (MMA N)
 #define TC_BK 64                // k elements per panel (128 bytes: one swizzle row)
-#define TC_THREADS 224
+#define TC_THREADS 352             // 11 warps, see the roles below
 #define TC_SPIN_LIMIT (1u << 24)
 #define TC_WPANEL (TC_BN * TC_BK * 2)
 #define TC_XTILE (128 * TC_BK * 2)
@@ -146,10 +147,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   const int u_end = min(u_begin + p.upc, p.total_units);
   const bool has_work = u_begin < u_end;
 
+  if (blockIdx.x == 0 && threadIdx.x == 0) trace_stamp(TR_none);     // CTA start, before any dependency
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.w_stages; ++s) { mbar_init(full_w + s, 1); mbar_init(empty_w + s, 1); }
     for (int s = 0; s < p.x_stages; ++s) { mbar_init(full_x + s, 1); mbar_init(empty_x + s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -250,9 +252,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         if (!ok) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
       }
     } else {
-      // ------------------------------------------------------------------ epilogue warps 2..5
+      // ------------------------------------------------------------------ epilogue warps 2..5, 7..10
       const int q = warp & 3;                   // TMEM lane quarter this warp may read
+      const int half = warp >= 7 ? 1 : 0;       // which 128 accumulator columns this warp drains
       pdl_wait();                               // the output buffer is read by the previous kernel
+      if (blockIdx.x == 0 && warp == 2 && lane == 0) trace_stamp(TR_k_gemm_tc);
       const bool inter = p.x_mode == TC_X_INTERLEAVED;
       const int row = q * 32 + lane;            // accumulator lane = X row
       const int token = inter ? row >> 1 : row;
@@ -272,26 +276,32 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         int slot = (int)blockIdx.x - first_cta;
         float *dst = p.out + (long long)slot * p.slot_stride + (long long)token * p.N + tile * TC_BN;
         uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * TC_BN;
-        for (int col0 = 0; col0 < TC_BN; col0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(taddr + (uint32_t)col0, r);
-          tmem_ld_wait();
-          if (inter) {
-            // lanes 2t and 2t+1 hold the products of token t's high and low parts: add them;
-            // both lanes then hold the sum and each stores half of the 32 columns
-            float v[32];
+        // four chunks of 32 columns; the TMEM load of chunk i+1 is in flight while chunk i is stored
+        uint32_t ra[32], rb[32];
+        tmem_ld32(taddr + (uint32_t)half * 128u, ra);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              float a = __uint_as_float(r[j]);
-              v[j] = a + __shfl_xor_sync(0xffffffffu, a, 1);
+        for (int ci = 0; ci < 4; ++ci) {
+          const int col0 = half * 128 + ci * 32;
+          uint32_t (&r)[32] = (ci & 1) ? rb : ra;
+          tmem_ld_wait();
+          if (ci + 1 < 4) tmem_ld32(taddr + (uint32_t)(col0 + 32), (ci & 1) ? ra : rb);
+          if (inter) {
+            // lanes 2t and 2t+1 hold the products of token t's high and low parts.  The even lane
+            // stores columns 0..15 of the chunk and the odd lane 16..31: each sends the partner
+            // the 16 values it needs and adds what it receives to its own.
+            float v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              float send = __uint_as_float(part ? r[j] : r[16 + j]);
+              float mine = __uint_as_float(part ? r[16 + j] : r[j]);
+              v[j] = mine + __shfl_xor_sync(0xffffffffu, send, 1);
             }
             if (token < p.n_tok) {
 #pragma unroll
               for (int j4 = 0; j4 < 4; ++j4) {
                 int jj = part * 16 + j4 * 4;
-                float4 o = part ? make_float4(v[16 + j4 * 4], v[17 + j4 * 4], v[18 + j4 * 4], v[19 + j4 * 4])
-                                : make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
-                if (tile * TC_BN + col0 + jj < p.N) *reinterpret_cast<float4 *>(dst + col0 + jj) = o;
+                if (tile * TC_BN + col0 + jj < p.N)
+                  *reinterpret_cast<float4 *>(dst + col0 + jj) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
               }
             }
           } else if (token < p.n_tok) {
@@ -410,7 +420,7 @@ static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const voi
   if (p.wp > p.KB) p.wp = p.KB;
   if (p.KB % p.wp == 0) p.upc = (p.upc + p.wp - 1) / p.wp * p.wp;   // CTA ranges cover whole W stages
   grid = (p.total_units + p.upc - 1) / p.upc;
-  p.x_stages = 2;
+  p.x_stages = x_mode == TC_X_PLANAR ? 2 : 4;
   int xstage = x_mode == TC_X_PLANAR ? 2 * TC_XTILE : TC_XTILE;
   int budget = pl->max_smem - 2048 - p.x_stages * xstage;
   p.w_stages = budget / (p.wp * TC_WPANEL);

@@ -6,16 +6,17 @@
 #include "common.cuh"
 
 // ---------------------------------------------------------------------------------------
-// x[r] = embed[tok[r]] (fp32 residual stream).  tok < 0 leaves a zero row.
+// x[r] = embed[tok[r]] (fp32 residual stream).  tok < 0 leaves a zero row.  One thread per four
+// elements: grid (rows, ceil(d / 1024)).
 template <typename T>
 __global__ void k_embed(const T *__restrict__ embed, const int *__restrict__ tok, float *x, int d,
                         int vocab, int *status) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_embed);
   int r = blockIdx.x, t = tok[r];
-  if (t >= vocab) { if (threadIdx.x == 0) atomicMax(status, DREAM_DEV_BAD_INDEX); t = -1; }
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    x[(long long)r * d + i] = t >= 0 ? to_f(embed[(long long)t * d + i]) : 0.f;
+  int i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+  if (t >= vocab) { if (threadIdx.x == 0 && blockIdx.y == 0) atomicMax(status, DREAM_DEV_BAD_INDEX); t = -1; }
+  if (i >= d) return;
+  *reinterpret_cast<float4 *>(x + (long long)r * d + i) = t >= 0 ? ld_f4(embed + (long long)t * d + i) : make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 // Prompt input rows of the prefill: visual embeddings inside [vis_start, vis_start+v),
@@ -24,8 +25,7 @@ template <typename T>
 __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict__ visual,
                                const int *__restrict__ ids, int vis_start, int v, float *x,
                                float *x0, int d, int vocab, int *status) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_build_prompt);
   int r = blockIdx.x;
   const T *src;
   if (r >= vis_start && r < vis_start + v) src = visual + (long long)(r - vis_start) * d;
@@ -54,9 +54,15 @@ k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
              float eps, int d, T *xn, float *copy, const int *row_seq,
              const int *tap_state, int layer, T *raw, XLayout lay) {
   __shared__ float sh[33];
-  pdl_trigger();
-  pdl_wait();
   int r = blockIdx.x, d4 = d >> 2;
+  // the gains are weights: they can be fetched before the predecessor has finished
+  float4 gq[NORM_NV];
+#pragma unroll
+  for (int j = 0; j < NORM_NV; ++j) {
+    int i = threadIdx.x + j * NORM_THREADS;
+    gq[j] = (xn && i < d4) ? ld_f4(gain + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  kernel_entry(TR_k_resid_norm);
   float *xr = x + (long long)r * d;
   float4 v[NORM_NV];
   float ss = 0.f;
@@ -94,21 +100,20 @@ k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
   float tot = block_sum(ss, sh);
   float inv = rsqrtf(tot / (float)d + eps);
   bool do_copy = copy != nullptr && (tap_state == nullptr || tap_state[row_seq[r]] == layer);
-  auto emit = [&](int i, float4 t) {
+  auto emit = [&](int i, float4 t, float4 gv) {
     if (do_copy) *reinterpret_cast<float4 *>(copy + (long long)r * d + 4 * i) = t;
     if (raw) store_split4<T>(raw + r * lay.row_stride + 4 * i, lay.lo_delta, t);
-    if (xn) {
-      float4 gq = ld_f4(gain + 4 * i);
+    if (xn)
       store_split4<T>(xn + r * lay.row_stride + 4 * i, lay.lo_delta,
-                      make_float4(t.x * inv * gq.x, t.y * inv * gq.y, t.z * inv * gq.z, t.w * inv * gq.w));
-    }
+                      make_float4(t.x * inv * gv.x, t.y * inv * gv.y, t.z * inv * gv.z, t.w * inv * gv.w));
   };
 #pragma unroll
   for (int j = 0; j < NORM_NV; ++j) {
     int i = threadIdx.x + j * NORM_THREADS;
-    if (i < d4) emit(i, v[j]);
+    if (i < d4) emit(i, v[j], gq[j]);
   }
-  for (int i = threadIdx.x + NORM_NV * NORM_THREADS; i < d4; i += NORM_THREADS) emit(i, ld_f4(xr + 4 * i));
+  for (int i = threadIdx.x + NORM_NV * NORM_THREADS; i < d4; i += NORM_THREADS)
+    emit(i, ld_f4(xr + 4 * i), xn ? ld_f4(gain + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -145,8 +150,7 @@ template <typename T>
 __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
                                   const int *__restrict__ row_pos, const int *__restrict__ row_slot,
                                   int row0, void *qbuf, PagedKV kv, int H, const double *__restrict__ inv_freq) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_qkv_post_target);
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int hd = kv.hd, half = hd >> 1, q4 = half >> 2, Hkv = kv.hkv;
   int w = blockIdx.y * blockDim.x + threadIdx.x;
@@ -197,8 +201,7 @@ struct FlatKV {
 __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
                                  const int *__restrict__ row_pos, const int *__restrict__ row_dst,
                                  int row0, int has_q, void *qbuf, FlatKV kv, int H, const double *__restrict__ inv_freq) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_qkv_post_draft);
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int hd = kv.hd, half = hd >> 1, q4 = half >> 2, Hkv = kv.hkv;
   int Hq = has_q ? H : 0;
@@ -232,8 +235,7 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
 // A GEMM output [rows][H * hd] becomes the query rows of the cross-attention (no rotary).
 // grid (rows, ceil(H * hd / 1024)).
 __global__ void k_gemm_to_q(GemmOut g, void *qbuf, int H, int hd, int split) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_gemm_to_q);
   int r = blockIdx.x, i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
   if (i >= H * hd) return;
   int h = i / hd;
@@ -247,8 +249,7 @@ __global__ void k_gemm_to_q(GemmOut g, void *qbuf, int H, int hd, int split) {
 __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
                              const int *__restrict__ row_dst, const int *__restrict__ row_in,
                              const int *__restrict__ nperm, int row0, FlatKV kv) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_mem_append);
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int seq = row_seq[r];
   int dst = nperm ? (row_in[r] < 0 ? -1 : nperm[seq] + row_in[r]) : row_dst[r];
@@ -265,8 +266,7 @@ __global__ void k_mem_append(GemmOut g, const int *__restrict__ row_seq,
 // grid (ceil(ff / 1024), rows).
 template <typename T>
 __global__ void k_silu_mul(GemmOut g, T *act, int ff, XLayout lay) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_silu_mul);
   int r = blockIdx.y;
   int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= ff) return;
@@ -279,8 +279,7 @@ __global__ void k_silu_mul(GemmOut g, T *act, int ff, XLayout lay) {
 // x += GEMM output; optional fp32 copy into a per-layer store (prefill tap candidates).
 // grid (rows, ceil(d / 1024)).
 __global__ void k_resid_add(float *x, GemmOut g, int d, float *copy) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_resid_add);
   int r = blockIdx.x, i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
   if (i >= d) return;
   float4 v = ld_f4(x + (long long)r * d + i), t = gemm_val4(g, r, i);
@@ -294,8 +293,7 @@ template <typename T>
 __global__ void k_gather_rows(const float *__restrict__ src, const int *__restrict__ idx, T *dst,
                               int d, const int *layer_ptr, int layer_lo, long long layer_stride,
                               XLayout lay) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_gather_rows);
   int r = blockIdx.x, s = idx[r];
   if (layer_ptr) src += (long long)(*layer_ptr - layer_lo) * layer_stride;
   for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4)
@@ -306,11 +304,13 @@ __global__ void k_gather_rows(const float *__restrict__ src, const int *__restri
 // ---------------------------------------------------------------------------------------
 // Per row of a [rows][V] GEMM output: the KTOP largest logits (ties -> lower id), in
 // descending order, and the log-sum-exp of the row.  grid (rows, nsplit): block (r, sp) scans
-// columns [sp * TOPK_COLS, (sp + 1) * TOPK_COLS) and leaves a sorted partial list and an (m, z)
-// pair; the block that finishes a row last merges the partials, always in the same order.
+// columns [sp * TOPK_COLS, (sp + 1) * TOPK_COLS), 16 per thread held in registers, and leaves a
+// sorted partial list and an (m, z) pair; the block that finishes a row last merges the partials,
+// always in the same order.  Selection is KTOP rounds of a block-wide "best remaining" search.
 #define TOPK_MAX 16
 #define TOPK_THREADS 256
 #define TOPK_COLS 4096
+#define TOPK_PER_THREAD (TOPK_COLS / TOPK_THREADS)
 struct TopkScratch {
   float *pv;       // [rows][nsplit][TOPK_MAX] partial values
   int *pi;         // [rows][nsplit][TOPK_MAX] partial ids
@@ -318,30 +318,36 @@ struct TopkScratch {
   int *counter;    // [rows] blocks done; zero between launches
 };
 
-// Block-wide selection of the `ktop` best heads of per-thread sorted lists kept in shared memory
-// (list t = sv/si[t * TOPK_MAX ..], `len` valid entries for t < nlists).  Round j's winner goes
-// to out_v/out_i[j].
-__device__ __forceinline__ void topk_merge_lists(const float *sv, const int *si, int nlists, int len, int ktop,
-                                                 float *out_v, int *out_i, float *cand_v, int *cand_i, int *cand_t) {
-  int tid = threadIdx.x, head = 0;
+// ktop rounds over NV register candidates per thread: round j's block-wide best goes to
+// out_v/out_i[j] and is retired.  sh_* hold one entry per warp.
+template <int NV>
+__device__ __forceinline__ void topk_rounds(const float (&v)[NV], const int (&id)[NV], int ktop, float *out_v, int *out_i,
+                                            float *sh_v, int *sh_i) {
+  int tid = threadIdx.x;
+  unsigned taken = 0u;
   for (int round = 0; round < ktop; ++round) {
-    bool live = tid < nlists && head < len;
-    float v = live ? sv[tid * TOPK_MAX + head] : -INFINITY;
-    int id = live ? si[tid * TOPK_MAX + head] : 0x7fffffff;
-    int t = tid;
+    float bv = -INFINITY;
+    int bi = 0x7fffffff, bj = -1;
+#pragma unroll
+    for (int j = 0; j < NV; ++j)
+      if (!((taken >> j) & 1u) && better(v[j], id[j], bv, bi)) { bv = v[j]; bi = id[j]; bj = j; }
+    float wv = bv;
+    int wi = bi;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, v, o);
-      int oi = __shfl_xor_sync(0xffffffffu, id, o), ot = __shfl_xor_sync(0xffffffffu, t, o);
-      if (better(ov, oi, v, id)) { v = ov; id = oi; t = ot; }
+      float ov = __shfl_xor_sync(0xffffffffu, wv, o);
+      int oi = __shfl_xor_sync(0xffffffffu, wi, o);
+      if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
     }
-    if ((tid & 31) == 0) { cand_v[tid >> 5] = v; cand_i[tid >> 5] = id; cand_t[tid >> 5] = t; }
+    if ((tid & 31) == 0) { sh_v[tid >> 5] = wv; sh_i[tid >> 5] = wi; }
     __syncthreads();
-    float bv = cand_v[0]; int bi = cand_i[0], bt = cand_t[0];
+    float gv = sh_v[0];
+    int gi = sh_i[0];
+#pragma unroll
     for (int w = 1; w < TOPK_THREADS / 32; ++w)
-      if (better(cand_v[w], cand_i[w], bv, bi)) { bv = cand_v[w]; bi = cand_i[w]; bt = cand_t[w]; }
-    if (tid == bt) ++head;
-    if (tid == 0) { out_v[round] = bv; out_i[round] = bi; }
+      if (better(sh_v[w], sh_i[w], gv, gi)) { gv = sh_v[w]; gi = sh_i[w]; }
+    if (bj >= 0 && bi == gi && bv == gv) taken |= 1u << bj;      // ids are unique: one owner
+    if (tid == 0) { out_v[round] = gv; out_i[round] = gi; }
     __syncthreads();
   }
 }
@@ -349,56 +355,57 @@ __device__ __forceinline__ void topk_merge_lists(const float *sv, const int *si,
 __global__ void __launch_bounds__(TOPK_THREADS)
 k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_val, int *top_id, float *lse,
            float *logits_out) {
-  __shared__ float sv[TOPK_THREADS * TOPK_MAX];
-  __shared__ int si[TOPK_THREADS * TOPK_MAX];
   __shared__ float red[33];
-  __shared__ float cand_v[TOPK_THREADS / 32];
-  __shared__ int cand_i[TOPK_THREADS / 32], cand_t[TOPK_THREADS / 32];
+  __shared__ float sh_v[TOPK_THREADS / 32];
+  __shared__ int sh_i[TOPK_THREADS / 32];
   __shared__ int is_last;
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_topk_lse);
   int r = blockIdx.x, sp = blockIdx.y, tid = threadIdx.x;
-  int c0 = sp * TOPK_COLS, c1 = min(V, c0 + TOPK_COLS);
-  float lv[TOPK_MAX];
-  int li[TOPK_MAX];
-  for (int j = 0; j < TOPK_MAX; ++j) { lv[j] = -INFINITY; li[j] = 0x7fffffff; }
-  float m = -INFINITY, z = 0.f;
-  auto consider = [&](float v, int c) {
-    if (v > m) { z = z * __expf(m - v) + 1.f; m = v; } else z += __expf(v - m);
-    if (better(v, c, lv[ktop - 1], li[ktop - 1])) {
-      int j = ktop - 1;
-      while (j > 0 && better(v, c, lv[j - 1], li[j - 1])) { lv[j] = lv[j - 1]; li[j] = li[j - 1]; --j; }
-      lv[j] = v; li[j] = c;
-    }
-  };
+  int c0 = sp * TOPK_COLS;
+  float v[TOPK_PER_THREAD];
+  int id[TOPK_PER_THREAD];
   if ((V & 3) == 0) {
-    for (int c = c0 + tid * 4; c < c1; c += TOPK_THREADS * 4) {
-      float4 v = gemm_val4(g, r, c);
-      if (logits_out) *reinterpret_cast<float4 *>(logits_out + (long long)r * V + c) = v;
-      consider(v.x, c); consider(v.y, c + 1); consider(v.z, c + 2); consider(v.w, c + 3);
+    float4 q[TOPK_PER_THREAD / 4];
+#pragma unroll
+    for (int j = 0; j < TOPK_PER_THREAD / 4; ++j) {
+      int c = c0 + (j * TOPK_THREADS + tid) * 4;
+      q[j] = c < V ? gemm_val4(g, r, c) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+#pragma unroll
+    for (int j = 0; j < TOPK_PER_THREAD / 4; ++j) {
+      int c = c0 + (j * TOPK_THREADS + tid) * 4;
+      if (logits_out && c < V) *reinterpret_cast<float4 *>(logits_out + (long long)r * V + c) = q[j];
+      v[4 * j] = q[j].x; v[4 * j + 1] = q[j].y; v[4 * j + 2] = q[j].z; v[4 * j + 3] = q[j].w;
+      id[4 * j] = c; id[4 * j + 1] = c + 1; id[4 * j + 2] = c + 2; id[4 * j + 3] = c + 3;
     }
   } else {
-    for (int c = c0 + tid; c < c1; c += TOPK_THREADS) {
-      float v = gemm_val(g, r, c);
-      if (logits_out) logits_out[(long long)r * V + c] = v;
-      consider(v, c);
+#pragma unroll
+    for (int j = 0; j < TOPK_PER_THREAD; ++j) {
+      int c = c0 + j * TOPK_THREADS + tid;
+      v[j] = c < V ? gemm_val(g, r, c) : -INFINITY;
+      id[j] = c;
+      if (logits_out && c < V) logits_out[(long long)r * V + c] = v[j];
     }
   }
+#pragma unroll
+  for (int j = 0; j < TOPK_PER_THREAD; ++j) if (id[j] >= V) id[j] = 0x7fffffff;
   // (m, z) of this block's columns, combined in a fixed order
+  float m = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < TOPK_PER_THREAD; ++j) m = fmaxf(m, v[j]);
   float bm = warp_max(m);
-  __syncthreads();
   if ((tid & 31) == 0) red[tid >> 5] = bm;
   __syncthreads();
   if (tid < 32) { float t = tid < TOPK_THREADS / 32 ? red[tid] : -INFINITY; t = warp_max(t); if (tid == 0) red[32] = t; }
   __syncthreads();
   float gm = red[32];
-  float tot = block_sum(m == -INFINITY ? 0.f : z * __expf(m - gm), red);
+  float z = 0.f;
+#pragma unroll
+  for (int j = 0; j < TOPK_PER_THREAD; ++j) z += __expf(v[j] - gm);        // exp(-inf) = 0 for padding
+  float tot = block_sum(z, red);
   long long po = (long long)r * nsplit + sp;
   if (tid == 0) { ts.pm[po] = gm; ts.pz[po] = tot; }
-  // this block's sorted top-ktop
-  for (int j = 0; j < ktop; ++j) { sv[tid * TOPK_MAX + j] = lv[j]; si[tid * TOPK_MAX + j] = li[j]; }
-  __syncthreads();
-  topk_merge_lists(sv, si, TOPK_THREADS, ktop, ktop, ts.pv + po * TOPK_MAX, ts.pi + po * TOPK_MAX, cand_v, cand_i, cand_t);
+  topk_rounds<TOPK_PER_THREAD>(v, id, ktop, ts.pv + po * TOPK_MAX, ts.pi + po * TOPK_MAX, sh_v, sh_i);
   // the last block of the row merges
   __threadfence();
   __syncthreads();
@@ -410,11 +417,17 @@ k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_va
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  if (tid < nsplit) {
-    for (int j = 0; j < ktop; ++j) {
-      sv[tid * TOPK_MAX + j] = __ldcg(ts.pv + ((long long)r * nsplit + tid) * TOPK_MAX + j);
-      si[tid * TOPK_MAX + j] = __ldcg(ts.pi + ((long long)r * nsplit + tid) * TOPK_MAX + j);
-    }
+  // candidates: nsplit lists of ktop entries, up to 4 per thread (nsplit * ktop <= 1024)
+  float cv[4];
+  int ci[4];
+  int ncand = nsplit * ktop;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    int e = j * TOPK_THREADS + tid;
+    bool ok = e < ncand;
+    int q = ok ? e / ktop : 0, w = ok ? e - q * ktop : 0;
+    cv[j] = ok ? __ldcg(ts.pv + ((long long)r * nsplit + q) * TOPK_MAX + w) : -INFINITY;
+    ci[j] = ok ? __ldcg(ts.pi + ((long long)r * nsplit + q) * TOPK_MAX + w) : 0x7fffffff;
   }
   if (tid == 0) {
     float mm = -INFINITY, zz = 0.f;
@@ -422,6 +435,5 @@ k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_va
     for (int q = 0; q < nsplit; ++q) zz += __ldcg(ts.pz + (long long)r * nsplit + q) * __expf(__ldcg(ts.pm + (long long)r * nsplit + q) - mm);
     lse[r] = mm + logf(zz);
   }
-  __syncthreads();
-  topk_merge_lists(sv, si, nsplit, ktop, ktop, top_val + (long long)r * ktop, top_id + (long long)r * ktop, cand_v, cand_i, cand_t);
+  topk_rounds<4>(cv, ci, ktop, top_val + (long long)r * ktop, top_id + (long long)r * ktop, sh_v, sh_i);
 }

@@ -59,8 +59,7 @@ struct TreeBatch { TreePtrs t[DREAM_MAX_BATCH]; int seq[DREAM_MAX_BATCH]; };
 // draft self-attention K/V rows.  One thread per sequence slot b.
 __global__ void k_draft_begin(TreeBatch tb, int B, SeqDev s, DraftTreeDev dt, TreeShape ts,
                               RowMeta rm, int rows_per_seq, int cap_rows, int *status) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_draft_begin);
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   int seq = tb.seq[b];
@@ -97,8 +96,7 @@ __global__ void k_tree_expand(TreeBatch tb, SeqDev s, DraftTreeDev dt, TreeShape
                               int rows_per_seq, const float *__restrict__ top_val,
                               const int *__restrict__ top_id, const float *__restrict__ lse,
                               RowMeta rm_next, int next_rows_per_seq) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_tree_expand);
   __shared__ float cum[256];
   int b = blockIdx.x, seq = tb.seq[b];
   int K = ts.K, m = ts.beam[p - 1], nnew = m * K;
@@ -141,8 +139,7 @@ __global__ void k_tree_expand(TreeBatch tb, SeqDev s, DraftTreeDev dt, TreeShape
 // earlier candidate), order them by creation index behind the root, remap parents, build
 // the ancestor-or-self masks.  One block per sequence slot.
 __global__ void k_tree_finalize(TreeBatch tb, SeqDev s, DraftTreeDev dt, TreeShape ts) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_tree_finalize);
   extern __shared__ int sm[];
   int NC = ts.NC, Nsel = ts.T - 1;
   int *sel = sm, *node_of = sm + NC;       // [NC] each
@@ -186,8 +183,7 @@ __global__ void k_tree_finalize(TreeBatch tb, SeqDev s, DraftTreeDev dt, TreeSha
 // Verification rows: node i of slot b is row b*T + i at position P + depth[i], KV slot P + i.
 __global__ void k_verify_setup(TreeBatch tb, int B, int T, SeqDev s, RowMeta rm, uint32_t *mask,
                                int max_seq, int *status) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_verify_setup);
   int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= B * T) return;
   int b = r / T, i = r - b * T, seq = tb.seq[b];
@@ -207,8 +203,7 @@ __global__ void k_verify_setup(TreeBatch tb, int B, int T, SeqDev s, RowMeta rm,
 // One warp per sequence slot.
 __global__ void k_accept(TreeBatch tb, int B, int T, int D, SeqDev s, const int *__restrict__ argmax,
                          int *accept_len, int *out_tokens, int *comp_src) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_accept);
   int b = blockIdx.x, lane = threadIdx.x, seq = tb.seq[b];
   TreePtrs tp = tb.t[b];
   const int *am = argmax + b * T;
@@ -251,8 +246,7 @@ __global__ void k_accept(TreeBatch tb, int B, int T, int D, SeqDev s, const int 
 template <typename T>
 __global__ void k_compact_kv(TreeBatch tb, SeqDev s, void *pool, long long layer_stride,
                              long long kv_stride, PagedKV kv) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_compact_kv);
   int b = blockIdx.y, seq = tb.seq[b];
   int layer = blockIdx.x >> 1, which = blockIdx.x & 1;
   T *base = (T *)pool + (long long)layer * layer_stride + (long long)which * kv_stride;
@@ -274,8 +268,7 @@ __global__ void k_compact_kv(TreeBatch tb, SeqDev s, void *pool, long long layer
 // nperm_m + j.  Then nperm_m advances.  One thread per sequence slot.
 __global__ void k_accept_rows(TreeBatch tb, int B, int T, int D, SeqDev s, int *gather_idx,
                               RowMeta rm, int cap_rows, int *status) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_accept_rows);
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   int seq = tb.seq[b], A = s.last_A[seq], nm = s.nperm_m[seq];
@@ -293,8 +286,7 @@ __global__ void k_accept_rows(TreeBatch tb, int B, int T, int D, SeqDev s, int *
 // Tap-layer selection (Section 3.2): argmin (or argmax) of AE over [lo, hi], ties -> lower layer.
 __global__ void k_select_tap(const float *__restrict__ ae, int mode, int fixed, int lo, int hi,
                              int *tap_out, int *tap_user) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_select_tap);
   if (threadIdx.x || blockIdx.x) return;
   int best = fixed;
   if (mode != 0) {
@@ -315,8 +307,7 @@ __global__ void k_select_visual(const float *__restrict__ scores_all, long long 
                                 const int *__restrict__ tap, int tap_lo, int v, int k, int vis_start,
                                 int n, const int *__restrict__ forced, int *kept, float *scores_out,
                                 int *ctx_pos, int *flags /* [n] scratch */) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_select_visual);
   const float *sc = scores_all + (long long)(*tap - tap_lo) * layer_stride;
   for (int j = threadIdx.x; j < n; j += blockDim.x) flags[j] = (j < vis_start || j >= vis_start + v) ? 1 : 0;
   __syncthreads();
@@ -349,8 +340,7 @@ __global__ void k_select_visual(const float *__restrict__ scores_all, long long 
 // ctx_pos[i] (or position i when the memory keeps every prompt position).
 __global__ void k_ctx_rows(const int *__restrict__ ctx_pos, int count, int identity, int seq,
                            RowMeta rm, int *gather_idx, int row0) {
-  pdl_trigger();
-  pdl_wait();
+  kernel_entry(TR_k_ctx_rows);
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
   int p = identity ? row0 + i : ctx_pos[i];
