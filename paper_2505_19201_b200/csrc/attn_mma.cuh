@@ -15,6 +15,7 @@
 #pragma once
 #include "common.cuh"
 #include "rows.cuh"
+#include "prologue.cuh"
 
 #define AM_ROWS 64
 #define AM_THREADS 128
@@ -70,6 +71,7 @@ struct AttnMmaArgs {
   float *part_o, *part_ml;          // [slot][chunk][kvh][rt][64][hd], [..][64][2]
   void *out;                        // [R][H*hd] rows in GEMM-input layout
   XLayout lay;
+  L2Prefetch next_w;                // weights of the GEMM that follows, pulled into L2 meanwhile
   PagedKV paged;                    // PAGED kernels
   FlatKV2 flat;                     // flat kernels
 };
@@ -95,7 +97,8 @@ k_attn_mma(AttnMmaArgs a) {
   bf16 *Qh = reinterpret_cast<bf16 *>(am_smem), *Ql = Qh + AM_ROWS * LD, *KV = Ql + AM_ROWS * LD;
   uint32_t *mwords = reinterpret_cast<uint32_t *>(KV + 2 * BUF_ELEMS);          // [64][4]
   int *row_r = reinterpret_cast<int *>(mwords + AM_ROWS * 4), *row_h = row_r + AM_ROWS;
-  kernel_entry(TR_k_attn_mma);
+  l2_prefetch_slice(a.next_w, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), gridDim.x * gridDim.y * gridDim.z);
+  kernel_entry_late(TR_k_attn_mma);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int chunk = blockIdx.x, kvh = blockIdx.y / a.n_rt, rt = blockIdx.y - kvh * a.n_rt, slot = blockIdx.z;
   const int Hkv = a.H / a.G;
@@ -272,6 +275,7 @@ k_attn_mma(AttnMmaArgs a) {
     }
     __syncthreads();
   }
+  pdl_trigger();                    // the keys are done: the GEMM kernel that follows may take the SMs
   l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1); l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
   l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1); l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
 
@@ -312,30 +316,9 @@ __global__ void __launch_bounds__(256)
 k_attn_combine(AttnMmaArgs a, int R) {
   kernel_entry(TR_k_attn_combine);
   long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  int c4 = (int)(idx % (HD / 4));
-  long long rh = idx / (HD / 4);
-  int h = (int)(rh % a.H), r = (int)(rh / a.H);
-  if (r >= R) return;
-  if (a.row_in && a.row_in[r] < 0) return;
-  const int Hkv = a.H / a.G;
-  int slot = r / a.rows_per_seq, node = r - slot * a.rows_per_seq;
-  int kvh = h / a.G, rr = node * a.G + (h - kvh * a.G);
-  int rt = rr / AM_ROWS, lr = rr - rt * AM_ROWS;
-  const long long cstride = (long long)Hkv * a.n_rt * AM_ROWS;
-  const long long p0 = (((long long)slot * a.n_chunks * Hkv + kvh) * a.n_rt + rt) * AM_ROWS + lr;
-  float M = -INFINITY;
-  for (int c = 0; c < a.n_chunks; ++c) M = fmaxf(M, __ldcg(a.part_ml + (p0 + c * cstride) * 2));
-  float L = 0.f;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int c = 0; c < a.n_chunks; ++c) {
-    long long pr = p0 + c * cstride;
-    float2 ml = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + pr * 2));
-    float4 o = __ldcg(reinterpret_cast<const float4 *>(a.part_o + pr * HD + c4 * 4));
-    float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
-    L += ml.y * w;
-    acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
-  }
-  float inv = L > 0.f ? 1.f / L : 0.f;
-  store_split4<bf16>(reinterpret_cast<bf16 *>(a.out) + r * a.lay.row_stride + h * HD + c4 * 4, a.lay.lo_delta,
-                     make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+  if (idx >= (long long)R * a.H * (HD / 4)) return;
+  ProCombine pc;
+  pc.part_o = a.part_o; pc.part_ml = a.part_ml; pc.row_in = a.row_in; pc.n_chunks = a.n_chunks; pc.n_rt = a.n_rt;
+  pc.H = a.H; pc.G = a.G; pc.rows_per_seq = a.rows_per_seq; pc.hd = HD; pc.out = reinterpret_cast<bf16 *>(a.out); pc.lay = a.lay;
+  pro_combine_item(pc, idx);
 }

@@ -90,6 +90,31 @@ __device__ __forceinline__ void kernel_entry(int id) {
   if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) trace_stamp(id);
 }
 
+// The same, for a kernel that wants its successor to start only when it is about to finish (a
+// successor that fills the SMs' shared memory would otherwise crowd it out): it calls
+// pdl_trigger() itself, late.
+__device__ __forceinline__ void kernel_entry_late(int id) {
+  pdl_wait();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) trace_stamp(id);
+}
+
+// Weights never change, so a kernel that leaves HBM idle can pull the next GEMM's weights into the
+// 126 MB L2 ahead of time, before its own grid dependency resolves.  Every CTA requests an equal
+// slice with bulk L2 prefetches issued by one thread.
+struct L2Prefetch {
+  const char *ptr;               // 128-byte aligned; null = nothing to fetch
+  unsigned long long bytes;
+};
+__device__ __forceinline__ void l2_prefetch_slice(const L2Prefetch &pf, unsigned cta, unsigned n_cta) {
+  if (!pf.ptr || threadIdx.x != 0) return;
+  unsigned long long per = ((pf.bytes + n_cta - 1) / n_cta + 127ull) & ~127ull;
+  unsigned long long lo = per * cta, hi = lo + per < pf.bytes ? lo + per : pf.bytes;
+  for (unsigned long long o = lo; o < hi; o += 32768ull) {
+    unsigned sz = (unsigned)((hi - o < 32768ull ? hi - o : 32768ull) & ~15ull);
+    if (sz) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(pf.ptr + o), "r"(sz) : "memory");
+  }
+}
+
 // A bf16 GEMM input row is stored as two bf16 rows, hi = bf16(v) and lo = bf16(v - hi), so the
 // tensor cores see the activation to ~16 mantissa bits while the weights stream once.  fp32
 // inputs have no lo part.  XLayout says where the rows of such a buffer live: token t starts at
@@ -133,20 +158,32 @@ __device__ __forceinline__ float gemm_val(const GemmOut &g, int r, int c) {
 }
 
 // Four consecutive columns c..c+3 (c a multiple of 4: they share a tile, hence a slot count).
+// The slots are added in slot order, but fetched four at a time so that a value made of many
+// partial sums costs a few memory round trips instead of one per slot.
+__device__ __forceinline__ void add4(float4 &s, const float4 &t) { s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w; }
+__device__ __forceinline__ int gemm_extra_slots(const GemmOut &g, int c) {
+  if (!g.upc) return 0;
+  unsigned u0 = (unsigned)(c >> 8) * (unsigned)g.kb;
+  return (int)((u0 + (unsigned)g.kb - 1u) / (unsigned)g.upc) - (int)(u0 / (unsigned)g.upc);
+}
 __device__ __forceinline__ float4 gemm_val4(const GemmOut &g, int r, int c) {
   int ch = r >> g.chunk_shift;
   const float4 *p = reinterpret_cast<const float4 *>(g.base + (long long)ch * g.chunk_stride +
                                                      (long long)(r - (ch << g.chunk_shift)) * g.ld + c);
   float4 s = *p;
-  if (g.upc) {
-    unsigned u0 = (unsigned)(c >> 8) * (unsigned)g.kb;
-    int extra = (int)((u0 + (unsigned)g.kb - 1u) / (unsigned)g.upc) - (int)(u0 / (unsigned)g.upc);
-    long long st4 = g.slot_stride >> 2;
-    for (int i = 1; i <= extra; ++i) {
-      float4 t = p[(long long)i * st4];
-      s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
-    }
+  const int extra = gemm_extra_slots(g, c);
+  const long long st4 = g.slot_stride >> 2;
+  int i = 1;
+  for (; i + 3 <= extra; i += 4) {
+    float4 t0 = p[(long long)i * st4], t1 = p[(long long)(i + 1) * st4], t2 = p[(long long)(i + 2) * st4], t3 = p[(long long)(i + 3) * st4];
+    add4(s, t0); add4(s, t1); add4(s, t2); add4(s, t3);
   }
+  if (i + 1 <= extra) {
+    float4 t0 = p[(long long)i * st4], t1 = p[(long long)(i + 1) * st4];
+    add4(s, t0); add4(s, t1);
+    i += 2;
+  }
+  if (i <= extra) { float4 t0 = p[(long long)i * st4]; add4(s, t0); }
   return s;
 }
 

@@ -32,6 +32,7 @@
 #include <tuple>
 
 #include "common.cuh"
+#include "prologue.cuh"
 
 #define TC_BN 256               // weight rows per tile (MMA N)
 #define TC_BK 64                // k elements per panel (128 bytes: one swizzle row)
@@ -42,16 +43,29 @@
 
 enum { TC_X_PLAIN = 0, TC_X_INTERLEAVED = 1, TC_X_PLANAR = 2 };
 
-struct TcParams {
+#define TC_MAX_STAGES 4
+
+// One GEMM of a chain, preceded by the row-wise work that produces its input.
+struct TcStage {
   float *out;
   long long slot_stride;        // floats between partial-sum slots
   int N, K, KB, n_tiles, total_units, upc;
-  int n_tok;                    // real token rows of this launch
+  int n_tok;                    // real token rows
   int x_mode;                   // TC_X_*
   int lo_rows;                  // TC_X_PLANAR: row of the first low part in the X tensor map
-  int wp, w_stages, x_stages;   // panels per W stage, ring depths
-  int *status;
+  Prologue pro;                 // kind PRO_NONE: the input was written by an earlier kernel
 };
+// A chain of up to TC_MAX_STAGES GEMMs run by one launch: stage k's prologue reads stage k-1's
+// output.  Grid-wide barriers (a counter in global memory that only grows) order the stages.
+struct TcChain {
+  int n_stages;
+  int wp, w_stages, x_stages;   // panels per ring stage, ring depths (shared by all stages)
+  int *status;
+  unsigned long long *bar_counter;
+  unsigned long long bar_base;  // value of the counter when this launch starts
+  TcStage st[TC_MAX_STAGES];
+};
+struct TcMaps { CUtensorMap w[TC_MAX_STAGES], x[TC_MAX_STAGES]; };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -126,15 +140,37 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+
+// Grid-wide barrier number `ord` of this launch: every CTA adds one to a counter that only grows
+// and waits until all of them have.  All CTAs of the grid are resident (one per SM), so the wait
+// ends; it is bounded all the same.  One thread per CTA calls it.
+#define TC_GRID_SPIN_LIMIT (1u << 22)
+__device__ __forceinline__ bool grid_barrier(const TcChain &p, int ord) {
+  __threadfence();
+  atomicAdd(p.bar_counter, 1ull);
+  const unsigned long long target = p.bar_base + (unsigned long long)(ord + 1) * gridDim.x;
+  for (uint32_t it = 0; it < TC_GRID_SPIN_LIMIT; ++it) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p.bar_counter) : "memory");
+    if (v >= target) return true;
+    __nanosleep(32);
+  }
+  return false;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 // ------------------------------------------------------------------------------------------ kernel
 // Dynamic shared memory (1024-byte aligned): W ring [w_stages][wp][32 KB], X ring
-// [x_stages][16 KB, or 32 KB = high tile | low tile when planar], then the barriers.
+// [x_stages][wp][16 KB, or 32 KB = high tile | low tile when planar], then the barriers.
 __global__ void __launch_bounds__(TC_THREADS, 1)
-k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, TcParams p) {
+k_gemm_tc(const __grid_constant__ TcMaps maps, const __grid_constant__ TcChain p) {
   extern __shared__ uint8_t smem_raw[];
+  __shared__ float pro_sh[8];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const bool planar = p.st[0].x_mode == TC_X_PLANAR;      // one layout per chain
   const uint32_t wstage_bytes = (uint32_t)p.wp * TC_WPANEL;
-  const uint32_t xstage_bytes = p.x_mode == TC_X_PLANAR ? 2u * TC_XTILE : (uint32_t)TC_XTILE;
+  const uint32_t xpanel_bytes = planar ? 2u * TC_XTILE : (uint32_t)TC_XTILE;
+  const uint32_t xstage_bytes = (uint32_t)p.wp * xpanel_bytes;
   uint8_t *wring = smem, *xring = smem + (size_t)p.w_stages * wstage_bytes;
   uint64_t *bars = (uint64_t *)(xring + (size_t)p.x_stages * xstage_bytes);
   uint64_t *full_w = bars, *empty_w = full_w + p.w_stages, *full_x = empty_w + p.w_stages, *empty_x = full_x + p.x_stages;
@@ -143,10 +179,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   volatile int *abort_flag = (volatile int *)(tmem_base_p + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u_begin = blockIdx.x * p.upc;
-  const int u_end = min(u_begin + p.upc, p.total_units);
-  const bool has_work = u_begin < u_end;
-
   if (blockIdx.x == 0 && threadIdx.x == 0) trace_stamp(TR_none);     // CTA start, before any dependency
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.w_stages; ++s) { mbar_init(full_w + s, 1); mbar_init(empty_w + s, 1); }
@@ -164,117 +196,163 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   tc_fence_after();
   pdl_trigger();
   const uint32_t tmem_base = *tmem_base_p;
+  // grid barriers of the launch, in order: [after stage 0's prologue], then for every later
+  // stage one before its prologue (the previous GEMM is complete) and one after it
+  const int bar0 = p.st[0].pro.kind != PRO_NONE ? 1 : 0;
 
-  if (has_work) {
-    if (warp == 0) {
-      // ------------------------------------------------------------------ W producer: weights are
-      // constant, so nothing here waits for the previous kernel
-      if (lane == 0) {
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-        const uint64_t pol = policy_evict_first();
-        uint32_t it = 0;
-        int u = u_begin;
+  if (warp == 0) {
+    // ------------------------------------------------------------------ W producer: weights are
+    // constant, so nothing here waits for anything but ring space; it runs ahead across stages
+    if (lane == 0) {
+      const uint64_t pol = policy_evict_first();
+      int s = 0;
+      uint32_t ph = 0;
+      bool wrapped = false, live = true;
+      for (int st = 0; st < p.n_stages && live; ++st) {
+        const TcStage &S = p.st[st];
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.w[st]) : "memory");
+        int u = blockIdx.x * S.upc;
+        const int u_end = min(u + S.upc, S.total_units);
         while (u < u_end) {
-          int tile = u / p.KB, kb = u - tile * p.KB;
-          int np = min(p.wp, min(p.KB - kb, u_end - u));
-          int s = it % p.w_stages;
-          if (it >= (uint32_t)p.w_stages && !mbar_wait(empty_w + s, ((it / p.w_stages) & 1) ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break; }
-          if (*abort_flag) break;
+          int tile = u / S.KB, kb = u - tile * S.KB;
+          int np = min(p.wp, min(S.KB - kb, u_end - u));
+          if (wrapped && !mbar_wait(empty_w + s, ph ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; live = false; break; }
+          if (*abort_flag) { live = false; break; }
           uint8_t *dst = wring + (size_t)s * wstage_bytes;
           mbar_expect_tx(full_w + s, (uint32_t)np * TC_WPANEL);
-          for (int q = 0; q < np; ++q) tma_load_2d(dst + (size_t)q * TC_WPANEL, &map_w, full_w + s, (kb + q) * TC_BK, tile * TC_BN, pol);
-          u += np; ++it;
+          for (int q = 0; q < np; ++q) tma_load_2d(dst + (size_t)q * TC_WPANEL, &maps.w[st], full_w + s, (kb + q) * TC_BK, tile * TC_BN, pol);
+          u += np;
+          if (++s == p.w_stages) { s = 0; ph ^= 1; wrapped = true; }
         }
       }
-    } else if (warp == 6) {
-      // ------------------------------------------------------------------ X producer
-      if (lane == 0) {
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
-        pdl_wait();
-        const uint64_t pol = policy_evict_last();
-        uint32_t it = 0;
-        for (int u = u_begin; u < u_end; ++u, ++it) {
-          int tile = u / p.KB, kb = u - tile * p.KB;
-          int s = it % p.x_stages;
-          if (it >= (uint32_t)p.x_stages && !mbar_wait(empty_x + s, ((it / p.x_stages) & 1) ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break; }
-          if (*abort_flag) break;
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ X producer: waits until the
+    // stage's input exists (previous kernel, or this stage's prologue on every CTA), then feeds
+    // one X stage per W stage
+    const uint64_t pol = policy_evict_last();
+    int s = 0;
+    uint32_t ph = 0;
+    bool wrapped = false, live = true;
+    for (int st = 0; st < p.n_stages; ++st) {
+      const TcStage &S = p.st[st];
+      if (S.pro.kind != PRO_NONE) {
+        named_bar_sync(1, PRO_THREADS + 32);                  // this CTA's share of the prologue is written
+        if (lane == 0 && live && !grid_barrier(p, st == 0 ? 0 : bar0 + 2 * (st - 1) + 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; live = false; }
+      } else if (st == 0 && lane == 0) pdl_wait();
+      if (lane == 0 && live) {
+        fence_proxy_async();                                  // rows written by ordinary stores, read by TMA
+        if (blockIdx.x == 0) trace_stamp(TR_k_gemm_tc);
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.x[st]) : "memory");
+        int u = blockIdx.x * S.upc;
+        const int u_end = min(u + S.upc, S.total_units);
+        while (u < u_end) {
+          int tile = u / S.KB, kb = u - tile * S.KB;
+          int np = min(p.wp, min(S.KB - kb, u_end - u));
+          if (wrapped && !mbar_wait(empty_x + s, ph ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; live = false; break; }
+          if (*abort_flag) { live = false; break; }
           uint8_t *dst = xring + (size_t)s * xstage_bytes;
-          mbar_expect_tx(full_x + s, xstage_bytes);
-          tma_load_2d(dst, &map_x, full_x + s, kb * TC_BK, 0, pol);
-          if (p.x_mode == TC_X_PLANAR) tma_load_2d(dst + TC_XTILE, &map_x, full_x + s, kb * TC_BK, p.lo_rows, pol);
+          mbar_expect_tx(full_x + s, (uint32_t)np * xpanel_bytes);
+          for (int q = 0; q < np; ++q) {
+            tma_load_2d(dst + (size_t)q * xpanel_bytes, &maps.x[st], full_x + s, (kb + q) * TC_BK, 0, pol);
+            if (planar) tma_load_2d(dst + (size_t)q * xpanel_bytes + TC_XTILE, &maps.x[st], full_x + s, (kb + q) * TC_BK, S.lo_rows, pol);
+          }
+          u += np;
+          if (++s == p.x_stages) { s = 0; ph ^= 1; wrapped = true; }
         }
       }
-    } else if (warp == 1) {
-      // ------------------------------------------------------------------ MMA issuer
-      if (lane == 0) {
-        // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        const bool planar = p.x_mode == TC_X_PLANAR;
-        uint32_t wit = 0, xit = 0, seg = 0;
-        int u = u_begin;
-        bool ok = true;
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      int ws = 0, xs = 0;
+      uint32_t wph = 0, xph = 0, seg = 0;
+      bool ok = true;
+      for (int st = 0; st < p.n_stages && ok; ++st) {
+        const TcStage &S = p.st[st];
+        int u = blockIdx.x * S.upc;
+        const int u_end = min(u + S.upc, S.total_units);
         while (u < u_end && ok) {
-          int tile = u / p.KB;
-          int seg_end = min((tile + 1) * p.KB, u_end);
+          int tile = u / S.KB;
+          int seg_end = min((tile + 1) * S.KB, u_end);
           int buf = seg & 1;
           if (seg >= 2 && !mbar_wait(acc_empty + buf, ((seg >> 1) & 1) ^ 1)) { ok = false; break; }
           tc_fence_after();
           uint32_t d_addr = tmem_base + (uint32_t)buf * TC_BN;
-          bool first = true;
+          uint32_t accum = 0u;
           while (u < seg_end) {
-            int kb = u - tile * p.KB;
-            int np = min(p.wp, min(p.KB - kb, u_end - u));
-            int s = wit % p.w_stages;
-            if (!mbar_wait(full_w + s, (wit / p.w_stages) & 1)) { ok = false; break; }
-            uint32_t sw0 = smem_u32(wring + (size_t)s * wstage_bytes);
-            for (int q = 0; q < np; ++q, ++xit) {
-              int t = xit % p.x_stages;
-              uint32_t sx = smem_u32(xring + (size_t)t * xstage_bytes);
-              if (!mbar_wait(full_x + t, (xit / p.x_stages) & 1)) { ok = false; break; }
-              tc_fence_after();
-              uint64_t ad = smem_desc(sx), al = smem_desc(sx + TC_XTILE), bd = smem_desc(sw0 + (uint32_t)q * TC_WPANEL);
+            int np = min(p.wp, seg_end - u);
+            if (!mbar_wait(full_w + ws, wph) || !mbar_wait(full_x + xs, xph)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t sw0 = smem_u32(wring + (size_t)ws * wstage_bytes), sx0 = smem_u32(xring + (size_t)xs * xstage_bytes);
+            for (int q = 0; q < np; ++q) {
+              uint64_t ad = smem_desc(sx0 + (uint32_t)q * xpanel_bytes), al = smem_desc(sx0 + (uint32_t)q * xpanel_bytes + TC_XTILE);
+              uint64_t bd = smem_desc(sw0 + (uint32_t)q * TC_WPANEL);
 #pragma unroll
               for (int k = 0; k < TC_BK / 16; ++k) {
-                mma_bf16(d_addr, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, (first && k == 0) ? 0u : 1u);
+                mma_bf16(d_addr, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, accum);
+                accum = 1u;
                 if (planar) mma_bf16(d_addr, al + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, 1u);
               }
-              first = false;
-              mma_commit(empty_x + t);          // frees the X stage once these MMAs have read it
             }
-            if (!ok) break;
-            mma_commit(empty_w + s);            // frees the W stage
-            u += np; ++wit;
+            mma_commit(empty_x + xs);           // frees both stages once these MMAs have read them
+            mma_commit(empty_w + ws);
+            u += np;
+            if (++ws == p.w_stages) { ws = 0; wph ^= 1; }
+            if (++xs == p.x_stages) { xs = 0; xph ^= 1; }
           }
           if (!ok) break;
           mma_commit(acc_full + buf);           // accumulator complete
           ++seg;
         }
-        if (!ok) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
       }
-    } else {
-      // ------------------------------------------------------------------ epilogue warps 2..5, 7..10
-      const int q = warp & 3;                   // TMEM lane quarter this warp may read
-      const int half = warp >= 7 ? 1 : 0;       // which 128 accumulator columns this warp drains
-      pdl_wait();                               // the output buffer is read by the previous kernel
-      if (blockIdx.x == 0 && warp == 2 && lane == 0) trace_stamp(TR_k_gemm_tc);
-      const bool inter = p.x_mode == TC_X_INTERLEAVED;
-      const int row = q * 32 + lane;            // accumulator lane = X row
-      const int token = inter ? row >> 1 : row;
-      const int part = inter ? lane & 1 : 0;
-      uint32_t seg = 0;
-      int u = u_begin;
-      while (u < u_end) {
-        int tile = u / p.KB;
-        int seg_end = min((tile + 1) * p.KB, u_end);
+      if (!ok) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
+    }
+  } else {
+    // ------------------------------------------------------------------ warps 2..5, 7..10: the
+    // stage's prologue, then the epilogue of its GEMM segments
+    const int q = warp & 3;                   // TMEM lane quarter this warp may read
+    const int half = warp >= 7 ? 1 : 0;       // which 128 accumulator columns this warp drains
+    const int ptid = (warp < 7 ? warp - 2 : warp - 3) * 32 + lane;      // 0..255 among these warps
+    pdl_wait();                               // inputs and the output buffer belong to earlier kernels
+    const bool inter = p.st[0].x_mode == TC_X_INTERLEAVED;
+    const int row = q * 32 + lane;            // accumulator lane = X row
+    const int token = inter ? row >> 1 : row;
+    const int part = inter ? lane & 1 : 0;
+    uint32_t seg = 0;
+    bool live = true;
+    for (int st = 0; st < p.n_stages; ++st) {
+      const TcStage &S = p.st[st];
+      if (st > 0) {
+        // every CTA's results of the previous GEMM must be in memory before this prologue reads them
+        __threadfence();
+        named_bar_sync(3, PRO_THREADS);
+        if (ptid == 0 && !grid_barrier(p, bar0 + 2 * (st - 1))) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
+        named_bar_sync(3, PRO_THREADS);
+      }
+      if (S.pro.kind != PRO_NONE) {
+        pro_run(S.pro, ptid, blockIdx.x, gridDim.x, pro_sh);
+        __threadfence();
+        fence_proxy_async();
+        named_bar_arrive(1, PRO_THREADS + 32);                // tells this CTA's X producer
+      }
+      int u = blockIdx.x * S.upc;
+      const int u_end = min(u + S.upc, S.total_units);
+      while (u < u_end && live) {
+        int tile = u / S.KB;
+        int seg_end = min((tile + 1) * S.KB, u_end);
         int buf = seg & 1;
         int ok = 1;
         if (lane == 0) ok = mbar_wait(acc_full + buf, (seg >> 1) & 1) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok || *abort_flag) { if (lane == 0) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; } break; }
+        if (!ok || *abort_flag) { if (lane == 0) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; } live = false; break; }
         tc_fence_after();
-        int first_cta = (tile * p.KB) / p.upc;
+        int first_cta = (tile * S.KB) / S.upc;
         int slot = (int)blockIdx.x - first_cta;
-        float *dst = p.out + (long long)slot * p.slot_stride + (long long)token * p.N + tile * TC_BN;
+        float *dst = S.out + (long long)slot * S.slot_stride + (long long)token * S.N + tile * TC_BN;
         uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * TC_BN;
         // four chunks of 32 columns; the TMEM load of chunk i+1 is in flight while chunk i is stored
         uint32_t ra[32], rb[32];
@@ -296,18 +374,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
               float mine = __uint_as_float(part ? r[16 + j] : r[j]);
               v[j] = mine + __shfl_xor_sync(0xffffffffu, send, 1);
             }
-            if (token < p.n_tok) {
+            if (token < S.n_tok) {
 #pragma unroll
               for (int j4 = 0; j4 < 4; ++j4) {
                 int jj = part * 16 + j4 * 4;
-                if (tile * TC_BN + col0 + jj < p.N)
+                if (tile * TC_BN + col0 + jj < S.N)
                   *reinterpret_cast<float4 *>(dst + col0 + jj) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
               }
             }
-          } else if (token < p.n_tok) {
+          } else if (token < S.n_tok) {
 #pragma unroll
             for (int j4 = 0; j4 < 8; ++j4) {
-              if (tile * TC_BN + col0 + j4 * 4 < p.N)
+              if (tile * TC_BN + col0 + j4 * 4 < S.N)
                 *reinterpret_cast<float4 *>(dst + col0 + j4 * 4) =
                     make_float4(__uint_as_float(r[j4 * 4]), __uint_as_float(r[j4 * 4 + 1]), __uint_as_float(r[j4 * 4 + 2]),
                                 __uint_as_float(r[j4 * 4 + 3]));
@@ -338,10 +416,12 @@ struct GemmTcPlan {
   int max_smem;
   int use_pdl;
   int *status;
+  unsigned long long *bar_counter;     // device: arrivals at grid barriers since the plan was made
+  unsigned long long bar_total;        // host mirror: what the counter reads once everything enqueued has run
   std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;
 };
 
-static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status, int use_pdl) {
+static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status, unsigned long long *bar_counter, int use_pdl) {
   void *fn = nullptr;
   cudaDriverEntryPointQueryResult qr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn)
@@ -351,9 +431,12 @@ static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status, int use
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&pl->n_sms, cudaDevAttrMultiProcessorCount, dev);
   cudaDeviceGetAttribute(&pl->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->max_smem) != cudaSuccess)
+  // the kernel also has a few bytes of static shared memory: leave room for them
+  if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->max_smem - 256) != cudaSuccess)
     return "cannot raise the dynamic shared memory limit";
   pl->status = status;
+  pl->bar_counter = bar_counter;       // zeroed by the caller
+  pl->bar_total = 0;
   pl->use_pdl = use_pdl;
   return nullptr;
 }
@@ -400,41 +483,80 @@ static inline long long gemm_tc_out_floats(int n_sms, int slot_rows, int N, int 
   return slots * (long long)slot_rows * N;
 }
 
-// Enqueue one GEMM of `rows` tokens (<= 64 when x_mode is interleaved, <= 128 otherwise).
+// One GEMM of a chain as the host describes it.
 //   X: bf16, row-major, K columns.  TC_X_PLAIN: row t = token t.  TC_X_INTERLEAVED: row 2t = high
 //   part of token t, row 2t+1 = low part.  TC_X_PLANAR: row t = high part, row lo_rows + t = low part.
-// Returns false if the launch could not be made (no tensor map, output too small).
-static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const void *W, const void *X, int x_mode, int lo_rows,
-                                  int rows, int slot_rows, int N, int K, float *out, long long out_floats, GemmOut *g) {
-  TcParams p;
-  p.n_tok = rows;
-  p.x_mode = x_mode;
-  p.lo_rows = lo_rows;
-  p.N = N; p.K = K; p.KB = K / TC_BK;
-  p.n_tiles = (N + TC_BN - 1) / TC_BN;
-  p.total_units = p.n_tiles * p.KB;
-  int grid = pl->n_sms < p.total_units ? pl->n_sms : p.total_units;
-  p.upc = (p.total_units + grid - 1) / grid;
+//   rows <= 64 when interleaved, <= 128 otherwise; every GEMM of a chain has the same rows and x_mode.
+//   pro: the row-wise work that writes X (kind PRO_NONE: an earlier kernel did); stages after the
+//   first must have one.
+struct GemmTcDesc {
+  const void *W, *X;
+  int x_mode, lo_rows, rows, slot_rows, N, K;
+  float *out;
+  long long out_floats;
+  Prologue pro;
+};
+
+// Enqueue a chain of n GEMMs as one launch.  g[i] receives the descriptor consumers read stage
+// i's result through; it depends on the shapes only, so a call with launch == false serves to
+// learn the descriptors that later stages' prologues need.  Returns false if the launch could not
+// be made.
+static inline bool gemm_tc_launch_chain(GemmTcPlan *pl, cudaStream_t stream, int n, const GemmTcDesc *d, GemmOut *g,
+                                        bool launch = true) {
+  if (n < 1 || n > TC_MAX_STAGES) return false;
+  TcChain p;
+  TcMaps maps;
+  p.n_stages = n;
+  const int x_mode = d[0].x_mode;
   // W stages of two panels (256-byte runs per weight row) unless the X ring needs the room
   p.wp = x_mode == TC_X_PLANAR ? 1 : 2;
-  if (p.wp > p.KB) p.wp = p.KB;
-  if (p.KB % p.wp == 0) p.upc = (p.upc + p.wp - 1) / p.wp * p.wp;   // CTA ranges cover whole W stages
-  grid = (p.total_units + p.upc - 1) / p.upc;
-  p.x_stages = x_mode == TC_X_PLANAR ? 2 : 4;
-  int xstage = x_mode == TC_X_PLANAR ? 2 * TC_XTILE : TC_XTILE;
+  int max_grid = 1;
+  for (int i = 0; i < n; ++i) {
+    TcStage &S = p.st[i];
+    if (d[i].x_mode != x_mode || d[i].rows != d[0].rows || (launch && i > 0 && d[i].pro.kind == PRO_NONE)) return false;
+    S.n_tok = d[i].rows; S.x_mode = x_mode; S.lo_rows = d[i].lo_rows;
+    S.N = d[i].N; S.K = d[i].K; S.KB = d[i].K / TC_BK;
+    S.n_tiles = (S.N + TC_BN - 1) / TC_BN;
+    S.total_units = S.n_tiles * S.KB;
+    if (S.KB < p.wp) p.wp = 1;
+  }
+  for (int i = 0; i < n; ++i) {
+    TcStage &S = p.st[i];
+    int grid = pl->n_sms < S.total_units ? pl->n_sms : S.total_units;
+    S.upc = (S.total_units + grid - 1) / grid;
+    if (S.KB % p.wp == 0) S.upc = (S.upc + p.wp - 1) / p.wp * p.wp;   // CTA ranges cover whole ring stages
+    grid = (S.total_units + S.upc - 1) / S.upc;
+    if (grid > max_grid) max_grid = grid;
+    S.out = d[i].out;
+    S.slot_stride = (long long)d[i].slot_rows * S.N;       // slot_rows >= rows: the same for every chunk of one GEMM
+    long long max_slots = (S.KB + S.upc - 1) / S.upc + 1;
+    if (S.slot_stride * max_slots > d[i].out_floats) return false;
+    S.pro = d[i].pro;
+    int x_rows = x_mode == TC_X_INTERLEAVED ? 2 * d[i].rows : (x_mode == TC_X_PLANAR ? d[i].lo_rows + d[i].rows : d[i].rows);
+    if (launch) {
+      const CUtensorMap *mw = tc_map(pl, d[i].W, S.N, S.K, TC_BN);
+      const CUtensorMap *mx = tc_map(pl, d[i].X, x_rows, S.K, 128);
+      if (!mw || !mx) return false;
+      maps.w[i] = *mw; maps.x[i] = *mx;
+    }
+    g[i].base = S.out; g[i].slot_stride = S.slot_stride; g[i].chunk_stride = 0; g[i].chunk_shift = 30; g[i].ld = S.N; g[i].kb = S.KB; g[i].upc = S.upc;
+  }
+  if (!launch) return true;
+  bool any_pro = false;
+  for (int i = 0; i < n; ++i) any_pro = any_pro || d[i].pro.kind != PRO_NONE;
+  // a launch with grid barriers needs every CTA resident: one per SM, never more CTAs than SMs
+  int grid = any_pro ? pl->n_sms : max_grid;
+  int xstage = p.wp * (x_mode == TC_X_PLANAR ? 2 * TC_XTILE : TC_XTILE);
+  p.x_stages = 2;
   int budget = pl->max_smem - 2048 - p.x_stages * xstage;
   p.w_stages = budget / (p.wp * TC_WPANEL);
   if (p.w_stages > 8) p.w_stages = 8;
   if (p.w_stages < 2) return false;
-  p.out = out;
-  p.slot_stride = (long long)slot_rows * N;       // slot_rows >= rows: the same for every chunk of one GEMM
-  long long max_slots = (p.KB + p.upc - 1) / p.upc + 1;
-  if (p.slot_stride * max_slots > out_floats) return false;
+  if (budget - p.w_stages * p.wp * TC_WPANEL >= xstage) p.x_stages = 3;   // room left over: a third X stage
   p.status = pl->status;
-  int x_rows = x_mode == TC_X_INTERLEAVED ? 2 * rows : (x_mode == TC_X_PLANAR ? lo_rows + rows : rows);
-  const CUtensorMap *mw = tc_map(pl, W, N, K, TC_BN);
-  const CUtensorMap *mx = tc_map(pl, X, x_rows, K, 128);
-  if (!mw || !mx) return false;
+  p.bar_counter = pl->bar_counter;
+  p.bar_base = pl->bar_total;
+  int n_bars = (d[0].pro.kind != PRO_NONE ? 1 : 0) + 2 * (n - 1);
   size_t smem = (size_t)p.w_stages * p.wp * TC_WPANEL + (size_t)p.x_stages * xstage + 1024 + 512;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
@@ -442,7 +564,16 @@ static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const voi
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = pl->use_pdl ? 1 : 0;
-  if (cudaLaunchKernelEx(&cfg, k_gemm_tc, *mw, *mx, p) != cudaSuccess) return false;
-  g->base = out; g->slot_stride = p.slot_stride; g->chunk_stride = 0; g->chunk_shift = 30; g->ld = N; g->kb = p.KB; g->upc = p.upc;
+  if (cudaLaunchKernelEx(&cfg, k_gemm_tc, maps, p) != cudaSuccess) return false;
+  pl->bar_total += (unsigned long long)n_bars * grid;
   return true;
+}
+
+// A single GEMM without a prologue.
+static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const void *W, const void *X, int x_mode, int lo_rows,
+                                  int rows, int slot_rows, int N, int K, float *out, long long out_floats, GemmOut *g) {
+  GemmTcDesc d;
+  d.W = W; d.X = X; d.x_mode = x_mode; d.lo_rows = lo_rows; d.rows = rows; d.slot_rows = slot_rows; d.N = N; d.K = K;
+  d.out = out; d.out_floats = out_floats; d.pro.kind = PRO_NONE; d.pro.rows = 0;
+  return gemm_tc_launch_chain(pl, stream, 1, &d, g);
 }

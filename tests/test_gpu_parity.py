@@ -42,3 +42,10 @@ def test_llava_shape_4_layers_bf16():
 def test_smolvlm_shape_full_bf16():
     """Config 2: SmolVLM-2B-shaped target, all 24 layers, 4 decode steps."""
     pr, s = _run("smolvlm2b", 4)
+
+
+def test_chained_gemm_launches(monkeypatch):
+    """The optional mode in which norms, gating and the attention merge run as prologues inside
+    chained GEMM launches (grid-wide barriers between stages) gives the same results."""
+    monkeypatch.setenv("DREAM_CHAIN", "1")
+    pr, s = _run("llava7b", 2, n_layers=2, decode_steps=4)
