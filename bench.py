@@ -158,9 +158,14 @@ def main():
     ap.add_argument("--workload", default="llava7b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-gemm", type=int, default=1)
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: cut the target to this many layers (the line's workload name says so)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     p = dict(configs.PRESETS[args.workload])
+    if args.layers:
+        p = configs.scaled(args.workload, n_layers=args.layers)
+        p["name"] = "%s[n_layers=%d]" % (p["name"], args.layers)
     if args.impl == "reference":
         return run_reference(args, p)
 

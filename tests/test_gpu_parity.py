@@ -44,6 +44,23 @@ def test_smolvlm_shape_full_bf16():
     pr, s = _run("smolvlm2b", 4)
 
 
+@pytest.mark.parametrize("batch", [2, 4])
+def test_llava_shape_batched(batch):
+    """Several sequences per call: 2 x 61 tree rows take the two-plane GEMM input layout, 4 x 61 rows
+    are cut into 64-row launches; every sequence is checked against its own oracle run."""
+    from tests.parity import Pair
+    pr = Pair("llava7b", max_batch=batch, n_layers=2, n_visual=192, k_visual=48, n_prompt=64, decode_steps=4)
+    try:
+        seqs = tuple(range(batch))
+        for s in seqs:
+            pr.prefill(seq=s, seq_seed=s)
+        for _ in range(2):
+            pr.step(seqs=seqs)
+        print(json.dumps(pr.summary(), default=float))
+    finally:
+        pr.close()
+
+
 def test_chained_gemm_launches(monkeypatch):
     """The optional mode in which norms, gating and the attention merge run as prologues inside
     chained GEMM launches (grid-wide barriers between stages) gives the same results."""
