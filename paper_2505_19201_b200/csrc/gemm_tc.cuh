@@ -44,6 +44,8 @@
 enum { TC_X_PLAIN = 0, TC_X_INTERLEAVED = 1, TC_X_PLANAR = 2 };
 
 #define TC_MAX_STAGES 4
+#define TC_STG_LD 36            // floats per row of an epilogue staging tile (32 + padding)
+#define TC_STG_BYTES (8 * 16 * TC_STG_LD * 4)
 
 // One GEMM of a chain, preceded by the row-wise work that produces its input.
 struct TcStage {
@@ -177,6 +179,7 @@ k_gemm_tc(const __grid_constant__ TcMaps maps, const __grid_constant__ TcChain p
   uint64_t *acc_full = empty_x + p.x_stages, *acc_empty = acc_full + 2;
   uint32_t *tmem_base_p = (uint32_t *)(acc_empty + 2);
   volatile int *abort_flag = (volatile int *)(tmem_base_p + 1);
+  float *stage_tiles = (float *)(bars + 64);               // 8 warps x [16][TC_STG_LD] floats, 512 bytes behind the barriers' start
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (blockIdx.x == 0 && threadIdx.x == 0) trace_stamp(TR_none);     // CTA start, before any dependency
@@ -317,10 +320,10 @@ k_gemm_tc(const __grid_constant__ TcMaps maps, const __grid_constant__ TcChain p
     const int q = warp & 3;                   // TMEM lane quarter this warp may read
     const int half = warp >= 7 ? 1 : 0;       // which 128 accumulator columns this warp drains
     const int ptid = (warp < 7 ? warp - 2 : warp - 3) * 32 + lane;      // 0..255 among these warps
+    float *stg = stage_tiles + (ptid >> 5) * (16 * TC_STG_LD);          // this warp's staging tile
     pdl_wait();                               // inputs and the output buffer belong to earlier kernels
     const bool inter = p.st[0].x_mode == TC_X_INTERLEAVED;
     const int row = q * 32 + lane;            // accumulator lane = X row
-    const int token = inter ? row >> 1 : row;
     const int part = inter ? lane & 1 : 0;
     uint32_t seg = 0;
     bool live = true;
@@ -352,9 +355,12 @@ k_gemm_tc(const __grid_constant__ TcMaps maps, const __grid_constant__ TcChain p
         tc_fence_after();
         int first_cta = (tile * S.KB) / S.upc;
         int slot = (int)blockIdx.x - first_cta;
-        float *dst = S.out + (long long)slot * S.slot_stride + (long long)token * S.N + tile * TC_BN;
+        float *dst0 = S.out + (long long)slot * S.slot_stride + tile * TC_BN;       // row 0 of this CTA's slot, first column of the tile
         uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * TC_BN;
-        // four chunks of 32 columns; the TMEM load of chunk i+1 is in flight while chunk i is stored
+        // four chunks of 32 columns; the TMEM load of chunk i+1 is in flight while chunk i is stored.
+        // A lane holds values of one row, but a store instruction is cheapest when the lanes of a
+        // warp cover whole 128-byte runs of a row: the chunk goes through a [16][32] tile in shared
+        // memory (rows padded to 36 floats) and leaves as 4 stores of 4 rows x 128 bytes.
         uint32_t ra[32], rb[32];
         tmem_ld32(taddr + (uint32_t)half * 128u, ra);
 #pragma unroll
@@ -363,32 +369,52 @@ k_gemm_tc(const __grid_constant__ TcMaps maps, const __grid_constant__ TcChain p
           uint32_t (&r)[32] = (ci & 1) ? rb : ra;
           tmem_ld_wait();
           if (ci + 1 < 4) tmem_ld32(taddr + (uint32_t)(col0 + 32), (ci & 1) ? ra : rb);
+          const int c4 = (lane & 7) * 4;
+          const bool col_ok = tile * TC_BN + col0 + c4 < S.N;
           if (inter) {
             // lanes 2t and 2t+1 hold the products of token t's high and low parts.  The even lane
-            // stores columns 0..15 of the chunk and the odd lane 16..31: each sends the partner
+            // keeps columns 0..15 of the chunk and the odd lane 16..31: each sends the partner
             // the 16 values it needs and adds what it receives to its own.
-            float v[16];
+            float4 *srow = reinterpret_cast<float4 *>(stg + (lane >> 1) * TC_STG_LD + part * 16);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              float send = __uint_as_float(part ? r[j] : r[16 + j]);
-              float mine = __uint_as_float(part ? r[16 + j] : r[j]);
-              v[j] = mine + __shfl_xor_sync(0xffffffffu, send, 1);
-            }
-            if (token < S.n_tok) {
+            for (int j4 = 0; j4 < 4; ++j4) {
+              float v[4];
 #pragma unroll
-              for (int j4 = 0; j4 < 4; ++j4) {
-                int jj = part * 16 + j4 * 4;
-                if (tile * TC_BN + col0 + jj < S.N)
-                  *reinterpret_cast<float4 *>(dst + col0 + jj) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
+              for (int e = 0; e < 4; ++e) {
+                const int j = j4 * 4 + e;
+                float send = __uint_as_float(part ? r[j] : r[16 + j]);
+                float mine = __uint_as_float(part ? r[16 + j] : r[j]);
+                v[e] = mine + __shfl_xor_sync(0xffffffffu, send, 1);
               }
+              srow[j4] = make_float4(v[0], v[1], v[2], v[3]);
             }
-          } else if (token < S.n_tok) {
+            __syncwarp();
 #pragma unroll
-            for (int j4 = 0; j4 < 8; ++j4) {
-              if (tile * TC_BN + col0 + j4 * 4 < S.N)
-                *reinterpret_cast<float4 *>(dst + col0 + j4 * 4) =
-                    make_float4(__uint_as_float(r[j4 * 4]), __uint_as_float(r[j4 * 4 + 1]), __uint_as_float(r[j4 * 4 + 2]),
-                                __uint_as_float(r[j4 * 4 + 3]));
+            for (int i = 0; i < 4; ++i) {
+              const int tl = i * 4 + (lane >> 3), tok = q * 16 + tl;
+              float4 val = *reinterpret_cast<const float4 *>(stg + tl * TC_STG_LD + c4);
+              if (tok < S.n_tok && col_ok) *reinterpret_cast<float4 *>(dst0 + (long long)tok * S.N + col0 + c4) = val;
+            }
+            __syncwarp();
+          } else {
+            // one row per lane: two halves of 16 rows through the same tile
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              if ((lane >> 4) == h) {
+                float4 *srow = reinterpret_cast<float4 *>(stg + (lane & 15) * TC_STG_LD);
+#pragma unroll
+                for (int j4 = 0; j4 < 8; ++j4)
+                  srow[j4] = make_float4(__uint_as_float(r[j4 * 4]), __uint_as_float(r[j4 * 4 + 1]), __uint_as_float(r[j4 * 4 + 2]),
+                                         __uint_as_float(r[j4 * 4 + 3]));
+              }
+              __syncwarp();
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int tl = i * 4 + (lane >> 3), tok = q * 32 + h * 16 + tl;
+                float4 val = *reinterpret_cast<const float4 *>(stg + tl * TC_STG_LD + c4);
+                if (tok < S.n_tok && col_ok) *reinterpret_cast<float4 *>(dst0 + (long long)tok * S.N + col0 + c4) = val;
+              }
+              __syncwarp();
             }
           }
         }
@@ -548,7 +574,7 @@ static inline bool gemm_tc_launch_chain(GemmTcPlan *pl, cudaStream_t stream, int
   int grid = any_pro ? pl->n_sms : max_grid;
   int xstage = p.wp * (x_mode == TC_X_PLANAR ? 2 * TC_XTILE : TC_XTILE);
   p.x_stages = 2;
-  int budget = pl->max_smem - 2048 - p.x_stages * xstage;
+  int budget = pl->max_smem - 2048 - TC_STG_BYTES - p.x_stages * xstage;
   p.w_stages = budget / (p.wp * TC_WPANEL);
   if (p.w_stages > 8) p.w_stages = 8;
   if (p.w_stages < 2) return false;
@@ -557,7 +583,7 @@ static inline bool gemm_tc_launch_chain(GemmTcPlan *pl, cudaStream_t stream, int
   p.bar_counter = pl->bar_counter;
   p.bar_base = pl->bar_total;
   int n_bars = (d[0].pro.kind != PRO_NONE ? 1 : 0) + 2 * (n - 1);
-  size_t smem = (size_t)p.w_stages * p.wp * TC_WPANEL + (size_t)p.x_stages * xstage + 1024 + 512;
+  size_t smem = (size_t)p.w_stages * p.wp * TC_WPANEL + (size_t)p.x_stages * xstage + 1024 + 512 + TC_STG_BYTES;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
   cudaLaunchAttribute attr[1];
