@@ -15,7 +15,6 @@
 #pragma once
 #include "common.cuh"
 #include "rows.cuh"
-#include "prologue.cuh"
 
 #define AM_ROWS 64
 #define AM_THREADS 128
@@ -59,7 +58,7 @@ struct FlatKV2 {
 
 struct AttnMmaArgs {
   const bf16 *q;                    // [R][H][2][hd] queries (rotary applied, unscaled): high row, low row
-  const int *row_seq;               // [R] sequence of each row
+  int slot_seq[DREAM_MAX_BATCH];    // sequence of each query-row slot (grid z)
   const int *row_in;                // [R] or null: rows with a negative entry are idle; index into anc
   const int *prefix_len;            // by sequence: keys [0, prefix) are visible to every row
   const uint32_t *mask;             // [R][4] visible tail keys, or null when anc is given
@@ -103,13 +102,42 @@ k_attn_mma(AttnMmaArgs a) {
   const int chunk = blockIdx.x, kvh = blockIdx.y / a.n_rt, rt = blockIdx.y - kvh * a.n_rt, slot = blockIdx.z;
   const int Hkv = a.H / a.G;
   const int r_base = slot * a.rows_per_seq;
-  const int seq = a.row_seq[r_base];
+  const int seq = a.slot_seq[slot];
+  if (PAGED && tid < a.blocks_per_chunk + 1) {       // page-table entries of this chunk's blocks, on their way to L1 meanwhile
+    const int j = min((chunk * a.blocks_per_chunk + tid) * KBLK, a.paged.pages_per_seq * a.paged.page_tokens - 1);
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(a.paged.page_table + seq * a.paged.pages_per_seq + (j >> a.paged.page_shift)));
+  }
   const int P = a.prefix_len[seq];
   const int total_keys = P + a.tail_len;
   const int nb = (total_keys + KBLK - 1) / KBLK;
   const int b0 = chunk * a.blocks_per_chunk, b1 = min(nb, b0 + a.blocks_per_chunk);
   const int rows_total = a.rows_per_seq * a.G;
 
+  auto load_block = [&](int blk, int buf, bool commit) {
+    bf16 *dstb = KV + buf * BUF_ELEMS;
+    for (int idx = tid; idx < KBLK * (HD / 8); idx += AM_THREADS) {
+      int row = idx / (HD / 8), sg = idx - row * (HD / 8);
+      int j = blk * KBLK + row;
+      bool ok = j < total_keys;
+      uint32_t dk = smem_addr(dstb + row * LD + sg * 8), dv = dk + PLANES * PLANE_ELEMS * 2;
+      if (PAGED) {
+        const bf16 *Kp = (const bf16 *)a.paged.base, *Vp = Kp + a.paged.kv_stride;
+        long long o = ok ? a.paged.off(seq, j, kvh) + sg * 8 : 0;
+        cp_async16(dk, Kp + o, ok ? 16 : 0);
+        cp_async16(dv, Vp + o, ok ? 16 : 0);
+      } else {
+        long long ok_ = ok ? a.flat.off(seq, 0, kvh, j) + sg * 8 : 0, ov_ = ok ? a.flat.off(seq, 1, kvh, j) + sg * 8 : 0;
+        cp_async16(dk, a.flat.base + ok_, ok ? 16 : 0);
+        cp_async16(dk + PLANE_ELEMS * 2, a.flat.base + ok_ + (ok ? HD : 0), ok ? 16 : 0);
+        cp_async16(dv, a.flat.base + ov_, ok ? 16 : 0);
+        cp_async16(dv + PLANE_ELEMS * 2, a.flat.base + ov_ + (ok ? HD : 0), ok ? 16 : 0);
+      }
+    }
+    if (commit) cp_async_commit();
+  };
+
+  // the first K/V block does not depend on the row table: its copies start before the table is built
+  if (b0 < b1) load_block(b0, 0, false);
   // ---- row table: global row, head and tail mask of each of the 64 rows
   if (tid < AM_ROWS) {
     int rr = rt * AM_ROWS + tid, r = -1, h = 0;
@@ -131,7 +159,7 @@ k_attn_mma(AttnMmaArgs a) {
     for (int wd = 0; wd < 4; ++wd) mwords[tid * 4 + wd] = mw[wd];
   }
   __syncthreads();
-  // ---- queries: high and low rows copied asynchronously (joins the first K/V block's group)
+  // ---- queries: high and low rows copied asynchronously (same group as the first K/V block)
   for (int idx = tid; idx < AM_ROWS * (HD / 8); idx += AM_THREADS) {
     int lr = idx / (HD / 8), sg = idx - lr * (HD / 8);
     int r = row_r[lr];
@@ -140,28 +168,7 @@ k_attn_mma(AttnMmaArgs a) {
     cp_async16(smem_addr(Ql + lr * LD + sg * 8), src + (r >= 0 ? HD : 0), r >= 0 ? 16 : 0);
   }
 
-  auto load_block = [&](int blk, int buf) {
-    bf16 *dstb = KV + buf * BUF_ELEMS;
-    for (int idx = tid; idx < KBLK * (HD / 8); idx += AM_THREADS) {
-      int row = idx / (HD / 8), sg = idx - row * (HD / 8);
-      int j = blk * KBLK + row;
-      bool ok = j < total_keys;
-      uint32_t dk = smem_addr(dstb + row * LD + sg * 8), dv = dk + PLANES * PLANE_ELEMS * 2;
-      if (PAGED) {
-        const bf16 *Kp = (const bf16 *)a.paged.base, *Vp = Kp + a.paged.kv_stride;
-        long long o = ok ? a.paged.off(seq, j, kvh) + sg * 8 : 0;
-        cp_async16(dk, Kp + o, ok ? 16 : 0);
-        cp_async16(dv, Vp + o, ok ? 16 : 0);
-      } else {
-        long long ok_ = ok ? a.flat.off(seq, 0, kvh, j) + sg * 8 : 0, ov_ = ok ? a.flat.off(seq, 1, kvh, j) + sg * 8 : 0;
-        cp_async16(dk, a.flat.base + ok_, ok ? 16 : 0);
-        cp_async16(dk + PLANE_ELEMS * 2, a.flat.base + ok_ + (ok ? HD : 0), ok ? 16 : 0);
-        cp_async16(dv, a.flat.base + ov_, ok ? 16 : 0);
-        cp_async16(dv + PLANE_ELEMS * 2, a.flat.base + ov_ + (ok ? HD : 0), ok ? 16 : 0);
-      }
-    }
-    cp_async_commit();
-  };
+  cp_async_commit();
 
   float o_acc[NT_O][4];
 #pragma unroll
@@ -177,10 +184,10 @@ k_attn_mma(AttnMmaArgs a) {
   const int k_row = l7 + (mi >> 1) * 8, k_col = (mi & 1) * 8;          // K fragments (non-transposed)
   const int v_row = l7 + (mi & 1) * 8, v_col = (mi >> 1) * 8;          // V fragments (transposed)
 
-  if (b0 < b1) load_block(b0, 0); else { cp_async_commit(); cp_async_wait<0>(); }
+  if (b0 >= b1) cp_async_wait<0>();
   for (int blk = b0; blk < b1; ++blk) {
     const int buf = (blk - b0) & 1;
-    if (blk + 1 < b1) { load_block(blk + 1, buf ^ 1); cp_async_wait<1>(); } else cp_async_wait<0>();
+    if (blk + 1 < b1) { load_block(blk + 1, buf ^ 1, true); cp_async_wait<1>(); } else cp_async_wait<0>();
     __syncthreads();
     const bf16 *Kb = KV + buf * BUF_ELEMS, *Vb = Kb + PLANES * PLANE_ELEMS;
     // ---- S = Q K^T
@@ -310,15 +317,51 @@ k_attn_mma(AttnMmaArgs a) {
 }
 
 // Merge of the chunk partials: out[r][h] = sum_c w_c O_c / sum_c w_c l_c with w_c = 2^(m_c - max m).
-// One thread per (row, head, four output columns); grid = ceil(R * H * hd / 4 / 256).
+// One thread per (row, head, four output columns); grid = ceil(R * H * hd / 4 / 256).  Partials are
+// laid out [slot][chunk][kv head][row tile][64][hd].
 template <int HD>
 __global__ void __launch_bounds__(256)
 k_attn_combine(AttnMmaArgs a, int R) {
   kernel_entry(TR_k_attn_combine);
   long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)R * a.H * (HD / 4)) return;
-  ProCombine pc;
-  pc.part_o = a.part_o; pc.part_ml = a.part_ml; pc.row_in = a.row_in; pc.n_chunks = a.n_chunks; pc.n_rt = a.n_rt;
-  pc.H = a.H; pc.G = a.G; pc.rows_per_seq = a.rows_per_seq; pc.hd = HD; pc.out = reinterpret_cast<bf16 *>(a.out); pc.lay = a.lay;
-  pro_combine_item(pc, idx);
+  constexpr int Q4 = HD >> 2;
+  int c4 = (int)(idx % Q4);
+  long long rh = idx / Q4;
+  int h = (int)(rh % a.H), r = (int)(rh / a.H);
+  if (a.row_in && a.row_in[r] < 0) return;
+  const int Hkv = a.H / a.G;
+  int slot = r / a.rows_per_seq, node = r - slot * a.rows_per_seq;
+  int kvh = h / a.G, rr = node * a.G + (h - kvh * a.G);
+  int rt = rr >> 6, lr = rr & 63;
+  const long long cstride = (long long)Hkv * a.n_rt * 64;
+  const long long p0 = (((long long)slot * a.n_chunks * Hkv + kvh) * a.n_rt + rt) * 64 + lr;
+  // chunks in rounds of four: (m, l) pairs and output vectors are fetched together, the running
+  // maximum rescales what has been accumulated (same result as a two-pass merge up to rounding)
+  float M = -INFINITY, L = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int c0 = 0; c0 < a.n_chunks; c0 += 4) {
+    float2 ml[4];
+    float4 o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      bool ok = c0 + k < a.n_chunks;
+      long long pr = p0 + (long long)(ok ? c0 + k : c0) * cstride;
+      ml[k] = ok ? __ldcg(reinterpret_cast<const float2 *>(a.part_ml + pr * 2)) : make_float2(-INFINITY, 0.f);
+      o[k] = ok ? __ldcg(reinterpret_cast<const float4 *>(a.part_o + pr * HD + c4 * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (ml[k].x == -INFINITY) continue;
+      float Mn = fmaxf(M, ml[k].x);
+      float sc = exp2f(M - Mn), w = exp2f(ml[k].x - Mn);       // exp2(-inf) = 0 on the first live chunk
+      L = L * sc + ml[k].y * w;
+      acc.x = acc.x * sc + o[k].x * w; acc.y = acc.y * sc + o[k].y * w;
+      acc.z = acc.z * sc + o[k].z * w; acc.w = acc.w * sc + o[k].w * w;
+      M = Mn;
+    }
+  }
+  float inv = L > 0.f ? 1.f / L : 0.f;
+  store_split4<bf16>(reinterpret_cast<bf16 *>(a.out) + r * a.lay.row_stride + h * HD + c4 * 4, a.lay.lo_delta,
+                     make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
 }

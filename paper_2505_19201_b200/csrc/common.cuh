@@ -7,6 +7,8 @@
 
 typedef __nv_bfloat16 bf16;
 
+#define DREAM_MAX_BATCH 8          // sequences one call may list
+
 #define DREAM_DEV_OK 0
 #define DREAM_DEV_TIMEOUT 1
 #define DREAM_DEV_BAD_INDEX 2

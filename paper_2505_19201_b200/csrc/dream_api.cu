@@ -43,8 +43,6 @@ struct dream_ctx {
   void *kv_pool;
   long long kv_stride, layer_stride;
   int *page_table, *status;
-  unsigned long long *bar_counter;     // grid-barrier arrivals of the chained GEMM launches
-  int use_chain;
   SeqDev sd;
   float *dself, *dmem;
   DraftTreeDev dt;
@@ -60,6 +58,7 @@ struct dream_ctx {
   float *am_part_o, *am_part_ml;       // split-K attention partials
   int am_rt_max;
   int key_ub[DREAM_MAX_BATCH];         // upper bound of the draft caches' permanent rows
+  int cur_seq[DREAM_MAX_BATCH];        // sequences of the call being enqueued, by slot
   int tk_nsplit;
   int *top_id, *argmax_i, *accept_len_i, *out_tokens_i, *comp_src_i;
   size_t gout_floats;
@@ -212,7 +211,6 @@ static size_t carve(dream_ctx *c, char *base) {
   c->kv_pool = a.take_bytes((size_t)f.n_layers * c->layer_stride * e);
   c->page_table = a.take<int>((size_t)MB * c->pps);
   c->status = a.take<int>(64);
-  c->bar_counter = a.take<unsigned long long>(32);
   int *st = a.take<int>((size_t)MB * (9 + 3 * (DREAM_MAX_DEPTH + 1)));
   if (base) {
     c->sd.P = st; c->sd.pending = st + MB; c->sd.tap = st + 2 * MB; c->sd.nperm_d = st + 3 * MB;
@@ -363,57 +361,6 @@ static GemmOut gemm(dream_ctx *c, const void *W, const void *X, XMode m, int row
   return g;
 }
 
-// Chained launches: up to TC_MAX_STAGES GEMMs, each with the row-wise work that makes its input
-// as a prologue, in one kernel.  Only for bf16 row sets that fit one launch.
-static bool chain_ok(const dream_ctx *c, int R) {
-  return c->use_chain && R <= (xmode(c, R).mode == TC_X_INTERLEAVED ? TC_ROWS_SPLIT_1MMA : TC_ROWS_MAX);
-}
-static Prologue pro_none() {
-  Prologue p;
-  memset(&p, 0, sizeof(p));
-  p.kind = PRO_NONE;
-  return p;
-}
-static Prologue pro_norm(dream_ctx *c, float *x, const GemmOut &gin, bool has_in, const void *gain, int rows, XMode m,
-                         float *copy = nullptr, const int *row_seq = nullptr, const int *tap = nullptr, int layer = 0,
-                         bool want_raw = false) {
-  Prologue p = pro_none();
-  p.kind = PRO_NORM; p.rows = rows;
-  p.norm.x = x; p.norm.gin = gin; p.norm.has_in = has_in ? 1 : 0; p.norm.gain = (const bf16 *)gain;
-  p.norm.eps = c->cfg.rms_eps; p.norm.d = c->cfg.d_model; p.norm.xn = (bf16 *)c->xn; p.norm.copy = copy;
-  p.norm.row_seq = row_seq; p.norm.tap_state = tap; p.norm.layer = layer;
-  p.norm.raw = want_raw ? (bf16 *)c->raw : nullptr; p.norm.lay = xlay(m, c->cfg.d_model);
-  return p;
-}
-static Prologue pro_silu(dream_ctx *c, const GemmOut &g, int rows, XMode m) {
-  Prologue p = pro_none();
-  p.kind = PRO_SILU; p.rows = rows;
-  p.silu.g = g; p.silu.act = (bf16 *)c->act; p.silu.ff = c->cfg.d_ff; p.silu.lay = xlay(m, c->cfg.d_ff);
-  return p;
-}
-struct ChainGemm { const void *W, *X; int N, K; Prologue pro; };
-// Launches the chain; out[i] describes GEMM i's result.  All results share the context's GEMM
-// output buffer: stage i's consumers are stage i+1's prologue, and the last one's the caller.
-static void gemm_chain(dream_ctx *c, int n, const ChainGemm *cg, XMode m, int rows, GemmOut *out, bool launch = true) {
-  GemmTcDesc d[TC_MAX_STAGES];
-  double bytes = 0.0;
-  for (int i = 0; i < n; ++i) {
-    d[i].W = cg[i].W; d[i].X = cg[i].X; d[i].x_mode = m.mode; d[i].lo_rows = m.lo_rows; d[i].rows = rows; d[i].slot_rows = rows;
-    d[i].N = cg[i].N; d[i].K = cg[i].K; d[i].out = c->gout; d[i].out_floats = (long long)c->gout_floats; d[i].pro = cg[i].pro;
-    bytes += 2.0 * cg[i].N * cg[i].K;
-  }
-  if (!launch) {                                   // only the output descriptors are wanted
-    if (!gemm_tc_launch_chain(&c->tc, c->stream, n, d, out, false)) c->gemm_failed = 1;
-    return;
-  }
-  bool timed = c->prof_on && 2 * (c->prof_n + 1) <= (int)c->prof_ev.size();
-  if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], c->stream);
-  if (!gemm_tc_launch_chain(&c->tc, c->stream, n, d, out)) c->gemm_failed = 1;
-  if (timed) { cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], c->stream); c->prof_n++; c->prof_bytes += bytes; }
-  c->launches++;
-  c->tc_launches++;
-}
-
 static PagedKV paged(dream_ctx *c, int layer) {
   PagedKV kv;
   kv.base = (char *)c->kv_pool + (size_t)layer * c->layer_stride * c->esz;
@@ -484,12 +431,8 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   const char *pdl = getenv("DREAM_PDL");              // "0" serialises every launch (debugging aid)
   c->use_pdl = !(pdl && !strcmp(pdl, "0"));
   c->use_tc = cfg->dtype == DREAM_BF16;
-  // "1": row-wise steps run as prologues inside chained GEMM launches (fewer kernels, grid-wide
-  // barriers instead); measured slower than one kernel per step on B200, so it is off by default
-  const char *chain = getenv("DREAM_CHAIN");
-  c->use_chain = c->use_tc && chain && !strcmp(chain, "1");
   if (c->use_tc) {
-    const char *why = gemm_tc_plan_init(&c->tc, c->status, c->bar_counter, c->use_pdl);
+    const char *why = gemm_tc_plan_init(&c->tc, c->status, c->use_pdl);
     if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
   }
   if (c->use_tc) {
@@ -601,9 +544,10 @@ template <typename T, int HD> struct AttnLaunch {
   }
   // Split-K plan and launch of the tensor-core attention (bf16 configurations).
   template <bool PAGED>
-  static void mma(dream_ctx *c, AttnMmaArgs a, int B, int rows_per_seq, int key_ub, Prologue *defer) {
+  static void mma(dream_ctx *c, AttnMmaArgs a, int B, int rows_per_seq, int key_ub) {
     const dream_config &f = c->cfg;
     constexpr int KBLK = AmShape<HD>::KBLK;
+    for (int b = 0; b < DREAM_MAX_BATCH; ++b) a.slot_seq[b] = b < B ? c->cur_seq[b] : 0;
     a.q = (const bf16 *)c->qbuf; a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
     a.n_rt = (rows_per_seq * a.G + AM_ROWS - 1) / AM_ROWS;
@@ -615,24 +559,18 @@ template <typename T, int HD> struct AttnLaunch {
     a.out = c->attn_out;
     dim3 grid(a.n_chunks, f.n_kv_heads * a.n_rt, B);
     LAUNCH(c, (k_attn_mma<HD, PAGED>), grid, AM_THREADS, (attn_mma_smem<HD, PAGED>()), a);
-    if (defer) *defer = pro_none();
-    if (a.n_chunks > 1 && defer) {            // the merge of the chunks becomes the next GEMM's prologue
-      defer->kind = PRO_COMBINE; defer->rows = B * rows_per_seq;
-      ProCombine &pc = defer->comb;
-      pc.part_o = a.part_o; pc.part_ml = a.part_ml; pc.row_in = a.row_in; pc.n_chunks = a.n_chunks; pc.n_rt = a.n_rt;
-      pc.H = a.H; pc.G = a.G; pc.rows_per_seq = rows_per_seq; pc.hd = HD; pc.out = (bf16 *)a.out; pc.lay = a.lay;
-    } else if (a.n_chunks > 1) {
+    if (a.n_chunks > 1) {
       long long items = (long long)B * rows_per_seq * f.n_heads * (HD / 4);
       LAUNCH(c, (k_attn_combine<HD>), (unsigned)((items + 255) / 256), 256, 0, a, B * rows_per_seq);
     }
   }
-  static void tree(dream_ctx *c, int layer, int R, XMode m, int B, int key_ub, Prologue *defer) {
+  static void tree(dream_ctx *c, int layer, int R, XMode m, int B, int key_ub) {
     if (sizeof(T) == 2) {
       AttnMmaArgs a = {};
       a.next_w.ptr = (const char *)c->wo[layer]; a.next_w.bytes = (unsigned long long)c->cfg.d_model * c->Hhd * 2;
-      a.row_seq = c->rm[0].seq; a.row_in = nullptr; a.prefix_len = c->sd.P; a.mask = c->vmask; a.anc = nullptr;
+      a.row_in = nullptr; a.prefix_len = c->sd.P; a.mask = c->vmask; a.anc = nullptr;
       a.tail_len = c->T; a.lay = xlay(m, c->Hhd); a.paged = paged(c, layer);
-      mma<true>(c, a, B, c->T, key_ub, defer);
+      mma<true>(c, a, B, c->T, key_ub);
       return;
     }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
@@ -640,13 +578,13 @@ template <typename T, int HD> struct AttnLaunch {
            c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
   }
   static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, XMode m, int B,
-                    int rows_per_seq, int key_ub, Prologue *defer) {
+                    int rows_per_seq, int key_ub) {
     if (sizeof(T) == 2) {
       AttnMmaArgs a = {};
-      a.row_seq = rm.seq; a.row_in = rm.in; a.prefix_len = nperm; a.mask = nullptr; a.anc = c->dt.in_anc;
+      a.row_in = rm.in; a.prefix_len = nperm; a.mask = nullptr; a.anc = c->dt.in_anc;
       a.anc_stride = c->ts.NI; a.strict = strict; a.tail_len = c->ts.NI; a.lay = xlay(m, c->Hhd);
       a.flat.base = (bf16 *)cache; a.flat.cap = c->cap_rows; a.flat.hkv = c->cfg.n_kv_heads; a.flat.hd = HD;
-      mma<false>(c, a, B, rows_per_seq, key_ub, defer);
+      mma<false>(c, a, B, rows_per_seq, key_ub);
       return;
     }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
@@ -848,6 +786,7 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
   const dream_config &f = c->cfg;
   const TreeShape &ts = c->ts;
   int d = f.d_model, cur = 0;
+  for (int b = 0; b < B; ++b) c->cur_seq[b] = tb.seq[b];
   int key_ub = 0;                 // most keys any listed sequence can hold in a draft cache
   for (int b = 0; b < B; ++b) key_ub = imax(key_ub, c->key_ub[tb.seq[b]] + ts.D + 1 + ts.NI);
   for (int p = 1; p <= ts.D; ++p) {
@@ -858,50 +797,23 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
     LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
     GemmOut g;
-    if (sizeof(T) == 2 && chain_ok(c, R)) {
-      // [norm -> QKV] | rotary | self-attention | [merge -> O] [norm -> cross Q] | cross-attention |
-      // [merge -> cross O] [norm -> gate/up] [SiLU -> down] | [final norm -> memory K/V] | append | LM head
-      ChainGemm a1 = {c->dw.wqkv, c->xn, c->qkvN, d, pro_norm(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm)};
-      gemm_chain(c, 1, &a1, xm, R, &g);
-      LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
-      Prologue merge;
-      HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub, &merge));
-      GemmOut go[3];
-      ChainGemm a2[2] = {{c->dw.wo, c->attn_out, d, c->Hhd, merge}, {c->dw.xq, c->xn, c->Hhd, d, pro_none()}};
-      gemm_chain(c, 2, a2, xm, R, go, false);
-      a2[1].pro = pro_norm(c, c->x, go[0], true, c->dw.lnx, R, xm);
-      gemm_chain(c, 2, a2, xm, R, go);
-      LAUNCH(c, k_gemm_to_q, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, go[1], c->qbuf, f.n_heads, f.head_dim, 1);
-      HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm, B, m, key_ub, &merge));
-      ChainGemm a3[3] = {{c->dw.xo, c->attn_out, d, c->Hhd, merge}, {c->dw.wgu, c->xn, 2 * f.d_ff, d, pro_none()}, {c->dw.wd, c->act, d, f.d_ff, pro_none()}};
-      gemm_chain(c, 3, a3, xm, R, go, false);
-      a3[1].pro = pro_norm(c, c->x, go[0], true, c->dw.ln2, R, xm);
-      a3[2].pro = pro_silu(c, go[1], R, xm);
-      gemm_chain(c, 3, a3, xm, R, go);
-      // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
-      ChainGemm a4 = {c->dw.xkv, c->raw, c->kvN, d, pro_norm(c, c->x, go[2], true, c->ln_f, R, xm, nullptr, nullptr, nullptr, 0, true)};
-      gemm_chain(c, 1, &a4, xm, R, &g);
-      LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
-      g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
-    } else {
-      norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
-      g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
-      LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
-      HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub, nullptr));
-      g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
-      norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
-      g = gemm<T>(c, c->dw.xq, c->xn, xm, R, c->Hhd, d);
-      LAUNCH(c, k_gemm_to_q, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, f.n_heads, f.head_dim, sizeof(T) == 2 ? 1 : 0);
-      HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm, B, m, key_ub, nullptr));
-      g = gemm<T>(c, c->dw.xo, c->attn_out, xm, R, d, c->Hhd);
-      norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, xm);
-      g = mlp_rows<T>(c, c->dw.wgu, c->dw.wd, R, xm);
-      // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
-      norm_rows<T>(c, c->x, g, true, c->ln_f, R, xm, nullptr, nullptr, nullptr, 0, true);
-      g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
-      LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
-      g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
-    }
+    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
+    g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
+    LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
+    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub));
+    g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
+    g = gemm<T>(c, c->dw.xq, c->xn, xm, R, c->Hhd, d);
+    LAUNCH(c, k_gemm_to_q, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, f.n_heads, f.head_dim, sizeof(T) == 2 ? 1 : 0);
+    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm, B, m, key_ub));
+    g = gemm<T>(c, c->dw.xo, c->attn_out, xm, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, xm);
+    g = mlp_rows<T>(c, c->dw.wgu, c->dw.wd, R, xm);
+    // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
+    norm_rows<T>(c, c->x, g, true, c->ln_f, R, xm, nullptr, nullptr, nullptr, 0, true);
+    g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
+    LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
+    g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
     LAUNCH(c, k_topk_lse, dim3(R, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, ts.K, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
     int next_m = p < ts.D ? ts.beam[p] : 1;
     LAUNCH(c, k_tree_expand, B, 128, 0, tb, c->sd, c->dt, ts, p, m, c->top_val, c->top_id, c->lse_rows, rn, next_m);
@@ -934,46 +846,22 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
   const XMode xm = xmode(c, R);
   RowMeta &rm = c->rm[0];
   int key_ub = 0;
-  for (int b = 0; b < B; ++b) key_ub = imax(key_ub, c->p_ub[tb.seq[b]] + c->T);
+  for (int b = 0; b < B; ++b) { key_ub = imax(key_ub, c->p_ub[tb.seq[b]] + c->T); c->cur_seq[b] = tb.seq[b]; }
   LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
   LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
   GemmOut gd = NO_GEMM, g;
-  const bool chained = sizeof(T) == 2 && chain_ok(c, R);
   for (int l = 0; l < L; ++l) {
     // the first norm completes S^l (for l >= 1) and captures it where a sequence taps layer l
-    if (chained) {
-      // [norm -> QKV] | rotary, cache append | attention | [merge -> O] [norm -> gate/up] [SiLU -> down]
-      ChainGemm a1 = {c->wqkv[l], c->xn, c->qkvN, d,
-                      pro_norm(c, c->x, gd, l > 0, c->ln1[l], R, xm, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l)};
-      gemm_chain(c, 1, &a1, xm, R, &g);
-      LAUNCH(c, (k_qkv_post_target<T>), dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv);
-      Prologue merge;
-      HD_DISPATCH(c, T, tree(c, l, R, xm, B, key_ub, &merge));
-      GemmOut go[3];
-      // the descriptors of stage i's output are known before the launch: they depend on shapes only
-      ChainGemm a3[3] = {{c->wo[l], c->attn_out, d, c->Hhd, merge}, {c->wgu[l], c->xn, 2 * f.d_ff, d, pro_none()}, {c->wd[l], c->act, d, f.d_ff, pro_none()}};
-      gemm_chain(c, 3, a3, xm, R, go, false);
-      a3[1].pro = pro_norm(c, c->x, go[0], true, c->ln2[l], R, xm);
-      a3[2].pro = pro_silu(c, go[1], R, xm);
-      gemm_chain(c, 3, a3, xm, R, go);
-      gd = go[2];
-      continue;
-    }
     norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, xm, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
     g = gemm<T>(c, c->wqkv[l], c->xn, xm, R, c->qkvN, d);
     LAUNCH(c, (k_qkv_post_target<T>), dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv);
-    HD_DISPATCH(c, T, tree(c, l, R, xm, B, key_ub, nullptr));
+    HD_DISPATCH(c, T, tree(c, l, R, xm, B, key_ub));
     g = gemm<T>(c, c->wo[l], c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->ln2[l], R, xm);
     gd = mlp_rows<T>(c, c->wgu[l], c->wd[l], R, xm);
   }
-  if (chained) {
-    ChainGemm a1 = {c->lm_head, c->xn, f.vocab, d, pro_norm(c, c->x, gd, true, c->ln_f, R, xm, c->tapbuf, rm.seq, c->sd.tap, L)};
-    gemm_chain(c, 1, &a1, xm, R, &g);
-  } else {
-    norm_rows<T>(c, c->x, gd, true, c->ln_f, R, xm, c->tapbuf, rm.seq, c->sd.tap, L);
-    g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
-  }
+  norm_rows<T>(c, c->x, gd, true, c->ln_f, R, xm, c->tapbuf, rm.seq, c->sd.tap, L);
+  g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
   LAUNCH(c, k_topk_lse, dim3(R, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, 2, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, logits);
   LAUNCH(c, k_argmax_out, (R + 127) / 128, 128, 0, c->top_id, c->top_val, R, argmax, margin,
          argmax == c->argmax_i ? (int *)nullptr : c->argmax_i);

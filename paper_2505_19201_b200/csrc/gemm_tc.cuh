@@ -11,8 +11,8 @@
 //       - 65..128 tokens: high and low parts are two A tiles and two MMAs per k-step accumulate
 //         into the same TMEM columns;
 //   * two independent shared-memory rings fed by TMA (cp.async.bulk.tensor.2d, 128-byte swizzle,
-//     no multicast): a deep one for W panels (256 rows x 64 k, evict-first) and a shallow one for
-//     X panels (128 rows x 64 k, served by L2, evict-last);
+//     no multicast): one for W panels (256 rows x 64 k, evict-first) and one for X panels
+//     (128 rows x 64 k, served by L2, evict-last);
 //   * persistent stream-K: the (tile, panel) units are dealt out in equal contiguous ranges to one
 //     CTA per SM; a CTA that covers part of a tile writes a partial sum to its own slot and the
 //     consumer adds the slots in a fixed order;
@@ -20,7 +20,8 @@
 //     dependency resolves; only the X producer and the epilogue wait for the previous kernel;
 //   * warp roles: 0 = W producer, 1 = MMA issuer and TMEM owner, 6 = X producer, 2..5 and 7..10 =
 //     epilogue (tcgen05.ld -> 128-bit stores; the first set drains accumulator columns 0..127, the
-//     second 128..255, loads software-pipelined); two TMEM accumulators alternate so that the
+//     second 128..255, loads software-pipelined, each chunk turned in shared memory so that a
+//     store covers whole 128-byte runs of a row); two TMEM accumulators alternate so that the
 //     epilogue of one segment overlaps the MMAs of the next;
 //   * every mbarrier wait is bounded: on expiry the kernel raises the status word and leaves.
 #pragma once
@@ -32,42 +33,28 @@
 #include <tuple>
 
 #include "common.cuh"
-#include "prologue.cuh"
 
 #define TC_BN 256               // weight rows per tile (MMA N)
 #define TC_BK 64                // k elements per panel (128 bytes: one swizzle row)
-#define TC_THREADS 352             // 11 warps, see the roles below
+#define TC_THREADS 352          // 11 warps, see the roles above
 #define TC_SPIN_LIMIT (1u << 24)
 #define TC_WPANEL (TC_BN * TC_BK * 2)
+#define TC_STG_LD 36            // floats per row of an epilogue staging tile (32 + padding)
+#define TC_STG_BYTES (8 * 16 * TC_STG_LD * 4)
 #define TC_XTILE (128 * TC_BK * 2)
 
 enum { TC_X_PLAIN = 0, TC_X_INTERLEAVED = 1, TC_X_PLANAR = 2 };
 
-#define TC_MAX_STAGES 4
-#define TC_STG_LD 36            // floats per row of an epilogue staging tile (32 + padding)
-#define TC_STG_BYTES (8 * 16 * TC_STG_LD * 4)
-
-// One GEMM of a chain, preceded by the row-wise work that produces its input.
-struct TcStage {
+struct TcParams {
   float *out;
   long long slot_stride;        // floats between partial-sum slots
   int N, K, KB, n_tiles, total_units, upc;
   int n_tok;                    // real token rows
   int x_mode;                   // TC_X_*
   int lo_rows;                  // TC_X_PLANAR: row of the first low part in the X tensor map
-  Prologue pro;                 // kind PRO_NONE: the input was written by an earlier kernel
-};
-// A chain of up to TC_MAX_STAGES GEMMs run by one launch: stage k's prologue reads stage k-1's
-// output.  Grid-wide barriers (a counter in global memory that only grows) order the stages.
-struct TcChain {
-  int n_stages;
-  int wp, w_stages, x_stages;   // panels per ring stage, ring depths (shared by all stages)
+  int wp, w_stages, x_stages;   // panels per ring stage, ring depths
   int *status;
-  unsigned long long *bar_counter;
-  unsigned long long bar_base;  // value of the counter when this launch starts
-  TcStage st[TC_MAX_STAGES];
 };
-struct TcMaps { CUtensorMap w[TC_MAX_STAGES], x[TC_MAX_STAGES]; };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -143,33 +130,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 
-// Grid-wide barrier number `ord` of this launch: every CTA adds one to a counter that only grows
-// and waits until all of them have.  All CTAs of the grid are resident (one per SM), so the wait
-// ends; it is bounded all the same.  One thread per CTA calls it.
-#define TC_GRID_SPIN_LIMIT (1u << 22)
-__device__ __forceinline__ bool grid_barrier(const TcChain &p, int ord) {
-  __threadfence();
-  atomicAdd(p.bar_counter, 1ull);
-  const unsigned long long target = p.bar_base + (unsigned long long)(ord + 1) * gridDim.x;
-  for (uint32_t it = 0; it < TC_GRID_SPIN_LIMIT; ++it) {
-    unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p.bar_counter) : "memory");
-    if (v >= target) return true;
-    __nanosleep(32);
-  }
-  return false;
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
-
 // ------------------------------------------------------------------------------------------ kernel
 // Dynamic shared memory (1024-byte aligned): W ring [w_stages][wp][32 KB], X ring
 // [x_stages][wp][16 KB, or 32 KB = high tile | low tile when planar], then the barriers.
 __global__ void __launch_bounds__(TC_THREADS, 1)
-k_gemm_tc(const __grid_constant__ TcMaps maps, const __grid_constant__ TcChain p) {
+k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ float pro_sh[8];
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const bool planar = p.st[0].x_mode == TC_X_PLANAR;      // one layout per chain
+  const bool planar = p.x_mode == TC_X_PLANAR;
   const uint32_t wstage_bytes = (uint32_t)p.wp * TC_WPANEL;
   const uint32_t xpanel_bytes = planar ? 2u * TC_XTILE : (uint32_t)TC_XTILE;
   const uint32_t xstage_bytes = (uint32_t)p.wp * xpanel_bytes;
@@ -199,231 +167,189 @@ k_gemm_tc(const __grid_constant__ TcMaps maps, const __grid_constant__ TcChain p
   tc_fence_after();
   pdl_trigger();
   const uint32_t tmem_base = *tmem_base_p;
-  // grid barriers of the launch, in order: [after stage 0's prologue], then for every later
-  // stage one before its prologue (the previous GEMM is complete) and one after it
-  const int bar0 = p.st[0].pro.kind != PRO_NONE ? 1 : 0;
+  const int u_begin = blockIdx.x * p.upc, u_end = min(u_begin + p.upc, p.total_units);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ W producer: weights are
-    // constant, so nothing here waits for anything but ring space; it runs ahead across stages
+    // constant, so nothing here waits for anything but ring space
     if (lane == 0) {
       const uint64_t pol = policy_evict_first();
-      int s = 0;
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+      int s = 0, u = u_begin;
       uint32_t ph = 0;
-      bool wrapped = false, live = true;
-      for (int st = 0; st < p.n_stages && live; ++st) {
-        const TcStage &S = p.st[st];
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.w[st]) : "memory");
-        int u = blockIdx.x * S.upc;
-        const int u_end = min(u + S.upc, S.total_units);
-        while (u < u_end) {
-          int tile = u / S.KB, kb = u - tile * S.KB;
-          int np = min(p.wp, min(S.KB - kb, u_end - u));
-          if (wrapped && !mbar_wait(empty_w + s, ph ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; live = false; break; }
-          if (*abort_flag) { live = false; break; }
-          uint8_t *dst = wring + (size_t)s * wstage_bytes;
-          mbar_expect_tx(full_w + s, (uint32_t)np * TC_WPANEL);
-          for (int q = 0; q < np; ++q) tma_load_2d(dst + (size_t)q * TC_WPANEL, &maps.w[st], full_w + s, (kb + q) * TC_BK, tile * TC_BN, pol);
-          u += np;
-          if (++s == p.w_stages) { s = 0; ph ^= 1; wrapped = true; }
-        }
+      bool wrapped = false;
+      while (u < u_end) {
+        int tile = u / p.KB, kb = u - tile * p.KB;
+        int np = min(p.wp, min(p.KB - kb, u_end - u));
+        if (wrapped && !mbar_wait(empty_w + s, ph ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break; }
+        if (*abort_flag) break;
+        uint8_t *dst = wring + (size_t)s * wstage_bytes;
+        mbar_expect_tx(full_w + s, (uint32_t)np * TC_WPANEL);
+        for (int q = 0; q < np; ++q) tma_load_2d(dst + (size_t)q * TC_WPANEL, &map_w, full_w + s, (kb + q) * TC_BK, tile * TC_BN, pol);
+        u += np;
+        if (++s == p.w_stages) { s = 0; ph ^= 1; wrapped = true; }
       }
     }
   } else if (warp == 6) {
     // ------------------------------------------------------------------ X producer: waits until the
-    // stage's input exists (previous kernel, or this stage's prologue on every CTA), then feeds
-    // one X stage per W stage
-    const uint64_t pol = policy_evict_last();
-    int s = 0;
-    uint32_t ph = 0;
-    bool wrapped = false, live = true;
-    for (int st = 0; st < p.n_stages; ++st) {
-      const TcStage &S = p.st[st];
-      if (S.pro.kind != PRO_NONE) {
-        named_bar_sync(1, PRO_THREADS + 32);                  // this CTA's share of the prologue is written
-        if (lane == 0 && live && !grid_barrier(p, st == 0 ? 0 : bar0 + 2 * (st - 1) + 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; live = false; }
-      } else if (st == 0 && lane == 0) pdl_wait();
-      if (lane == 0 && live) {
-        fence_proxy_async();                                  // rows written by ordinary stores, read by TMA
-        if (blockIdx.x == 0) trace_stamp(TR_k_gemm_tc);
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.x[st]) : "memory");
-        int u = blockIdx.x * S.upc;
-        const int u_end = min(u + S.upc, S.total_units);
-        while (u < u_end) {
-          int tile = u / S.KB, kb = u - tile * S.KB;
-          int np = min(p.wp, min(S.KB - kb, u_end - u));
-          if (wrapped && !mbar_wait(empty_x + s, ph ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; live = false; break; }
-          if (*abort_flag) { live = false; break; }
-          uint8_t *dst = xring + (size_t)s * xstage_bytes;
-          mbar_expect_tx(full_x + s, (uint32_t)np * xpanel_bytes);
-          for (int q = 0; q < np; ++q) {
-            tma_load_2d(dst + (size_t)q * xpanel_bytes, &maps.x[st], full_x + s, (kb + q) * TC_BK, 0, pol);
-            if (planar) tma_load_2d(dst + (size_t)q * xpanel_bytes + TC_XTILE, &maps.x[st], full_x + s, (kb + q) * TC_BK, S.lo_rows, pol);
-          }
-          u += np;
-          if (++s == p.x_stages) { s = 0; ph ^= 1; wrapped = true; }
+    // input exists (previous kernel), then feeds one X stage per W stage
+    if (lane == 0) {
+      const uint64_t pol = policy_evict_last();
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+      pdl_wait();
+      if (blockIdx.x == 0) trace_stamp(TR_k_gemm_tc);
+      int s = 0, u = u_begin;
+      uint32_t ph = 0;
+      bool wrapped = false;
+      while (u < u_end) {
+        int tile = u / p.KB, kb = u - tile * p.KB;
+        int np = min(p.wp, min(p.KB - kb, u_end - u));
+        if (wrapped && !mbar_wait(empty_x + s, ph ^ 1)) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break; }
+        if (*abort_flag) break;
+        uint8_t *dst = xring + (size_t)s * xstage_bytes;
+        mbar_expect_tx(full_x + s, (uint32_t)np * xpanel_bytes);
+        for (int q = 0; q < np; ++q) {
+          tma_load_2d(dst + (size_t)q * xpanel_bytes, &map_x, full_x + s, (kb + q) * TC_BK, 0, pol);
+          if (planar) tma_load_2d(dst + (size_t)q * xpanel_bytes + TC_XTILE, &map_x, full_x + s, (kb + q) * TC_BK, p.lo_rows, pol);
         }
+        u += np;
+        if (++s == p.x_stages) { s = 0; ph ^= 1; wrapped = true; }
       }
-      __syncwarp();
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = 256, M = 128
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-      int ws = 0, xs = 0;
+      int ws = 0, xs = 0, u = u_begin;
       uint32_t wph = 0, xph = 0, seg = 0;
       bool ok = true;
-      for (int st = 0; st < p.n_stages && ok; ++st) {
-        const TcStage &S = p.st[st];
-        int u = blockIdx.x * S.upc;
-        const int u_end = min(u + S.upc, S.total_units);
-        while (u < u_end && ok) {
-          int tile = u / S.KB;
-          int seg_end = min((tile + 1) * S.KB, u_end);
-          int buf = seg & 1;
-          if (seg >= 2 && !mbar_wait(acc_empty + buf, ((seg >> 1) & 1) ^ 1)) { ok = false; break; }
+      while (u < u_end && ok) {
+        int tile = u / p.KB;
+        int seg_end = min((tile + 1) * p.KB, u_end);
+        int buf = seg & 1;
+        if (seg >= 2 && !mbar_wait(acc_empty + buf, ((seg >> 1) & 1) ^ 1)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t d_addr = tmem_base + (uint32_t)buf * TC_BN;
+        uint32_t accum = 0u;
+        while (u < seg_end) {
+          int np = min(p.wp, seg_end - u);
+          if (!mbar_wait(full_w + ws, wph) || !mbar_wait(full_x + xs, xph)) { ok = false; break; }
           tc_fence_after();
-          uint32_t d_addr = tmem_base + (uint32_t)buf * TC_BN;
-          uint32_t accum = 0u;
-          while (u < seg_end) {
-            int np = min(p.wp, seg_end - u);
-            if (!mbar_wait(full_w + ws, wph) || !mbar_wait(full_x + xs, xph)) { ok = false; break; }
-            tc_fence_after();
-            uint32_t sw0 = smem_u32(wring + (size_t)ws * wstage_bytes), sx0 = smem_u32(xring + (size_t)xs * xstage_bytes);
-            for (int q = 0; q < np; ++q) {
-              uint64_t ad = smem_desc(sx0 + (uint32_t)q * xpanel_bytes), al = smem_desc(sx0 + (uint32_t)q * xpanel_bytes + TC_XTILE);
-              uint64_t bd = smem_desc(sw0 + (uint32_t)q * TC_WPANEL);
+          uint32_t sw0 = smem_u32(wring + (size_t)ws * wstage_bytes), sx0 = smem_u32(xring + (size_t)xs * xstage_bytes);
+          for (int q = 0; q < np; ++q) {
+            uint64_t ad = smem_desc(sx0 + (uint32_t)q * xpanel_bytes), al = smem_desc(sx0 + (uint32_t)q * xpanel_bytes + TC_XTILE);
+            uint64_t bd = smem_desc(sw0 + (uint32_t)q * TC_WPANEL);
 #pragma unroll
-              for (int k = 0; k < TC_BK / 16; ++k) {
-                mma_bf16(d_addr, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, accum);
-                accum = 1u;
-                if (planar) mma_bf16(d_addr, al + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, 1u);
-              }
+            for (int k = 0; k < TC_BK / 16; ++k) {
+              mma_bf16(d_addr, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, accum);
+              accum = 1u;
+              if (planar) mma_bf16(d_addr, al + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, 1u);
             }
-            mma_commit(empty_x + xs);           // frees both stages once these MMAs have read them
-            mma_commit(empty_w + ws);
-            u += np;
-            if (++ws == p.w_stages) { ws = 0; wph ^= 1; }
-            if (++xs == p.x_stages) { xs = 0; xph ^= 1; }
           }
-          if (!ok) break;
-          mma_commit(acc_full + buf);           // accumulator complete
-          ++seg;
+          mma_commit(empty_x + xs);           // frees both stages once these MMAs have read them
+          mma_commit(empty_w + ws);
+          u += np;
+          if (++ws == p.w_stages) { ws = 0; wph ^= 1; }
+          if (++xs == p.x_stages) { xs = 0; xph ^= 1; }
         }
+        if (!ok) break;
+        mma_commit(acc_full + buf);           // accumulator complete
+        ++seg;
       }
       if (!ok) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
     }
   } else {
-    // ------------------------------------------------------------------ warps 2..5, 7..10: the
-    // stage's prologue, then the epilogue of its GEMM segments
+    // ------------------------------------------------------------------ warps 2..5, 7..10: epilogue
+    // of the CTA's segments (partial sums to this CTA's slot)
     const int q = warp & 3;                   // TMEM lane quarter this warp may read
     const int half = warp >= 7 ? 1 : 0;       // which 128 accumulator columns this warp drains
-    const int ptid = (warp < 7 ? warp - 2 : warp - 3) * 32 + lane;      // 0..255 among these warps
-    float *stg = stage_tiles + (ptid >> 5) * (16 * TC_STG_LD);          // this warp's staging tile
-    pdl_wait();                               // inputs and the output buffer belong to earlier kernels
-    const bool inter = p.st[0].x_mode == TC_X_INTERLEAVED;
-    const int row = q * 32 + lane;            // accumulator lane = X row
+    const int pwarp = warp < 7 ? warp - 2 : warp - 3;                   // 0..7 among these warps
+    float *stg = stage_tiles + pwarp * (16 * TC_STG_LD);                // this warp's staging tile
+    pdl_wait();                               // the output buffer belongs to earlier kernels
+    const bool inter = p.x_mode == TC_X_INTERLEAVED;
     const int part = inter ? lane & 1 : 0;
     uint32_t seg = 0;
-    bool live = true;
-    for (int st = 0; st < p.n_stages; ++st) {
-      const TcStage &S = p.st[st];
-      if (st > 0) {
-        // every CTA's results of the previous GEMM must be in memory before this prologue reads them
-        __threadfence();
-        named_bar_sync(3, PRO_THREADS);
-        if (ptid == 0 && !grid_barrier(p, bar0 + 2 * (st - 1))) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
-        named_bar_sync(3, PRO_THREADS);
-      }
-      if (S.pro.kind != PRO_NONE) {
-        pro_run(S.pro, ptid, blockIdx.x, gridDim.x, pro_sh);
-        __threadfence();
-        fence_proxy_async();
-        named_bar_arrive(1, PRO_THREADS + 32);                // tells this CTA's X producer
-      }
-      int u = blockIdx.x * S.upc;
-      const int u_end = min(u + S.upc, S.total_units);
-      while (u < u_end && live) {
-        int tile = u / S.KB;
-        int seg_end = min((tile + 1) * S.KB, u_end);
-        int buf = seg & 1;
-        int ok = 1;
-        if (lane == 0) ok = mbar_wait(acc_full + buf, (seg >> 1) & 1) ? 1 : 0;
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok || *abort_flag) { if (lane == 0) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; } live = false; break; }
-        tc_fence_after();
-        int first_cta = (tile * S.KB) / S.upc;
-        int slot = (int)blockIdx.x - first_cta;
-        float *dst0 = S.out + (long long)slot * S.slot_stride + tile * TC_BN;       // row 0 of this CTA's slot, first column of the tile
-        uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * TC_BN;
-        // four chunks of 32 columns; the TMEM load of chunk i+1 is in flight while chunk i is stored.
-        // A lane holds values of one row, but a store instruction is cheapest when the lanes of a
-        // warp cover whole 128-byte runs of a row: the chunk goes through a [16][32] tile in shared
-        // memory (rows padded to 36 floats) and leaves as 4 stores of 4 rows x 128 bytes.
-        uint32_t ra[32], rb[32];
-        tmem_ld32(taddr + (uint32_t)half * 128u, ra);
+    int u = u_begin;
+    while (u < u_end) {
+      int tile = u / p.KB;
+      int seg_end = min((tile + 1) * p.KB, u_end);
+      int buf = seg & 1;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(acc_full + buf, (seg >> 1) & 1) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok || *abort_flag) { if (lane == 0) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; } break; }
+      tc_fence_after();
+      int first_cta = (tile * p.KB) / p.upc;
+      int slot = (int)blockIdx.x - first_cta;
+      float *dst0 = p.out + (long long)slot * p.slot_stride + tile * TC_BN;       // row 0 of this CTA's slot, first column of the tile
+      uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * TC_BN;
+      // four chunks of 32 columns; the TMEM load of chunk i+1 is in flight while chunk i is stored.
+      // A lane holds values of one row, but a store instruction is cheapest when the lanes of a
+      // warp cover whole 128-byte runs of a row: the chunk goes through a [16][32] tile in shared
+      // memory (rows padded to 36 floats) and leaves as 4 stores of 4 rows x 128 bytes.
+      uint32_t ra[32], rb[32];
+      tmem_ld32(taddr + (uint32_t)half * 128u, ra);
 #pragma unroll
-        for (int ci = 0; ci < 4; ++ci) {
-          const int col0 = half * 128 + ci * 32;
-          uint32_t (&r)[32] = (ci & 1) ? rb : ra;
-          tmem_ld_wait();
-          if (ci + 1 < 4) tmem_ld32(taddr + (uint32_t)(col0 + 32), (ci & 1) ? ra : rb);
-          const int c4 = (lane & 7) * 4;
-          const bool col_ok = tile * TC_BN + col0 + c4 < S.N;
-          if (inter) {
-            // lanes 2t and 2t+1 hold the products of token t's high and low parts.  The even lane
-            // keeps columns 0..15 of the chunk and the odd lane 16..31: each sends the partner
-            // the 16 values it needs and adds what it receives to its own.
-            float4 *srow = reinterpret_cast<float4 *>(stg + (lane >> 1) * TC_STG_LD + part * 16);
+      for (int ci = 0; ci < 4; ++ci) {
+        const int col0 = half * 128 + ci * 32;
+        uint32_t (&r)[32] = (ci & 1) ? rb : ra;
+        tmem_ld_wait();
+        if (ci + 1 < 4) tmem_ld32(taddr + (uint32_t)(col0 + 32), (ci & 1) ? ra : rb);
+        const int c4 = (lane & 7) * 4;
+        const bool col_ok = tile * TC_BN + col0 + c4 < p.N;
+        if (inter) {
+          // lanes 2t and 2t+1 hold the products of token t's high and low parts.  The even lane
+          // keeps columns 0..15 of the chunk and the odd lane 16..31: each sends the partner
+          // the 16 values it needs and adds what it receives to its own.
+          float4 *srow = reinterpret_cast<float4 *>(stg + (lane >> 1) * TC_STG_LD + part * 16);
 #pragma unroll
-            for (int j4 = 0; j4 < 4; ++j4) {
-              float v[4];
+          for (int j4 = 0; j4 < 4; ++j4) {
+            float v[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int j = j4 * 4 + e;
-                float send = __uint_as_float(part ? r[j] : r[16 + j]);
-                float mine = __uint_as_float(part ? r[16 + j] : r[j]);
-                v[e] = mine + __shfl_xor_sync(0xffffffffu, send, 1);
-              }
-              srow[j4] = make_float4(v[0], v[1], v[2], v[3]);
+            for (int e = 0; e < 4; ++e) {
+              const int j = j4 * 4 + e;
+              float send = __uint_as_float(part ? r[j] : r[16 + j]);
+              float mine = __uint_as_float(part ? r[16 + j] : r[j]);
+              v[e] = mine + __shfl_xor_sync(0xffffffffu, send, 1);
+            }
+            srow[j4] = make_float4(v[0], v[1], v[2], v[3]);
+          }
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int tl = i * 4 + (lane >> 3), tok = q * 16 + tl;
+            float4 val = *reinterpret_cast<const float4 *>(stg + tl * TC_STG_LD + c4);
+            if (tok < p.n_tok && col_ok) *reinterpret_cast<float4 *>(dst0 + (long long)tok * p.N + col0 + c4) = val;
+          }
+          __syncwarp();
+        } else {
+          // one row per lane: two halves of 16 rows through the same tile
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            if ((lane >> 4) == h) {
+              float4 *srow = reinterpret_cast<float4 *>(stg + (lane & 15) * TC_STG_LD);
+#pragma unroll
+              for (int j4 = 0; j4 < 8; ++j4)
+                srow[j4] = make_float4(__uint_as_float(r[j4 * 4]), __uint_as_float(r[j4 * 4 + 1]), __uint_as_float(r[j4 * 4 + 2]),
+                                       __uint_as_float(r[j4 * 4 + 3]));
             }
             __syncwarp();
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const int tl = i * 4 + (lane >> 3), tok = q * 16 + tl;
+              const int tl = i * 4 + (lane >> 3), tok = q * 32 + h * 16 + tl;
               float4 val = *reinterpret_cast<const float4 *>(stg + tl * TC_STG_LD + c4);
-              if (tok < S.n_tok && col_ok) *reinterpret_cast<float4 *>(dst0 + (long long)tok * S.N + col0 + c4) = val;
+              if (tok < p.n_tok && col_ok) *reinterpret_cast<float4 *>(dst0 + (long long)tok * p.N + col0 + c4) = val;
             }
             __syncwarp();
-          } else {
-            // one row per lane: two halves of 16 rows through the same tile
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              if ((lane >> 4) == h) {
-                float4 *srow = reinterpret_cast<float4 *>(stg + (lane & 15) * TC_STG_LD);
-#pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4)
-                  srow[j4] = make_float4(__uint_as_float(r[j4 * 4]), __uint_as_float(r[j4 * 4 + 1]), __uint_as_float(r[j4 * 4 + 2]),
-                                         __uint_as_float(r[j4 * 4 + 3]));
-              }
-              __syncwarp();
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const int tl = i * 4 + (lane >> 3), tok = q * 32 + h * 16 + tl;
-                float4 val = *reinterpret_cast<const float4 *>(stg + tl * TC_STG_LD + c4);
-                if (tok < S.n_tok && col_ok) *reinterpret_cast<float4 *>(dst0 + (long long)tok * S.N + col0 + c4) = val;
-              }
-              __syncwarp();
-            }
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty + buf);
-        u = seg_end;
-        ++seg;
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty + buf);
+      u = seg_end;
+      ++seg;
     }
   }
   tc_fence_before();
@@ -442,12 +368,10 @@ struct GemmTcPlan {
   int max_smem;
   int use_pdl;
   int *status;
-  unsigned long long *bar_counter;     // device: arrivals at grid barriers since the plan was made
-  unsigned long long bar_total;        // host mirror: what the counter reads once everything enqueued has run
   std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;
 };
 
-static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status, unsigned long long *bar_counter, int use_pdl) {
+static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status, int use_pdl) {
   void *fn = nullptr;
   cudaDriverEntryPointQueryResult qr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn)
@@ -457,12 +381,9 @@ static inline const char *gemm_tc_plan_init(GemmTcPlan *pl, int *status, unsigne
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&pl->n_sms, cudaDevAttrMultiProcessorCount, dev);
   cudaDeviceGetAttribute(&pl->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  // the kernel also has a few bytes of static shared memory: leave room for them
-  if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->max_smem - 256) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->max_smem) != cudaSuccess)
     return "cannot raise the dynamic shared memory limit";
   pl->status = status;
-  pl->bar_counter = bar_counter;       // zeroed by the caller
-  pl->bar_total = 0;
   pl->use_pdl = use_pdl;
   return nullptr;
 }
@@ -509,69 +430,34 @@ static inline long long gemm_tc_out_floats(int n_sms, int slot_rows, int N, int 
   return slots * (long long)slot_rows * N;
 }
 
-// One GEMM of a chain as the host describes it.
+// Enqueue one GEMM.
 //   X: bf16, row-major, K columns.  TC_X_PLAIN: row t = token t.  TC_X_INTERLEAVED: row 2t = high
 //   part of token t, row 2t+1 = low part.  TC_X_PLANAR: row t = high part, row lo_rows + t = low part.
-//   rows <= 64 when interleaved, <= 128 otherwise; every GEMM of a chain has the same rows and x_mode.
-//   pro: the row-wise work that writes X (kind PRO_NONE: an earlier kernel did); stages after the
-//   first must have one.
-struct GemmTcDesc {
-  const void *W, *X;
-  int x_mode, lo_rows, rows, slot_rows, N, K;
-  float *out;
-  long long out_floats;
-  Prologue pro;
-};
-
-// Enqueue a chain of n GEMMs as one launch.  g[i] receives the descriptor consumers read stage
-// i's result through; it depends on the shapes only, so a call with launch == false serves to
-// learn the descriptors that later stages' prologues need.  Returns false if the launch could not
-// be made.
-static inline bool gemm_tc_launch_chain(GemmTcPlan *pl, cudaStream_t stream, int n, const GemmTcDesc *d, GemmOut *g,
-                                        bool launch = true) {
-  if (n < 1 || n > TC_MAX_STAGES) return false;
-  TcChain p;
-  TcMaps maps;
-  p.n_stages = n;
-  const int x_mode = d[0].x_mode;
+//   rows <= 64 when interleaved, <= 128 otherwise.  slot_rows >= rows: rows of a partial-sum slot.
+// *g receives the descriptor consumers read the result through.  Returns false if the launch could
+// not be made.
+static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const void *W, const void *X, int x_mode, int lo_rows,
+                                  int rows, int slot_rows, int N, int K, float *out, long long out_floats, GemmOut *g) {
+  TcParams p;
+  p.n_tok = rows; p.x_mode = x_mode; p.lo_rows = lo_rows;
+  p.N = N; p.K = K; p.KB = K / TC_BK;
+  p.n_tiles = (N + TC_BN - 1) / TC_BN;
+  p.total_units = p.n_tiles * p.KB;
   // W stages of two panels (256-byte runs per weight row) unless the X ring needs the room
-  p.wp = x_mode == TC_X_PLANAR ? 1 : 2;
-  int max_grid = 1;
-  for (int i = 0; i < n; ++i) {
-    TcStage &S = p.st[i];
-    if (d[i].x_mode != x_mode || d[i].rows != d[0].rows || (launch && i > 0 && d[i].pro.kind == PRO_NONE)) return false;
-    S.n_tok = d[i].rows; S.x_mode = x_mode; S.lo_rows = d[i].lo_rows;
-    S.N = d[i].N; S.K = d[i].K; S.KB = d[i].K / TC_BK;
-    S.n_tiles = (S.N + TC_BN - 1) / TC_BN;
-    S.total_units = S.n_tiles * S.KB;
-    if (S.KB < p.wp) p.wp = 1;
-  }
-  for (int i = 0; i < n; ++i) {
-    TcStage &S = p.st[i];
-    int grid = pl->n_sms < S.total_units ? pl->n_sms : S.total_units;
-    S.upc = (S.total_units + grid - 1) / grid;
-    if (S.KB % p.wp == 0) S.upc = (S.upc + p.wp - 1) / p.wp * p.wp;   // CTA ranges cover whole ring stages
-    grid = (S.total_units + S.upc - 1) / S.upc;
-    if (grid > max_grid) max_grid = grid;
-    S.out = d[i].out;
-    S.slot_stride = (long long)d[i].slot_rows * S.N;       // slot_rows >= rows: the same for every chunk of one GEMM
-    long long max_slots = (S.KB + S.upc - 1) / S.upc + 1;
-    if (S.slot_stride * max_slots > d[i].out_floats) return false;
-    S.pro = d[i].pro;
-    int x_rows = x_mode == TC_X_INTERLEAVED ? 2 * d[i].rows : (x_mode == TC_X_PLANAR ? d[i].lo_rows + d[i].rows : d[i].rows);
-    if (launch) {
-      const CUtensorMap *mw = tc_map(pl, d[i].W, S.N, S.K, TC_BN);
-      const CUtensorMap *mx = tc_map(pl, d[i].X, x_rows, S.K, 128);
-      if (!mw || !mx) return false;
-      maps.w[i] = *mw; maps.x[i] = *mx;
-    }
-    g[i].base = S.out; g[i].slot_stride = S.slot_stride; g[i].chunk_stride = 0; g[i].chunk_shift = 30; g[i].ld = S.N; g[i].kb = S.KB; g[i].upc = S.upc;
-  }
-  if (!launch) return true;
-  bool any_pro = false;
-  for (int i = 0; i < n; ++i) any_pro = any_pro || d[i].pro.kind != PRO_NONE;
-  // a launch with grid barriers needs every CTA resident: one per SM, never more CTAs than SMs
-  int grid = any_pro ? pl->n_sms : max_grid;
+  p.wp = (x_mode == TC_X_PLANAR || p.KB < 2) ? 1 : 2;
+  int grid = pl->n_sms < p.total_units ? pl->n_sms : p.total_units;
+  p.upc = (p.total_units + grid - 1) / grid;
+  if (p.KB % p.wp == 0) p.upc = (p.upc + p.wp - 1) / p.wp * p.wp;       // CTA ranges cover whole ring stages
+  grid = (p.total_units + p.upc - 1) / p.upc;
+  p.out = out;
+  p.slot_stride = (long long)slot_rows * N;
+  long long max_slots = (p.KB + p.upc - 1) / p.upc + 1;
+  if (p.slot_stride * max_slots > out_floats) return false;
+  int x_rows = x_mode == TC_X_INTERLEAVED ? 2 * rows : (x_mode == TC_X_PLANAR ? lo_rows + rows : rows);
+  const CUtensorMap *mw = tc_map(pl, W, N, K, TC_BN);
+  const CUtensorMap *mx = tc_map(pl, X, x_rows, K, 128);
+  if (!mw || !mx) return false;
+  g->base = p.out; g->slot_stride = p.slot_stride; g->chunk_stride = 0; g->chunk_shift = 30; g->ld = N; g->kb = p.KB; g->upc = p.upc;
   int xstage = p.wp * (x_mode == TC_X_PLANAR ? 2 * TC_XTILE : TC_XTILE);
   p.x_stages = 2;
   int budget = pl->max_smem - 2048 - TC_STG_BYTES - p.x_stages * xstage;
@@ -580,9 +466,6 @@ static inline bool gemm_tc_launch_chain(GemmTcPlan *pl, cudaStream_t stream, int
   if (p.w_stages < 2) return false;
   if (budget - p.w_stages * p.wp * TC_WPANEL >= xstage) p.x_stages = 3;   // room left over: a third X stage
   p.status = pl->status;
-  p.bar_counter = pl->bar_counter;
-  p.bar_base = pl->bar_total;
-  int n_bars = (d[0].pro.kind != PRO_NONE ? 1 : 0) + 2 * (n - 1);
   size_t smem = (size_t)p.w_stages * p.wp * TC_WPANEL + (size_t)p.x_stages * xstage + 1024 + 512 + TC_STG_BYTES;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
@@ -590,16 +473,5 @@ static inline bool gemm_tc_launch_chain(GemmTcPlan *pl, cudaStream_t stream, int
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = pl->use_pdl ? 1 : 0;
-  if (cudaLaunchKernelEx(&cfg, k_gemm_tc, maps, p) != cudaSuccess) return false;
-  pl->bar_total += (unsigned long long)n_bars * grid;
-  return true;
-}
-
-// A single GEMM without a prologue.
-static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const void *W, const void *X, int x_mode, int lo_rows,
-                                  int rows, int slot_rows, int N, int K, float *out, long long out_floats, GemmOut *g) {
-  GemmTcDesc d;
-  d.W = W; d.X = X; d.x_mode = x_mode; d.lo_rows = lo_rows; d.rows = rows; d.slot_rows = slot_rows; d.N = N; d.K = K;
-  d.out = out; d.out_floats = out_floats; d.pro.kind = PRO_NONE; d.pro.rows = 0;
-  return gemm_tc_launch_chain(pl, stream, 1, &d, g);
+  return cudaLaunchKernelEx(&cfg, k_gemm_tc, *mw, *mx, p) == cudaSuccess;
 }

@@ -5,7 +5,6 @@
 #include "common.cuh"
 #include "rows.cuh"
 
-#define DREAM_MAX_BATCH 8
 #define DREAM_MAX_DEPTH 15
 
 // Per-sequence device state (arrays indexed by sequence id).

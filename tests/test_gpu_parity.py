@@ -77,10 +77,3 @@ def test_llava_shape_batched(batch):
         print(json.dumps(pr.summary(), default=float))
     finally:
         pr.close()
-
-
-def test_chained_gemm_launches(monkeypatch):
-    """The optional mode in which norms, gating and the attention merge run as prologues inside
-    chained GEMM launches (grid-wide barriers between stages) gives the same results."""
-    monkeypatch.setenv("DREAM_CHAIN", "1")
-    pr, s = _run("llava7b", 2, n_layers=2, decode_steps=4)
