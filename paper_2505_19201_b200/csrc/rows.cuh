@@ -318,46 +318,69 @@ struct TopkScratch {
   int *counter;    // [rows] blocks done; zero between launches
 };
 
-// ktop rounds over NV register candidates per thread: round j's block-wide best goes to
-// out_v/out_i[j] and is retired.  sh_* hold one entry per warp.
+// The ktop best of a block's candidates (NV per thread, in registers), in order, to out_v/out_i.
+// Two levels, so that only one block-wide step is needed: every warp selects its own ktop best in
+// ktop rounds of "best remaining" (a scan of the thread's candidates and a warp reduction), then
+// warp 0 selects from the warps' lists the same way.  Ids are unique, so a winner has one owner.
+// sh_* hold TOPK_THREADS / 32 * TOPK_MAX entries.
+template <int NV>
+__device__ __forceinline__ void topk_round(const float (&v)[NV], const int (&id)[NV], unsigned &taken, float &wv, int &wi) {
+  float bv = -INFINITY;
+  int bi = 0x7fffffff, bj = -1;
+#pragma unroll
+  for (int j = 0; j < NV; ++j)
+    if (!((taken >> j) & 1u) && better(v[j], id[j], bv, bi)) { bv = v[j]; bi = id[j]; bj = j; }
+  wv = bv; wi = bi;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, wv, o);
+    int oi = __shfl_xor_sync(0xffffffffu, wi, o);
+    if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
+  }
+  if (bj >= 0 && bi == wi && bv == wv) taken |= 1u << bj;
+}
 template <int NV>
 __device__ __forceinline__ void topk_rounds(const float (&v)[NV], const int (&id)[NV], int ktop, float *out_v, int *out_i,
                                             float *sh_v, int *sh_i) {
-  int tid = threadIdx.x;
+  constexpr int NW = TOPK_THREADS / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned taken = 0u;
   for (int round = 0; round < ktop; ++round) {
-    float bv = -INFINITY;
-    int bi = 0x7fffffff, bj = -1;
-#pragma unroll
-    for (int j = 0; j < NV; ++j)
-      if (!((taken >> j) & 1u) && better(v[j], id[j], bv, bi)) { bv = v[j]; bi = id[j]; bj = j; }
-    float wv = bv;
-    int wi = bi;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, wv, o);
-      int oi = __shfl_xor_sync(0xffffffffu, wi, o);
-      if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; }
-    }
-    if ((tid & 31) == 0) { sh_v[tid >> 5] = wv; sh_i[tid >> 5] = wi; }
-    __syncthreads();
-    float gv = sh_v[0];
-    int gi = sh_i[0];
-#pragma unroll
-    for (int w = 1; w < TOPK_THREADS / 32; ++w)
-      if (better(sh_v[w], sh_i[w], gv, gi)) { gv = sh_v[w]; gi = sh_i[w]; }
-    if (bj >= 0 && bi == gi && bv == gv) taken |= 1u << bj;      // ids are unique: one owner
-    if (tid == 0) { out_v[round] = gv; out_i[round] = gi; }
-    __syncthreads();
+    float wv;
+    int wi;
+    topk_round<NV>(v, id, taken, wv, wi);
+    if (lane == 0) { sh_v[warp * TOPK_MAX + round] = wv; sh_i[warp * TOPK_MAX + round] = wi; }
   }
+  __syncthreads();
+  if (warp == 0) {
+    constexpr int NC = NW * TOPK_MAX / 32;           // candidates per lane
+    float cv[NC];
+    int ci[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+      int e = j * 32 + lane;
+      bool ok = e < NW * ktop;
+      int q = ok ? e / ktop : 0, w = ok ? e - q * ktop : 0;
+      cv[j] = ok ? sh_v[q * TOPK_MAX + w] : -INFINITY;
+      ci[j] = ok ? sh_i[q * TOPK_MAX + w] : 0x7fffffff;
+    }
+    unsigned tk = 0u;
+    for (int round = 0; round < ktop; ++round) {
+      float wv;
+      int wi;
+      topk_round<NC>(cv, ci, tk, wv, wi);
+      if (lane == 0) { out_v[round] = wv; out_i[round] = wi; }
+    }
+  }
+  __syncthreads();
 }
 
 __global__ void __launch_bounds__(TOPK_THREADS)
 k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_val, int *top_id, float *lse,
            float *logits_out) {
   __shared__ float red[33];
-  __shared__ float sh_v[TOPK_THREADS / 32];
-  __shared__ int sh_i[TOPK_THREADS / 32];
+  __shared__ float sh_v[TOPK_THREADS / 32 * TOPK_MAX];
+  __shared__ int sh_i[TOPK_THREADS / 32 * TOPK_MAX];
   __shared__ int is_last;
   kernel_entry(TR_k_topk_lse);
   int r = blockIdx.x, sp = blockIdx.y, tid = threadIdx.x;
