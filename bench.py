@@ -33,7 +33,7 @@ from paper_2505_19201_b200 import configs, synth  # noqa: E402
 # capture ran on the 4-layer cut of the workload (same layer shapes); traffic grows in proportion
 # to the weight bytes, so a step's mean launch is scaled by this ratio.  None for workloads without
 # a capture, and to be reset to None whenever the kernel changes.
-TRAFFIC_RATIO = {"llava7b": (105.45 + 34.67 + 186.46 + 97.00) / (100.66 + 33.55 + 180.36 + 90.18)}
+TRAFFIC_RATIO = {"llava7b": (105.50 + 34.62 + 186.71 + 96.32) / (100.66 + 33.55 + 180.36 + 90.18)}
 
 METRIC = "verified_tree_tokens_per_s"
 UNIT = "tokens/s"
@@ -185,7 +185,7 @@ def run_reference(args, p):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--workload", default="llava7b")
