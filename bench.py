@@ -155,6 +155,26 @@ def oracle_sample(p, twg, dwg, T, budget_s=12.0, max_steps=8):
                        f"state filled with random values (no CPU prefill); {dt_s:.1f} s per step", seconds=dt_s)
 
 
+def slowest_rank(times_ms, world, device):
+    """Element-wise maximum over the ranks of a list of durations (every rank calls this)."""
+    ms = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    return [float(x) for x in ms]
+
+
+def job_value(world, batch, tree_nodes, ms_per_step):
+    """Whole-job throughput: every rank runs an independent replica of the same workload, so the
+    job verifies world * batch * tree_nodes tree tokens per step of the slowest rank."""
+    return world * batch * tree_nodes / (ms_per_step / 1e3)
+
+
+def request_seed(seq, rank):
+    """Input seed of sequence `seq` on rank `rank`: replicas decode different requests."""
+    return seq + 100 * rank
+
+
 def run_reference(args, p):
     """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -219,7 +239,7 @@ def main():
     T = ctx.T
     seqs = list(range(B))
     for s in seqs:
-        vis, ids = synth.request_inputs(p, s + 100 * rank, dev)
+        vis, ids = synth.request_inputs(p, request_seed(s, rank), dev)
         ctx.dream_prefill(s, vis, 0, ids)
         ctx.dream_compress_visual(s, p["k_visual"])
     ctx.dream_poll()
@@ -300,16 +320,13 @@ def main():
             gemm = dict(kernel="k_gemm_tc", launches=n_l, launches_per_step=n_l / nprof, bytes_per_launch=g_bytes / n_l,
                         us_per_launch=1e3 * g_ms / n_l, gbs=g_bytes / g_ms / 1e6, ms_per_step=g_ms / nprof,
                         bytes_per_step=g_bytes / nprof)
-    ms = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(ms[0]), float(ms[1])
+    total_ms, e2e_ms = slowest_rank([total_ms, e2e_ms], world, dev)
     if rank != 0:
         return
     pk, pk_src = peaks()
     sb = step_bytes(p, T, P0)
     ms_step = total_ms / args.steps
-    value = world * B * T / (ms_step / 1e3)
+    value = job_value(world, B, T, ms_step)
     step_gbs = sb["total"] / (ms_step / 1e3) / 1e9
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None,
@@ -320,7 +337,7 @@ def main():
                 step_bytes=sb["total"], step_gbs=step_gbs,
                 step_roofline_frac=step_gbs / pk["hbm_gbs"], step_roofline_frac_nominal_8tbs=step_gbs / 8000.0,
                 clocks=sampler.summary(), gpu_launches=int(launches),
-                e2e=dict(value=world * B * T / (e2e_ms / args.steps / 1e3), unit=UNIT,
+                e2e=dict(value=job_value(world, B, T, e2e_ms / args.steps), unit=UNIT,
                          h2d_bytes_per_step=4 * B, d2h_bytes_per_step=4 * B * (p["tree_depth"] + 2)))
     if gemm:
         line["roofline"] = dict(bound="hbm", achieved=gemm["gbs"], peak=pk["hbm_gbs"], unit="GB/s",
