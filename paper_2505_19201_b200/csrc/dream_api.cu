@@ -264,7 +264,8 @@ static size_t carve(dream_ctx *c, char *base) {
         long long per = (gemm_tc_out_floats(192, TC_ROWS_SPLIT_1MMA, N, K) + 63) & ~63LL;
         long long per2 = (gemm_tc_out_floats(192, TC_ROWS_MAX, N, K) + 63) & ~63LL;
         fl = (size_t)imax(1, ROW_CHUNK / TC_ROWS_SPLIT_1MMA) * per;
-        if ((size_t)per2 > fl) fl = per2;
+        size_t fl2 = (size_t)imax(1, ROW_CHUNK / TC_ROWS_MAX) * per2;
+        if (fl2 > fl) fl = fl2;
       } else fl = (size_t)ROW_CHUNK * N;
       if (fl > need) need = fl;
     }
@@ -315,12 +316,13 @@ extern "C" dream_status dream_arena_bytes(const dream_config *cfg, size_t *bytes
 // ------------------------------------------------------------------------------------- GEMM dispatch
 
 // How the rows of a bf16 GEMM input buffer are laid out for a launch set of R rows: up to 64 rows
-// (and beyond 128, in chunks of 64) high and low rows alternate; 65..128 rows use two planes.
+// high and low rows alternate; more rows use two planes (high parts first, low parts lo_rows rows
+// further on) and go through the GEMM 128 at a time, so the weights stream once per 128 rows.
 struct XMode { int mode, lo_rows; };
 static XMode xmode(const dream_ctx *c, int R) {
   if (c->cfg.dtype != DREAM_BF16) return XMode{TC_X_PLAIN, 0};
-  if (R <= TC_ROWS_SPLIT_1MMA || R > TC_ROWS_MAX) return XMode{TC_X_INTERLEAVED, 0};
-  return XMode{TC_X_PLANAR, TC_ROWS_MAX};
+  if (R <= TC_ROWS_SPLIT_1MMA) return XMode{TC_X_INTERLEAVED, 0};
+  return XMode{TC_X_PLANAR, R <= TC_ROWS_MAX ? TC_ROWS_MAX : ROW_CHUNK};
 }
 static XLayout xlay(XMode m, long long width) {
   if (m.mode == TC_X_INTERLEAVED) return XLayout{2 * width, width};
