@@ -178,6 +178,10 @@ k_attn_mma(AttnMmaArgs a) {
 #pragma unroll
   for (int wd = 0; wd < 4; ++wd) { mw0[wd] = mwords[(warp * 16 + g) * 4 + wd]; mw1[wd] = mwords[(warp * 16 + g + 8) * 4 + wd]; }
 
+  // a warp whose sixteen rows are all idle (few query rows: the draft's passes) only keeps the
+  // copies and barriers going
+  const bool warp_live = __any_sync(0xffffffffu, row_r[warp * 16 + (lane & 15)] >= 0);
+
   const int mi = lane >> 3, l7 = lane & 7;
   const uint32_t qh_addr = smem_addr(Qh + (warp * 16 + l7 + (mi & 1) * 8) * LD + (mi >> 1) * 8);
   const uint32_t ql_addr = qh_addr + AM_ROWS * LD * 2;
@@ -190,6 +194,7 @@ k_attn_mma(AttnMmaArgs a) {
     if (blk + 1 < b1) { load_block(blk + 1, buf ^ 1, true); cp_async_wait<1>(); } else cp_async_wait<0>();
     __syncthreads();
     const bf16 *Kb = KV + buf * BUF_ELEMS, *Vb = Kb + PLANES * PLANE_ELEMS;
+    if (!warp_live) { __syncthreads(); continue; }
     // ---- S = Q K^T
     float s[NT_S][4];
 #pragma unroll
@@ -286,6 +291,7 @@ k_attn_mma(AttnMmaArgs a) {
   l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1); l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
   l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1); l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
 
+  if (!warp_live) return;
   bf16 *out = reinterpret_cast<bf16 *>(a.out);
   if (a.n_chunks == 1) {
 #pragma unroll
