@@ -56,7 +56,7 @@ enum { DREAM_TAP_FIXED = 0, DREAM_TAP_ENTROPY_MIN = 1, DREAM_TAP_ENTROPY_MAX = 2
 
 /* Shapes and hyper-parameters; plain data, copied by dream_init. */
 typedef struct {
-  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ff, vocab;
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ff, vocab;   /* d_model <= 16384 */
   int32_t dtype;                 /* DREAM_F32 or DREAM_BF16: weights, KV caches, GEMM inputs */
   float rms_eps, rope_theta;
   int32_t max_batch;             /* sequences resident at once */

@@ -189,6 +189,26 @@ __device__ __forceinline__ float4 gemm_val4(const GemmOut &g, int r, int c) {
   return s;
 }
 
+// The same with up to MAXS extra slots fetched per round trip (more registers; for consumers that
+// read values made of many partial sums, such as the outputs of the narrow projections).
+template <int MAXS>
+__device__ __forceinline__ float4 gemm_val4_wide(const GemmOut &g, int r, int c) {
+  int ch = r >> g.chunk_shift;
+  const float4 *p = reinterpret_cast<const float4 *>(g.base + (long long)ch * g.chunk_stride +
+                                                     (long long)(r - (ch << g.chunk_shift)) * g.ld + c);
+  float4 s = *p;
+  const int extra = gemm_extra_slots(g, c);
+  const long long st4 = g.slot_stride >> 2;
+  for (int i = 1; i <= extra; i += MAXS) {
+    float4 t[MAXS];
+#pragma unroll
+    for (int k = 0; k < MAXS; ++k) t[k] = i + k <= extra ? p[(long long)(i + k) * st4] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int k = 0; k < MAXS; ++k) add4(s, t[k]);
+  }
+  return s;
+}
+
 // Four consecutive elements of a GEMM input row, high (and low) parts, as 8-byte stores.
 template <typename T> __device__ __forceinline__ void store_split4(T *p, long long lo_delta, float4 v);
 template <> __device__ __forceinline__ void store_split4<float>(float *p, long long, float4 v) {

@@ -152,6 +152,7 @@ static dream_status check_config(const dream_config *c, TreeShape *ts) {
       c->n_heads % c->n_kv_heads || c->d_ff < 8 || c->vocab < 2)
     return fail(nullptr, DREAM_E_ARG, "model shape");
   if (c->d_model % 8 || c->d_ff % 8) return fail(nullptr, DREAM_E_UNSUPPORTED, "d_model, d_ff must be multiples of 8");
+  if (c->d_model > 16384) return fail(nullptr, DREAM_E_UNSUPPORTED, "d_model above 16384");
   if (c->vocab > TOPK_THREADS * TOPK_COLS) return fail(nullptr, DREAM_E_UNSUPPORTED, "vocab above 1048576");
   if (c->dtype == DREAM_BF16 && (c->d_model % 64 || c->d_ff % 64 || (c->n_heads * c->head_dim) % 64 || c->vocab % 8))
     return fail(nullptr, DREAM_E_UNSUPPORTED, "bf16: d_model, d_ff, n_heads*head_dim must be multiples of 64 and vocab of 8");
@@ -607,7 +608,15 @@ template <typename T>
 static void norm_rows(dream_ctx *c, float *x, const GemmOut &gin, bool has_in, const void *gain, int rows, XMode m,
                       float *copy = nullptr, const int *row_seq = nullptr, const int *tap = nullptr, int layer = 0,
                       bool want_raw = false) {
-  LAUNCH(c, (k_resid_norm<T>), rows, NORM_THREADS, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+  const int d4 = c->cfg.d_model / 4;
+  int nv = 1;
+  while ((d4 + nv - 1) / nv > 1024) nv *= 2;                 // d_model <= 16384 by check_config
+  const int threads = ((d4 + nv - 1) / nv + 31) & ~31;
+  if (nv == 1) LAUNCH(c, (k_resid_norm<T, 1>), rows, threads, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
+  else if (nv == 2) LAUNCH(c, (k_resid_norm<T, 2>), rows, threads, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
+  else LAUNCH(c, (k_resid_norm<T, 4>), rows, threads, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
          (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
 }
 template <typename T>

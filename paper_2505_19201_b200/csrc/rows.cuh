@@ -46,74 +46,63 @@ __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict_
 // Optional side outputs of the updated residual: `copy` (fp32; when tap_state is given the
 // row is copied only if its sequence's tap layer equals `layer`) and `raw` (element type,
 // unnormalised: the memory side of Eq. 1 takes features without a norm).
-#define NORM_THREADS 512
-#define NORM_NV 4                // float4 groups a thread keeps in registers (rows up to 8192 wide)
-template <typename T>
-__global__ void __launch_bounds__(NORM_THREADS)
+// Block size: ceil(d / 4 / NV) threads rounded up to a warp (at most 1024); a thread keeps NV
+// groups of four elements, so rows of up to 4096 * NV elements fit.  The partial-sum slots of a
+// value are all fetched at once (up to 12 per round trip).
+template <typename T, int NV>
+__global__ void __launch_bounds__(1024)
 k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
              float eps, int d, T *xn, float *copy, const int *row_seq,
              const int *tap_state, int layer, T *raw, XLayout lay) {
   __shared__ float sh[33];
-  int r = blockIdx.x, d4 = d >> 2;
+  const int r = blockIdx.x, d4 = d >> 2, nt = blockDim.x;
   // the gains are weights: they can be fetched before the predecessor has finished
-  float4 gq[NORM_NV];
+  float4 gq[NV];
 #pragma unroll
-  for (int j = 0; j < NORM_NV; ++j) {
-    int i = threadIdx.x + j * NORM_THREADS;
+  for (int j = 0; j < NV; ++j) {
+    int i = threadIdx.x + j * nt;
     gq[j] = (xn && i < d4) ? ld_f4(gain + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   kernel_entry(TR_k_resid_norm);
   float *xr = x + (long long)r * d;
-  float4 v[NORM_NV];
+  float4 v[NV];
   float ss = 0.f;
   // every load of the row is issued before the first use
 #pragma unroll
-  for (int j = 0; j < NORM_NV; ++j) {
-    int i = threadIdx.x + j * NORM_THREADS;
+  for (int j = 0; j < NV; ++j) {
+    int i = threadIdx.x + j * nt;
     v[j] = i < d4 ? ld_f4(xr + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   if (has_in) {
-    float4 gv[NORM_NV];
+    float4 gv[NV];
 #pragma unroll
-    for (int j = 0; j < NORM_NV; ++j) {
-      int i = threadIdx.x + j * NORM_THREADS;
-      gv[j] = i < d4 ? gemm_val4(gin, r, 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < NV; ++j) {
+      int i = threadIdx.x + j * nt;
+      gv[j] = i < d4 ? gemm_val4_wide<12 / NV>(gin, r, 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
-    for (int j = 0; j < NORM_NV; ++j) {
-      int i = threadIdx.x + j * NORM_THREADS;
+    for (int j = 0; j < NV; ++j) {
+      int i = threadIdx.x + j * nt;
       v[j].x += gv[j].x; v[j].y += gv[j].y; v[j].z += gv[j].z; v[j].w += gv[j].w;
       if (i < d4) *reinterpret_cast<float4 *>(xr + 4 * i) = v[j];
     }
   }
 #pragma unroll
-  for (int j = 0; j < NORM_NV; ++j) ss += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
-  for (int i = threadIdx.x + NORM_NV * NORM_THREADS; i < d4; i += NORM_THREADS) {      // rows wider than 8192
-    float4 t = ld_f4(xr + 4 * i);
-    if (has_in) {
-      float4 gq = gemm_val4(gin, r, 4 * i);
-      t.x += gq.x; t.y += gq.y; t.z += gq.z; t.w += gq.w;
-      *reinterpret_cast<float4 *>(xr + 4 * i) = t;
-    }
-    ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
-  }
+  for (int j = 0; j < NV; ++j) ss += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
   float tot = block_sum(ss, sh);
   float inv = rsqrtf(tot / (float)d + eps);
   bool do_copy = copy != nullptr && (tap_state == nullptr || tap_state[row_seq[r]] == layer);
-  auto emit = [&](int i, float4 t, float4 gv) {
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int i = threadIdx.x + j * nt;
+    if (i >= d4) continue;
+    float4 t = v[j];
     if (do_copy) *reinterpret_cast<float4 *>(copy + (long long)r * d + 4 * i) = t;
     if (raw) store_split4<T>(raw + r * lay.row_stride + 4 * i, lay.lo_delta, t);
     if (xn)
       store_split4<T>(xn + r * lay.row_stride + 4 * i, lay.lo_delta,
-                      make_float4(t.x * inv * gv.x, t.y * inv * gv.y, t.z * inv * gv.z, t.w * inv * gv.w));
-  };
-#pragma unroll
-  for (int j = 0; j < NORM_NV; ++j) {
-    int i = threadIdx.x + j * NORM_THREADS;
-    if (i < d4) emit(i, v[j], gq[j]);
+                      make_float4(t.x * inv * gq[j].x, t.y * inv * gq[j].y, t.z * inv * gq[j].z, t.w * inv * gq[j].w));
   }
-  for (int i = threadIdx.x + NORM_NV * NORM_THREADS; i < d4; i += NORM_THREADS)
-    emit(i, ld_f4(xr + 4 * i), xn ? ld_f4(gain + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f));
 }
 
 // ---------------------------------------------------------------------------------------
