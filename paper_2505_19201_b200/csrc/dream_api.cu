@@ -555,7 +555,8 @@ template <typename T, int HD> struct AttnLaunch {
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
     a.n_rt = (rows_per_seq * a.G + AM_ROWS - 1) / AM_ROWS;
     int nb_ub = imax(1, (key_ub + KBLK - 1) / KBLK), ctas = f.n_kv_heads * a.n_rt * B;
-    int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, (2 * c->tc.n_sms + ctas - 1) / ctas));
+    // two CTAs fit an SM: as many key chunks as keep the whole grid in one wave
+    int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, 2 * c->tc.n_sms / ctas));
     a.blocks_per_chunk = (nb_ub + want - 1) / want;
     a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
     a.part_o = c->am_part_o; a.part_ml = c->am_part_ml;
