@@ -59,7 +59,7 @@ struct dream_ctx {
   int am_rt_max;
   int key_ub[DREAM_MAX_BATCH];         // upper bound of the draft caches' permanent rows
   int cur_seq[DREAM_MAX_BATCH];        // sequences of the call being enqueued, by slot
-  int tk_nsplit;
+  int tk_nsplit, tk_nv;                // vocabulary blocks of the top-k kernel, columns per thread (4 or 16)
   int *top_id, *argmax_i, *accept_len_i, *out_tokens_i, *comp_src_i;
   size_t gout_floats;
   // host side
@@ -106,6 +106,11 @@ static inline void launch_k(dream_ctx *c, void (*kernel)(P...), dim3 grid, dim3 
   c->launches++;
 }
 #define LAUNCH(c, kernel, grid, block, smem, ...) launch_k(c, kernel, dim3(grid), dim3(block), (size_t)(smem), __VA_ARGS__)
+#define TOPK_LAUNCH(c, grid, ...)                                                        \
+  do {                                                                                   \
+    if ((c)->tk_nv == 4) LAUNCH(c, (k_topk_lse<4>), grid, TOPK_THREADS, 0, __VA_ARGS__); \
+    else LAUNCH(c, (k_topk_lse<16>), grid, TOPK_THREADS, 0, __VA_ARGS__);                \
+  } while (0)
 
 // ------------------------------------------------------------------------------------- shapes
 
@@ -289,7 +294,9 @@ static size_t carve(dream_ctx *c, char *base) {
     c->am_part_o = a.take<float>(prow * f.head_dim);
     c->am_part_ml = a.take<float>(prow * 2);
   } else { c->am_part_o = nullptr; c->am_part_ml = nullptr; }
-  c->tk_nsplit = (f.vocab + TOPK_COLS - 1) / TOPK_COLS;
+  // small blocks (1024 columns) while the merge of the blocks' lists stays within 1024 candidates
+  c->tk_nv = (f.vocab + 1023) / 1024 * TOPK_MAX <= 1024 ? 4 : 16;
+  c->tk_nsplit = (f.vocab + c->tk_nv * TOPK_THREADS - 1) / (c->tk_nv * TOPK_THREADS);
   c->tks.pv = a.take<float>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
   c->tks.pi = a.take<int>((size_t)ROW_CHUNK * c->tk_nsplit * TOPK_MAX);
   c->tks.pm = a.take<float>((size_t)ROW_CHUNK * c->tk_nsplit);
@@ -667,7 +674,7 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
   // first token: LM head on the last prompt row
   norm_rows<T>(c, c->x + (size_t)(n - 1) * d, NO_GEMM, false, c->ln_f, 1, m1);
   GemmOut g = gemm<T>(c, c->lm_head, c->xn, m1, 1, f.vocab, d);
-  LAUNCH(c, k_topk_lse, dim3(1, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, 2, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
+  TOPK_LAUNCH(c, dim3(1, c->tk_nsplit), g, f.vocab, 2, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
   LAUNCH(c, k_first_token, 1, 32, 0, c->top_id, c->top_val, first_token, first_margin);
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, n, c->top_id, -1, -1);
   LAUNCH(c, k_select_tap, 1, 32, 0, c->ae, f.tap_mode, f.tap_layer, f.tap_lo, f.tap_hi, c->sd.tap + seq, tap_layer);
@@ -826,7 +833,7 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
     LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
     g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
-    LAUNCH(c, k_topk_lse, dim3(R, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, ts.K, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
+    TOPK_LAUNCH(c, dim3(R, c->tk_nsplit), g, f.vocab, ts.K, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
     int next_m = p < ts.D ? ts.beam[p] : 1;
     LAUNCH(c, k_tree_expand, B, 128, 0, tb, c->sd, c->dt, ts, p, m, c->top_val, c->top_id, c->lse_rows, rn, next_m);
     cur ^= 1;
@@ -874,7 +881,7 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
   }
   norm_rows<T>(c, c->x, gd, true, c->ln_f, R, xm, c->tapbuf, rm.seq, c->sd.tap, L);
   g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
-  LAUNCH(c, k_topk_lse, dim3(R, c->tk_nsplit), TOPK_THREADS, 0, g, f.vocab, 2, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, logits);
+  TOPK_LAUNCH(c, dim3(R, c->tk_nsplit), g, f.vocab, 2, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, logits);
   LAUNCH(c, k_argmax_out, (R + 127) / 128, 128, 0, c->top_id, c->top_val, R, argmax, margin,
          argmax == c->argmax_i ? (int *)nullptr : c->argmax_i);
   return DREAM_OK;
@@ -1095,7 +1102,7 @@ extern "C" dream_status dream_topk_lse_static(const float *logits, int32_t rows,
   GemmOut g;                                   // a plain [rows][vocab] matrix: one slot, one chunk
   g.base = logits; g.slot_stride = 0; g.chunk_stride = 0; g.chunk_shift = 30; g.ld = vocab; g.kb = 0; g.upc = 0;
   int nsplit = (vocab + TOPK_COLS - 1) / TOPK_COLS;
-  k_topk_lse<<<dim3(rows, nsplit), TOPK_THREADS, 0, stream>>>(g, vocab, ktop, nsplit, ts, top_val, top_id, lse, (float *)nullptr);
+  k_topk_lse<TOPK_COLS / TOPK_THREADS><<<dim3(rows, nsplit), TOPK_THREADS, 0, stream>>>(g, vocab, ktop, nsplit, ts, top_val, top_id, lse, (float *)nullptr);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(nullptr, DREAM_E_CUDA, "k_topk_lse launch: %s", cudaGetErrorString(e));
   return DREAM_OK;

@@ -293,7 +293,7 @@ __global__ void k_gather_rows(const float *__restrict__ src, const int *__restri
 // ---------------------------------------------------------------------------------------
 // Per row of a [rows][V] GEMM output: the KTOP largest logits (ties -> lower id), in
 // descending order, and the log-sum-exp of the row.  grid (rows, nsplit): block (r, sp) scans
-// columns [sp * TOPK_COLS, (sp + 1) * TOPK_COLS), 16 per thread held in registers, and leaves a
+// columns [sp * NV * 256, (sp + 1) * NV * 256), NV (4 or 16) per thread held in registers, and leaves a
 // sorted partial list and an (m, z) pair; the block that finishes a row last merges the partials,
 // always in the same order.  Selection is KTOP rounds of a block-wide "best remaining" search.
 #define TOPK_MAX 16
@@ -364,6 +364,7 @@ __device__ __forceinline__ void topk_rounds(const float (&v)[NV], const int (&id
   __syncthreads();
 }
 
+template <int NV>
 __global__ void __launch_bounds__(TOPK_THREADS)
 k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_val, int *top_id, float *lse,
            float *logits_out) {
@@ -373,18 +374,18 @@ k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_va
   __shared__ int is_last;
   kernel_entry(TR_k_topk_lse);
   int r = blockIdx.x, sp = blockIdx.y, tid = threadIdx.x;
-  int c0 = sp * TOPK_COLS;
-  float v[TOPK_PER_THREAD];
-  int id[TOPK_PER_THREAD];
+  int c0 = sp * (NV * TOPK_THREADS);
+  float v[NV];
+  int id[NV];
   if ((V & 3) == 0) {
-    float4 q[TOPK_PER_THREAD / 4];
+    float4 q[NV / 4];
 #pragma unroll
-    for (int j = 0; j < TOPK_PER_THREAD / 4; ++j) {
+    for (int j = 0; j < NV / 4; ++j) {
       int c = c0 + (j * TOPK_THREADS + tid) * 4;
       q[j] = c < V ? gemm_val4(g, r, c) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
 #pragma unroll
-    for (int j = 0; j < TOPK_PER_THREAD / 4; ++j) {
+    for (int j = 0; j < NV / 4; ++j) {
       int c = c0 + (j * TOPK_THREADS + tid) * 4;
       if (logits_out && c < V) *reinterpret_cast<float4 *>(logits_out + (long long)r * V + c) = q[j];
       v[4 * j] = q[j].x; v[4 * j + 1] = q[j].y; v[4 * j + 2] = q[j].z; v[4 * j + 3] = q[j].w;
@@ -392,7 +393,7 @@ k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_va
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < TOPK_PER_THREAD; ++j) {
+    for (int j = 0; j < NV; ++j) {
       int c = c0 + j * TOPK_THREADS + tid;
       v[j] = c < V ? gemm_val(g, r, c) : -INFINITY;
       id[j] = c;
@@ -400,11 +401,11 @@ k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_va
     }
   }
 #pragma unroll
-  for (int j = 0; j < TOPK_PER_THREAD; ++j) if (id[j] >= V) id[j] = 0x7fffffff;
+  for (int j = 0; j < NV; ++j) if (id[j] >= V) id[j] = 0x7fffffff;
   // (m, z) of this block's columns, combined in a fixed order
   float m = -INFINITY;
 #pragma unroll
-  for (int j = 0; j < TOPK_PER_THREAD; ++j) m = fmaxf(m, v[j]);
+  for (int j = 0; j < NV; ++j) m = fmaxf(m, v[j]);
   float bm = warp_max(m);
   if ((tid & 31) == 0) red[tid >> 5] = bm;
   __syncthreads();
@@ -413,11 +414,11 @@ k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_va
   float gm = red[32];
   float z = 0.f;
 #pragma unroll
-  for (int j = 0; j < TOPK_PER_THREAD; ++j) z += __expf(v[j] - gm);        // exp(-inf) = 0 for padding
+  for (int j = 0; j < NV; ++j) z += __expf(v[j] - gm);        // exp(-inf) = 0 for padding
   float tot = block_sum(z, red);
   long long po = (long long)r * nsplit + sp;
   if (tid == 0) { ts.pm[po] = gm; ts.pz[po] = tot; }
-  topk_rounds<TOPK_PER_THREAD>(v, id, ktop, ts.pv + po * TOPK_MAX, ts.pi + po * TOPK_MAX, sh_v, sh_i);
+  topk_rounds<NV>(v, id, ktop, ts.pv + po * TOPK_MAX, ts.pi + po * TOPK_MAX, sh_v, sh_i);
   // the last block of the row merges
   __threadfence();
   __syncthreads();
