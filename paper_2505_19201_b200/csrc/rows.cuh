@@ -442,11 +442,22 @@ k_topk_lse(GemmOut g, int V, int ktop, int nsplit, TopkScratch ts, float *top_va
     cv[j] = ok ? __ldcg(ts.pv + ((long long)r * nsplit + q) * TOPK_MAX + w) : -INFINITY;
     ci[j] = ok ? __ldcg(ts.pi + ((long long)r * nsplit + q) * TOPK_MAX + w) : 0x7fffffff;
   }
-  if (tid == 0) {
-    float mm = -INFINITY, zz = 0.f;
-    for (int q = 0; q < nsplit; ++q) mm = fmaxf(mm, __ldcg(ts.pm + (long long)r * nsplit + q));
-    for (int q = 0; q < nsplit; ++q) zz += __ldcg(ts.pz + (long long)r * nsplit + q) * __expf(__ldcg(ts.pm + (long long)r * nsplit + q) - mm);
-    lse[r] = mm + logf(zz);
+  if (tid < 32) {                 // log-sum-exp of the row from the blocks' (max, sum) pairs, one warp, fixed order
+    float pm[8], pz[8];           // up to 256 blocks
+    float mm = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      int q = k * 32 + tid;
+      pm[k] = q < nsplit ? __ldcg(ts.pm + (long long)r * nsplit + q) : -INFINITY;
+      pz[k] = q < nsplit ? __ldcg(ts.pz + (long long)r * nsplit + q) : 0.f;
+      mm = fmaxf(mm, pm[k]);
+    }
+    mm = warp_max(mm);
+    float zz = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) zz += pz[k] * __expf(pm[k] - mm);         // exp(-inf) = 0 for the padding
+    zz = warp_sum(zz);
+    if (tid == 0) lse[r] = mm + logf(zz);
   }
   topk_rounds<4>(cv, ci, ktop, top_val + (long long)r * ktop, top_id + (long long)r * ktop, sh_v, sh_i);
 }
