@@ -272,6 +272,8 @@ static size_t carve(dream_ctx *c, char *base) {
         fl = (size_t)imax(1, ROW_CHUNK / TC_ROWS_SPLIT_1MMA) * per;
         size_t fl2 = (size_t)imax(1, ROW_CHUNK / TC_ROWS_MAX) * per2;
         if (fl2 > fl) fl = fl2;
+        size_t fl3 = (size_t)((gemm_tc_out_floats(192, ROW_CHUNK, N, K) + 63) & ~63LL);
+        if (fl3 > fl) fl = fl3;
       } else fl = (size_t)ROW_CHUNK * N;
       if (fl > need) need = fl;
     }
@@ -325,7 +327,7 @@ extern "C" dream_status dream_arena_bytes(const dream_config *cfg, size_t *bytes
 
 // How the rows of a bf16 GEMM input buffer are laid out for a launch set of R rows: up to 64 rows
 // high and low rows alternate; more rows use two planes (high parts first, low parts lo_rows rows
-// further on) and go through the GEMM 128 at a time, so the weights stream once per 128 rows.
+// further on); up to 256 rows go through a GEMM in one launch (two token tiles per weight panel).
 struct XMode { int mode, lo_rows; };
 static XMode xmode(const dream_ctx *c, int R) {
   if (c->cfg.dtype != DREAM_BF16) return XMode{TC_X_PLAIN, 0};
@@ -344,7 +346,8 @@ template <typename T>
 static GemmOut gemm(dream_ctx *c, const void *W, const void *X, XMode m, int rows, int N, int K) {
   GemmOut g;
   if (sizeof(T) == 2) {
-    int chunk = m.mode == TC_X_INTERLEAVED ? TC_ROWS_SPLIT_1MMA : TC_ROWS_MAX;
+    // rows per launch: 64 (interleaved), 128 (two planes), 256 (two planes with room for two token tiles)
+    int chunk = m.mode == TC_X_INTERLEAVED ? TC_ROWS_SPLIT_1MMA : (m.mode == TC_X_PLANAR && m.lo_rows >= 2 * TC_ROWS_MAX ? 2 * TC_ROWS_MAX : TC_ROWS_MAX);
     int nch = (rows + chunk - 1) / chunk;
     int slot_rows = nch > 1 ? chunk : rows;
     long long per = (gemm_tc_out_floats(c->tc.n_sms, slot_rows, N, K) + 63) & ~63LL;
@@ -361,7 +364,7 @@ static GemmOut gemm(dream_ctx *c, const void *W, const void *X, XMode m, int row
       c->launches++;
       c->tc_launches++;
     }
-    g.base = c->gout; g.chunk_stride = per; g.chunk_shift = chunk == 64 ? 6 : 7;
+    g.base = c->gout; g.chunk_stride = per; g.chunk_shift = chunk == 64 ? 6 : (chunk == 128 ? 7 : 8);
     return g;
   }
   c->simt_launches++;

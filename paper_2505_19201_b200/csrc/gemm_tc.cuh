@@ -52,6 +52,7 @@ struct TcParams {
   int n_tok;                    // real token rows
   int x_mode;                   // TC_X_*
   int lo_rows;                  // TC_X_PLANAR: row of the first low part in the X tensor map
+  int m_tiles;                  // token tiles of 128 rows per launch: 1, or 2 (TC_X_PLANAR, 129..256 tokens)
   int wp, w_stages, x_stages;   // panels per ring stage, ring depths
   int *status;
 };
@@ -139,7 +140,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const bool planar = p.x_mode == TC_X_PLANAR;
   const uint32_t wstage_bytes = (uint32_t)p.wp * TC_WPANEL;
-  const uint32_t xpanel_bytes = planar ? 2u * TC_XTILE : (uint32_t)TC_XTILE;
+  const uint32_t xpanel_bytes = planar ? 2u * TC_XTILE * (uint32_t)p.m_tiles : (uint32_t)TC_XTILE;   // per token tile: high | low
+  const int n_buf = p.m_tiles == 2 ? 1 : 2;                // two token tiles fill all 512 TMEM columns: one accumulator set
   const uint32_t xstage_bytes = (uint32_t)p.wp * xpanel_bytes;
   uint8_t *wring = smem, *xring = smem + (size_t)p.w_stages * wstage_bytes;
   uint64_t *bars = (uint64_t *)(xring + (size_t)p.x_stages * xstage_bytes);
@@ -209,8 +211,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         uint8_t *dst = xring + (size_t)s * xstage_bytes;
         mbar_expect_tx(full_x + s, (uint32_t)np * xpanel_bytes);
         for (int q = 0; q < np; ++q) {
-          tma_load_2d(dst + (size_t)q * xpanel_bytes, &map_x, full_x + s, (kb + q) * TC_BK, 0, pol);
-          if (planar) tma_load_2d(dst + (size_t)q * xpanel_bytes + TC_XTILE, &map_x, full_x + s, (kb + q) * TC_BK, p.lo_rows, pol);
+          if (!planar) tma_load_2d(dst + (size_t)q * xpanel_bytes, &map_x, full_x + s, (kb + q) * TC_BK, 0, pol);
+          else
+            for (int mt = 0; mt < p.m_tiles; ++mt) {
+              uint8_t *dt = dst + (size_t)q * xpanel_bytes + (size_t)mt * 2 * TC_XTILE;
+              tma_load_2d(dt, &map_x, full_x + s, (kb + q) * TC_BK, mt * 128, pol);
+              tma_load_2d(dt + TC_XTILE, &map_x, full_x + s, (kb + q) * TC_BK, p.lo_rows + mt * 128, pol);
+            }
         }
         u += np;
         if (++s == p.x_stages) { s = 0; ph ^= 1; wrapped = true; }
@@ -227,8 +234,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       while (u < u_end && ok) {
         int tile = u / p.KB;
         int seg_end = min((tile + 1) * p.KB, u_end);
-        int buf = seg & 1;
-        if (seg >= 2 && !mbar_wait(acc_empty + buf, ((seg >> 1) & 1) ^ 1)) { ok = false; break; }
+        const int buf = (int)seg % n_buf, use = (int)seg / n_buf;       // use: earlier segments in this accumulator set
+        if (use >= 1 && !mbar_wait(acc_empty + buf, (uint32_t)(use - 1) & 1u)) { ok = false; break; }
         tc_fence_after();
         uint32_t d_addr = tmem_base + (uint32_t)buf * TC_BN;
         uint32_t accum = 0u;
@@ -238,14 +245,20 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
           tc_fence_after();
           uint32_t sw0 = smem_u32(wring + (size_t)ws * wstage_bytes), sx0 = smem_u32(xring + (size_t)xs * xstage_bytes);
           for (int q = 0; q < np; ++q) {
-            uint64_t ad = smem_desc(sx0 + (uint32_t)q * xpanel_bytes), al = smem_desc(sx0 + (uint32_t)q * xpanel_bytes + TC_XTILE);
             uint64_t bd = smem_desc(sw0 + (uint32_t)q * TC_WPANEL);
+            for (int mt = 0; mt < p.m_tiles; ++mt) {
+              const uint32_t xa = sx0 + (uint32_t)q * xpanel_bytes + (uint32_t)mt * 2u * TC_XTILE;
+              const uint64_t ad = smem_desc(xa), al = smem_desc(xa + TC_XTILE);
+              const uint32_t dm = d_addr + (uint32_t)mt * TC_BN;
+              uint32_t acc = accum;
 #pragma unroll
-            for (int k = 0; k < TC_BK / 16; ++k) {
-              mma_bf16(d_addr, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, accum);
-              accum = 1u;
-              if (planar) mma_bf16(d_addr, al + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, 1u);
+              for (int k = 0; k < TC_BK / 16; ++k) {
+                mma_bf16(dm, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, acc);
+                acc = 1u;
+                if (planar) mma_bf16(dm, al + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, 1u);
+              }
             }
+            accum = 1u;
           }
           mma_commit(empty_x + xs);           // frees both stages once these MMAs have read them
           mma_commit(empty_w + ws);
@@ -274,16 +287,17 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
     while (u < u_end) {
       int tile = u / p.KB;
       int seg_end = min((tile + 1) * p.KB, u_end);
-      int buf = seg & 1;
+      const int buf = (int)seg % n_buf, use = (int)seg / n_buf;
       int ok = 1;
-      if (lane == 0) ok = mbar_wait(acc_full + buf, (seg >> 1) & 1) ? 1 : 0;
+      if (lane == 0) ok = mbar_wait(acc_full + buf, (uint32_t)use & 1u) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok || *abort_flag) { if (lane == 0) { atomicMax(p.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; } break; }
       tc_fence_after();
       int first_cta = (tile * p.KB) / p.upc;
       int slot = (int)blockIdx.x - first_cta;
       float *dst0 = p.out + (long long)slot * p.slot_stride + tile * TC_BN;       // row 0 of this CTA's slot, first column of the tile
-      uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * TC_BN;
+      for (int mt = 0; mt < p.m_tiles; ++mt) {      // token tiles: rows mt * 128 .. of the output, accumulator columns mt * 256 ..
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf + mt) * TC_BN;
       // four chunks of 32 columns; the TMEM load of chunk i+1 is in flight while chunk i is stored.
       // A lane holds values of one row, but a store instruction is cheapest when the lanes of a
       // warp cover whole 128-byte runs of a row: the chunk goes through a [16][32] tile in shared
@@ -337,13 +351,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
             __syncwarp();
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const int tl = i * 4 + (lane >> 3), tok = q * 32 + h * 16 + tl;
+              const int tl = i * 4 + (lane >> 3), tok = mt * 128 + q * 32 + h * 16 + tl;
               float4 val = *reinterpret_cast<const float4 *>(stg + tl * TC_STG_LD + c4);
               if (tok < p.n_tok && col_ok) *reinterpret_cast<float4 *>(dst0 + (long long)tok * p.N + col0 + c4) = val;
             }
             __syncwarp();
           }
         }
+      }
       }
       tc_fence_before();
       __syncwarp();
@@ -433,13 +448,18 @@ static inline long long gemm_tc_out_floats(int n_sms, int slot_rows, int N, int 
 // Enqueue one GEMM.
 //   X: bf16, row-major, K columns.  TC_X_PLAIN: row t = token t.  TC_X_INTERLEAVED: row 2t = high
 //   part of token t, row 2t+1 = low part.  TC_X_PLANAR: row t = high part, row lo_rows + t = low part.
-//   rows <= 64 when interleaved, <= 128 otherwise.  slot_rows >= rows: rows of a partial-sum slot.
+//   rows <= 64 when interleaved, <= 128 otherwise, except that TC_X_PLANAR with lo_rows >= 256 takes
+//   up to 256 rows as two token tiles that share every weight panel (the weights stream once;
+//   both accumulators fill the TMEM, so epilogues no longer overlap the next segment's MMAs).
+//   slot_rows >= rows: rows of a partial-sum slot.
 // *g receives the descriptor consumers read the result through.  Returns false if the launch could
 // not be made.
 static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const void *W, const void *X, int x_mode, int lo_rows,
                                   int rows, int slot_rows, int N, int K, float *out, long long out_floats, GemmOut *g) {
   TcParams p;
   p.n_tok = rows; p.x_mode = x_mode; p.lo_rows = lo_rows;
+  p.m_tiles = rows > TC_ROWS_MAX ? 2 : 1;
+  if (rows > 2 * TC_ROWS_MAX || (p.m_tiles == 2 && (x_mode != TC_X_PLANAR || lo_rows < 2 * TC_ROWS_MAX))) return false;
   p.N = N; p.K = K; p.KB = K / TC_BK;
   p.n_tiles = (N + TC_BN - 1) / TC_BN;
   p.total_units = p.n_tiles * p.KB;
@@ -458,7 +478,7 @@ static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const voi
   const CUtensorMap *mx = tc_map(pl, X, x_rows, K, 128);
   if (!mw || !mx) return false;
   g->base = p.out; g->slot_stride = p.slot_stride; g->chunk_stride = 0; g->chunk_shift = 30; g->ld = N; g->kb = p.KB; g->upc = p.upc;
-  int xstage = p.wp * (x_mode == TC_X_PLANAR ? 2 * TC_XTILE : TC_XTILE);
+  int xstage = p.wp * (x_mode == TC_X_PLANAR ? 2 * TC_XTILE * p.m_tiles : TC_XTILE);
   p.x_stages = 2;
   int budget = pl->max_smem - 2048 - TC_STG_BYTES - p.x_stages * xstage;
   p.w_stages = budget / (p.wp * TC_WPANEL);
