@@ -34,6 +34,7 @@ struct dream_ctx {
   int use_tc, use_pdl, gemm_failed;
   int chunk;                           // prompt rows per pass of the prefill loop
   double *rope_inv;                    // [head_dim / 2] rotary inverse frequencies
+  float2 *rope_tab;                    // [ROW_CHUNK][head_dim / 2] rotary (cos, sin) of the rows of the call being enqueued
   std::vector<const void *> ln1, wqkv, wo, ln2, wgu, wd;
   const void *embed, *ln_f, *lm_head;
   dream_draft_weights dw;
@@ -281,6 +282,7 @@ static size_t carve(dream_ctx *c, char *base) {
   }
   c->gout = a.take<float>(c->gout_floats);
   c->rope_inv = a.take<double>(f.head_dim / 2);
+  c->rope_tab = a.take<float2>((size_t)ROW_CHUNK * (f.head_dim / 2));
   c->lse_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
   c->ent_pre = a.take<float>((size_t)f.n_heads * f.max_prompt);
   c->ae = a.take<float>(f.n_layers);
@@ -657,7 +659,7 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
       norm_rows<T>(c, c->x + (size_t)r0 * d, NO_GEMM, false, c->ln1[l], rows, m1);
       GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, m1, rows, c->qkvN, d);
       LAUNCH(c, (k_qkv_post_target<T>), dim3(rows, (c->qkvN / 8 + 255) / 256), 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
-             paged(c, l), f.n_heads, c->rope_inv);
+             paged(c, l), f.n_heads, c->rope_inv, (const float2 *)nullptr);
     }
     HD_DISPATCH(c, T, prefill(c, l, seq, n));
     LAUNCH(c, k_entropy_mean, 1, 1024, 0, c->ent_pre, f.n_heads * n, c->ae + l);
@@ -744,7 +746,7 @@ static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *force
     norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, rows, m1);
     GemmOut g = gemm<T>(c, wkv, c->xn, m1, rows, c->kvN, d);
     LAUNCH(c, k_qkv_post_draft, dim3(rows, (c->kvN / 8 + 255) / 256), 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].dst, 0, 0, (float *)nullptr,
-           flat(c, c->dself), f.n_heads, c->rope_inv);
+           flat(c, c->dself), f.n_heads, c->rope_inv, (const float2 *)nullptr);
   }
   // cross-attention memory: tapped features at the context positions, projected (Eq. 1)
   int nm = f.xattn_full_memory ? n : nc;
@@ -817,11 +819,12 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     const XMode xm = xmode(c, R);
     RowMeta &rm = c->rm[cur], &rn = c->rm[cur ^ 1];
     if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
-    LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
+    LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status,
+           (const int *)rm.pos, (const double *)c->rope_inv, c->rope_tab, f.head_dim / 2);
     GemmOut g;
     norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
     g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
-    LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv);
+    LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv, (const float2 *)c->rope_tab);
     HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub));
     g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
@@ -870,13 +873,14 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
   int key_ub = 0;
   for (int b = 0; b < B; ++b) { key_ub = imax(key_ub, c->p_ub[tb.seq[b]] + c->T); c->cur_seq[b] = tb.seq[b]; }
   LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
-  LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status);
+  LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status,
+           (const int *)rm.pos, (const double *)c->rope_inv, c->rope_tab, f.head_dim / 2);
   GemmOut gd = NO_GEMM, g;
   for (int l = 0; l < L; ++l) {
     // the first norm completes S^l (for l >= 1) and captures it where a sequence taps layer l
     norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, xm, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
     g = gemm<T>(c, c->wqkv[l], c->xn, xm, R, c->qkvN, d);
-    LAUNCH(c, (k_qkv_post_target<T>), dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv);
+    LAUNCH(c, (k_qkv_post_target<T>), dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv, (const float2 *)c->rope_tab);
     HD_DISPATCH(c, T, tree(c, l, R, xm, B, key_ub));
     g = gemm<T>(c, c->wo[l], c->attn_out, xm, R, d, c->Hhd);
     norm_rows<T>(c, c->x, g, true, c->ln2[l], R, xm);

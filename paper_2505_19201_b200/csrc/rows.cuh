@@ -6,13 +6,23 @@
 #include "common.cuh"
 
 // ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void rope_cs(int pos, double inv, float *c, float *s);
 // x[r] = embed[tok[r]] (fp32 residual stream).  tok < 0 leaves a zero row.  One thread per four
-// elements: grid (rows, ceil(d / 1024)).
+// elements: grid (rows, ceil(d / 1024)).  With rope_tab the first block of a row also tabulates
+// the row's rotary factors for every layer of the call: rope_tab[r][i] = (cos, sin)(pos[r] *
+// inv_freq[i]), i < half.
 template <typename T>
 __global__ void k_embed(const T *__restrict__ embed, const int *__restrict__ tok, float *x, int d,
-                        int vocab, int *status) {
+                        int vocab, int *status, const int *__restrict__ pos, const double *__restrict__ inv_freq,
+                        float2 *rope_tab, int half) {
   kernel_entry(TR_k_embed);
   int r = blockIdx.x, t = tok[r];
+  if (rope_tab && blockIdx.y == 0)
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+      float c, s;
+      rope_cs(pos[r], inv_freq[i], &c, &s);
+      rope_tab[(long long)r * half + i] = make_float2(c, s);
+    }
   int i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
   if (t >= vocab) { if (threadIdx.x == 0 && blockIdx.y == 0) atomicMax(status, DREAM_DEV_BAD_INDEX); t = -1; }
   if (i >= d) return;
@@ -120,6 +130,19 @@ __device__ __forceinline__ void rope_cs(int pos, double inv, float *c, float *s)
   sincosf((float)a, s, c);
 }
 
+// (cos, sin) of four neighbouring rotary indices i..i+3 (i a multiple of 4) of row r: from the
+// table k_embed made for the call's rows, or computed when there is none (prefill).
+__device__ __forceinline__ void rope_cs4(const float2 *tab, int r, int half, int pos, const double *inv_freq, int i,
+                                         float4 &cs01, float4 &cs23) {
+  if (tab) {
+    const float4 *t = reinterpret_cast<const float4 *>(tab + (long long)r * half + i);
+    cs01 = t[0]; cs23 = t[1];
+  } else {
+    rope_cs(pos, inv_freq[i], &cs01.x, &cs01.y); rope_cs(pos, inv_freq[i + 1], &cs01.z, &cs01.w);
+    rope_cs(pos, inv_freq[i + 2], &cs23.x, &cs23.y); rope_cs(pos, inv_freq[i + 3], &cs23.z, &cs23.w);
+  }
+}
+
 // Where a row's K/V go.  Target cache: pages [layer][2][page][H_kv][page_tokens][hd].
 struct PagedKV {
   void *base;                    // this layer's K pool; V pool = base + kv_stride elements
@@ -138,7 +161,8 @@ struct PagedKV {
 template <typename T>
 __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
                                   const int *__restrict__ row_pos, const int *__restrict__ row_slot,
-                                  int row0, void *qbuf, PagedKV kv, int H, const double *__restrict__ inv_freq) {
+                                  int row0, void *qbuf, PagedKV kv, int H, const double *__restrict__ inv_freq,
+                                  const float2 *__restrict__ rope_tab) {
   kernel_entry(TR_k_qkv_post_target);
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int hd = kv.hd, half = hd >> 1, q4 = half >> 2, Hkv = kv.hkv;
@@ -147,11 +171,11 @@ __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
   int hh = w / q4, i = (w - hh * q4) * 4;
   int seq = row_seq[r], pos = row_pos[r], slot = row_slot[r];
   T *Kp = (T *)kv.base, *Vp = (T *)kv.base + kv.kv_stride;
-  float4 a = gemm_val4(g, lr, hh * hd + i), b = gemm_val4(g, lr, hh * hd + i + half);
+  float4 cs01 = make_float4(1.f, 0.f, 1.f, 0.f), cs23 = cs01;
+  if (hh < H + Hkv) rope_cs4(rope_tab, r, half, pos, inv_freq, i, cs01, cs23);      // fetched along with the slots
+  float4 a = gemm_val4_wide<4>(g, lr, hh * hd + i), b = gemm_val4_wide<4>(g, lr, hh * hd + i + half);
   if (hh < H + Hkv) {
-    float c0, s0, c1, s1, c2, s2, c3, s3;
-    rope_cs(pos, inv_freq[i], &c0, &s0); rope_cs(pos, inv_freq[i + 1], &c1, &s1);
-    rope_cs(pos, inv_freq[i + 2], &c2, &s2); rope_cs(pos, inv_freq[i + 3], &c3, &s3);
+    const float c0 = cs01.x, s0 = cs01.y, c1 = cs01.z, s1 = cs01.w, c2 = cs23.x, s2 = cs23.y, c3 = cs23.z, s3 = cs23.w;
     float4 ra = make_float4(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1, a.z * c2 - b.z * s2, a.w * c3 - b.w * s3);
     float4 rb = make_float4(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1, b.z * c2 + a.z * s2, b.w * c3 + a.w * s3);
     if (hh < H) {
@@ -189,7 +213,8 @@ struct FlatKV {
 // row_dst[r] (skipped when < 0).  Work items and grid as in k_qkv_post_target.
 __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
                                  const int *__restrict__ row_pos, const int *__restrict__ row_dst,
-                                 int row0, int has_q, void *qbuf, FlatKV kv, int H, const double *__restrict__ inv_freq) {
+                                 int row0, int has_q, void *qbuf, FlatKV kv, int H, const double *__restrict__ inv_freq,
+                                 const float2 *__restrict__ rope_tab) {
   kernel_entry(TR_k_qkv_post_draft);
   int r = blockIdx.x + row0, lr = blockIdx.x;
   int hd = kv.hd, half = hd >> 1, q4 = half >> 2, Hkv = kv.hkv;
@@ -199,11 +224,11 @@ __global__ void k_qkv_post_draft(GemmOut g, const int *__restrict__ row_seq,
   int hh = w / q4, i = (w - hh * q4) * 4;
   int dst = row_dst[r], seq = row_seq[r], pos = row_pos[r];
   if (hh >= Hq && dst < 0) return;
-  float4 a = gemm_val4(g, lr, hh * hd + i), b = gemm_val4(g, lr, hh * hd + i + half);
+  float4 cs01 = make_float4(1.f, 0.f, 1.f, 0.f), cs23 = cs01;
+  if (hh < Hq + Hkv) rope_cs4(rope_tab, r, half, pos, inv_freq, i, cs01, cs23);
+  float4 a = gemm_val4_wide<4>(g, lr, hh * hd + i), b = gemm_val4_wide<4>(g, lr, hh * hd + i + half);
   if (hh < Hq + Hkv) {
-    float c0, s0, c1, s1, c2, s2, c3, s3;
-    rope_cs(pos, inv_freq[i], &c0, &s0); rope_cs(pos, inv_freq[i + 1], &c1, &s1);
-    rope_cs(pos, inv_freq[i + 2], &c2, &s2); rope_cs(pos, inv_freq[i + 3], &c3, &s3);
+    const float c0 = cs01.x, s0 = cs01.y, c1 = cs01.z, s1 = cs01.w, c2 = cs23.x, s2 = cs23.y, c3 = cs23.z, s3 = cs23.w;
     float4 ra = make_float4(a.x * c0 - b.x * s0, a.y * c1 - b.y * s1, a.z * c2 - b.z * s2, a.w * c3 - b.w * s3);
     float4 rb = make_float4(b.x * c0 + a.x * s0, b.y * c1 + a.y * s1, b.z * c2 + a.z * s2, b.w * c3 + a.w * s3);
     if (hh < Hq) {
