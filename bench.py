@@ -213,12 +213,26 @@ def main():
     ap.add_argument("--profile-gemm", type=int, default=1)
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: cut the target to this many layers (the line's workload name says so)")
+    ap.add_argument("--keep", type=float, default=0.0,
+                    help="sweep aid: fraction of the visual tokens the compression keeps (the preset's k otherwise)")
+    ap.add_argument("--chain", action="store_true",
+                    help="sweep aid: a chain-shaped draft (one child per node, depth D) instead of the tree")
+    ap.add_argument("--batch", type=int, default=0, help="sweep aid: number of sequences per step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     p = dict(configs.PRESETS[args.workload])
     if args.layers:
         p = configs.scaled(args.workload, n_layers=args.layers)
         p["name"] = "%s[n_layers=%d]" % (p["name"], args.layers)
+    if args.keep:
+        p["k_visual"] = max(1, min(p["n_visual"], int(p["n_visual"] * args.keep + 0.5)))
+        p["name"] = "%s[k_visual=%d]" % (p["name"], p["k_visual"])
+    if args.chain:
+        p.update(tree_topk=1, tree_beam=1, tree_max_nodes=p["tree_depth"])
+        p["name"] = "%s[chain]" % p["name"]
+    if args.batch:
+        p["batch"] = args.batch
+        p["name"] = "%s[batch=%d]" % (p["name"], args.batch)
     if args.impl == "reference":
         return run_reference(args, p)
 

@@ -42,6 +42,10 @@ PRESETS = {
                           576, 144, 256, 6, 8, 60, 256, 4, TAP_ENTROPY_MAX),
     "pixtral12b": _preset("pixtral12b", "bf16", 40, 5120, 32, 8, 128, 14336, 131072,
                           1024, 256, 512, 6, 8, 60, 64, 1, TAP_ENTROPY_MIN),
+    # LLaVA-1.5-13B-shaped target (Section 4 lists the 13B model among the targets): same prompt and
+    # tree as the 7B-shaped workload.
+    "llava13b": _preset("llava13b", "bf16", 40, 5120, 40, 40, 128, 13824, 32000,
+                        576, 144, 256, 6, 8, 60, 256, 1, TAP_ENTROPY_MAX),
     "gemma3_12b": _preset("gemma3_12b", "bf16", 48, 3840, 16, 8, 256, 15360, 262144,
                           256, 64, 4096, 7, 10, 80, 64, 1, TAP_ENTROPY_MIN),
 }

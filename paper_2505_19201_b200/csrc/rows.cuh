@@ -56,6 +56,16 @@ __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict_
 // Optional side outputs of the updated residual: `copy` (fp32; when tap_state is given the
 // row is copied only if its sequence's tap layer equals `layer`) and `raw` (element type,
 // unnormalised: the memory side of Eq. 1 takes features without a norm).
+// With an EmbedSrc the rows do not come from x but from the embedding table (x is written), and
+// the rows' rotary factors are tabulated as k_embed does: lookup and first norm in one kernel.
+struct EmbedSrc {
+  const void *embed;             // null: the rows are in x already
+  const int *tok, *pos;
+  const double *inv_freq;
+  float2 *rope_tab;
+  int *status;
+  int vocab, half;
+};
 // Block size: ceil(d / 4 / NV) threads rounded up to a warp (at most 1024); a thread keeps NV
 // groups of four elements, so rows of up to 4096 * NV elements fit.  The partial-sum slots of a
 // value are all fetched at once (up to 12 per round trip).
@@ -63,7 +73,7 @@ template <typename T, int NV>
 __global__ void __launch_bounds__(1024)
 k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
              float eps, int d, T *xn, float *copy, const int *row_seq,
-             const int *tap_state, int layer, T *raw, XLayout lay) {
+             const int *tap_state, int layer, T *raw, XLayout lay, EmbedSrc es) {
   __shared__ float sh[33];
   const int r = blockIdx.x, d4 = d >> 2, nt = blockDim.x;
   // the gains are weights: they can be fetched before the predecessor has finished
@@ -77,11 +87,29 @@ k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
   float *xr = x + (long long)r * d;
   float4 v[NV];
   float ss = 0.f;
-  // every load of the row is issued before the first use
+  if (es.embed) {
+    int t = es.tok[r];
+    if (t >= es.vocab) { if (threadIdx.x == 0) atomicMax(es.status, DREAM_DEV_BAD_INDEX); t = -1; }
+    const T *src = (const T *)es.embed + (long long)(t < 0 ? 0 : t) * d;
 #pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    int i = threadIdx.x + j * nt;
-    v[j] = i < d4 ? ld_f4(xr + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < NV; ++j) {
+      int i = threadIdx.x + j * nt;
+      v[j] = (i < d4 && t >= 0) ? ld_f4(src + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < d4) *reinterpret_cast<float4 *>(xr + 4 * i) = v[j];
+    }
+    if (es.rope_tab)
+      for (int i = threadIdx.x; i < es.half; i += nt) {
+        float cs, sn;
+        rope_cs(es.pos[r], es.inv_freq[i], &cs, &sn);
+        es.rope_tab[(long long)r * es.half + i] = make_float2(cs, sn);
+      }
+  } else {
+    // every load of the row is issued before the first use
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      int i = threadIdx.x + j * nt;
+      v[j] = i < d4 ? ld_f4(xr + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
   }
   if (has_in) {
     float4 gv[NV];
