@@ -468,6 +468,58 @@ class DreamOracle:
             path.append(cur)
             out.append(tree["tokens"][cur])
 
+    # ------------------------------------------------------------------ O8, sampling form
+    @staticmethod
+    def accept_sample(tree, logits, temp, uniforms):
+        """Stochastic acceptance at temperature `temp` > 0 (Section 2.1: a draft token d is kept
+        with probability min(1, P_target(d) / P_draft(d)), which holds at any temperature;
+        Section 4 evaluates Temp = 1).
+
+        Reading for a tree whose children are the draft's top-K choices (no draw on the draft
+        side): every child is a point-mass proposal, P_draft = 1, so child c of the current node
+        is kept with probability p(token_c), p = softmax(logits[cur] / temp) with the tokens
+        already refused at this node taken out and the rest renormalised (the residual
+        max(p - P_draft, 0) of a point mass is p without that token).  Children are tried in
+        node order.  When every child is refused, or the node has none, the emitted token is
+        drawn from what is left of p by inverting its cumulative sum in token order.  The
+        emitted token then follows p exactly, whatever the draft proposed.
+
+        uniforms[j][r]: the number in [0, 1) used at path step j for the r-th child tried
+        (r < K), uniforms[j][-1] for the final draw.  Returns (A, out_tokens, path, slack) with
+        slack = the smallest distance of a used uniform from the threshold it was compared with.
+        """
+        T = len(tree["tokens"])
+        lg = torch.as_tensor(logits, dtype=torch.float64)
+        cur, path, out, slack, j = 0, [0], [], 1.0, 0
+        while True:
+            p = torch.softmax(lg[cur] / temp, 0)
+            kids = [i for i in range(T) if tree["parent"][i] == cur]
+            left, taken = 1.0, None
+            for r, c in enumerate(kids):
+                pc = float(p[tree["tokens"][c]]) / left
+                u = float(uniforms[j][r])
+                slack = min(slack, abs(u - pc))
+                if u < pc:
+                    taken = c
+                    break
+                left -= float(p[tree["tokens"][c]])
+                p[tree["tokens"][c]] = 0.0
+            if taken is None:
+                cdf = torch.cumsum(p, 0)
+                target = float(uniforms[j][-1]) * float(cdf[-1])
+                g = int(torch.searchsorted(cdf, torch.tensor(target, dtype=torch.float64), right=True))
+                g = min(g, len(p) - 1)
+                while float(p[g]) == 0.0:        # a refused token or an underflowed tail entry
+                    g -= 1
+                lo = float(cdf[g - 1]) if g > 0 else 0.0
+                slack = min(slack, (target - lo) / float(cdf[-1]), (float(cdf[g]) - target) / float(cdf[-1]))
+                out.append(g)
+                return len(path) - 1, out, path, slack
+            cur = taken
+            path.append(cur)
+            out.append(tree["tokens"][cur])
+            j += 1
+
     # ------------------------------------------------------------------ O9
     def commit(self, st, tree, ver, path, out_tokens):
         """Compact the target KV to the accepted path and extend the draft's caches."""
@@ -487,12 +539,16 @@ class DreamOracle:
         st.pending = out_tokens[-1]
         return path
 
-    def step(self, st, tree=None):
-        """One draft + verify + accept + commit round; `tree` overrides the draft's tree."""
+    def step(self, st, tree=None, temp=0.0, uniforms=None):
+        """One draft + verify + accept + commit round; `tree` overrides the draft's tree.
+        temp > 0 takes the sampling form of the acceptance with the given uniforms."""
         drafted = self.draft_tree(st)
         tree = drafted if tree is None else tree
         ver = self.verify_tree(st, tree)
-        A, out, path = self.accept(tree, ver["argmax"])
+        if temp > 0:
+            A, out, path, _ = self.accept_sample(tree, ver["logits"], temp, uniforms)
+        else:
+            A, out, path = self.accept(tree, ver["argmax"])
         self.commit(st, tree, ver, path, out)
         return dict(tree=tree, drafted=drafted, ver=ver, A=A, out=out, path=path)
 
