@@ -218,6 +218,9 @@ def main():
     ap.add_argument("--chain", action="store_true",
                     help="sweep aid: a chain-shaped draft (one child per node, depth D) instead of the tree")
     ap.add_argument("--batch", type=int, default=0, help="sweep aid: number of sequences per step")
+    ap.add_argument("--temp", type=float, default=0.0,
+                    help="acceptance by the sampling rule at this temperature (greedy otherwise); the verify "
+                         "call then also writes the logits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     p = dict(configs.PRESETS[args.workload])
@@ -233,6 +236,8 @@ def main():
     if args.batch:
         p["batch"] = args.batch
         p["name"] = "%s[batch=%d]" % (p["name"], args.batch)
+    if args.temp > 0:
+        p["name"] = "%s[temp=%g]" % (p["name"], args.temp)
     if args.impl == "reference":
         return run_reference(args, p)
 
@@ -264,6 +269,10 @@ def main():
     alen = torch.zeros(B, dtype=torch.int32, device=dev)
     outt = torch.zeros(B * (p["tree_depth"] + 1), dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream(dev)
+    if args.temp > 0:
+        lg = torch.zeros(B * T, p["vocab"], dtype=torch.float32, device=dev)
+        uni = torch.rand(B, p["tree_depth"] + 1, T, dtype=torch.float32, device=dev,
+                         generator=torch.Generator(dev).manual_seed(rank))
 
     def one_step(ev=None):
         if ev:
@@ -271,10 +280,13 @@ def main():
         ctx.dream_draft_tree(seqs, trees)
         if ev:
             ev[1].record(stream)
-        ctx.dream_verify_tree(seqs, trees, am)
+        ctx.dream_verify_tree(seqs, trees, am, None, lg if args.temp > 0 else None)
         if ev:
             ev[2].record(stream)
-        ctx.dream_accept(seqs, trees, am, alen, outt)
+        if args.temp > 0:
+            ctx.dream_accept_sample(seqs, trees, lg, args.temp, uni, alen, outt)
+        else:
+            ctx.dream_accept(seqs, trees, am, alen, outt)
         if ev:
             ev[3].record(stream)
 

@@ -167,6 +167,26 @@ dream_status dream_accept(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
                           const dream_tree *trees, const int32_t *node_argmax,
                           int32_t *accept_len, int32_t *out_tokens, int32_t *compaction_src);
 
+/* Acceptance at a sampling temperature above zero, and the same state update as dream_accept
+ * (Section 2.1: a draft token d is accepted with probability min(1, P_target(d) / P_draft(d)), a
+ * rule that holds at any temperature; Section 4 reports Temp = 1).  The tree's children are the
+ * draft's top-K choices, so each is a point-mass proposal (P_draft = 1): child c of the current
+ * node, tried in node order, is kept when u < p(token_c), where p = softmax(logits[cur] /
+ * temperature) without the tokens already refused at this node, renormalised.  When every child
+ * is refused, or the node has none, the emitted token is drawn from what is left of p by
+ * inverting its cumulative sum in token order.  The emitted tokens follow the target's own
+ * sampling distribution whatever the tree proposed.
+ *   logits      : device float [n_seqs][T][vocab], e.g. the dump of dream_verify_tree
+ *   temperature : > 0 (DREAM_E_ARG otherwise)
+ *   uniforms    : device float [n_seqs][D+1][T], numbers in [0, 1) drawn by the caller: [b][j][r]
+ *                 decides the r-th child tried at path step j, [b][j][T-1] is the final draw
+ * Outputs as in dream_accept.  Follows dream_verify_tree (DREAM_E_STATE otherwise); enqueues on the
+ * context's stream and returns. */
+dream_status dream_accept_sample(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
+                                 const dream_tree *trees, const float *logits, float temperature,
+                                 const float *uniforms, int32_t *accept_len, int32_t *out_tokens,
+                                 int32_t *compaction_src);
+
 /* One whole round (draft, verify, accept) with HOST result buffers: runs the three calls
  * above on the context's internal tree buffers, copies accept_len [n_seqs] and out_tokens
  * [n_seqs][D+1] to host memory and waits for them.  This is the call a serving loop makes. */

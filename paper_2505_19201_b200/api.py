@@ -71,6 +71,7 @@ def lib():
             "dream_draft_tree": [vp, i32p, i32, C.POINTER(dream_tree)],
             "dream_verify_tree": [vp, i32p, i32, C.POINTER(dream_tree), vp, vp, vp],
             "dream_accept": [vp, i32p, i32, C.POINTER(dream_tree), vp, vp, vp, vp],
+            "dream_accept_sample": [vp, i32p, i32, C.POINTER(dream_tree), vp, C.c_float, vp, vp, vp, vp],
             "dream_step_host": [vp, i32p, i32, vp, vp],
             "dream_seq_state": [vp, i32, i32p, i32p, i32p],
             "dream_debug_read": [vp, i32, i32, i32, i32, vp],
@@ -255,6 +256,11 @@ class Context:
         a, n = self._seqs(seqs)
         _check(self.h, lib().dream_accept(self.h, a, n, self._trees(trees), _ptr(node_argmax), _ptr(accept_len),
                                           _ptr(out_tokens), _ptr(compaction_src)))
+
+    def dream_accept_sample(self, seqs, trees, logits, temperature, uniforms, accept_len, out_tokens, compaction_src=None):
+        a, n = self._seqs(seqs)
+        _check(self.h, lib().dream_accept_sample(self.h, a, n, self._trees(trees), _ptr(logits), float(temperature),
+                                                 _ptr(uniforms), _ptr(accept_len), _ptr(out_tokens), _ptr(compaction_src)))
 
     def dream_step_host(self, seqs, accept_len_host, out_tokens_host):
         """accept_len_host / out_tokens_host: CPU int32 tensors (HOST buffers)."""

@@ -924,12 +924,16 @@ extern "C" dream_status dream_verify_tree(dream_ctx *c, const int32_t *seqs, int
 // ------------------------------------------------------------------------------------- accept
 
 template <typename T>
+// `logits` null: greedy acceptance on `argmax`; otherwise the sampling form on `logits` at
+// temperature `temp` with the caller's `uniforms`.
 static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const int *argmax, int *accept_len,
-                                int *out_tokens, int *comp_src) {
+                                int *out_tokens, int *comp_src, const float *logits = nullptr, float temp = 0.f,
+                                const float *uniforms = nullptr) {
   const dream_config &f = c->cfg;
   int D = c->ts.D, d = f.d_model, R = B * (D + 1);
   RowMeta &rm = c->rm[0];
-  LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
+  if (logits) LAUNCH(c, k_accept_sample, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src);
+  else LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
   LAUNCH(c, (k_compact_kv<T>), dim3(f.n_layers * 2, B), 256, 0, tb, c->sd, c->kv_pool, c->layer_stride, c->kv_stride, paged(c, 0));
   LAUNCH(c, k_accept_rows, 1, 32, 0, tb, B, c->T, D, c->sd, c->gather_idx, rm, c->cap_rows - c->ts.NI, c->status);
   const XMode xm = xmode(c, R);
@@ -950,6 +954,25 @@ extern "C" dream_status dream_accept(dream_ctx *c, const int32_t *seqs, int32_t 
     if (c->phase[seqs[b]] != PH_VERIFIED) return fail(c, DREAM_E_STATE, "sequence %d: dream_accept follows dream_verify_tree", seqs[b]);
   s = c->cfg.dtype == DREAM_BF16 ? accept_impl<bf16>(c, tb, n_seqs, node_argmax, accept_len, out_tokens, comp_src)
                                  : accept_impl<float>(c, tb, n_seqs, node_argmax, accept_len, out_tokens, comp_src);
+  if (s) return s;
+  CUDA_OK(c, cudaGetLastError());
+  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
+  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; c->key_ub[seqs[b]] += c->ts.D + 1; }
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_accept_sample(dream_ctx *c, const int32_t *seqs, int32_t n_seqs, const dream_tree *trees,
+                                            const float *logits, float temperature, const float *uniforms,
+                                            int32_t *accept_len, int32_t *out_tokens, int32_t *comp_src) {
+  TreeBatch tb;
+  dream_status s = make_batch(c, seqs, n_seqs, trees, false, &tb);
+  if (s) return s;
+  if (!logits || !uniforms || !accept_len || !out_tokens) return fail(c, DREAM_E_ARG, "logits, uniforms, accept_len, out_tokens are required");
+  if (!(temperature > 0.f)) return fail(c, DREAM_E_ARG, "temperature must be above zero (dream_accept is the greedy form)");
+  for (int b = 0; b < n_seqs; ++b)
+    if (c->phase[seqs[b]] != PH_VERIFIED) return fail(c, DREAM_E_STATE, "sequence %d: dream_accept_sample follows dream_verify_tree", seqs[b]);
+  s = c->cfg.dtype == DREAM_BF16 ? accept_impl<bf16>(c, tb, n_seqs, nullptr, accept_len, out_tokens, comp_src, logits, temperature, uniforms)
+                                 : accept_impl<float>(c, tb, n_seqs, nullptr, accept_len, out_tokens, comp_src, logits, temperature, uniforms);
   if (s) return s;
   CUDA_OK(c, cudaGetLastError());
   if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");

@@ -178,6 +178,29 @@ __global__ void k_tree_finalize(TreeBatch tb, SeqDev s, DraftTreeDev dt, TreeSha
   }
 }
 
+
+// What an acceptance leaves behind for sequence slot b: the emitted tokens (A accepted draft
+// tokens, then the target's own token g), the compaction map, the tokens that still lack draft
+// K/V rows, and the advanced prefix.  One thread.
+__device__ __forceinline__ void accept_commit(const TreePtrs &tp, int b, int seq, int D, const SeqDev &s, const int *path,
+                                              int A, int g, int *accept_len, int *out_tokens, int *comp_src) {
+  int P = s.P[seq];
+  out_tokens[b * (D + 1) + A] = g;
+  for (int j = A + 1; j <= D; ++j) out_tokens[b * (D + 1) + j] = -1;
+  accept_len[b] = A;
+  for (int j = 0; j <= D; ++j) {
+    if (comp_src) comp_src[b * (D + 1) + j] = j <= A ? path[j] : -1;
+    if (j <= A) {
+      s.new_tok[seq * (DREAM_MAX_DEPTH + 1) + j] = tp.tokens[path[j]];
+      s.new_pos[seq * (DREAM_MAX_DEPTH + 1) + j] = P + j;
+    }
+  }
+  s.n_new[seq] = A + 1;
+  s.last_P[seq] = P; s.last_A[seq] = A;
+  s.P[seq] = P + A + 1;
+  s.pending[seq] = g;
+}
+
 // ---------------------------------------------------------------------------------------
 // Verification rows: node i of slot b is row b*T + i at position P + depth[i], KV slot P + i.
 __global__ void k_verify_setup(TreeBatch tb, int B, int T, SeqDev s, RowMeta rm, uint32_t *mask,
@@ -219,23 +242,138 @@ __global__ void k_accept(TreeBatch tb, int B, int T, int D, SeqDev s, const int 
     cur = found; ++A;
     if (lane == 0) { path[A] = cur; out_tokens[b * (D + 1) + A - 1] = tp.tokens[cur]; }
   }
-  if (lane == 0) {
-    int g = am[cur], P = s.P[seq];
-    out_tokens[b * (D + 1) + A] = g;
-    for (int j = A + 1; j <= D; ++j) out_tokens[b * (D + 1) + j] = -1;
-    accept_len[b] = A;
-    for (int j = 0; j <= D; ++j) {
-      if (comp_src) comp_src[b * (D + 1) + j] = j <= A ? path[j] : -1;
-      if (j <= A) {
-        s.new_tok[seq * (DREAM_MAX_DEPTH + 1) + j] = tp.tokens[path[j]];
-        s.new_pos[seq * (DREAM_MAX_DEPTH + 1) + j] = P + j;
+  if (lane == 0) accept_commit(tp, b, seq, D, s, path, A, am[cur], accept_len, out_tokens, comp_src);
+}
+
+// ---------------------------------------------------------------------------------------
+// Acceptance at a temperature above zero (Section 2.1: a draft token is kept with probability
+// min(1, P_target / P_draft); Section 4 evaluates Temp = 1).  The tree's children are the draft's
+// top-K choices, i.e. point-mass proposals (P_draft = 1): child c of the current node is kept
+// when u < p(token_c), p = softmax(logits[cur] / temp) without the tokens already refused at this
+// node, renormalised; children are tried in node order.  When every child is refused (or there is
+// none) the emitted token is drawn from what is left of p by inverting its cumulative sum in
+// token order.  uniforms[b][j][r]: the number used at path step j for the r-th child tried
+// (r < T - 1), [j][T - 1] for the final draw.  One block of 1024 threads per sequence slot; warp
+// w owns the tokens [w * seg, (w + 1) * seg).
+#define SAMPLE_MAX_REFUSED 128
+__global__ void __launch_bounds__(1024)
+k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float *__restrict__ logits, float temp,
+                const float *__restrict__ uniforms, int *accept_len, int *out_tokens, int *comp_src) {
+  kernel_entry(TR_k_accept);
+  __shared__ float sh[33];
+  __shared__ float wtot[32];
+  __shared__ int refused[SAMPLE_MAX_REFUSED];
+  __shared__ int sh_i[4];
+  __shared__ float sh_f[2];
+  const int b = blockIdx.x, seq = tb.seq[b], lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const TreePtrs tp = tb.t[b];
+  const float inv_t = 1.f / temp;
+  const int seg = (((V + 31) / 32) + 31) & ~31;
+  const int v0 = w * seg, v1 = min(V, v0 + seg);
+  int *path = s.path + seq * (DREAM_MAX_DEPTH + 1);
+  if (threadIdx.x == 0) path[0] = 0;
+  int cur = 0, A = 0, emitted = -1;
+  while (emitted < 0) {
+    const float *row = logits + ((long long)b * T + cur) * V;
+    const float *u = uniforms + ((long long)b * (D + 1) + A) * T;
+    // the row's maximum (of the scaled logits)
+    float m = -INFINITY;
+    for (int v = threadIdx.x; v < V; v += blockDim.x) m = fmaxf(m, row[v] * inv_t);
+    m = warp_max(m);
+    __syncthreads();
+    if (lane == 0) sh[w] = m;
+    __syncthreads();
+    m = sh[0];
+    for (int i = 1; i < 32; ++i) m = fmaxf(m, sh[i]);
+    int n_ref = 0, last_kid = 0, tried = 0, taken = -1;
+    for (;;) {
+      // mass of every token not refused so far, per warp segment, then the whole row
+      float acc = 0.f;
+      for (int v = v0 + lane; v < v1; v += 32) {
+        float e = __expf(row[v] * inv_t - m);
+        for (int i = 0; i < n_ref; ++i) if (refused[i] == v) e = 0.f;
+        acc += e;
       }
+      acc = warp_sum(acc);
+      __syncthreads();
+      if (lane == 0) wtot[w] = acc;
+      // next child of cur in node order
+      int kid = 0x7fffffff;
+      if (A < D)
+        for (int i = last_kid + 1 + (int)threadIdx.x; i < T; i += blockDim.x)
+          if (tp.parent[i] == cur) kid = min(kid, i);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) kid = min(kid, __shfl_xor_sync(0xffffffffu, kid, o));
+      if (lane == 0) sh[w] = __int_as_float(kid);
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        float Z = 0.f;
+        for (int i = 0; i < 32; ++i) Z += wtot[i];
+        int k = 0x7fffffff;
+        for (int i = 0; i < 32; ++i) k = min(k, __float_as_int(sh[i]));
+        int decision = 0;                                   // 0 = final draw, 1 = kept, 2 = refused
+        if (k != 0x7fffffff && n_ref < SAMPLE_MAX_REFUSED) {
+          int tok = tp.tokens[k];
+          float e = (tok >= 0 && tok < V) ? __expf(row[tok] * inv_t - m) : 0.f;
+          for (int i = 0; i < n_ref; ++i) if (refused[i] == tok) e = 0.f;
+          decision = u[tried] * Z < e ? 1 : 2;
+          if (decision == 2) refused[n_ref] = tok;
+        }
+        sh_i[0] = decision; sh_i[1] = k; sh_f[0] = Z;
+      }
+      __syncthreads();
+      const int decision = sh_i[0];
+      if (decision == 0) break;
+      last_kid = sh_i[1];
+      ++tried;
+      if (decision == 1) { taken = last_kid; break; }
+      ++n_ref;
     }
-    s.n_new[seq] = A + 1;
-    s.last_P[seq] = P; s.last_A[seq] = A;
-    s.P[seq] = P + A + 1;
-    s.pending[seq] = g;
+    if (taken >= 0) {
+      cur = taken; ++A;
+      if (threadIdx.x == 0) { path[A] = cur; out_tokens[b * (D + 1) + A - 1] = tp.tokens[cur]; }
+      continue;
+    }
+    // final draw: the first token, in token order, at which the running mass exceeds u * Z
+    const float target = u[T - 1] * sh_f[0];
+    if (threadIdx.x == 0) {
+      float c = 0.f;
+      int ws = -1;
+      for (int i = 0; i < 32; ++i) { if (c + wtot[i] > target) { ws = i; break; } c += wtot[i]; }
+      if (ws < 0) {                                         // rounding pushed the target past the end:
+        ws = 31;                                            // the last token that has mass
+        while (ws > 0 && wtot[ws] <= 0.f) --ws;
+        c = -INFINITY;
+      }
+      sh_i[2] = ws; sh_f[1] = c;
+    }
+    __syncthreads();
+    if (w == sh_i[2]) {
+      float c = sh_f[1];
+      int found = -1, last_pos = -1;
+      for (int base = v0; base < v1 && found < 0; base += 32) {
+        int v = base + lane;
+        float e = 0.f;
+        if (v < v1) {
+          e = __expf(row[v] * inv_t - m);
+          for (int i = 0; i < n_ref; ++i) if (refused[i] == v) e = 0.f;
+        }
+        float inc = e;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { float t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+        unsigned hit = __ballot_sync(0xffffffffu, e > 0.f && c + inc > target);
+        unsigned pos = __ballot_sync(0xffffffffu, e > 0.f);
+        if (pos) last_pos = base + 31 - __clz(pos);
+        if (hit) found = base + __ffs(hit) - 1;
+        c += __shfl_sync(0xffffffffu, inc, 31);
+      }
+      if (found < 0) found = last_pos;                      // the segment's last token with mass
+      if (lane == 0) sh_i[3] = found;
+    }
+    __syncthreads();
+    emitted = sh_i[3];
   }
+  if (threadIdx.x == 0) accept_commit(tp, b, seq, D, s, path, A, emitted, accept_len, out_tokens, comp_src);
 }
 
 // KV compaction: the rows of path node j move from tail slot P + path[j] to P + j, for every

@@ -88,6 +88,9 @@ class Pair:
         self.ctx = api.Context(self.cfg, self.twg, self.dwg, device)
         self.T = self.ctx.T
         self.report = dict(exempt=0, decisions=0)
+        # sampling form of the acceptance: both sides read the same fp32 logits and uniforms; the GPU
+        # sums a row's exp() in fp32 in another order than the oracle's fp64 (relative 1e-6 or so)
+        self.samp_slack = 1e-4
         self.st = {}
 
     def _decide(self, same, margin, what):
@@ -138,8 +141,11 @@ class Pair:
         return st
 
     # ------------------------------------------------------------------ one round
-    def step(self, seqs=(0,), inject=None, check_cache_rows=2):
-        """Draft, verify, accept on both sides; `inject` maps seq -> oracle-format tree to verify instead."""
+    def step(self, seqs=(0,), inject=None, check_cache_rows=2, temp=0.0, gen=None):
+        """Draft, verify, accept on both sides; `inject` maps seq -> oracle-format tree to verify instead.
+        temp > 0 takes the sampling form of the acceptance: both sides get the oracle's logits
+        (as fp32) and the same uniforms from `gen`, so the walk itself is what is compared; a
+        mismatch is accepted only where a uniform fell within `samp_slack` of its threshold."""
         p, dev, tol, T, ctx, orc = self.p, self.device, self.tol, self.T, self.ctx, self.orc
         B, D, V = len(seqs), p["tree_depth"], p["vocab"]
         trees = [ctx.new_tree() for _ in seqs]
@@ -185,12 +191,18 @@ class Pair:
         gam, glg = am.cpu().tolist(), lg.cpu()
         hid = {(b, i): ctx.dream_debug_read(seqs[b], 7, 0, b * T + i) for b in range(B) for i in (0, T - 1)}
         tapr = {(b, i): ctx.dream_debug_read(seqs[b], 6, 0, b * T + i) for b in range(B) for i in (0, T - 1)}
-        ctx.dream_accept(list(seqs), trees, am, alen, outt, csrc)
+        vers = [orc.verify_tree(self.st[s], use[b]) for b, s in enumerate(seqs)]
+        if temp > 0:
+            olg = torch.stack([v["logits"].float() for v in vers]).contiguous()
+            uni = torch.rand(B, D + 1, T, generator=gen, dtype=torch.float32)
+            ctx.dream_accept_sample(list(seqs), trees, olg.to(dev), temp, uni.to(dev), alen, outt, csrc)
+        else:
+            ctx.dream_accept(list(seqs), trees, am, alen, outt, csrc)
         ctx.dream_poll()
         results = []
         for b, s in enumerate(seqs):
             st, tree = self.st[s], use[b]
-            ver = orc.verify_tree(st, tree)
+            ver = vers[b]
             close(glg[b * T:(b + 1) * T], ver["logits"], tol, "verify logits", self.report)
             for i in (0, T - 1):
                 close(hid[(b, i)], ver["hidden"][i], tol, "final hidden", self.report)
@@ -198,7 +210,17 @@ class Pair:
             for i in range(T):
                 if not self._decide(gam[b * T + i] == ver["argmax"][i], ver["margin"][i], f"argmax of node {i}"):
                     ver["argmax"][i] = gam[b * T + i]
-            A, out, path = orc.accept(tree, ver["argmax"])
+            if temp > 0:
+                A, out, path, slack = orc.accept_sample(tree, olg[b].double(), temp, uni[b].double())
+                gA = int(alen[b])
+                g_out = outt.cpu().tolist()[b * (D + 1):b * (D + 1) + gA + 1]
+                g_path = csrc.cpu().tolist()[b * (D + 1):b * (D + 1) + gA + 1]
+                if not self._decide((gA, g_out, g_path) == (A, out, path), slack * (tol.dec / self.samp_slack), "sampled acceptance"):
+                    assert g_path[0] == 0 and all(tree["parent"][c] == q for q, c in zip(g_path, g_path[1:]))
+                    assert g_out[:-1] == [tree["tokens"][c] for c in g_path[1:]] and 0 <= g_out[-1] < V
+                    A, out, path = gA, g_out, g_path
+            else:
+                A, out, path = orc.accept(tree, ver["argmax"])
             P0 = st.P
             orc.commit(st, tree, ver, path, out)
             assert int(alen[b]) == A, f"accept length {int(alen[b])} != {A}"
