@@ -33,7 +33,7 @@ from paper_2505_19201_b200 import configs, synth  # noqa: E402
 # capture ran on the 4-layer cut of the workload (same layer shapes); traffic grows in proportion
 # to the weight bytes, so a step's mean launch is scaled by this ratio.  None for workloads without
 # a capture, and to be reset to None whenever the kernel changes.
-TRAFFIC_RATIO = {"llava7b": (105.50 + 34.62 + 186.71 + 96.32) / (100.66 + 33.55 + 180.36 + 90.18)}
+TRAFFIC_RATIO = {"llava7b": (105.94 + 34.63 + 187.11 + 96.19) / (100.66 + 33.55 + 180.36 + 90.18)}
 
 METRIC = "verified_tree_tokens_per_s"
 UNIT = "tokens/s"
