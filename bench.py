@@ -257,10 +257,16 @@ def main():
     ctx = api.Context(cfg, twg, dwg, dev)
     T = ctx.T
     seqs = list(range(B))
+    setup_ms = []                      # per sequence: prefill (with entropy and tap choice) + compression
     for s in seqs:
         vis, ids = synth.request_inputs(p, request_seed(s, rank), dev)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(torch.cuda.current_stream(dev))
         ctx.dream_prefill(s, vis, 0, ids)
         ctx.dream_compress_visual(s, p["k_visual"])
+        s1.record(torch.cuda.current_stream(dev))
+        torch.cuda.synchronize(dev)
+        setup_ms.append(s0.elapsed_time(s1))
     ctx.dream_poll()
     P0 = p["n_visual"] + p["n_prompt"]
 
@@ -360,6 +366,7 @@ def main():
                 config=dict(workload=p["name"], batch=B, tree_nodes=T, prefix=P0, parallelism=f"replicas{world}",
                             l2="step working set (weights, %.1f GB) exceeds the 126 MB L2" % (sb["gemm_weights"] / 1e9)),
                 draft_us=draft_us, verify_us=verify_us, accept_us=accept_us,
+                setup_ms_per_sequence=statistics.median(setup_ms),
                 step_bytes=sb["total"], step_gbs=step_gbs,
                 step_roofline_frac=step_gbs / pk["hbm_gbs"], step_roofline_frac_nominal_8tbs=step_gbs / 8000.0,
                 clocks=sampler.summary(), gpu_launches=int(launches),

@@ -104,3 +104,16 @@ def test_llava_full_size_output_does_not_depend_on_the_tree():
                               min_margin=min(ma))))
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("preset", ["pixtral12b", "gemma3_12b"])
+def test_large_presets_full_size_against_the_oracle(preset):
+    """The Pixtral-12B-shaped and Gemma3-12B-shaped workloads at full size (40 / 48 layers, prefixes
+    of 1536 / 4352 tokens) against the oracle: prefill, compression and one round, element by
+    element.  The oracle needs about one and two minutes of CPU time for them on 16 cores;
+    DREAM_SKIP_LARGE=1 leaves them out."""
+    import os
+    if os.environ.get("DREAM_SKIP_LARGE") == "1":
+        pytest.skip("DREAM_SKIP_LARGE=1")
+    from tests.test_gpu_parity import _run
+    _run(preset, 1, decode_steps=4)
