@@ -95,3 +95,36 @@ def test_emitted_tokens_follow_the_target_distribution():
         assert abs(float(second[v]) / n1 - float(p1[v])) < 4.5 * sd
     # node 1 proposes token 3: it is walked into exactly when token 3 is emitted first
     assert n1 == int(first[3])
+
+
+def test_sampled_rounds_leave_the_state_of_a_fresh_prefill():
+    """Whole loop with the sampling rule: after several rounds whose trees hold plausible
+    proposals, the target KV cache equals that of a fresh prefill of prompt + emitted tokens, and
+    every emitted token was drawn from the target's row at its position (it has non-zero
+    probability there and the pending token is the last one emitted)."""
+    from tests.test_oracle_pins import _setup
+    p, orc, st, vis, ids = _setup(scale=30.0)
+    g = torch.Generator().manual_seed(21)
+    D, V = p["tree_depth"], p["vocab"]
+    emitted, lens = [st.pending], []
+    for _ in range(5):
+        # proposals: the two most likely tokens under the target at each level of a depth-D chain
+        toks, par, last = [st.pending], [-1], 0
+        for _lvl in range(D):
+            ver = orc.verify_tree(st, O.make_tree(toks, par))
+            top = torch.topk(ver["logits"][last], 2).indices.tolist()
+            toks += top
+            par += [last, last]
+            last = len(toks) - 2
+        T = len(toks)
+        u = torch.rand(D + 1, T, dtype=torch.float64, generator=g)
+        r = orc.step(st, O.make_tree(toks, par), temp=0.7, uniforms=u.tolist())
+        assert len(r["out"]) == r["A"] + 1 and r["out"][-1] == st.pending
+        emitted += r["out"]
+        lens.append(r["A"])
+    assert max(lens) >= 1
+    st2, tok2, _ = orc.prefill(vis, 0, ids, extra_ids=emitted[:-1])
+    assert st2.P == st.P
+    for l in range(p["n_layers"]):
+        assert torch.allclose(st.K[l], st2.K[l], atol=1e-10)
+        assert torch.allclose(st.V[l], st2.V[l], atol=1e-10)
