@@ -131,32 +131,53 @@ __global__ void k_entropy_mean(const float *__restrict__ ent, int count, float *
 
 // Importance of visual token j at this layer (Section 3.3): the attention weight it receives,
 // summed over the later query rows (and its own row when include_self) and over heads.
-// One warp per visual column; heads outer, rows inner, both ascending: a fixed order.
+// One warp per (visual column, head), grid (ceil(v / 8), H): rows ascending, four in flight at a
+// time, added in row order; k_colsum_heads then adds the heads in ascending order: a fixed order.
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_colsum(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
-         const float *__restrict__ lse, int vis_start, int v, int include_self, float *score) {
+         const float *__restrict__ lse, int vis_start, int v, int include_self, float *part /* [H][v] */) {
   constexpr int EPL = HD / 32;
   kernel_entry(TR_k_colsum);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  int jv = blockIdx.x * ATT_WARPS + w;
+  int jv = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (jv >= v) return;
   int j = vis_start + jv;
-  const T *Kp = (const T *)kv.base;
-  float tot = 0.f;
-  for (int h = 0; h < H; ++h) {
-    int kvh = h / (H / kv.hkv);
-    float k[EPL], q[EPL];
-    RowLoad<EPL, T>::ld(Kp + kv.off(seq, j, kvh), lane, k);
-    float hs = 0.f;
-    for (int i = include_self ? j : j + 1; i < n; ++i) {
-      QLoad<EPL, T>::ld(qbuf, (long long)i * H + h, lane, q);
-      float s = dot_lane<EPL>(q, k) * scale;
-      hs += __expf(s - lse[(long long)h * n + i]);
-    }
-    tot += hs;
+  int kvh = h / (H / kv.hkv);
+  float k[EPL];
+  RowLoad<EPL, T>::ld((const T *)kv.base + kv.off(seq, j, kvh), lane, k);
+  const float *lse_h = lse + (long long)h * n;
+  float hs = 0.f;
+  int i = include_self ? j : j + 1;
+  for (; i + 3 < n; i += 4) {
+    float q0[EPL], q1[EPL], q2[EPL], q3[EPL];
+    QLoad<EPL, T>::ld(qbuf, (long long)i * H + h, lane, q0);
+    QLoad<EPL, T>::ld(qbuf, (long long)(i + 1) * H + h, lane, q1);
+    QLoad<EPL, T>::ld(qbuf, (long long)(i + 2) * H + h, lane, q2);
+    QLoad<EPL, T>::ld(qbuf, (long long)(i + 3) * H + h, lane, q3);
+    float l0 = lse_h[i], l1 = lse_h[i + 1], l2 = lse_h[i + 2], l3 = lse_h[i + 3];
+    float s0 = dot_lane<EPL>(q0, k), s1 = dot_lane<EPL>(q1, k), s2 = dot_lane<EPL>(q2, k), s3 = dot_lane<EPL>(q3, k);
+    hs += __expf(s0 * scale - l0);
+    hs += __expf(s1 * scale - l1);
+    hs += __expf(s2 * scale - l2);
+    hs += __expf(s3 * scale - l3);
   }
-  if (lane == 0) score[jv] = tot;
+  for (; i < n; ++i) {
+    float q[EPL];
+    QLoad<EPL, T>::ld(qbuf, (long long)i * H + h, lane, q);
+    hs += __expf(dot_lane<EPL>(q, k) * scale - lse_h[i]);
+  }
+  if (lane == 0) part[(long long)h * v + jv] = hs;
+}
+
+// score[jv] = sum over heads, ascending, of the per-head column sums.
+__global__ void k_colsum_heads(const float *__restrict__ part, int H, int v, float *score) {
+  kernel_entry(TR_k_colsum);
+  int jv = blockIdx.x * blockDim.x + threadIdx.x;
+  if (jv >= v) return;
+  float tot = 0.f;
+  for (int h = 0; h < H; ++h) tot += part[(long long)h * v + jv];
+  score[jv] = tot;
 }
 
 // ---------------------------------------------------------------------------------------

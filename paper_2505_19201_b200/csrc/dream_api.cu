@@ -554,8 +554,11 @@ template <typename T, int HD> struct AttnLaunch {
   }
   static void colsum(dream_ctx *c, int layer, int seq, int n, int vis_start, int v, float *score) {
     if (v == 0) return;
-    LAUNCH(c, (k_colsum<T, HD>), (v + ATT_WARPS - 1) / ATT_WARPS, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n,
-           c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, score);
+    // the per-head sums land in the entropy buffer, which is idle between this layer's entropy mean
+    // and the next layer's attention ([H][n] floats, v <= n)
+    LAUNCH(c, (k_colsum<T, HD>), dim3((v + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads), ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n,
+           c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, c->ent_pre);
+    LAUNCH(c, k_colsum_heads, (v + 255) / 256, 256, 0, (const float *)c->ent_pre, c->cfg.n_heads, v, score);
   }
   // Split-K plan and launch of the tensor-core attention (bf16 configurations).
   template <bool PAGED>
