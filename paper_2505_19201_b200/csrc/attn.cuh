@@ -103,7 +103,23 @@ k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H,
   for (int e = 0; e < EPL; ++e) q[e] *= scale;
   Soft<EPL> st;
   st.init();
-  for (int j = 0; j <= i; ++j) {
+  // four keys in flight at a time (their loads and butterfly reductions overlap); the softmax
+  // state still takes them one by one in ascending order
+  int j = 0;
+  for (; j + 3 <= i; j += 4) {
+    float k4[4][EPL], v4[4][EPL], s4[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      long long o = kv.off(seq, j + u, kvh);
+      RowLoad<EPL, T>::ld(Kp + o, lane, k4[u]);
+      RowLoad<EPL, T>::ld(Vp + o, lane, v4[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) s4[u] = dot_lane<EPL>(q, k4[u]);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) st.template push<true>(s4[u], v4[u]);
+  }
+  for (; j <= i; ++j) {
     long long o = kv.off(seq, j, kvh);
     RowLoad<EPL, T>::ld(Kp + o, lane, k);
     RowLoad<EPL, T>::ld(Vp + o, lane, v);
