@@ -84,12 +84,13 @@ __device__ __forceinline__ float dot_lane(const float (&a)[EPL], const float (&b
 
 // ---------------------------------------------------------------------------------------
 // Causal self-attention of the n prompt rows at one layer.  grid (ceil(n/8), H).
-// Outputs: attn_out [n][H*hd] (element type, input of the O projection), lse [H][n] (row
+// Outputs: attn_out, rows of H*hd values (element type, input of the O projection) in chunks of
+// chunk_rows rows, chunk_stride elements apart, each laid out as `lay` says; lse [H][n] (row
 // log-sum-exp of the scaled scores, for the importance pass), ent [H][n] row entropies.
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
-               T *attn_out, XLayout lay, float *lse, float *ent) {
+               T *attn_out, XLayout lay, int chunk_rows, long long chunk_stride, float *lse, float *ent) {
   constexpr int EPL = HD / 32;
   kernel_entry(TR_k_attn_prefill);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -128,7 +129,8 @@ k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H,
   float inv = 1.f / st.z;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
-    store_split<T>(attn_out + i * lay.row_stride + h * HD + lane * EPL + e, lay.lo_delta, st.acc[e] * inv);
+    store_split<T>(attn_out + (i / chunk_rows) * chunk_stride + (i % chunk_rows) * lay.row_stride + h * HD + lane * EPL + e,
+                   lay.lo_delta, st.acc[e] * inv);
   if (lane == 0) {
     lse[(long long)h * n + i] = st.m + logf(st.z);
     ent[(long long)h * n + i] = logf(st.z) - st.u / st.z;

@@ -204,7 +204,7 @@ static void derive(dream_ctx *c) {
   c->pps = (f.max_seq + f.page_tokens - 1) / f.page_tokens;
   c->n_pages = c->pps * f.max_batch;
   c->chunk = f.dtype == DREAM_BF16 ? TC_ROWS_SPLIT_1MMA : ROW_CHUNK;
-  c->RM = (imax(ROW_CHUNK, f.max_prompt) + 15) & ~15;
+  c->RM = (imax(ROW_CHUNK, f.max_prompt) + ROW_CHUNK - 1) / ROW_CHUNK * ROW_CHUNK;     // whole prefill chunks
   c->XR = c->RM;
 }
 
@@ -546,11 +546,18 @@ __global__ void k_read_row(const T *src, float *dst, int n) {
   if (i < n) dst[i] = to_f(src[i]);
 }
 
+// Elements between the attention outputs of consecutive prefill chunks (ROW_CHUNK rows each; bf16
+// configurations keep a plane of high and a plane of low rows per chunk).
+static long long prefill_chunk_stride(const dream_ctx *c) {
+  return (long long)(c->cfg.dtype == DREAM_BF16 ? 2 : 1) * ROW_CHUNK * c->Hhd;
+}
 template <typename T, int HD> struct AttnLaunch {
+  // The output rows are laid out per prefill chunk of ROW_CHUNK rows (the O projection's input).
   static void prefill(dream_ctx *c, int layer, int seq, int n) {
     dim3 grid((n + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
+    const XMode m = xmode(c, ROW_CHUNK);
     LAUNCH(c, (k_attn_prefill<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n, c->cfg.n_heads,
-           1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(xmode(c, 1), c->Hhd), c->lse_pre, c->ent_pre);
+           1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd), ROW_CHUNK, prefill_chunk_stride(c), c->lse_pre, c->ent_pre);
   }
   static void colsum(dream_ctx *c, int layer, int seq, int n, int vis_start, int v, float *score) {
     if (v == 0) return;
@@ -660,17 +667,20 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
                                  const int *ids, int q, int *first_token, float *first_margin,
                                  float *layer_entropy, int *tap_layer) {
   const dream_config &f = c->cfg;
-  int n = q + v, d = f.d_model, L = f.n_layers, CH = c->chunk;
+  // The prompt goes through the projections ROW_CHUNK rows at a time: the weights stream once per
+  // chunk (bf16: two token tiles of 128 rows share every weight panel).
+  int n = q + v, d = f.d_model, L = f.n_layers, CH = ROW_CHUNK;
   LAUNCH(c, k_iota_rows, (n + 255) / 256, 256, 0, c->rm[0], seq, n);
   LAUNCH(c, (k_build_prompt<T>), n, 256, 0, (const T *)c->embed, (const T *)visual, ids, vis_start, v, c->x, c->x0,
          d, f.vocab, c->status);
-  const XMode m1 = xmode(c, 1);            // the layout of at most one chunk of rows
-  const XLayout att = xlay(m1, c->Hhd);
+  const XMode mp = xmode(c, CH);           // the layout of a full chunk of rows
+  const XMode m1 = xmode(c, 1);
+  const long long att_chunk = prefill_chunk_stride(c);
   for (int l = 0; l < L; ++l) {
     for (int r0 = 0; r0 < n; r0 += CH) {
       int rows = imin(CH, n - r0);
-      norm_rows<T>(c, c->x + (size_t)r0 * d, NO_GEMM, false, c->ln1[l], rows, m1);
-      GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, m1, rows, c->qkvN, d);
+      norm_rows<T>(c, c->x + (size_t)r0 * d, NO_GEMM, false, c->ln1[l], rows, mp);
+      GemmOut g = gemm<T>(c, c->wqkv[l], c->xn, mp, rows, c->qkvN, d);
       LAUNCH(c, (k_qkv_post_target<T>), dim3(rows, (c->qkvN / 8 + 255) / 256), 256, 0, g, c->rm[0].seq, c->rm[0].pos, c->rm[0].slot, r0, c->qbuf,
              paged(c, l), f.n_heads, c->rope_inv, (const float2 *)nullptr);
     }
@@ -682,9 +692,9 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
     for (int r0 = 0; r0 < n; r0 += CH) {
       int rows = imin(CH, n - r0);
       float *xr = c->x + (size_t)r0 * d;
-      GemmOut g = gemm<T>(c, c->wo[l], (const T *)c->attn_out + (long long)r0 * att.row_stride, m1, rows, d, c->Hhd);
-      norm_rows<T>(c, xr, g, true, c->ln2[l], rows, m1);
-      g = mlp_rows<T>(c, c->wgu[l], c->wd[l], rows, m1);
+      GemmOut g = gemm<T>(c, c->wo[l], (const T *)c->attn_out + (long long)(r0 / CH) * att_chunk, mp, rows, d, c->Hhd);
+      norm_rows<T>(c, xr, g, true, c->ln2[l], rows, mp);
+      g = mlp_rows<T>(c, c->wgu[l], c->wd[l], rows, mp);
       float *copy = is_cand ? c->taps_store + ((size_t)cand * f.max_prompt + r0) * d : nullptr;
       LAUNCH(c, k_resid_add, dim3(rows, (d + 1023) / 1024), 256, 0, xr, g, d, copy);
     }
