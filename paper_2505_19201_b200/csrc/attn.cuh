@@ -83,57 +83,65 @@ __device__ __forceinline__ float dot_lane(const float (&a)[EPL], const float (&b
 #define ATT_WARPS 8
 
 // ---------------------------------------------------------------------------------------
-// Causal self-attention of the n prompt rows at one layer.  grid (ceil(n/8), H).
+// Causal self-attention of the n prompt rows at one layer.  A warp owns ATT_PF_ROWS consecutive
+// rows of one head, so a key/value row fetched from the cache serves all of them; two keys are
+// in flight at a time (their loads and butterfly reductions overlap) and each row's softmax state
+// takes its keys one by one in ascending order.  grid (ceil(n / (8 * ATT_PF_ROWS)), H).
 // Outputs: attn_out, rows of H*hd values (element type, input of the O projection) in chunks of
 // chunk_rows rows, chunk_stride elements apart, each laid out as `lay` says; lse [H][n] (row
 // log-sum-exp of the scaled scores, for the importance pass), ent [H][n] row entropies.
+#define ATT_PF_ROWS 4
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H, float scale,
                T *attn_out, XLayout lay, int chunk_rows, long long chunk_stride, float *lse, float *ent) {
-  constexpr int EPL = HD / 32;
+  constexpr int EPL = HD / 32, RW = ATT_PF_ROWS;
   kernel_entry(TR_k_attn_prefill);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  int i = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
-  if (i >= n) return;
+  int i0 = (blockIdx.x * ATT_WARPS + w) * RW, h = blockIdx.y;
+  if (i0 >= n) return;
+  const int nr = min(RW, n - i0);
   int kvh = h / (H / kv.hkv);
   const T *Kp = (const T *)kv.base, *Vp = (const T *)kv.base + kv.kv_stride;
-  float q[EPL], k[EPL], v[EPL];
-  QLoad<EPL, T>::ld(qbuf, (long long)i * H + h, lane, q);
+  float q[RW][EPL];
+  Soft<EPL> st[RW];
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) q[e] *= scale;
-  Soft<EPL> st;
-  st.init();
-  // four keys in flight at a time (their loads and butterfly reductions overlap); the softmax
-  // state still takes them one by one in ascending order
-  int j = 0;
-  for (; j + 3 <= i; j += 4) {
-    float k4[4][EPL], v4[4][EPL], s4[4];
+  for (int r = 0; r < RW; ++r) {
+    QLoad<EPL, T>::ld(qbuf, (long long)min(i0 + r, n - 1) * H + h, lane, q[r]);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      long long o = kv.off(seq, j + u, kvh);
-      RowLoad<EPL, T>::ld(Kp + o, lane, k4[u]);
-      RowLoad<EPL, T>::ld(Vp + o, lane, v4[u]);
+    for (int e = 0; e < EPL; ++e) q[r][e] *= scale;
+    st[r].init();
+  }
+  const int jmax = i0 + nr - 1;
+  for (int j = 0; j <= jmax; j += 2) {
+    float k0[EPL], v0[EPL], k1[EPL], v1[EPL], s0[RW], s1[RW];
+    const bool two = j + 1 <= jmax;
+    long long o0 = kv.off(seq, j, kvh), o1 = kv.off(seq, two ? j + 1 : j, kvh);
+    RowLoad<EPL, T>::ld(Kp + o0, lane, k0);
+    RowLoad<EPL, T>::ld(Vp + o0, lane, v0);
+    RowLoad<EPL, T>::ld(Kp + o1, lane, k1);
+    RowLoad<EPL, T>::ld(Vp + o1, lane, v1);
+#pragma unroll
+    for (int r = 0; r < RW; ++r) { s0[r] = dot_lane<EPL>(q[r], k0); s1[r] = dot_lane<EPL>(q[r], k1); }
+#pragma unroll
+    for (int r = 0; r < RW; ++r) {
+      if (r < nr && j <= i0 + r) st[r].template push<true>(s0[r], v0);
+      if (r < nr && two && j + 1 <= i0 + r) st[r].template push<true>(s1[r], v1);
     }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) s4[u] = dot_lane<EPL>(q, k4[u]);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) st.template push<true>(s4[u], v4[u]);
   }
-  for (; j <= i; ++j) {
-    long long o = kv.off(seq, j, kvh);
-    RowLoad<EPL, T>::ld(Kp + o, lane, k);
-    RowLoad<EPL, T>::ld(Vp + o, lane, v);
-    st.template push<true>(dot_lane<EPL>(q, k), v);
-  }
-  float inv = 1.f / st.z;
 #pragma unroll
-  for (int e = 0; e < EPL; ++e)
-    store_split<T>(attn_out + (i / chunk_rows) * chunk_stride + (i % chunk_rows) * lay.row_stride + h * HD + lane * EPL + e,
-                   lay.lo_delta, st.acc[e] * inv);
-  if (lane == 0) {
-    lse[(long long)h * n + i] = st.m + logf(st.z);
-    ent[(long long)h * n + i] = logf(st.z) - st.u / st.z;
+  for (int r = 0; r < RW; ++r) {
+    if (r >= nr) break;
+    const int i = i0 + r;
+    float inv = 1.f / st[r].z;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e)
+      store_split<T>(attn_out + (i / chunk_rows) * chunk_stride + (i % chunk_rows) * lay.row_stride + h * HD + lane * EPL + e,
+                     lay.lo_delta, st[r].acc[e] * inv);
+    if (lane == 0) {
+      lse[(long long)h * n + i] = st[r].m + logf(st[r].z);
+      ent[(long long)h * n + i] = logf(st[r].z) - st[r].u / st[r].z;
+    }
   }
 }
 

@@ -554,7 +554,7 @@ static long long prefill_chunk_stride(const dream_ctx *c) {
 template <typename T, int HD> struct AttnLaunch {
   // The output rows are laid out per prefill chunk of ROW_CHUNK rows (the O projection's input).
   static void prefill(dream_ctx *c, int layer, int seq, int n) {
-    dim3 grid((n + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
+    dim3 grid((n + ATT_WARPS * ATT_PF_ROWS - 1) / (ATT_WARPS * ATT_PF_ROWS), c->cfg.n_heads);
     const XMode m = xmode(c, ROW_CHUNK);
     LAUNCH(c, (k_attn_prefill<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n, c->cfg.n_heads,
            1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd), ROW_CHUNK, prefill_chunk_stride(c), c->lse_pre, c->ent_pre);
