@@ -204,7 +204,7 @@ static void derive(dream_ctx *c) {
   c->pps = (f.max_seq + f.page_tokens - 1) / f.page_tokens;
   c->n_pages = c->pps * f.max_batch;
   c->chunk = f.dtype == DREAM_BF16 ? TC_ROWS_SPLIT_1MMA : ROW_CHUNK;
-  c->RM = (imax(ROW_CHUNK, f.max_prompt) + ROW_CHUNK - 1) / ROW_CHUNK * ROW_CHUNK;     // whole prefill chunks
+  c->RM = (imax(ROW_CHUNK, f.max_prompt) + 15) & ~15;
   c->XR = c->RM;
 }
 
@@ -253,7 +253,8 @@ static size_t carve(dream_ctx *c, char *base) {
   c->x0 = a.take<float>((size_t)f.max_prompt * d);
   c->qbuf = a.take<float>((size_t)c->XR * c->Hhd);
   int planes = f.dtype == DREAM_BF16 ? 2 : 1;      // bf16 GEMM inputs: a high and a low row per token
-  c->attn_out = a.take_bytes((size_t)planes * c->XR * c->Hhd * e);
+  // attention outputs: whole prefill chunks of ROW_CHUNK rows
+  c->attn_out = a.take_bytes((size_t)planes * ((c->XR + ROW_CHUNK - 1) / ROW_CHUNK * ROW_CHUNK) * c->Hhd * e);
   c->xn = a.take_bytes((size_t)planes * ROW_CHUNK * d * e);
   c->raw = a.take_bytes((size_t)planes * ROW_CHUNK * d * e);
   c->act = a.take_bytes((size_t)planes * ROW_CHUNK * f.d_ff * e);
@@ -630,27 +631,17 @@ template <typename T, int HD> struct AttnLaunch {
 template <typename T>
 static void norm_rows(dream_ctx *c, float *x, const GemmOut &gin, bool has_in, const void *gain, int rows, XMode m,
                       float *copy = nullptr, const int *row_seq = nullptr, const int *tap = nullptr, int layer = 0,
-                      bool want_raw = false, const EmbedSrc *embed = nullptr) {
+                      bool want_raw = false) {
   const int d4 = c->cfg.d_model / 4;
   int nv = 1;
   while ((d4 + nv - 1) / nv > 1024) nv *= 2;                 // d_model <= 16384 by check_config
   const int threads = ((d4 + nv - 1) / nv + 31) & ~31;
-  EmbedSrc es = {};
-  if (embed) es = *embed;
-#define NORM_ARGS x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model, (T *)c->xn, copy, row_seq, tap, layer, \
-                  want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model), es
-  if (nv == 1) LAUNCH(c, (k_resid_norm<T, 1>), rows, threads, 0, NORM_ARGS);
-  else if (nv == 2) LAUNCH(c, (k_resid_norm<T, 2>), rows, threads, 0, NORM_ARGS);
-  else LAUNCH(c, (k_resid_norm<T, 4>), rows, threads, 0, NORM_ARGS);
-#undef NORM_ARGS
-}
-// Embedding lookup of a call's rows (and their rotary table) fused with the first norm.
-template <typename T>
-static void embed_norm_rows(dream_ctx *c, const RowMeta &rm, const void *gain, int rows, XMode m) {
-  EmbedSrc es;
-  es.embed = c->embed; es.tok = rm.tok; es.pos = rm.pos; es.inv_freq = c->rope_inv; es.rope_tab = c->rope_tab;
-  es.status = c->status; es.vocab = c->cfg.vocab; es.half = c->cfg.head_dim / 2;
-  norm_rows<T>(c, c->x, NO_GEMM, false, gain, rows, m, nullptr, nullptr, nullptr, 0, false, &es);
+  if (nv == 1) LAUNCH(c, (k_resid_norm<T, 1>), rows, threads, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
+  else if (nv == 2) LAUNCH(c, (k_resid_norm<T, 2>), rows, threads, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
+  else LAUNCH(c, (k_resid_norm<T, 4>), rows, threads, 0, x, gin, has_in ? 1 : 0, (const T *)gain, c->cfg.rms_eps, c->cfg.d_model,
+         (T *)c->xn, copy, row_seq, tap, layer, want_raw ? (T *)c->raw : (T *)nullptr, xlay(m, c->cfg.d_model));
 }
 template <typename T>
 static GemmOut mlp_rows(dream_ctx *c, const void *wgu, const void *wd, int rows, XMode m) {
@@ -842,8 +833,10 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     const XMode xm = xmode(c, R);
     RowMeta &rm = c->rm[cur], &rn = c->rm[cur ^ 1];
     if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
+    LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status,
+           (const int *)rm.pos, (const double *)c->rope_inv, c->rope_tab, f.head_dim / 2);
     GemmOut g;
-    embed_norm_rows<T>(c, rm, c->dw.ln1, R, xm);
+    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
     g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
     LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv, (const float2 *)c->rope_tab);
     HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub));
@@ -894,12 +887,12 @@ static dream_status verify_impl(dream_ctx *c, const TreeBatch &tb, int B, int *a
   int key_ub = 0;
   for (int b = 0; b < B; ++b) { key_ub = imax(key_ub, c->p_ub[tb.seq[b]] + c->T); c->cur_seq[b] = tb.seq[b]; }
   LAUNCH(c, k_verify_setup, (R + 127) / 128, 128, 0, tb, B, c->T, c->sd, rm, c->vmask, f.max_seq, c->status);
+  LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status,
+           (const int *)rm.pos, (const double *)c->rope_inv, c->rope_tab, f.head_dim / 2);
   GemmOut gd = NO_GEMM, g;
   for (int l = 0; l < L; ++l) {
-    // the first norm completes S^l (for l >= 1) and captures it where a sequence taps layer l;
-    // layer 0's norm also looks the tree tokens up in the embedding table
-    if (l == 0) embed_norm_rows<T>(c, rm, c->ln1[0], R, xm);
-    else norm_rows<T>(c, c->x, gd, true, c->ln1[l], R, xm, c->tapbuf, rm.seq, c->sd.tap, l);
+    // the first norm completes S^l (for l >= 1) and captures it where a sequence taps layer l
+    norm_rows<T>(c, c->x, gd, l > 0, c->ln1[l], R, xm, l > 0 ? c->tapbuf : nullptr, rm.seq, c->sd.tap, l);
     g = gemm<T>(c, c->wqkv[l], c->xn, xm, R, c->qkvN, d);
     LAUNCH(c, (k_qkv_post_target<T>), dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.slot, 0, c->qbuf, paged(c, l), f.n_heads, c->rope_inv, (const float2 *)c->rope_tab);
     HD_DISPATCH(c, T, tree(c, l, R, xm, B, key_ub));

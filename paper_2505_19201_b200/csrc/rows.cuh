@@ -7,6 +7,28 @@
 
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ void rope_cs(int pos, double inv, float *c, float *s);
+// x[r] = embed[tok[r]] (fp32 residual stream).  tok < 0 leaves a zero row.  One thread per four
+// elements: grid (rows, ceil(d / 1024)).  With rope_tab the first block of a row also tabulates
+// the row's rotary factors for every layer of the call: rope_tab[r][i] = (cos, sin)(pos[r] *
+// inv_freq[i]), i < half.
+template <typename T>
+__global__ void k_embed(const T *__restrict__ embed, const int *__restrict__ tok, float *x, int d,
+                        int vocab, int *status, const int *__restrict__ pos, const double *__restrict__ inv_freq,
+                        float2 *rope_tab, int half) {
+  kernel_entry(TR_k_embed);
+  int r = blockIdx.x, t = tok[r];
+  if (rope_tab && blockIdx.y == 0)
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+      float c, s;
+      rope_cs(pos[r], inv_freq[i], &c, &s);
+      rope_tab[(long long)r * half + i] = make_float2(c, s);
+    }
+  int i = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
+  if (t >= vocab) { if (threadIdx.x == 0 && blockIdx.y == 0) atomicMax(status, DREAM_DEV_BAD_INDEX); t = -1; }
+  if (i >= d) return;
+  *reinterpret_cast<float4 *>(x + (long long)r * d + i) = t >= 0 ? ld_f4(embed + (long long)t * d + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 // Prompt input rows of the prefill: visual embeddings inside [vis_start, vis_start+v),
 // token embeddings elsewhere.  Writes the running residual x and a kept copy x0.
 template <typename T>
@@ -34,18 +56,6 @@ __global__ void k_build_prompt(const T *__restrict__ embed, const T *__restrict_
 // Optional side outputs of the updated residual: `copy` (fp32; when tap_state is given the
 // row is copied only if its sequence's tap layer equals `layer`) and `raw` (element type,
 // unnormalised: the memory side of Eq. 1 takes features without a norm).
-// With an EmbedSrc the rows do not come from x but from the embedding table: x[r] = embed[tok[r]]
-// is written (tok < 0 leaves a zero row), and the rows' rotary factors are tabulated for every
-// layer of the call, rope_tab[r][i] = (cos, sin)(pos[r] * inv_freq[i]), i < half: lookup and first
-// norm in one kernel.
-struct EmbedSrc {
-  const void *embed;             // null: the rows are in x already
-  const int *tok, *pos;
-  const double *inv_freq;
-  float2 *rope_tab;
-  int *status;
-  int vocab, half;
-};
 // Block size: ceil(d / 4 / NV) threads rounded up to a warp (at most 1024); a thread keeps NV
 // groups of four elements, so rows of up to 4096 * NV elements fit.  The partial-sum slots of a
 // value are all fetched at once (up to 12 per round trip).
@@ -53,7 +63,7 @@ template <typename T, int NV>
 __global__ void __launch_bounds__(1024)
 k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
              float eps, int d, T *xn, float *copy, const int *row_seq,
-             const int *tap_state, int layer, T *raw, XLayout lay, EmbedSrc es) {
+             const int *tap_state, int layer, T *raw, XLayout lay) {
   __shared__ float sh[33];
   const int r = blockIdx.x, d4 = d >> 2, nt = blockDim.x;
   // the gains are weights: they can be fetched before the predecessor has finished
@@ -67,29 +77,11 @@ k_resid_norm(float *x, GemmOut gin, int has_in, const T *__restrict__ gain,
   float *xr = x + (long long)r * d;
   float4 v[NV];
   float ss = 0.f;
-  if (es.embed) {
-    int t = es.tok[r];
-    if (t >= es.vocab) { if (threadIdx.x == 0) atomicMax(es.status, DREAM_DEV_BAD_INDEX); t = -1; }
-    const T *src = (const T *)es.embed + (long long)(t < 0 ? 0 : t) * d;
+  // every load of the row is issued before the first use
 #pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      int i = threadIdx.x + j * nt;
-      v[j] = (i < d4 && t >= 0) ? ld_f4(src + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
-      if (i < d4) *reinterpret_cast<float4 *>(xr + 4 * i) = v[j];
-    }
-    if (es.rope_tab)
-      for (int i = threadIdx.x; i < es.half; i += nt) {
-        float cs, sn;
-        rope_cs(es.pos[r], es.inv_freq[i], &cs, &sn);
-        es.rope_tab[(long long)r * es.half + i] = make_float2(cs, sn);
-      }
-  } else {
-    // every load of the row is issued before the first use
-#pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      int i = threadIdx.x + j * nt;
-      v[j] = i < d4 ? ld_f4(xr + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+  for (int j = 0; j < NV; ++j) {
+    int i = threadIdx.x + j * nt;
+    v[j] = i < d4 ? ld_f4(xr + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   if (has_in) {
     float4 gv[NV];
@@ -139,7 +131,7 @@ __device__ __forceinline__ void rope_cs(int pos, double inv, float *c, float *s)
 }
 
 // (cos, sin) of four neighbouring rotary indices i..i+3 (i a multiple of 4) of row r: from the
-// table the call's first norm kernel made for its rows, or computed when there is none (prefill).
+// table k_embed made for the call's rows, or computed when there is none (prefill).
 __device__ __forceinline__ void rope_cs4(const float2 *tab, int r, int half, int pos, const double *inv_freq, int i,
                                          float4 &cs01, float4 &cs23) {
   if (tab) {
