@@ -938,7 +938,8 @@ static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const 
   const dream_config &f = c->cfg;
   int D = c->ts.D, d = f.d_model, R = B * (D + 1);
   RowMeta &rm = c->rm[0];
-  if (logits) LAUNCH(c, k_accept_sample, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src);
+  if (logits && f.vocab <= 32 * 32 * SAMPLE_CACHE) LAUNCH(c, k_accept_sample<true>, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src);
+  else if (logits) LAUNCH(c, k_accept_sample<false>, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src);
   else LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
   LAUNCH(c, (k_compact_kv<T>), dim3(f.n_layers * 2, B), 256, 0, tb, c->sd, c->kv_pool, c->layer_stride, c->kv_stride, paged(c, 0));
   LAUNCH(c, k_accept_rows, 1, 32, 0, tb, B, c->T, D, c->sd, c->gather_idx, rm, c->cap_rows - c->ts.NI, c->status);

@@ -255,7 +255,11 @@ __global__ void k_accept(TreeBatch tb, int B, int T, int D, SeqDev s, const int 
 // token order.  uniforms[b][j][r]: the number used at path step j for the r-th child tried
 // (r < T - 1), [j][T - 1] for the final draw.  One block of 1024 threads per sequence slot; warp
 // w owns the tokens [w * seg, (w + 1) * seg).
+// CACHED (vocab <= 32768): a thread keeps the exponentials of its up to 32 tokens of the current row
+// in registers, so a trial costs no pass over memory; a refused token is zeroed in place.
 #define SAMPLE_MAX_REFUSED 128
+#define SAMPLE_CACHE 32
+template <bool CACHED>
 __global__ void __launch_bounds__(1024)
 k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float *__restrict__ logits, float temp,
                 const float *__restrict__ uniforms, int *accept_len, int *out_tokens, int *comp_src) {
@@ -273,26 +277,45 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
   int *path = s.path + seq * (DREAM_MAX_DEPTH + 1);
   if (threadIdx.x == 0) path[0] = 0;
   int cur = 0, A = 0, emitted = -1;
+  float ev[CACHED ? SAMPLE_CACHE : 1];
   while (emitted < 0) {
     const float *row = logits + ((long long)b * T + cur) * V;
     const float *u = uniforms + ((long long)b * (D + 1) + A) * T;
     // the row's maximum (of the scaled logits)
     float m = -INFINITY;
-    for (int v = threadIdx.x; v < V; v += blockDim.x) m = fmaxf(m, row[v] * inv_t);
+    if (CACHED) {
+#pragma unroll
+      for (int k = 0; k < SAMPLE_CACHE; ++k) {
+        int v = v0 + 32 * k + lane;
+        ev[k] = v < v1 ? row[v] * inv_t : -INFINITY;
+        m = fmaxf(m, ev[k]);
+      }
+    } else {
+      for (int v = threadIdx.x; v < V; v += blockDim.x) m = fmaxf(m, row[v] * inv_t);
+    }
     m = warp_max(m);
     __syncthreads();
     if (lane == 0) sh[w] = m;
     __syncthreads();
     m = sh[0];
     for (int i = 1; i < 32; ++i) m = fmaxf(m, sh[i]);
+    if (CACHED) {
+#pragma unroll
+      for (int k = 0; k < SAMPLE_CACHE; ++k) ev[k] = v0 + 32 * k + lane < v1 ? __expf(ev[k] - m) : 0.f;
+    }
     int n_ref = 0, last_kid = 0, tried = 0, taken = -1;
     for (;;) {
       // mass of every token not refused so far, per warp segment, then the whole row
       float acc = 0.f;
-      for (int v = v0 + lane; v < v1; v += 32) {
-        float e = __expf(row[v] * inv_t - m);
-        for (int i = 0; i < n_ref; ++i) if (refused[i] == v) e = 0.f;
-        acc += e;
+      if (CACHED) {
+#pragma unroll
+        for (int k = 0; k < SAMPLE_CACHE; ++k) acc += ev[k];
+      } else {
+        for (int v = v0 + lane; v < v1; v += 32) {
+          float e = __expf(row[v] * inv_t - m);
+          for (int i = 0; i < n_ref; ++i) if (refused[i] == v) e = 0.f;
+          acc += e;
+        }
       }
       acc = warp_sum(acc);
       __syncthreads();
@@ -327,6 +350,13 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
       last_kid = sh_i[1];
       ++tried;
       if (decision == 1) { taken = last_kid; break; }
+      if (CACHED) {                                         // the owner of the refused token drops it
+        const int off = refused[n_ref] - v0;
+        if (off >= 0 && off < seg && (off & 31) == lane) {
+#pragma unroll
+          for (int k = 0; k < SAMPLE_CACHE; ++k) if (k == (off >> 5)) ev[k] = 0.f;
+        }
+      }
       ++n_ref;
     }
     if (taken >= 0) {
@@ -351,21 +381,30 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
     if (w == sh_i[2]) {
       float c = sh_f[1];
       int found = -1, last_pos = -1;
-      for (int base = v0; base < v1 && found < 0; base += 32) {
-        int v = base + lane;
-        float e = 0.f;
-        if (v < v1) {
-          e = __expf(row[v] * inv_t - m);
-          for (int i = 0; i < n_ref; ++i) if (refused[i] == v) e = 0.f;
-        }
+      auto group = [&](int base, float e) {
         float inc = e;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { float t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
         unsigned hit = __ballot_sync(0xffffffffu, e > 0.f && c + inc > target);
         unsigned pos = __ballot_sync(0xffffffffu, e > 0.f);
         if (pos) last_pos = base + 31 - __clz(pos);
-        if (hit) found = base + __ffs(hit) - 1;
+        if (hit && found < 0) found = base + __ffs(hit) - 1;
         c += __shfl_sync(0xffffffffu, inc, 31);
+      };
+      if (CACHED) {
+#pragma unroll
+        for (int k = 0; k < SAMPLE_CACHE; ++k)
+          if (found < 0 && v0 + 32 * k < v1) group(v0 + 32 * k, ev[k]);
+      } else {
+        for (int base = v0; base < v1 && found < 0; base += 32) {
+          int v = base + lane;
+          float e = 0.f;
+          if (v < v1) {
+            e = __expf(row[v] * inv_t - m);
+            for (int i = 0; i < n_ref; ++i) if (refused[i] == v) e = 0.f;
+          }
+          group(base, e);
+        }
       }
       if (found < 0) found = last_pos;                      // the segment's last token with mass
       if (lane == 0) sh_i[3] = found;

@@ -71,11 +71,14 @@ def test_toy_sampled_acceptance():
         pr.close()
 
 
-def test_llava_shape_sampled_and_greedy_acceptance():
-    """LLaVA-7B-shaped widths (vocab 32000, 61 tree rows), 2 layers: injected continuation of depth
-    2, greedy rule, then the sampling rule near greedy and at temperature 1."""
+@pytest.mark.parametrize("preset", ["llava7b", "smolvlm2b"])
+def test_bf16_shapes_sampled_and_greedy_acceptance(preset):
+    """LLaVA-7B-shaped (vocab 32000: the sampling kernel keeps a row's exponentials in registers) and
+    SmolVLM-2B-shaped widths (vocab 49152: it re-reads the row per trial), 61 tree rows, 2 layers:
+    injected continuation of depth 2, greedy rule, then the sampling rule near greedy and at
+    temperature 1."""
     from tests.parity import Pair
-    pr = Pair("llava7b", n_layers=2, n_visual=96, k_visual=24, n_prompt=32, decode_steps=8)
+    pr = Pair(preset, n_layers=2, n_visual=96, k_visual=24, n_prompt=32, decode_steps=8)
     try:
         pr.prefill()
         gen = torch.Generator().manual_seed(12)
