@@ -110,10 +110,13 @@ def test_llava_full_size_output_does_not_depend_on_the_tree():
 def test_large_presets_full_size_against_the_oracle(preset):
     """The Pixtral-12B-shaped and Gemma3-12B-shaped workloads at full size (40 / 48 layers, prefixes
     of 1536 / 4352 tokens) against the oracle: prefill, compression and one round, element by
-    element.  The oracle needs about one and two minutes of CPU time for them on 16 cores;
-    DREAM_SKIP_LARGE=1 leaves them out."""
+    element.  The oracle needs about one and two minutes of CPU time for them on 16 cores, so they
+    run when DREAM_FULL_SIZE=1 is set:
+
+        DREAM_FULL_SIZE=1 python -m pytest tests/test_gpu_fullsize.py -q -k large
+    """
     import os
-    if os.environ.get("DREAM_SKIP_LARGE") == "1":
-        pytest.skip("DREAM_SKIP_LARGE=1")
+    if os.environ.get("DREAM_FULL_SIZE") != "1":
+        pytest.skip("set DREAM_FULL_SIZE=1 to run the full-size 12B-shaped cases (three minutes of oracle time)")
     from tests.test_gpu_parity import _run
     _run(preset, 1, decode_steps=4)
