@@ -5,11 +5,11 @@ from oracle.dream_oracle import DreamOracle, OracleConfig
 from paper_2505_19201_b200 import configs, synth
 
 
-def make_oracle(preset, dtype=torch.float64, seed=0, **over):
+def make_oracle(preset, dtype=torch.float64, seed=0, kv_dtype=None, **over):
     p = configs.scaled(preset, **over) if isinstance(preset, str) else dict(preset, **over)
     tw = synth.target_weights(p, seed)
     dw = synth.draft_weights(p, seed)
-    return p, DreamOracle(OracleConfig.from_preset(p), tw, dw, dtype)
+    return p, DreamOracle(OracleConfig.from_preset(p), tw, dw, dtype, kv_dtype=kv_dtype)
 
 
 def tiny_preset(**over):
