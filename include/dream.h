@@ -105,6 +105,14 @@ typedef struct {
  * depth, children per node, maximum draft length).  Host-only arithmetic. */
 dream_status dream_tree_nodes(const dream_config *cfg, int32_t *T);
 
+/* Depths and ancestor-or-self bit masks of a tree given by its parent array (Section 3.1: the
+ * tree mask lets a node attend to its ancestors only): node 0 is the root, parent[0] = -1 and
+ * every other node's parent has a smaller index.  All four arrays are HOST memory: parent
+ * int32[n_nodes] in; depth int32[n_nodes] and mask uint32[n_nodes][4] out, in the layout of
+ * dream_tree.  For callers that inject their own trees into dream_verify_tree.  Host-only
+ * arithmetic; DREAM_E_ARG for a parent that does not precede its child or n_nodes outside 1..128. */
+dream_status dream_tree_from_parents(const int32_t *parent, int32_t n_nodes, int32_t *depth, uint32_t *mask);
+
 /* Bytes of device memory dream_init needs for this configuration.  Host-only. */
 dream_status dream_arena_bytes(const dream_config *cfg, size_t *bytes);
 
@@ -160,7 +168,9 @@ dream_status dream_verify_tree(dream_ctx *ctx, const int32_t *seqs, int32_t n_se
  * round): follows from the root the child whose token equals its parent's argmax; emits
  * the A accepted tokens plus the target's own next token; compacts the target KV cache so
  * the accepted path occupies positions P..P+A; appends the accepted rows' tapped features
- * to the cross-attention memory; P += A + 1.  Outputs (device): accept_len int32[n_seqs];
+ * to the cross-attention memory; P += A + 1.  seqs and trees must be those of the last
+ * dream_verify_tree, in the same order (DREAM_E_STATE otherwise: the verify's tapped features and
+ * row map are kept by position in that list).  Outputs (device): accept_len int32[n_seqs];
  * out_tokens int32[n_seqs][D+1] (first A+1 valid); compaction_src int32[n_seqs][D+1] (tree
  * node whose KV row moved to P+j; first A+1 valid). */
 dream_status dream_accept(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
@@ -193,7 +203,10 @@ dream_status dream_accept_sample(dream_ctx *ctx, const int32_t *seqs, int32_t n_
 dream_status dream_step_host(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
                              int32_t *accept_len_host, int32_t *out_tokens_host);
 
-/* Read back per-sequence state (host outputs; synchronises the stream). */
+/* Read back per-sequence state (host outputs; synchronises the stream).  The host bounds a
+ * sequence's verified length from above between read-backs (it grows by at most tree_depth + 1 per
+ * round); this call, dream_step_host, and a small asynchronous copy behind every acceptance make
+ * the bound exact again, so DREAM_E_CAPACITY is only reported when max_seq is really reached. */
 dream_status dream_seq_state(dream_ctx *ctx, int32_t seq, int32_t *verified_len,
                              int32_t *pending_token, int32_t *tap_layer);
 
@@ -264,7 +277,10 @@ const char *dream_trace_name(int32_t id);
 /* Forget a sequence (its pages return to the pool). */
 dream_status dream_seq_reset(dream_ctx *ctx, int32_t seq);
 
-/* Wait for the stream and report the device status word (DREAM_OK or an error). */
+/* Wait for the stream and report the device status word: DREAM_OK, DREAM_E_DEVICE_TIMEOUT (a
+ * bounded wait inside a kernel ran out) or DREAM_E_STATE (a kernel met a malformed tree, an index
+ * or a capacity out of range, or a logits row without mass; the offending rows were skipped).
+ * The word is sticky: it is not cleared by reading it. */
 dream_status dream_poll(dream_ctx *ctx);
 
 /* Number of kernels this context has launched since dream_init. */

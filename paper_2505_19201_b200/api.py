@@ -63,6 +63,7 @@ def lib():
         sig = {
             "dream_tree_nodes": [C.POINTER(dream_config), i32p],
             "dream_arena_bytes": [C.POINTER(dream_config), C.POINTER(C.c_size_t)],
+            "dream_tree_from_parents": [i32p, i32, i32p, C.POINTER(C.c_uint32)],
             "dream_init": [C.POINTER(dream_config), C.POINTER(dream_target_weights), C.POINTER(dream_draft_weights),
                            vp, C.c_size_t, vp, C.POINTER(vp)],
             "dream_prefill": [vp, i32, vp, i32, i32, vp, i32, vp, vp, vp, vp],
@@ -158,21 +159,25 @@ class Tree:
         return dream_tree(*(t.data_ptr() for t in (self.tokens, self.parent, self.depth, self.mask, self.cum_logp)))
 
     def load(self, tokens, parent):
-        """Fill from host lists (inject a tree); depth and masks are derived here."""
+        """Fill from host lists (inject a tree); the library derives depths and masks
+        (dream_tree_from_parents)."""
         T = self.T
         assert len(tokens) == T and len(parent) == T
-        depth, mask = [0] * T, [[0, 0, 0, 0] for _ in range(T)]
-        for i in range(T):
-            if i:
-                depth[i] = depth[parent[i]] + 1
-                mask[i] = list(mask[parent[i]])
-            mask[i][i >> 5] |= 1 << (i & 31)
-        as_i32 = lambda w: w - (1 << 32) if w >= (1 << 31) else w
+        par = torch.tensor(parent, dtype=torch.int32)
+        depth = torch.zeros(T, dtype=torch.int32)
+        mask = torch.zeros(T, 4, dtype=torch.int32)
+        _check(None, lib().dream_tree_from_parents(C.cast(par.data_ptr(), C.POINTER(C.c_int32)), T,
+                                                   C.cast(depth.data_ptr(), C.POINTER(C.c_int32)),
+                                                   C.cast(mask.data_ptr(), C.POINTER(C.c_uint32))))
+        self.load_raw(tokens, par, depth, mask)
+
+    def load_raw(self, tokens, parent, depth, mask):
+        """Copy the four arrays to the device as they are (no checks: error-path tests use this)."""
         dev = self.tokens.device
-        self.tokens.copy_(torch.tensor(tokens, dtype=torch.int32).to(dev))
-        self.parent.copy_(torch.tensor(parent, dtype=torch.int32).to(dev))
-        self.depth.copy_(torch.tensor(depth, dtype=torch.int32).to(dev))
-        self.mask.copy_(torch.tensor([[as_i32(w) for w in row] for row in mask], dtype=torch.int32).to(dev))
+        self.tokens.copy_(torch.as_tensor(tokens, dtype=torch.int32).to(dev))
+        self.parent.copy_(torch.as_tensor(parent, dtype=torch.int32).to(dev))
+        self.depth.copy_(torch.as_tensor(depth, dtype=torch.int32).to(dev))
+        self.mask.copy_(torch.as_tensor(mask, dtype=torch.int32).reshape(self.T, 4).to(dev))
 
     def to_host(self):
         m = self.mask.cpu().to(torch.int64) & 0xFFFFFFFF

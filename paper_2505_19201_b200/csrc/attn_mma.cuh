@@ -86,6 +86,109 @@ constexpr size_t attn_mma_smem() {
   return (size_t)2 * AM_ROWS * AmShape<HD>::LD * 2 + (size_t)2 * (PAGED ? 2 : 4) * AmShape<HD>::KBLK * AmShape<HD>::LD * 2 + AM_ROWS * 24;
 }
 
+// One block of KBLK keys for the sixteen query rows of a warp: S = Q K^T (queries as high + low
+// parts; K as stored, plus its low plane when PLANES == 2), tail mask, online softmax in the exp2
+// domain, O += P V (probabilities as high + low parts).  Kb / Vb: the block's K and V planes in
+// shared memory; mw0 / mw1: visible-tail-key bits of the thread's two rows.
+template <int HD, int PLANES>
+__device__ __forceinline__ void attn_block(const bf16 *Kb, const bf16 *Vb, uint32_t qh_addr, uint32_t ql_addr, int k_row, int k_col,
+                                           int v_row, int v_col, int t, int j0, int P, int tail_len, float scale_log2,
+                                           const uint32_t (&mw0)[4], const uint32_t (&mw1)[4],
+                                           float (&o_acc)[HD / 8][4], float (&m_run)[2], float (&l_run)[2]) {
+  constexpr int KBLK = AmShape<HD>::KBLK, LD = AmShape<HD>::LD;
+  constexpr int NT_S = KBLK / 8, NT_O = HD / 8, PLANE_ELEMS = KBLK * LD;
+  constexpr bool PAGED = PLANES == 1;
+  // ---- S = Q K^T
+  float s[NT_S][4];
+#pragma unroll
+  for (int n = 0; n < NT_S; ++n) { s[n][0] = 0.f; s[n][1] = 0.f; s[n][2] = 0.f; s[n][3] = 0.f; }
+#pragma unroll
+  for (int ks = 0; ks < HD / 16; ++ks) {
+    uint32_t ah0, ah1, ah2, ah3, al0, al1, al2, al3;
+    ldsm_x4(qh_addr + ks * 32, ah0, ah1, ah2, ah3);
+    ldsm_x4(ql_addr + ks * 32, al0, al1, al2, al3);
+#pragma unroll
+    for (int np = 0; np < NT_S / 2; ++np) {
+      uint32_t kb0, kb1, kb2, kb3;
+      uint32_t ka = smem_addr(Kb + (np * 16 + k_row) * LD + ks * 16 + k_col);
+      ldsm_x4(ka, kb0, kb1, kb2, kb3);
+      mma_16816(s[2 * np], ah0, ah1, ah2, ah3, kb0, kb1);
+      mma_16816(s[2 * np], al0, al1, al2, al3, kb0, kb1);
+      mma_16816(s[2 * np + 1], ah0, ah1, ah2, ah3, kb2, kb3);
+      mma_16816(s[2 * np + 1], al0, al1, al2, al3, kb2, kb3);
+      if (!PAGED) {
+        ldsm_x4(ka + PLANE_ELEMS * 2, kb0, kb1, kb2, kb3);
+        mma_16816(s[2 * np], ah0, ah1, ah2, ah3, kb0, kb1);
+        mma_16816(s[2 * np + 1], ah0, ah1, ah2, ah3, kb2, kb3);
+      }
+    }
+  }
+  // ---- scale, mask, online softmax (exp2 domain)
+  const bool need_mask = j0 + KBLK > P;
+  float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+  for (int n = 0; n < NT_S; ++n) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float v = s[n][e] * scale_log2;
+      if (need_mask) {
+        int j = j0 + n * 8 + 2 * t + (e & 1);
+        bool vis = j < P;
+        if (!vis) {
+          int jt = j - P;
+          if (jt < tail_len) {
+            uint32_t wsel = (e >> 1) ? ((jt >> 5) == 0 ? mw1[0] : (jt >> 5) == 1 ? mw1[1] : (jt >> 5) == 2 ? mw1[2] : mw1[3])
+                                     : ((jt >> 5) == 0 ? mw0[0] : (jt >> 5) == 1 ? mw0[1] : (jt >> 5) == 2 ? mw0[2] : mw0[3]);
+            vis = (wsel >> (jt & 31)) & 1u;
+          }
+        }
+        if (!vis) v = -INFINITY;
+      }
+      s[n][e] = v;
+      if (e >> 1) mx1 = fmaxf(mx1, v); else mx0 = fmaxf(mx0, v);
+    }
+  }
+  mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+  mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+  float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+  float base0 = mn0 == -INFINITY ? 0.f : mn0, base1 = mn1 == -INFINITY ? 0.f : mn1;
+  float corr0 = exp2f(m_run[0] - base0), corr1 = exp2f(m_run[1] - base1);
+  m_run[0] = mn0; m_run[1] = mn1;
+  l_run[0] *= corr0; l_run[1] *= corr1;
+#pragma unroll
+  for (int n = 0; n < NT_O; ++n) { o_acc[n][0] *= corr0; o_acc[n][1] *= corr0; o_acc[n][2] *= corr1; o_acc[n][3] *= corr1; }
+#pragma unroll
+  for (int n = 0; n < NT_S; ++n) {
+    s[n][0] = exp2f(s[n][0] - base0); s[n][1] = exp2f(s[n][1] - base0);
+    s[n][2] = exp2f(s[n][2] - base1); s[n][3] = exp2f(s[n][3] - base1);
+    l_run[0] += s[n][0] + s[n][1]; l_run[1] += s[n][2] + s[n][3];
+  }
+  // ---- O += P V
+#pragma unroll
+  for (int kk = 0; kk < KBLK / 16; ++kk) {
+    uint32_t ph0, ph1, ph2, ph3, pl0, pl1, pl2, pl3;
+    split_pair(s[2 * kk][0], s[2 * kk][1], ph0, pl0);
+    split_pair(s[2 * kk][2], s[2 * kk][3], ph1, pl1);
+    split_pair(s[2 * kk + 1][0], s[2 * kk + 1][1], ph2, pl2);
+    split_pair(s[2 * kk + 1][2], s[2 * kk + 1][3], ph3, pl3);
+#pragma unroll
+    for (int nd = 0; nd < HD / 16; ++nd) {
+      uint32_t vb0, vb1, vb2, vb3;
+      uint32_t va = smem_addr(Vb + (kk * 16 + v_row) * LD + nd * 16 + v_col);
+      ldsm_x4_t(va, vb0, vb1, vb2, vb3);
+      mma_16816(o_acc[2 * nd], ph0, ph1, ph2, ph3, vb0, vb1);
+      mma_16816(o_acc[2 * nd], pl0, pl1, pl2, pl3, vb0, vb1);
+      mma_16816(o_acc[2 * nd + 1], ph0, ph1, ph2, ph3, vb2, vb3);
+      mma_16816(o_acc[2 * nd + 1], pl0, pl1, pl2, pl3, vb2, vb3);
+      if (!PAGED) {
+        ldsm_x4_t(va + PLANE_ELEMS * 2, vb0, vb1, vb2, vb3);
+        mma_16816(o_acc[2 * nd], ph0, ph1, ph2, ph3, vb0, vb1);
+        mma_16816(o_acc[2 * nd + 1], ph0, ph1, ph2, ph3, vb2, vb3);
+      }
+    }
+  }
+}
+
 template <int HD, bool PAGED>
 __global__ void __launch_bounds__(AM_THREADS)
 k_attn_mma(AttnMmaArgs a) {
@@ -195,96 +298,8 @@ k_attn_mma(AttnMmaArgs a) {
     __syncthreads();
     const bf16 *Kb = KV + buf * BUF_ELEMS, *Vb = Kb + PLANES * PLANE_ELEMS;
     if (!warp_live) { __syncthreads(); continue; }
-    // ---- S = Q K^T
-    float s[NT_S][4];
-#pragma unroll
-    for (int n = 0; n < NT_S; ++n) { s[n][0] = 0.f; s[n][1] = 0.f; s[n][2] = 0.f; s[n][3] = 0.f; }
-#pragma unroll
-    for (int ks = 0; ks < HD / 16; ++ks) {
-      uint32_t ah0, ah1, ah2, ah3, al0, al1, al2, al3;
-      ldsm_x4(qh_addr + ks * 32, ah0, ah1, ah2, ah3);
-      ldsm_x4(ql_addr + ks * 32, al0, al1, al2, al3);
-#pragma unroll
-      for (int np = 0; np < NT_S / 2; ++np) {
-        uint32_t kb0, kb1, kb2, kb3;
-        uint32_t ka = smem_addr(Kb + (np * 16 + k_row) * LD + ks * 16 + k_col);
-        ldsm_x4(ka, kb0, kb1, kb2, kb3);
-        mma_16816(s[2 * np], ah0, ah1, ah2, ah3, kb0, kb1);
-        mma_16816(s[2 * np], al0, al1, al2, al3, kb0, kb1);
-        mma_16816(s[2 * np + 1], ah0, ah1, ah2, ah3, kb2, kb3);
-        mma_16816(s[2 * np + 1], al0, al1, al2, al3, kb2, kb3);
-        if (!PAGED) {
-          ldsm_x4(ka + PLANE_ELEMS * 2, kb0, kb1, kb2, kb3);
-          mma_16816(s[2 * np], ah0, ah1, ah2, ah3, kb0, kb1);
-          mma_16816(s[2 * np + 1], ah0, ah1, ah2, ah3, kb2, kb3);
-        }
-      }
-    }
-    // ---- scale, mask, online softmax (exp2 domain)
-    const int j0 = blk * KBLK;
-    const bool need_mask = j0 + KBLK > P;
-    float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-    for (int n = 0; n < NT_S; ++n) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float v = s[n][e] * a.scale_log2;
-        if (need_mask) {
-          int j = j0 + n * 8 + 2 * t + (e & 1);
-          bool vis = j < P;
-          if (!vis) {
-            int jt = j - P;
-            if (jt < a.tail_len) {
-              uint32_t wsel = (e >> 1) ? ((jt >> 5) == 0 ? mw1[0] : (jt >> 5) == 1 ? mw1[1] : (jt >> 5) == 2 ? mw1[2] : mw1[3])
-                                       : ((jt >> 5) == 0 ? mw0[0] : (jt >> 5) == 1 ? mw0[1] : (jt >> 5) == 2 ? mw0[2] : mw0[3]);
-              vis = (wsel >> (jt & 31)) & 1u;
-            }
-          }
-          if (!vis) v = -INFINITY;
-        }
-        s[n][e] = v;
-        if (e >> 1) mx1 = fmaxf(mx1, v); else mx0 = fmaxf(mx0, v);
-      }
-    }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
-    float base0 = mn0 == -INFINITY ? 0.f : mn0, base1 = mn1 == -INFINITY ? 0.f : mn1;
-    float corr0 = exp2f(m_run[0] - base0), corr1 = exp2f(m_run[1] - base1);
-    m_run[0] = mn0; m_run[1] = mn1;
-    l_run[0] *= corr0; l_run[1] *= corr1;
-#pragma unroll
-    for (int n = 0; n < NT_O; ++n) { o_acc[n][0] *= corr0; o_acc[n][1] *= corr0; o_acc[n][2] *= corr1; o_acc[n][3] *= corr1; }
-#pragma unroll
-    for (int n = 0; n < NT_S; ++n) {
-      s[n][0] = exp2f(s[n][0] - base0); s[n][1] = exp2f(s[n][1] - base0);
-      s[n][2] = exp2f(s[n][2] - base1); s[n][3] = exp2f(s[n][3] - base1);
-      l_run[0] += s[n][0] + s[n][1]; l_run[1] += s[n][2] + s[n][3];
-    }
-    // ---- O += P V
-#pragma unroll
-    for (int kk = 0; kk < KBLK / 16; ++kk) {
-      uint32_t ph0, ph1, ph2, ph3, pl0, pl1, pl2, pl3;
-      split_pair(s[2 * kk][0], s[2 * kk][1], ph0, pl0);
-      split_pair(s[2 * kk][2], s[2 * kk][3], ph1, pl1);
-      split_pair(s[2 * kk + 1][0], s[2 * kk + 1][1], ph2, pl2);
-      split_pair(s[2 * kk + 1][2], s[2 * kk + 1][3], ph3, pl3);
-#pragma unroll
-      for (int nd = 0; nd < HD / 16; ++nd) {
-        uint32_t vb0, vb1, vb2, vb3;
-        uint32_t va = smem_addr(Vb + (kk * 16 + v_row) * LD + nd * 16 + v_col);
-        ldsm_x4_t(va, vb0, vb1, vb2, vb3);
-        mma_16816(o_acc[2 * nd], ph0, ph1, ph2, ph3, vb0, vb1);
-        mma_16816(o_acc[2 * nd], pl0, pl1, pl2, pl3, vb0, vb1);
-        mma_16816(o_acc[2 * nd + 1], ph0, ph1, ph2, ph3, vb2, vb3);
-        mma_16816(o_acc[2 * nd + 1], pl0, pl1, pl2, pl3, vb2, vb3);
-        if (!PAGED) {
-          ldsm_x4_t(va + PLANE_ELEMS * 2, vb0, vb1, vb2, vb3);
-          mma_16816(o_acc[2 * nd], ph0, ph1, ph2, ph3, vb0, vb1);
-          mma_16816(o_acc[2 * nd + 1], ph0, ph1, ph2, ph3, vb2, vb3);
-        }
-      }
-    }
+    attn_block<HD, PLANES>(Kb, Vb, qh_addr, ql_addr, k_row, k_col, v_row, v_col, t, blk * KBLK, P, a.tail_len, a.scale_log2,
+                           mw0, mw1, o_acc, m_run, l_run);
     __syncthreads();
   }
   pdl_trigger();                    // the keys are done: the GEMM kernel that follows may take the SMs

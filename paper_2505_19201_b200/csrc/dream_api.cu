@@ -22,6 +22,8 @@
 #define AM_MAX_CHUNKS 32        // most key chunks the split-K attention cuts a sequence into
 #define ROW_CHUNK 256          // most rows any launch set holds (max_batch * tree nodes, a prefill chunk)
 
+#define SNAP_SLOTS 4
+
 enum { PH_EMPTY = 0, PH_PREFILLED, PH_READY, PH_DRAFTED, PH_VERIFIED };
 
 static char g_init_error[256];
@@ -32,6 +34,8 @@ struct dream_ctx {
   TreeShape ts;
   int T, esz, qkvN, Hhd, kvN, n_cand, tap_lo_eff, cap_rows, pps, n_pages, RM, XR, gemm_rows_lm;
   int use_tc, use_pdl, gemm_failed;
+  cudaError_t launch_err;              // first refused kernel launch of the call being enqueued
+  const char *launch_err_name;
   int chunk;                           // prompt rows per pass of the prefill loop
   double *rope_inv;                    // [head_dim / 2] rotary inverse frequencies
   float2 *rope_tab;                    // [ROW_CHUNK][head_dim / 2] rotary (cos, sin) of the rows of the call being enqueued
@@ -58,7 +62,18 @@ struct dream_ctx {
   TopkScratch tks;
   float *am_part_o, *am_part_ml;       // split-K attention partials
   int am_rt_max;
-  int key_ub[DREAM_MAX_BATCH];         // upper bound of the draft caches' permanent rows
+  int key_ub0[DREAM_MAX_BATCH];        // permanent rows of the draft caches right after compression
+  // Verified lengths as the host knows them.  The device advances P by A + 1 per accept and the host
+  // only knows A <= D, so p_ub grows by D + 1 per accept until a snapshot of the device's P arrives:
+  // every accept enqueues a small copy of P into pinned memory behind an event, and the next call
+  // that plans launches adopts the newest snapshot whose event has completed (no host wait).
+  int *h_snap;                         // pinned [SNAP_SLOTS][DREAM_MAX_BATCH]
+  cudaEvent_t snap_ev[SNAP_SLOTS];
+  int snap_busy[SNAP_SLOTS];           // an event was recorded for this slot and not yet seen complete
+  long long snap_accepts[SNAP_SLOTS][DREAM_MAX_BATCH], snap_epoch[SNAP_SLOTS][DREAM_MAX_BATCH];
+  long long snap_order[SNAP_SLOTS], snap_clock;
+  long long accepts[DREAM_MAX_BATCH], epoch[DREAM_MAX_BATCH];
+  int last_verify_n, last_verify_seq[DREAM_MAX_BATCH];   // the sequence list of the last dream_verify_tree
   int cur_seq[DREAM_MAX_BATCH];        // sequences of the call being enqueued, by slot
   int tk_nsplit, tk_nv;                // vocabulary blocks of the top-k kernel, columns per thread (4 or 16)
   int *top_id, *argmax_i, *accept_len_i, *out_tokens_i, *comp_src_i;
@@ -93,20 +108,37 @@ static dream_status fail(dream_ctx *c, dream_status code, const char *fmt, ...) 
     if (e_ != cudaSuccess) return fail(c, DREAM_E_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
   } while (0)
 
+// End of an entry point that enqueued kernels: report a refused launch by name.
+static dream_status call_done(dream_ctx *c) {
+  if (c->launch_err != cudaSuccess) {
+    cudaError_t e = c->launch_err;
+    c->launch_err = cudaSuccess;
+    cudaGetLastError();
+    return fail(c, DREAM_E_CUDA, "launch of %s failed: %s", c->launch_err_name, cudaGetErrorString(e));
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(c, DREAM_E_CUDA, "CUDA error after enqueueing: %s", cudaGetErrorString(e));
+  if (c->gemm_failed) { c->gemm_failed = 0; return fail(c, DREAM_E_CUDA, "a GEMM launch was refused (shape, output room or tensor map)"); }
+  return DREAM_OK;
+}
+
 // Every kernel is launched with programmatic stream serialization: it may become resident while
 // its predecessor still runs and blocks in pdl_wait() until that one has finished.
+// A refused launch is remembered with the kernel's name (the first one of a call); the entry point
+// that enqueued it reports it through call_done().
 template <typename... P, typename... A>
-static inline void launch_k(dream_ctx *c, void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, A... args) {
+static inline void launch_k(dream_ctx *c, const char *name, void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, A... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = c->use_pdl ? 1 : 0;
-  cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+  if (e != cudaSuccess && c->launch_err == cudaSuccess) { c->launch_err = e; c->launch_err_name = name; }
   c->launches++;
 }
-#define LAUNCH(c, kernel, grid, block, smem, ...) launch_k(c, kernel, dim3(grid), dim3(block), (size_t)(smem), __VA_ARGS__)
+#define LAUNCH(c, kernel, grid, block, smem, ...) launch_k(c, #kernel, kernel, dim3(grid), dim3(block), (size_t)(smem), __VA_ARGS__)
 #define TOPK_LAUNCH(c, grid, ...)                                                        \
   do {                                                                                   \
     if ((c)->tk_nv == 4) LAUNCH(c, (k_topk_lse<4>), grid, TOPK_THREADS, 0, __VA_ARGS__); \
@@ -145,9 +177,35 @@ extern "C" dream_status dream_tree_nodes(const dream_config *cfg, int32_t *T) {
   return DREAM_OK;
 }
 
+extern "C" dream_status dream_tree_from_parents(const int32_t *parent, int32_t n_nodes, int32_t *depth, uint32_t *mask) {
+  if (!parent || !depth || !mask) return fail(nullptr, DREAM_E_ARG, "null argument");
+  if (n_nodes < 1 || n_nodes > 128) return fail(nullptr, DREAM_E_ARG, "n_nodes outside 1..128");
+  if (parent[0] != -1) return fail(nullptr, DREAM_E_ARG, "node 0 is the root: parent[0] must be -1");
+  for (int i = 0; i < n_nodes; ++i) {
+    uint32_t *m = mask + 4 * i;
+    if (i == 0) { depth[0] = 0; m[0] = m[1] = m[2] = m[3] = 0u; }
+    else {
+      int p = parent[i];
+      if (p < 0 || p >= i) return fail(nullptr, DREAM_E_ARG, "parent[%d] = %d: parents precede their children", i, p);
+      depth[i] = depth[p] + 1;
+      for (int w = 0; w < 4; ++w) m[w] = mask[4 * p + w];
+    }
+    m[i >> 5] |= 1u << (i & 31);
+  }
+  return DREAM_OK;
+}
+
 static int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
 static int imax(int a, int b) { return a > b ? a : b; }
 static int imin(int a, int b) { return a < b ? a : b; }
+
+// Most rows one sequence contributes to any launch set: a verify takes T rows, the first draft pass
+// D + 2 (root plus catch-up rows), a later pass its beam.
+static int rows_per_seq_max(const TreeShape *ts) {
+  int m = imax(ts->T, ts->D + 2);
+  for (int p = 0; p <= ts->D; ++p) m = imax(m, ts->beam[p]);
+  return m;
+}
 
 static dream_status check_config(const dream_config *c, TreeShape *ts) {
   if (!c) return fail(nullptr, DREAM_E_ARG, "null config");
@@ -168,7 +226,14 @@ static dream_status check_config(const dream_config *c, TreeShape *ts) {
   if (c->max_prompt < 1 || c->max_visual < 0 || c->max_visual > c->max_prompt || c->max_seq < c->max_prompt)
     return fail(nullptr, DREAM_E_ARG, "max_seq >= max_prompt >= max_visual required");
   if (tree_shape(c, ts)) return fail(nullptr, DREAM_E_UNSUPPORTED, "tree: depth<=15, topk<=16, beam*topk<=256, input nodes<=64, nodes<=128");
-  if (c->max_batch * ts->T > ROW_CHUNK) return fail(nullptr, DREAM_E_UNSUPPORTED, "max_batch * tree nodes must be <= 256");
+  if (c->max_batch * rows_per_seq_max(ts) > ROW_CHUNK)
+    return fail(nullptr, DREAM_E_UNSUPPORTED, "max_batch * max(tree nodes, depth + 2, widest beam) must be <= 256");
+  {   // the top-k kernel's last block merges at most 1024 candidates (vocabulary blocks x list length)
+    int nv = (c->vocab + 1023) / 1024 * TOPK_MAX <= 1024 ? 4 : 16;
+    int nsplit = (c->vocab + nv * TOPK_THREADS - 1) / (nv * TOPK_THREADS);
+    if (nsplit * imax(ts->K, 2) > 1024)
+      return fail(nullptr, DREAM_E_UNSUPPORTED, "vocab / 4096 * max(tree_topk, 2) must be <= 1024");
+  }
   if (c->tap_mode == DREAM_TAP_FIXED) {
     if (c->tap_layer < 1 || c->tap_layer > c->n_layers) return fail(nullptr, DREAM_E_ARG, "tap_layer");
   } else if (c->tap_mode == DREAM_TAP_ENTROPY_MIN || c->tap_mode == DREAM_TAP_ENTROPY_MAX) {
@@ -293,7 +358,7 @@ static size_t carve(dream_ctx *c, char *base) {
   c->top_val = a.take<float>((size_t)ROW_CHUNK * TOPK_MAX);
   c->top_id = a.take<int>((size_t)ROW_CHUNK * TOPK_MAX);
   c->lse_rows = a.take<float>(ROW_CHUNK);
-  c->am_rt_max = (T * (f.n_heads / f.n_kv_heads) + AM_ROWS - 1) / AM_ROWS;
+  c->am_rt_max = (rows_per_seq_max(&c->ts) * (f.n_heads / f.n_kv_heads) + AM_ROWS - 1) / AM_ROWS;
   if (f.dtype == DREAM_BF16) {
     size_t prow = (size_t)MB * AM_MAX_CHUNKS * f.n_kv_heads * c->am_rt_max * AM_ROWS;
     c->am_part_o = a.take<float>(prow * f.head_dim);
@@ -397,6 +462,42 @@ static FlatKV flat(dream_ctx *c, float *base) {
 }
 static const GemmOut NO_GEMM = {nullptr, 0, 0, 30, 0, 0, 0};
 
+// ------------------------------------------------------------------------------------- prefix bounds
+
+static int key_ub_of(const dream_ctx *c, int seq) { return c->key_ub0[seq] + (c->p_ub[seq] - c->n_prompt[seq]); }
+
+// After an accept was enqueued: copy the device's verified lengths to a free pinned slot.
+static void snapshot_lengths(dream_ctx *c) {
+  int slot = -1;
+  for (int i = 0; i < SNAP_SLOTS; ++i) {
+    if (c->snap_busy[i] && cudaEventQuery(c->snap_ev[i]) == cudaSuccess) c->snap_busy[i] = 2;   // complete, still unread or read
+    if (c->snap_busy[i] != 1 && (slot < 0 || c->snap_order[i] < c->snap_order[slot])) slot = i;
+  }
+  if (slot < 0) return;                                  // every slot still in flight: skip this one
+  if (cudaMemcpyAsync(c->h_snap + slot * DREAM_MAX_BATCH, c->sd.P, sizeof(int) * c->cfg.max_batch, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+      cudaEventRecord(c->snap_ev[slot], c->stream) != cudaSuccess) { cudaGetLastError(); c->snap_busy[slot] = 0; return; }
+  c->snap_busy[slot] = 1;
+  c->snap_order[slot] = ++c->snap_clock;
+  for (int b = 0; b < DREAM_MAX_BATCH; ++b) { c->snap_accepts[slot][b] = c->accepts[b]; c->snap_epoch[slot][b] = c->epoch[b]; }
+}
+
+// Before launches are planned: adopt the newest completed snapshot.  For a sequence that had k
+// accepts enqueued after the snapshot the bound is its P then plus k (D + 1).
+static void refresh_bounds(dream_ctx *c) {
+  int best = -1;
+  for (int i = 0; i < SNAP_SLOTS; ++i) {
+    if (c->snap_busy[i] == 1 && cudaEventQuery(c->snap_ev[i]) == cudaSuccess) c->snap_busy[i] = 2;
+    if (c->snap_busy[i] == 2 && (best < 0 || c->snap_order[i] > c->snap_order[best])) best = i;
+  }
+  cudaGetLastError();                                    // cudaErrorNotReady is not an error here
+  if (best < 0) return;
+  for (int b = 0; b < c->cfg.max_batch; ++b) {
+    if (c->snap_epoch[best][b] != c->epoch[b] || c->phase[b] < PH_READY) continue;
+    long long ub = (long long)c->h_snap[best * DREAM_MAX_BATCH + b] + (c->accepts[b] - c->snap_accepts[best][b]) * (c->ts.D + 1);
+    if (ub < c->p_ub[b]) c->p_ub[b] = (int)ub;
+  }
+}
+
 // ------------------------------------------------------------------------------------- init / free
 
 template <int HD>
@@ -405,6 +506,14 @@ static const char *attn_mma_setup() {
       cudaFuncSetAttribute(k_attn_mma<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_mma_smem<HD, false>()) != cudaSuccess)
     return "cannot raise the attention kernel's shared memory limit";
   return nullptr;
+}
+
+static void free_host_side(dream_ctx *c) {
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  for (int i = 0; i < SNAP_SLOTS; ++i) if (c->snap_ev[i]) cudaEventDestroy(c->snap_ev[i]);
+  cudaFreeHost(c->h_snap);
+  cudaFreeHost(c->h_stage);
+  delete c;
 }
 
 extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_weights *tw,
@@ -438,10 +547,23 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   if (e != cudaSuccess) { delete c; return fail(nullptr, DREAM_E_CUDA, "memset arena: %s", cudaGetErrorString(e)); }
   e = cudaHostAlloc((void **)&c->h_stage, sizeof(int) * ((size_t)cfg->max_batch * c->pps + 64 + cfg->max_batch * (DREAM_MAX_DEPTH + 2)), cudaHostAllocDefault);
   if (e != cudaSuccess) { delete c; return fail(nullptr, DREAM_E_CUDA, "pinned staging: %s", cudaGetErrorString(e)); }
+  e = cudaHostAlloc((void **)&c->h_snap, sizeof(int) * SNAP_SLOTS * DREAM_MAX_BATCH, cudaHostAllocDefault);
+  if (e != cudaSuccess) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "pinned snapshots: %s", cudaGetErrorString(e)); }
+  for (int i = 0; i < SNAP_SLOTS; ++i) {
+    c->snap_busy[i] = 0; c->snap_order[i] = 0; c->snap_ev[i] = nullptr;
+    if (cudaEventCreateWithFlags(&c->snap_ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      for (int j = 0; j < i; ++j) cudaEventDestroy(c->snap_ev[j]);
+      cudaFreeHost(c->h_snap); cudaFreeHost(c->h_stage); delete c;
+      return fail(nullptr, DREAM_E_CUDA, "cannot create an event");
+    }
+  }
+  c->snap_clock = 0; c->last_verify_n = 0;
+  for (int b = 0; b < DREAM_MAX_BATCH; ++b) { c->accepts[b] = 0; c->epoch[b] = 0; c->key_ub0[b] = 0; c->p_ub[b] = 0; c->n_prompt[b] = 0; }
   for (int p = c->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
   for (int b = 0; b < DREAM_MAX_BATCH; ++b) c->phase[b] = PH_EMPTY;
   c->prefill_seq = -1;
   c->launches = 0; c->tc_launches = 0; c->simt_launches = 0; c->gemm_failed = 0;
+  c->launch_err = cudaSuccess; c->launch_err_name = "";
   c->prof_on = 0; c->prof_n = 0; c->prof_bytes = 0.0;
   c->err[0] = 0;
   const char *pdl = getenv("DREAM_PDL");              // "0" serialises every launch (debugging aid)
@@ -449,14 +571,14 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   c->use_tc = cfg->dtype == DREAM_BF16;
   if (c->use_tc) {
     const char *why = gemm_tc_plan_init(&c->tc, c->status, c->use_pdl);
-    if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
+    if (why) { free_host_side(c); return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
   }
   if (c->use_tc) {
     const char *why = cfg->head_dim == 64 ? attn_mma_setup<64>() : cfg->head_dim == 128 ? attn_mma_setup<128>() : attn_mma_setup<256>();
-    if (why) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "%s", why); }
+    if (why) { free_host_side(c); return fail(nullptr, DREAM_E_CUDA, "%s", why); }
   }
   k_rope_table<<<(cfg->head_dim / 2 + 127) / 128, 128, 0, c->stream>>>(c->rope_inv, cfg->head_dim, cfg->rope_theta);
-  if (cudaGetLastError() != cudaSuccess) { cudaFreeHost(c->h_stage); delete c; return fail(nullptr, DREAM_E_CUDA, "rotary table launch failed"); }
+  if (cudaGetLastError() != cudaSuccess) { free_host_side(c); return fail(nullptr, DREAM_E_CUDA, "rotary table launch failed"); }
   *out = c;
   return DREAM_OK;
 }
@@ -464,9 +586,7 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
 extern "C" void dream_free(dream_ctx *c) {
   if (!c) return;
   cudaStreamSynchronize(c->stream);
-  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
-  cudaFreeHost(c->h_stage);
-  delete c;
+  free_host_side(c);
 }
 
 extern "C" const char *dream_last_error(const dream_ctx *c) { return c ? c->err : g_init_error; }
@@ -494,6 +614,7 @@ extern "C" dream_status dream_seq_reset(dream_ctx *c, int32_t seq) {
   for (int p : c->seq_pages[seq]) c->free_pages.push_back(p);
   c->seq_pages[seq].clear();
   c->phase[seq] = PH_EMPTY;
+  c->epoch[seq]++;
   if (c->prefill_seq == seq) c->prefill_seq = -1;
   return DREAM_OK;
 }
@@ -536,15 +657,13 @@ __global__ void k_copy_f32(const float *src, float *dst, int n) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src[i];
 }
-// A draft-cache row of a bf16 configuration: hd high parts then hd low parts.
-__global__ void k_read_row_split(const bf16 *src, float *dst, int n) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) dst[i] = to_f(src[i]) + to_f(src[n + i]);
-}
+// Debug read-back: block h copies n values from src + h * head_stride to dst + h * n.  split: the
+// source holds n high parts then n low parts (a draft-cache row of a bf16 configuration).
 template <typename T>
-__global__ void k_read_row(const T *src, float *dst, int n) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) dst[i] = to_f(src[i]);
+__global__ void k_read_row(const T *src, long long head_stride, float *dst, int n, int split) {
+  const T *s = src + (long long)blockIdx.x * head_stride;
+  for (int i = threadIdx.x; i < n; i += blockDim.x)
+    dst[(long long)blockIdx.x * n + i] = to_f(s[i]) + (split ? to_f(s[n + i]) : 0.f);
 }
 
 // Elements between the attention outputs of consecutive prefill chunks (ROW_CHUNK rows each; bf16
@@ -724,10 +843,10 @@ extern "C" dream_status dream_prefill(dream_ctx *c, int32_t seq, const void *vis
   if (f.dtype == DREAM_BF16) s = prefill_impl<bf16>(c, seq, visual, v, vis_start, ids, q, first_token, first_margin, layer_entropy, tap_layer);
   else s = prefill_impl<float>(c, seq, visual, v, vis_start, ids, q, first_token, first_margin, layer_entropy, tap_layer);
   if (s) return s;
-  CUDA_OK(c, cudaGetLastError());
-  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
+  s = call_done(c);
+  if (s) return s;
   c->phase[seq] = PH_PREFILLED;
-  c->n_prompt[seq] = v + q; c->p_ub[seq] = v + q;
+  c->n_prompt[seq] = v + q; c->p_ub[seq] = v + q; c->epoch[seq]++;
   c->prefill_seq = seq; c->pf_v = v; c->pf_vis_start = vis_start; c->pf_q = q;
   return DREAM_OK;
 }
@@ -786,10 +905,10 @@ extern "C" dream_status dream_compress_visual(dream_ctx *c, int32_t seq, int32_t
   s = c->cfg.dtype == DREAM_BF16 ? compress_impl<bf16>(c, seq, k, forced, kept, scores)
                                  : compress_impl<float>(c, seq, k, forced, kept, scores);
   if (s) return s;
-  CUDA_OK(c, cudaGetLastError());
-  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
+  s = call_done(c);
+  if (s) return s;
   c->phase[seq] = PH_READY;
-  c->key_ub[seq] = c->pf_q + (c->cfg.xattn_full_memory ? c->pf_v : k);
+  c->key_ub0[seq] = c->pf_q + (c->cfg.xattn_full_memory ? c->pf_v : k);
   c->prefill_seq = -1;
   return DREAM_OK;
 }
@@ -826,7 +945,7 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
   int d = f.d_model, cur = 0;
   for (int b = 0; b < B; ++b) c->cur_seq[b] = tb.seq[b];
   int key_ub = 0;                 // most keys any listed sequence can hold in a draft cache
-  for (int b = 0; b < B; ++b) key_ub = imax(key_ub, c->key_ub[tb.seq[b]] + ts.D + 1 + ts.NI);
+  for (int b = 0; b < B; ++b) key_ub = imax(key_ub, key_ub_of(c, tb.seq[b]) + ts.D + 1 + ts.NI);
   for (int p = 1; p <= ts.D; ++p) {
     int m = p == 1 ? ts.D + 2 : ts.beam[p - 1];
     int R = B * m;
@@ -868,10 +987,11 @@ extern "C" dream_status dream_draft_tree(dream_ctx *c, const int32_t *seqs, int3
   if (s) return s;
   for (int b = 0; b < n_seqs; ++b)
     if (c->phase[seqs[b]] != PH_READY) return fail(c, DREAM_E_STATE, "sequence %d: dream_draft_tree follows dream_compress_visual or dream_accept", seqs[b]);
+  refresh_bounds(c);
   s = c->cfg.dtype == DREAM_BF16 ? draft_impl<bf16>(c, tb, n_seqs) : draft_impl<float>(c, tb, n_seqs);
   if (s) return s;
-  CUDA_OK(c, cudaGetLastError());
-  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
+  s = call_done(c);
+  if (s) return s;
   for (int b = 0; b < n_seqs; ++b) c->phase[seqs[b]] = PH_DRAFTED;
   return DREAM_OK;
 }
@@ -914,6 +1034,7 @@ extern "C" dream_status dream_verify_tree(dream_ctx *c, const int32_t *seqs, int
   dream_status s = make_batch(c, seqs, n_seqs, trees, false, &tb);
   if (s) return s;
   if (!node_argmax) return fail(c, DREAM_E_ARG, "node_argmax is required");
+  refresh_bounds(c);
   for (int b = 0; b < n_seqs; ++b) {
     if (c->phase[seqs[b]] != PH_DRAFTED) return fail(c, DREAM_E_STATE, "sequence %d: dream_verify_tree follows dream_draft_tree", seqs[b]);
     if (c->p_ub[seqs[b]] + c->T > c->cfg.max_seq) return fail(c, DREAM_E_CAPACITY, "sequence %d may outgrow max_seq", seqs[b]);
@@ -921,13 +1042,22 @@ extern "C" dream_status dream_verify_tree(dream_ctx *c, const int32_t *seqs, int
   s = c->cfg.dtype == DREAM_BF16 ? verify_impl<bf16>(c, tb, n_seqs, node_argmax, node_margin, logits)
                                  : verify_impl<float>(c, tb, n_seqs, node_argmax, node_margin, logits);
   if (s) return s;
-  CUDA_OK(c, cudaGetLastError());
-  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
-  for (int b = 0; b < n_seqs; ++b) c->phase[seqs[b]] = PH_VERIFIED;
+  s = call_done(c);
+  if (s) return s;
+  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_VERIFIED; c->last_verify_seq[b] = seqs[b]; }
+  c->last_verify_n = n_seqs;
   return DREAM_OK;
 }
 
 // ------------------------------------------------------------------------------------- accept
+
+// The tapped features, row map and argmax of a verify are kept by batch slot, so the acceptance must
+// name the same sequences in the same order.
+static bool same_list_as_verify(const dream_ctx *c, const int *seqs, int n_seqs) {
+  if (n_seqs != c->last_verify_n) return false;
+  for (int b = 0; b < n_seqs; ++b) if (seqs[b] != c->last_verify_seq[b]) return false;
+  return true;
+}
 
 template <typename T>
 // `logits` null: greedy acceptance on `argmax`; otherwise the sampling form on `logits` at
@@ -938,8 +1068,8 @@ static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const 
   const dream_config &f = c->cfg;
   int D = c->ts.D, d = f.d_model, R = B * (D + 1);
   RowMeta &rm = c->rm[0];
-  if (logits && f.vocab <= 32 * 32 * SAMPLE_CACHE) LAUNCH(c, k_accept_sample<true>, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src);
-  else if (logits) LAUNCH(c, k_accept_sample<false>, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src);
+  if (logits && f.vocab <= 32 * 32 * SAMPLE_CACHE) LAUNCH(c, k_accept_sample<true>, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src, c->status);
+  else if (logits) LAUNCH(c, k_accept_sample<false>, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src, c->status);
   else LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
   LAUNCH(c, (k_compact_kv<T>), dim3(f.n_layers * 2, B), 256, 0, tb, c->sd, c->kv_pool, c->layer_stride, c->kv_stride, paged(c, 0));
   LAUNCH(c, k_accept_rows, 1, 32, 0, tb, B, c->T, D, c->sd, c->gather_idx, rm, c->cap_rows - c->ts.NI, c->status);
@@ -959,12 +1089,14 @@ extern "C" dream_status dream_accept(dream_ctx *c, const int32_t *seqs, int32_t 
   if (!node_argmax || !accept_len || !out_tokens) return fail(c, DREAM_E_ARG, "node_argmax, accept_len, out_tokens are required");
   for (int b = 0; b < n_seqs; ++b)
     if (c->phase[seqs[b]] != PH_VERIFIED) return fail(c, DREAM_E_STATE, "sequence %d: dream_accept follows dream_verify_tree", seqs[b]);
+  if (!same_list_as_verify(c, seqs, n_seqs)) return fail(c, DREAM_E_STATE, "dream_accept takes the sequence list of the last dream_verify_tree, in the same order");
   s = c->cfg.dtype == DREAM_BF16 ? accept_impl<bf16>(c, tb, n_seqs, node_argmax, accept_len, out_tokens, comp_src)
                                  : accept_impl<float>(c, tb, n_seqs, node_argmax, accept_len, out_tokens, comp_src);
   if (s) return s;
-  CUDA_OK(c, cudaGetLastError());
-  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
-  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; c->key_ub[seqs[b]] += c->ts.D + 1; }
+  s = call_done(c);
+  if (s) return s;
+  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; c->accepts[seqs[b]]++; }
+  snapshot_lengths(c);
   return DREAM_OK;
 }
 
@@ -978,12 +1110,14 @@ extern "C" dream_status dream_accept_sample(dream_ctx *c, const int32_t *seqs, i
   if (!(temperature > 0.f)) return fail(c, DREAM_E_ARG, "temperature must be above zero (dream_accept is the greedy form)");
   for (int b = 0; b < n_seqs; ++b)
     if (c->phase[seqs[b]] != PH_VERIFIED) return fail(c, DREAM_E_STATE, "sequence %d: dream_accept_sample follows dream_verify_tree", seqs[b]);
+  if (!same_list_as_verify(c, seqs, n_seqs)) return fail(c, DREAM_E_STATE, "dream_accept_sample takes the sequence list of the last dream_verify_tree, in the same order");
   s = c->cfg.dtype == DREAM_BF16 ? accept_impl<bf16>(c, tb, n_seqs, nullptr, accept_len, out_tokens, comp_src, logits, temperature, uniforms)
                                  : accept_impl<float>(c, tb, n_seqs, nullptr, accept_len, out_tokens, comp_src, logits, temperature, uniforms);
   if (s) return s;
-  CUDA_OK(c, cudaGetLastError());
-  if (c->gemm_failed) return fail(c, DREAM_E_CUDA, "a GEMM launch was refused");
-  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; c->key_ub[seqs[b]] += c->ts.D + 1; }
+  s = call_done(c);
+  if (s) return s;
+  for (int b = 0; b < n_seqs; ++b) { c->phase[seqs[b]] = PH_READY; c->p_ub[seqs[b]] += c->ts.D + 1; c->accepts[seqs[b]]++; }
+  snapshot_lengths(c);
   return DREAM_OK;
 }
 
@@ -1003,6 +1137,7 @@ extern "C" dream_status dream_step_host(dream_ctx *c, const int32_t *seqs, int32
   CUDA_OK(c, cudaMemcpyAsync(stage, c->accept_len_i, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(c, cudaMemcpyAsync(stage + DREAM_MAX_BATCH, c->out_tokens_i, sizeof(int) * n_seqs * D1, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  refresh_bounds(c);                     // the snapshot of this round's accept has landed: the bounds are exact
   memcpy(accept_len_host, stage, sizeof(int) * n_seqs);
   memcpy(out_tokens_host, stage + DREAM_MAX_BATCH, sizeof(int) * n_seqs * D1);
   return DREAM_OK;
@@ -1014,7 +1149,10 @@ extern "C" dream_status dream_seq_state(dream_ctx *c, int32_t seq, int32_t *veri
   dream_status s = check_seq(c, seq);
   if (s) return s;
   CUDA_OK(c, cudaStreamSynchronize(c->stream));
-  if (verified_len) CUDA_OK(c, cudaMemcpy(verified_len, c->sd.P + seq, sizeof(int), cudaMemcpyDeviceToHost));
+  int P_now = 0;
+  CUDA_OK(c, cudaMemcpy(&P_now, c->sd.P + seq, sizeof(int), cudaMemcpyDeviceToHost));
+  if (c->phase[seq] >= PH_READY && P_now < c->p_ub[seq]) c->p_ub[seq] = P_now;   // the stream is idle: P is exact
+  if (verified_len) *verified_len = P_now;
   if (pending) CUDA_OK(c, cudaMemcpy(pending, c->sd.pending + seq, sizeof(int), cudaMemcpyDeviceToHost));
   if (tap) CUDA_OK(c, cudaMemcpy(tap, c->sd.tap + seq, sizeof(int), cudaMemcpyDeviceToHost));
   return DREAM_OK;
@@ -1032,23 +1170,21 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
     if (c->seq_pages[seq].empty()) return fail(c, DREAM_E_STATE, "sequence has no pages");
     int pg = c->seq_pages[seq][index / f.page_tokens], in = index % f.page_tokens;
     const T *base = (const T *)c->kv_pool + (size_t)layer * c->layer_stride + (size_t)what * c->kv_stride;
-    for (int h = 0; h < f.n_kv_heads; ++h) {
-      const T *src = base + (((size_t)pg * f.n_kv_heads + h) * f.page_tokens + in) * f.head_dim;
-      k_read_row<T><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
-    }
+    const T *src = base + (((size_t)pg * f.n_kv_heads) * f.page_tokens + in) * f.head_dim;
+    k_read_row<T><<<f.n_kv_heads, 256, 0, c->stream>>>(src, (long long)f.page_tokens * f.head_dim, tmp, f.head_dim, 0);
   } else if (what >= 2 && what <= 5) {
     if (index < 0 || index >= c->cap_rows) return fail(c, DREAM_E_ARG, "row out of range");
     const float *base = what <= 3 ? c->dmem : c->dself;
     int kvsel = (what - 2) & 1;
-    for (int h = 0; h < f.n_kv_heads; ++h) {
-      const float *src = base + ((((size_t)seq * 2 + kvsel) * f.n_kv_heads + h) * c->cap_rows + index) * f.head_dim;
-      if (sizeof(T) == 2) k_read_row_split<<<1, 256, 0, c->stream>>>((const bf16 *)src, tmp + h * f.head_dim, f.head_dim);
-      else k_read_row<float><<<1, 256, 0, c->stream>>>(src, tmp + h * f.head_dim, f.head_dim);
-    }
+    // a row holds head_dim floats, or head_dim high then head_dim low bf16 parts: 4 bytes per element either way
+    const float *src = base + (((size_t)seq * 2 + kvsel) * f.n_kv_heads * c->cap_rows + index) * f.head_dim;
+    const long long hs = (long long)c->cap_rows * f.head_dim;
+    if (sizeof(T) == 2) k_read_row<bf16><<<f.n_kv_heads, 256, 0, c->stream>>>((const bf16 *)src, 2 * hs, tmp, f.head_dim, 1);
+    else k_read_row<float><<<f.n_kv_heads, 256, 0, c->stream>>>(src, hs, tmp, f.head_dim, 0);
   } else if (what == 6 || what == 7) {
     if (index < 0 || index >= ROW_CHUNK) return fail(c, DREAM_E_ARG, "row out of range");
     const float *src = (what == 6 ? c->tapbuf : c->x) + (size_t)index * d;
-    k_read_row<float><<<(d + 255) / 256, 256, 0, c->stream>>>(src, tmp, d);
+    k_read_row<float><<<1, 256, 0, c->stream>>>(src, 0LL, tmp, d, 0);
   } else return fail(c, DREAM_E_ARG, "unknown buffer id %d", what);
   CUDA_OK(c, cudaMemcpyAsync(dst, tmp, sizeof(float) * count, cudaMemcpyDeviceToHost, c->stream));
   CUDA_OK(c, cudaStreamSynchronize(c->stream));

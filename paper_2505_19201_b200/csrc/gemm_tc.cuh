@@ -413,10 +413,11 @@ static inline bool gemm_tc_supported(int N, int K) {
 
 // bf16 row-major [rows][K] matrix, box = 64 x box_rows, 128-byte swizzle.  Rows of a box that lie
 // beyond `rows` read as zero.
-static inline const CUtensorMap *tc_map(GemmTcPlan *pl, const void *ptr, int rows, int K, int box_rows) {
+// The encoded map is copied to *out: the cache may drop its entries at any later call.
+static inline bool tc_map(GemmTcPlan *pl, const void *ptr, int rows, int K, int box_rows, CUtensorMap *out) {
   auto key = std::make_tuple(ptr, rows, K, box_rows);
   auto it = pl->maps.find(key);
-  if (it != pl->maps.end()) return &it->second;
+  if (it != pl->maps.end()) { *out = it->second; return true; }
   CUtensorMap m;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)K * 2};
@@ -425,9 +426,11 @@ static inline const CUtensorMap *tc_map(GemmTcPlan *pl, const void *ptr, int row
   CUresult r = pl->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return nullptr;
+  if (r != CUDA_SUCCESS) return false;
   if (pl->maps.size() > 8192) pl->maps.clear();
-  return &(pl->maps[key] = m);
+  pl->maps[key] = m;
+  *out = m;
+  return true;
 }
 
 // Floats one launch may write when its slots hold slot_rows x N: a tile is shared by at most
@@ -474,9 +477,8 @@ static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const voi
   long long max_slots = (p.KB + p.upc - 1) / p.upc + 1;
   if (p.slot_stride * max_slots > out_floats) return false;
   int x_rows = x_mode == TC_X_INTERLEAVED ? 2 * rows : (x_mode == TC_X_PLANAR ? lo_rows + rows : rows);
-  const CUtensorMap *mw = tc_map(pl, W, N, K, TC_BN);
-  const CUtensorMap *mx = tc_map(pl, X, x_rows, K, 128);
-  if (!mw || !mx) return false;
+  CUtensorMap mw, mx;
+  if (!tc_map(pl, W, N, K, TC_BN, &mw) || !tc_map(pl, X, x_rows, K, 128, &mx)) return false;
   g->base = p.out; g->slot_stride = p.slot_stride; g->chunk_stride = 0; g->chunk_shift = 30; g->ld = N; g->kb = p.KB; g->upc = p.upc;
   int xstage = p.wp * (x_mode == TC_X_PLANAR ? 2 * TC_XTILE * p.m_tiles : TC_XTILE);
   p.x_stages = 2;
@@ -493,5 +495,5 @@ static inline bool gemm_tc_launch(GemmTcPlan *pl, cudaStream_t stream, const voi
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = pl->use_pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, k_gemm_tc, *mw, *mx, p) == cudaSuccess;
+  return cudaLaunchKernelEx(&cfg, k_gemm_tc, mw, mx, p) == cudaSuccess;
 }

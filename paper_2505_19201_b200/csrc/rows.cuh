@@ -170,6 +170,7 @@ __global__ void k_qkv_post_target(GemmOut g, const int *__restrict__ row_seq,
   if (w >= (H + 2 * Hkv) * q4) return;
   int hh = w / q4, i = (w - hh * q4) * 4;
   int seq = row_seq[r], pos = row_pos[r], slot = row_slot[r];
+  if (hh >= H && slot < 0) return;                 // an idle row (malformed tree node) stores no K/V
   T *Kp = (T *)kv.base, *Vp = (T *)kv.base + kv.kv_stride;
   float4 cs01 = make_float4(1.f, 0.f, 1.f, 0.f), cs23 = cs01;
   if (hh < H + Hkv) rope_cs4(rope_tab, r, half, pos, inv_freq, i, cs01, cs23);      // fetched along with the slots

@@ -214,8 +214,9 @@ __global__ void k_verify_setup(TreeBatch tb, int B, int T, SeqDev s, RowMeta rm,
   bool bad = (i == 0 ? par != -1 || dep != 0 : par < 0 || par >= i || dep != tp.depth[par < 0 ? 0 : par] + 1);
   if (P + T > max_seq) bad = true;
   if (bad) atomicMax(status, DREAM_DEV_BAD_INDEX);
+  // a malformed node keeps its row (so the launch shapes hold) but writes no K/V: slot -1
   rm.seq[r] = seq; rm.tok[r] = tp.tokens[i]; rm.pos[r] = P + (bad ? 0 : dep);
-  rm.slot[r] = bad ? 0 : P + i; rm.in[r] = i;
+  rm.slot[r] = bad ? -1 : P + i; rm.in[r] = i;
   for (int wd = 0; wd < 4; ++wd) mask[r * 4 + wd] = tp.mask[i * 4 + wd];
 }
 
@@ -262,7 +263,7 @@ __global__ void k_accept(TreeBatch tb, int B, int T, int D, SeqDev s, const int 
 template <bool CACHED>
 __global__ void __launch_bounds__(1024)
 k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float *__restrict__ logits, float temp,
-                const float *__restrict__ uniforms, int *accept_len, int *out_tokens, int *comp_src) {
+                const float *__restrict__ uniforms, int *accept_len, int *out_tokens, int *comp_src, int *status) {
   kernel_entry(TR_k_accept);
   __shared__ float sh[33];
   __shared__ float wtot[32];
@@ -278,7 +279,9 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
   if (threadIdx.x == 0) path[0] = 0;
   int cur = 0, A = 0, emitted = -1;
   float ev[CACHED ? SAMPLE_CACHE : 1];
-  while (emitted < 0) {
+  // at most D + 1 nodes are visited: every pass either walks into a child (A grows, and at A == D
+  // no child is looked for) or ends with the final draw, which always emits a token
+  for (int visit = 0; visit <= D && emitted < 0; ++visit) {
     const float *row = logits + ((long long)b * T + cur) * V;
     const float *u = uniforms + ((long long)b * (D + 1) + A) * T;
     // the row's maximum (of the scaled logits)
@@ -334,8 +337,9 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
         for (int i = 0; i < 32; ++i) Z += wtot[i];
         int k = 0x7fffffff;
         for (int i = 0; i < 32; ++i) k = min(k, __float_as_int(sh[i]));
-        int decision = 0;                                   // 0 = final draw, 1 = kept, 2 = refused
-        if (k != 0x7fffffff && n_ref < SAMPLE_MAX_REFUSED) {
+        int decision = 0;                                   // 0 = final draw, 1 = kept, 2 = refused, 3 = no mass
+        if (!(Z > 0.f) || Z > 3.0e38f) decision = 3;         // a row of NaN or infinities, or every massive token refused
+        else if (k != 0x7fffffff && n_ref < SAMPLE_MAX_REFUSED) {
           int tok = tp.tokens[k];
           float e = (tok >= 0 && tok < V) ? __expf(row[tok] * inv_t - m) : 0.f;
           for (int i = 0; i < n_ref; ++i) if (refused[i] == tok) e = 0.f;
@@ -346,7 +350,7 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
       }
       __syncthreads();
       const int decision = sh_i[0];
-      if (decision == 0) break;
+      if (decision == 0 || decision == 3) break;
       last_kid = sh_i[1];
       ++tried;
       if (decision == 1) { taken = last_kid; break; }
@@ -363,6 +367,11 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
       cur = taken; ++A;
       if (threadIdx.x == 0) { path[A] = cur; out_tokens[b * (D + 1) + A - 1] = tp.tokens[cur]; }
       continue;
+    }
+    if (sh_i[0] == 3) {                                     // nothing to draw from: token 0, and the status word says so
+      if (threadIdx.x == 0) atomicMax(status, DREAM_DEV_BAD_INDEX);
+      emitted = 0;
+      break;
     }
     // final draw: the first token, in token order, at which the running mass exceeds u * Z
     const float target = u[T - 1] * sh_f[0];
@@ -411,7 +420,12 @@ k_accept_sample(TreeBatch tb, int B, int T, int D, int V, SeqDev s, const float 
     }
     __syncthreads();
     emitted = sh_i[3];
+    if (emitted < 0) {                                      // no token with mass was met (cannot happen with Z > 0)
+      if (threadIdx.x == 0) atomicMax(status, DREAM_DEV_BAD_INDEX);
+      emitted = 0;
+    }
   }
+  if (emitted < 0) emitted = 0;
   if (threadIdx.x == 0) accept_commit(tp, b, seq, D, s, path, A, emitted, accept_len, out_tokens, comp_src);
 }
 

@@ -25,18 +25,27 @@ class Tol:
         self.score_rel = 5e-3 if bf else 1e-5
 
 
-def close(a, b, tol, what, report):
-    """max_abs is stated for values of unit scale (logits, normalised states).  The residual
-    stream of a deep randomly initialised model grows with depth, so for a tensor whose oracle
-    root-mean-square exceeds 1 the bound scales with it: the error of an element is relative
-    (one differently rounded bf16 K/V entry moves an attention output by 2^-9 of its size, and
-    such shifts add up like a random walk over the layers)."""
+# Tensors that are NOT of unit scale: rows of the unnormalised residual stream (final hidden state,
+# tapped features S^{l*}) and what Eq. 1 derives from them without a norm (the cross-attention
+# memory).  In a deep randomly initialised model their root-mean-square grows with depth (about 5
+# after 32 layers, 13 for the projected memory rows), so their max-abs bound is relative to it;
+# every other tensor (logits, log-probabilities, K/V rows of normalised inputs) takes the flat bound.
+RESIDUAL_SCALE = ("final hidden", "tapped features", "memory K row", "memory V row")
+
+
+def close(a, b, tol, what, report, stated_miss=None):
+    """max-abs (flat, or times the oracle tensor's root-mean-square for RESIDUAL_SCALE tensors) and
+    relative L2.  `stated_miss` maps a tensor name to the wider bound of a documented miss of the
+    flat tolerance; the raw numbers of every comparison go to report["float"]."""
     a, b = a.double().flatten(), b.double().flatten()
     ma = float((a - b).abs().max()) if a.numel() else 0.0
     rl = float((a - b).norm() / (b.norm() + 1e-30))
     rms = float(b.norm() / max(b.numel(), 1) ** 0.5)
-    bound = tol.max_abs * max(1.0, rms)
-    report.setdefault("float", []).append((what, ma, rl))
+    bound = tol.max_abs * max(1.0, rms) if what in RESIDUAL_SCALE else tol.max_abs
+    report.setdefault("float", []).append((what, ma, rl, rms))
+    if ma > bound and stated_miss and what in stated_miss:
+        report.setdefault("misses", []).append((what, ma, bound))
+        bound = stated_miss[what]
     assert ma <= bound, f"{what}: max-abs {ma:.3e} > {bound:.3e} (oracle rms {rms:.3e}, rel-L2 {rl:.3e})"
     assert rl <= tol.rel_l2, f"{what}: rel-L2 {rl:.3e} > {tol.rel_l2} (max-abs {ma:.3e})"
 
@@ -49,7 +58,7 @@ def close_stored(a, b, tol, what, report, bf16_store, where=""):
     a, b = a.double().flatten(), b.double().flatten()
     gap = (a - b).abs()
     rl = float(gap.norm() / (b.norm() + 1e-30))
-    report.setdefault("float", []).append((what, float(gap.max()), rl))
+    report.setdefault("float", []).append((what, float(gap.max()), rl, float(b.norm() / max(b.numel(), 1) ** 0.5)))
     bad = gap > b.abs() * 2.0 ** -7 + tol.max_abs
     if bool(bad.any()):
         i = int(torch.argmax(gap - b.abs() * 2.0 ** -7))
@@ -72,7 +81,12 @@ def valid_tree(t, T):
 class Pair:
     """One model on both sides: the oracle on the CPU and a library context on the GPU."""
 
-    def __init__(self, preset, oracle_dtype=None, device="cuda:0", seed=0, max_batch=None, **over):
+    def __init__(self, preset, oracle_dtype=None, device="cuda:0", seed=0, max_batch=None, oracle_kv="bf16",
+                 stated_miss=None, **over):
+        """oracle_kv: "bf16" = the oracle keeps its target K/V cache as a bf16 store like the GPU
+        (the reading of Section 4's "KV caching enabled" for bf16 models); "plain" = the oracle keeps
+        K/V in its arithmetic type, which shows how much that reading absorbs.
+        stated_miss: {tensor name: bound} for documented misses of the flat max-abs tolerance."""
         self.p = p = configs.scaled(preset, **over) if isinstance(preset, str) else dict(preset, **over)
         self.tol = Tol(p["dtype"])
         self.device = device
@@ -82,8 +96,9 @@ class Pair:
         cpu = lambda w: [t.cpu() for t in w] if isinstance(w, list) else w.cpu()
         self.orc = DreamOracle(OracleConfig.from_preset(p), {k: cpu(v) for k, v in self.twg.items()},
                                {k: cpu(v) for k, v in self.dwg.items()}, odt,
-                               kv_dtype=torch.bfloat16 if p["dtype"] == "bf16" else None)
+                               kv_dtype=torch.bfloat16 if p["dtype"] == "bf16" and oracle_kv == "bf16" else None)
         self.odt = odt
+        self.stated_miss = stated_miss or {}
         self.cfg = api.make_config(p, max_batch=max_batch)
         self.ctx = api.Context(self.cfg, self.twg, self.dwg, device)
         self.T = self.ctx.T
@@ -102,8 +117,14 @@ class Pair:
         return False
 
     # ------------------------------------------------------------------ prefill + compression
-    def prefill(self, seq=0, seq_seed=0, vis_start=0, k=None):
-        p, dev, tol = self.p, self.device, self.tol
+    def prefill(self, seq=0, seq_seed=0, vis_start=0, k=None, n_visual=None, n_prompt=None):
+        """n_visual / n_prompt shorten this sequence's prompt below the preset's (the context's capacity)."""
+        dev, tol = self.device, self.tol
+        p = dict(self.p)
+        if n_visual is not None:
+            p["n_visual"] = n_visual
+        if n_prompt is not None:
+            p["n_prompt"] = n_prompt
         vis, ids = synth.request_inputs(p, seq_seed, dev)
         tok = torch.zeros(1, dtype=torch.int32, device=dev)
         mg = torch.zeros(1, dtype=torch.float32, device=dev)
@@ -130,8 +151,10 @@ class Pair:
         self.report["score_gap_rel"] = rel
         assert rel <= tol.score_rel, f"importance: per-element relative gap {rel:.3e} > {tol.score_rel}"
         gk = kept.cpu().tolist()[:k]
-        cut = float(torch.sort(o64, descending=True).values[k - 1]) if 0 < k < p["n_visual"] else 1.0
-        exempt_below = 2 * tol.score_rel * max(cut, 1e-3 * scale)
+        # two scores may swap places only when they are closer than the two sides' measured
+        # disagreement allows: twice the largest per-element gap of this very comparison
+        exempt_below = 2.0 * float((g64 - o64).abs().max()) + 1e-30 if osc.numel() else 1.0
+        self.report["score_window_rel"] = exempt_below / max(scale, 1e-30)
         if not self._decide(gk == okept.tolist(), omargin * (tol.dec / exempt_below), "kept visual tokens"):
             assert gk == sorted(set(gk)) and all(0 <= j < p["n_visual"] for j in gk)
             self.orc.compress_visual(st, k, forced_idx=gk)
@@ -158,19 +181,24 @@ class Pair:
             valid_tree(gd, T)
             same = all(gd[k] == od[k] for k in ("tokens", "parent", "depth", "mask"))
             self._decide(same, od["min_margin"], "draft tree")
-            # a cumulative score is a sum of `depth` log-probabilities, each held to max_abs where the
-            # draft's cross-attention memory is of unit scale.  The memory holds unnormalised residual
-            # rows of the tapped layer (Eq. 1 has no norm on the key/value side), whose size grows with
-            # that layer's depth; the scores q.k / sqrt(hd) and with them the sensitivity of the draft's
-            # output to a relative difference of the memory rows grow in proportion, so the bound
-            # scales with the memory's root-mean-square like the bound of any tensor above unit scale.
+            # a cumulative score is a sum of `depth` log-probabilities, each held to the flat max_abs.
+            # Where the tapped layer is deep the memory holds large unnormalised rows (Eq. 1 has no norm
+            # on the key/value side), the softmax over it is sharply peaked and the draft's output is
+            # sensitive to the memory's relative error: a full-size case that exceeds the flat bound says
+            # so through `stated_miss` instead of scaling the bound.
             mem_rms = float(st.mK.double().norm() / max(st.mK.numel(), 1) ** 0.5)
-            lp_bound = tol.max_abs * max(1.0, mem_rms)
             self.report["memory_rms"] = mem_rms
+            lp_what = "draft logp (per level)"
+
+            def lp_check(gap):
+                self.report.setdefault("float", []).append((lp_what, gap, gap, 1.0))
+                bound = tol.max_abs
+                if gap > bound and lp_what in self.stated_miss:
+                    self.report.setdefault("misses", []).append((lp_what, gap, bound))
+                    bound = self.stated_miss[lp_what]
+                assert gap <= bound, f"draft cum_logp: {gap:.3e} per level > {bound:.3e} (memory rms {mem_rms:.2f})"
             if same:
-                gap = max(abs(g - o) / max(dd, 1) for g, o, dd in zip(gd["cum"], od["cum"], od["depth"]))
-                self.report.setdefault("float", []).append(("draft logp (per level)", gap, gap))
-                assert gap <= lp_bound, f"draft cum_logp: {gap:.3e} per level > {lp_bound:.3e}"
+                lp_check(max(abs(g - o) / max(dd, 1) for g, o, dd in zip(gd["cum"], od["cum"], od["depth"])))
                 g64, o64 = torch.tensor(gd["cum"], dtype=torch.float64), torch.tensor(od["cum"], dtype=torch.float64)
                 rl = float((g64 - o64).norm() / (o64.norm() + 1e-30))
                 assert rl <= tol.rel_l2, f"draft cum_logp: rel-L2 {rl:.3e} > {tol.rel_l2}"
@@ -179,9 +207,7 @@ class Pair:
                 om = {key(od, i): od["cum"][i] for i in range(len(od["tokens"]))}
                 common = [(gd["cum"][i], om[key(gd, i)], gd["depth"][i]) for i in range(T) if key(gd, i) in om]
                 self.report.setdefault("tree_overlap", []).append(len(common) / T)
-                gap = max(abs(g - o) / max(dd, 1) for g, o, dd in common)
-                self.report.setdefault("float", []).append(("draft logp (per level)", gap, gap))
-                assert gap <= lp_bound, f"draft cum_logp (common nodes): {gap:.3e} per level > {lp_bound:.3e}"
+                lp_check(max(abs(g - o) / max(dd, 1) for g, o, dd in common))
                 g64, o64 = torch.tensor([c[0] for c in common], dtype=torch.float64), torch.tensor([c[1] for c in common], dtype=torch.float64)
                 rl = float((g64 - o64).norm() / (o64.norm() + 1e-30))
                 assert rl <= tol.rel_l2, f"draft cum_logp (common nodes): rel-L2 {rl:.3e} > {tol.rel_l2}"
@@ -201,7 +227,7 @@ class Pair:
         outt = torch.zeros(B * (D + 1), dtype=torch.int32, device=dev)
         csrc = torch.zeros(B * (D + 1), dtype=torch.int32, device=dev)
         ctx.dream_poll()
-        gam, glg = am.cpu().tolist(), lg.cpu()
+        gam, glg, gmg = am.cpu().tolist(), lg.cpu(), mg.cpu().tolist()
         hid = {(b, i): ctx.dream_debug_read(seqs[b], 7, 0, b * T + i) for b in range(B) for i in (0, T - 1)}
         tapr = {(b, i): ctx.dream_debug_read(seqs[b], 6, 0, b * T + i) for b in range(B) for i in (0, T - 1)}
         vers = [orc.verify_tree(self.st[s], use[b]) for b, s in enumerate(seqs)]
@@ -216,11 +242,15 @@ class Pair:
         for b, s in enumerate(seqs):
             st, tree = self.st[s], use[b]
             ver = vers[b]
-            close(glg[b * T:(b + 1) * T], ver["logits"], tol, "verify logits", self.report)
+            close(glg[b * T:(b + 1) * T], ver["logits"], tol, "verify logits", self.report, self.stated_miss)
             for i in (0, T - 1):
                 close(hid[(b, i)], ver["hidden"][i], tol, "final hidden", self.report)
                 close(tapr[(b, i)], ver["tap_rows"][i], tol, "tapped features", self.report)
             for i in range(T):
+                # top-1 minus top-2 logit: a difference of two logits, each within max_abs
+                mgap = abs(gmg[b * T + i] - ver["margin"][i])
+                assert mgap <= 2 * tol.max_abs, f"margin of node {i}: {gmg[b * T + i]} vs {ver['margin'][i]}"
+                self.report["margin_gap"] = max(self.report.get("margin_gap", 0.0), mgap)
                 if not self._decide(gam[b * T + i] == ver["argmax"][i], ver["margin"][i], f"argmax of node {i}"):
                     ver["argmax"][i] = gam[b * T + i]
             if temp > 0:
@@ -243,7 +273,7 @@ class Pair:
             assert (gP, gpend) == (st.P, st.pending), "sequence state"
             # cache rows after compaction: the accepted path, a prefix row, the newest memory rows
             L = p["n_layers"]
-            for l in sorted({0, L - 1}):
+            for l in sorted({0, L // 2, L - 1}):
                 for pos in sorted({0, P0 - 1, P0, st.P - 1})[:2 + check_cache_rows]:
                     bf = p["dtype"] == "bf16"
                     close_stored(ctx.dream_debug_read(s, 0, l, pos), st.K[l][pos].flatten(), tol, "target K row", self.report, bf, f"(layer {l}, pos {pos}, P0 {P0}, A {A})")
@@ -274,11 +304,13 @@ class Pair:
     def summary(self):
         r = self.report
         worst = {}
-        for what, ma, rl in r.get("float", []):
-            w = worst.setdefault(what, [0.0, 0.0])
-            w[0], w[1] = max(w[0], ma), max(w[1], rl)
+        for what, ma, rl, rms in r.get("float", []):
+            w = worst.setdefault(what, [0.0, 0.0, 0.0])          # max-abs, rel-L2, oracle rms
+            w[0], w[1], w[2] = max(w[0], ma), max(w[1], rl), max(w[2], rms)
         return dict(decisions=r["decisions"], exempt=r["exempt"], worst=worst,
-                    tree_overlap=r.get("tree_overlap", []))
+                    misses_of_flat_max_abs=r.get("misses", []), margin_gap=r.get("margin_gap"),
+                    score_gap_rel=r.get("score_gap_rel"), score_window_rel=r.get("score_window_rel"),
+                    memory_rms=r.get("memory_rms"), tree_overlap=r.get("tree_overlap", []))
 
     def close(self):
         self.ctx.close()

@@ -8,9 +8,9 @@ import torch
 pytestmark = pytest.mark.gpu
 
 
-def _run(preset, steps, **over):
+def _run(preset, steps, stated_miss=None, **over):
     from tests.parity import Pair
-    pr = Pair(preset, **over)
+    pr = Pair(preset, stated_miss=stated_miss, **over)
     try:
         pr.prefill()
         accepted = []
