@@ -13,6 +13,7 @@
 #include "../../include/dream.h"
 #include "attn.cuh"
 #include "attn_mma.cuh"
+#include "attn_tc.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
@@ -87,6 +88,7 @@ struct dream_ctx {
   int *h_stage;                        // pinned: page-table staging + step_host results
   long long launches, tc_launches, simt_launches;
   GemmTcPlan tc;
+  AtMapCache at_maps;
   // per-launch timing of the weight-streaming GEMM (dream_gemm_timing)
   int prof_on, prof_n;
   double prof_bytes;
@@ -220,6 +222,8 @@ static dream_status check_config(const dream_config *c, TreeShape *ts) {
   if (c->vocab > TOPK_THREADS * TOPK_COLS) return fail(nullptr, DREAM_E_UNSUPPORTED, "vocab above 1048576");
   if (c->dtype == DREAM_BF16 && (c->d_model % 64 || c->d_ff % 64 || (c->n_heads * c->head_dim) % 64 || c->vocab % 8))
     return fail(nullptr, DREAM_E_UNSUPPORTED, "bf16: d_model, d_ff, n_heads*head_dim must be multiples of 64 and vocab of 8");
+  if (c->dtype == DREAM_BF16 && 64 % (c->n_heads / c->n_kv_heads))
+    return fail(nullptr, DREAM_E_UNSUPPORTED, "bf16: query heads per KV head must divide 64");
   if (c->max_batch < 1 || c->max_batch > DREAM_MAX_BATCH) return fail(nullptr, DREAM_E_ARG, "max_batch in 1..8");
   if (c->page_tokens < 16 || c->page_tokens > 256 || (c->page_tokens & (c->page_tokens - 1)))
     return fail(nullptr, DREAM_E_ARG, "page_tokens must be a power of two in 16..256");
@@ -501,6 +505,12 @@ static void refresh_bounds(dream_ctx *c) {
 // ------------------------------------------------------------------------------------- init / free
 
 template <int HD>
+static const char *attn_tc_setup_all() {
+  const char *w = attn_tc_setup<HD, false>();
+  return w ? w : attn_tc_setup<HD, true>();
+}
+
+template <int HD>
 static const char *attn_mma_setup() {
   if (cudaFuncSetAttribute(k_attn_mma<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_mma_smem<HD, true>()) != cudaSuccess ||
       cudaFuncSetAttribute(k_attn_mma<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_mma_smem<HD, false>()) != cudaSuccess)
@@ -575,6 +585,7 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   }
   if (c->use_tc) {
     const char *why = cfg->head_dim == 64 ? attn_mma_setup<64>() : cfg->head_dim == 128 ? attn_mma_setup<128>() : attn_mma_setup<256>();
+    if (!why) why = cfg->head_dim == 64 ? attn_tc_setup_all<64>() : cfg->head_dim == 128 ? attn_tc_setup_all<128>() : attn_tc_setup_all<256>();
     if (why) { free_host_side(c); return fail(nullptr, DREAM_E_CUDA, "%s", why); }
   }
   k_rope_table<<<(cfg->head_dim / 2 + 127) / 128, 128, 0, c->stream>>>(c->rope_inv, cfg->head_dim, cfg->rope_theta);
@@ -710,13 +721,68 @@ template <typename T, int HD> struct AttnLaunch {
       LAUNCH(c, (k_attn_combine<HD>), (unsigned)((items + 255) / 256), 256, 0, a, B * rows_per_seq);
     }
   }
+  // The tcgen05 attention (bf16 configurations): split-K plan, tensor maps, launch, merge of the chunks.
+  // cache: null = the paged target cache of `layer`, else a flat draft cache.
+  static void tc(dream_ctx *c, AttnTcArgs a, int layer, const float *cache, int B, int rows_per_seq, int key_ub, const int *row_in) {
+    const dream_config &f = c->cfg;
+    const bool flat_kv = cache != nullptr;
+    const int GROUP = flat_kv ? AtShape<HD, true>::GROUP : AtShape<HD, false>::GROUP;
+    for (int b = 0; b < DREAM_MAX_BATCH; ++b) a.slot_seq[b] = b < B ? c->cur_seq[b] : 0;
+    a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq; a.row_in = row_in;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+    a.n_rt = (rows_per_seq * a.G + 63) / 64;
+    const int nb_ub = imax(1, (key_ub + AT_KBLK - 1) / AT_KBLK), ng = (nb_ub + GROUP - 1) / GROUP;
+    const int tiles = f.n_kv_heads * a.n_rt * B;
+    // one CTA per SM: as many key chunks (of whole groups) as keep the grid in one wave
+    const int want = imin(imin(AM_MAX_CHUNKS, ng), imax(1, c->tc.n_sms / tiles));
+    a.blocks_per_chunk = (ng + want - 1) / want * GROUP;
+    a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
+    a.part_o = c->am_part_o; a.part_ml = c->am_part_ml; a.out = c->attn_out; a.status = c->status;
+    a.hkv = f.n_kv_heads;
+    CUtensorMap mq, mk, mv;
+    bool ok;
+    {
+      const unsigned long long dims[4] = {(unsigned long long)HD, 2ull, (unsigned long long)f.n_heads, (unsigned long long)c->XR};
+      const unsigned long long st[3] = {(unsigned long long)HD * 2, (unsigned long long)HD * 4, (unsigned long long)f.n_heads * HD * 4};
+      const unsigned box[4] = {64u, 2u, (unsigned)a.G, (unsigned)(64 / a.G)};
+      ok = at_map(&c->tc, &c->at_maps, c->qbuf, 4, dims, st, box, &mq);
+    }
+    if (flat_kv) {
+      const unsigned long long dims[3] = {(unsigned long long)HD, 2ull, (unsigned long long)f.max_batch * 2 * f.n_kv_heads * c->cap_rows};
+      const unsigned long long st[2] = {(unsigned long long)HD * 2, (unsigned long long)HD * 4};
+      const unsigned box[3] = {64u, 1u, 64u};
+      ok = ok && at_map(&c->tc, &c->at_maps, cache, 3, dims, st, box, &mk);
+      mv = mk;
+      a.flat_rows_per_head = c->cap_rows;
+    } else {
+      const PagedKV kv = paged(c, layer);
+      const unsigned long long dims[2] = {(unsigned long long)HD, (unsigned long long)c->n_pages * f.n_kv_heads * f.page_tokens};
+      const unsigned long long st[1] = {(unsigned long long)HD * 2};
+      const unsigned box[2] = {64u, (unsigned)imin(64, f.page_tokens)};
+      ok = ok && at_map(&c->tc, &c->at_maps, kv.base, 2, dims, st, box, &mk);
+      ok = ok && at_map(&c->tc, &c->at_maps, (const bf16 *)kv.base + kv.kv_stride, 2, dims, st, box, &mv);
+      a.page_table = kv.page_table; a.pages_per_seq = kv.pages_per_seq; a.page_tokens = kv.page_tokens; a.page_shift = kv.page_shift;
+    }
+    if (!ok) { c->gemm_failed = 1; return; }
+    cudaError_t e = flat_kv ? attn_tc_launch<HD, true>(c->stream, c->use_pdl, mq, mk, mv, a, B)
+                            : attn_tc_launch<HD, false>(c->stream, c->use_pdl, mq, mk, mv, a, B);
+    if (e != cudaSuccess && c->launch_err == cudaSuccess) { c->launch_err = e; c->launch_err_name = "k_attn_tc"; }
+    c->launches++;
+    if (a.n_chunks > 1) {
+      AttnMmaArgs m = {};
+      m.row_in = row_in; m.rows_per_seq = rows_per_seq; m.H = a.H; m.G = a.G; m.n_chunks = a.n_chunks; m.n_rt = a.n_rt;
+      m.part_o = a.part_o; m.part_ml = a.part_ml; m.out = a.out; m.lay = a.lay;
+      long long items = (long long)B * rows_per_seq * f.n_heads * (HD / 4);
+      LAUNCH(c, (k_attn_combine<HD>), (unsigned)((items + 255) / 256), 256, 0, m, B * rows_per_seq);
+    }
+  }
   static void tree(dream_ctx *c, int layer, int R, XMode m, int B, int key_ub) {
     if (sizeof(T) == 2) {
-      AttnMmaArgs a = {};
+      AttnTcArgs a = {};
+      a.mode = AT_VERIFY;
       a.next_w.ptr = (const char *)c->wo[layer]; a.next_w.bytes = (unsigned long long)c->cfg.d_model * c->Hhd * 2;
-      a.row_in = nullptr; a.prefix_len = c->sd.P; a.mask = c->vmask; a.anc = nullptr;
-      a.tail_len = c->T; a.lay = xlay(m, c->Hhd); a.paged = paged(c, layer);
-      mma<true>(c, a, B, c->T, key_ub);
+      a.prefix_len = c->sd.P; a.mask = c->vmask; a.tail_len = c->T; a.lay = xlay(m, c->Hhd);
+      tc(c, a, layer, nullptr, B, c->T, key_ub, nullptr);
       return;
     }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
@@ -726,11 +792,11 @@ template <typename T, int HD> struct AttnLaunch {
   static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, XMode m, int B,
                     int rows_per_seq, int key_ub) {
     if (sizeof(T) == 2) {
-      AttnMmaArgs a = {};
-      a.row_in = rm.in; a.prefix_len = nperm; a.mask = nullptr; a.anc = c->dt.in_anc;
-      a.anc_stride = c->ts.NI; a.strict = strict; a.tail_len = c->ts.NI; a.lay = xlay(m, c->Hhd);
-      a.flat.base = (bf16 *)cache; a.flat.cap = c->cap_rows; a.flat.hkv = c->cfg.n_kv_heads; a.flat.hd = HD;
-      mma<false>(c, a, B, rows_per_seq, key_ub);
+      AttnTcArgs a = {};
+      a.mode = AT_DRAFT;
+      a.prefix_len = nperm; a.anc = c->dt.in_anc; a.anc_stride = c->ts.NI; a.strict = strict; a.tail_len = c->ts.NI;
+      a.lay = xlay(m, c->Hhd);
+      tc(c, a, 0, cache, B, rows_per_seq, key_ub, rm.in);
       return;
     }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);

