@@ -175,6 +175,28 @@ def request_seed(seq, rank):
     return seq + 100 * rank
 
 
+def spawn_ranks(n):
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script on this node
+    (one per GPU, rendezvous on 127.0.0.1) and pass their output through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def setup_flops(p):
+    """Floating-point operations of one request's set-up (prefill): projections and MLP over the n
+    prompt rows of every layer, causal attention (QK^T and PV over n (n + 1) / 2 pairs), LM head on one row."""
+    d, H, Hkv, hd, ff, V, L = (p[k] for k in ("d_model", "n_heads", "n_kv_heads", "head_dim", "d_ff", "vocab", "n_layers"))
+    n = p["n_visual"] + p["n_prompt"]
+    layer_params = (H + 2 * Hkv) * hd * d + d * H * hd + 3 * d * ff
+    attn = 2 * 2 * H * hd * n * (n + 1) / 2
+    return L * (2 * layer_params * n + attn) + 2 * V * d
+
+
 def run_reference(args, p):
     """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -205,7 +227,8 @@ def run_reference(args, p):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=0,
+                    help="timed steps; 0 = the workload's decode length (256 for the LLaVA-7B-shaped one), at most 256")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--workload", default="llava7b")
@@ -223,7 +246,11 @@ def main():
                          "call then also writes the logits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        return spawn_ranks(args.gpus)
     p = dict(configs.PRESETS[args.workload])
+    if args.steps <= 0:
+        args.steps = min(256, int(p["decode_steps"]))
     if args.layers:
         p = configs.scaled(args.workload, n_layers=args.layers)
         p["name"] = "%s[n_layers=%d]" % (p["name"], args.layers)
@@ -251,7 +278,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
     B = p["batch"]
-    p["decode_steps"] = args.steps + args.warmup + 16 + 2 * args.steps   # room for every timed pass
+    p["decode_steps"] = args.steps + args.warmup + 16 + 2 * args.steps   # room for every timed pass (the end-to-end pass and the profiled pass follow)
     twg, dwg = synth.target_weights(p, 0, dev), synth.draft_weights(p, 0, dev)
     cfg = api.make_config(p)
     ctx = api.Context(cfg, twg, dwg, dev)
@@ -324,6 +351,9 @@ def main():
     draft_us = statistics.median(e[0].elapsed_time(e[1]) for e in evs) * 1e3
     verify_us = statistics.median(e[1].elapsed_time(e[2]) for e in evs) * 1e3
     accept_us = statistics.median(e[2].elapsed_time(e[3]) for e in evs) * 1e3
+    per_step_ms = [e[0].elapsed_time(e[3]) for e in evs]
+    k50 = min(50, len(per_step_ms))
+    first_ms, last_ms = statistics.median(per_step_ms[:k50]), statistics.median(per_step_ms[-k50:])
     ctx.dream_poll()
     # ---- end to end: the serving call with host result buffers, synchronising every step
     alen_h = torch.zeros(B, dtype=torch.int32).pin_memory()
@@ -366,9 +396,14 @@ def main():
                 config=dict(workload=p["name"], batch=B, tree_nodes=T, prefix=P0, parallelism=f"replicas{world}",
                             l2="step working set (weights, %.1f GB) exceeds the 126 MB L2" % (sb["gemm_weights"] / 1e9)),
                 draft_us=draft_us, verify_us=verify_us, accept_us=accept_us,
+                first_steps_ms=first_ms, last_steps_ms=last_ms,
                 setup_ms_per_sequence=statistics.median(setup_ms),
+                setup_tflops=setup_flops(p) / (statistics.median(setup_ms) / 1e3) / 1e12,
+                setup_frac_of_bf16_sustained=(setup_flops(p) / (statistics.median(setup_ms) / 1e3) / 1e12 / pk["bf16_tflops_sustained"]
+                                              if pk.get("bf16_tflops_sustained") else None),
                 step_bytes=sb["total"], step_gbs=step_gbs,
                 step_roofline_frac=step_gbs / pk["hbm_gbs"], step_roofline_frac_nominal_8tbs=step_gbs / 8000.0,
+                step_bytes_note="weights of every GEMM of the step + prefix KV of the verify + the draft's two caches (4 B per element)",
                 clocks=sampler.summary(), gpu_launches=int(launches),
                 e2e=dict(value=job_value(world, B, T, e2e_ms / args.steps), unit=UNIT,
                          h2d_bytes_per_step=4 * B, d2h_bytes_per_step=4 * B * (p["tree_depth"] + 2)))

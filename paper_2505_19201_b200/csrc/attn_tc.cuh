@@ -93,6 +93,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
         "r"(r[30]), "r"(r[31]) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // Makes this thread's shared-memory stores visible to the asynchronous proxy (the MMA reads P through it).
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -148,9 +155,11 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_p;
-  // every thread waits for the predecessor: the sequence state, the queries and the newest K/V rows are its outputs
-  pdl_wait();
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) trace_stamp(TR_k_attn_mma);
+  // Verification reads the verified prefix and its length, which were written rounds ago (hundreds
+  // of kernels back in the stream): its K/V blocks below the prefix length are fetched before the
+  // grid dependency resolves.  Everything else is an output of the immediate predecessors.
+  const bool early = a.mode == AT_VERIFY;
+  if (!early) pdl_wait();
 
   // ---- the chunk's blocks
   const int rows_total = a.rows_per_seq * a.G;              // entries of this sequence slot
@@ -168,75 +177,95 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const int b0 = chunk * a.blocks_per_chunk, b1 = min(nb, b0 + a.blocks_per_chunk);
   const int n_blk = max(0, b1 - b0);
 
+  // K and V of the chunk's block `it` into ring stage it % GROUP (producer thread only)
+  const uint64_t pol_kv = policy_evict_first();
+  auto issue_kv = [&](int it) {
+    const int st = it % GROUP, j0 = (b0 + it) * AT_KBLK;
+    // K: [plane][panel][stage][64 keys], so the blocks of a group form one operand of 64 x blocks keys
+    uint8_t *kd = k_s + st * AT_KVTILE, *vd = v_s + st * Sh::KV_STAGE;
+    constexpr int KSTEP = GROUP * AT_KVTILE;                 // bytes between consecutive (plane, panel) of K
+    mbar_expect_tx(k_full + st, (uint32_t)Sh::KV_STAGE);
+    mbar_expect_tx(v_full + st, (uint32_t)Sh::KV_STAGE);
+    if (FLAT) {
+      // rows of the map: (sequence, K | V, KV head, key); the second coordinate selects the plane
+      const long long rk = (((long long)seq * 2 + 0) * a.hkv + kvh) * a.flat_rows_per_head + j0;
+      const long long rv = (((long long)seq * 2 + 1) * a.hkv + kvh) * a.flat_rows_per_head + j0;
+      for (int pl = 0; pl < PLANES; ++pl)
+        for (int kp = 0; kp < KP; ++kp) {
+          tma_load_3d(kd + (pl * KP + kp) * KSTEP, &map_k, k_full + st, kp * 64, pl, (int)rk, pol_kv);
+          tma_load_3d(vd + (pl * KP + kp) * AT_KVTILE, &map_v, v_full + st, kp * 64, pl, (int)rv, pol_kv);
+        }
+    } else {
+      const int sub_rows = min(64, a.page_tokens), n_sub = 64 / sub_rows;
+      for (int sb = 0; sb < n_sub; ++sb) {
+        const int j = min(j0 + sb * sub_rows, a.pages_per_seq * a.page_tokens - 1);
+        const int pg = a.page_table[seq * a.pages_per_seq + (j >> a.page_shift)];
+        const int row = (pg * a.hkv + kvh) * a.page_tokens + (j & (a.page_tokens - 1));
+        for (int kp = 0; kp < KP; ++kp) {
+          tma_load_2d(kd + kp * KSTEP + sb * sub_rows * 128, &map_k, k_full + st, kp * 64, row, pol_kv);
+          tma_load_2d(vd + kp * AT_KVTILE + sb * sub_rows * 128, &map_v, v_full + st, kp * 64, row, pol_kv);
+        }
+      }
+    }
+  };
+  int n_pre = 0;                                            // blocks of the first group already under way
+  if (early) {
+    if (threadIdx.x == 0 && n_blk > 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+      while (n_pre < min(n_blk, GROUP) && (b0 + n_pre + 1) * AT_KBLK <= P) { issue_kv(n_pre); ++n_pre; }
+    }
+    pdl_wait();
+  }
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) trace_stamp(TR_k_attn_mma);
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && n_blk > 0) {
-      const uint64_t pol_q = policy_evict_last(), pol_kv = policy_evict_first();
+      const uint64_t pol_q = policy_evict_last();
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
       // queries: box (64 columns, high | low, G heads, 64 / G rows) -> row 2 e + part of the tile
       mbar_expect_tx(q_full, (uint32_t)Sh::Q_BYTES);
       const int node0 = slot * a.rows_per_seq + e_base / a.G;
       for (int kp = 0; kp < KP; ++kp) tma_load_4d(q_s + kp * AT_QTILE, &map_q, q_full, kp * 64, 0, kvh * a.G, node0, pol_q);
-      const int sub_rows = FLAT ? 64 : min(64, a.page_tokens), n_sub = 64 / sub_rows;
-      for (int it = 0; it < n_blk; ++it) {
-        const int st = it % GROUP, use = it / GROUP, j0 = (b0 + it) * AT_KBLK;
+      for (int it = n_pre; it < n_blk; ++it) {
+        const int st = it % GROUP, use = it / GROUP;
         if (use >= 1 && (!mbar_wait(k_empty + st, (uint32_t)(use - 1) & 1u) || !mbar_wait(v_empty + st, (uint32_t)(use - 1) & 1u))) {
           atomicMax(a.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; break;
         }
         if (*abort_flag) break;
-        uint8_t *kd = k_s + st * Sh::KV_STAGE, *vd = v_s + st * Sh::KV_STAGE;
-        mbar_expect_tx(k_full + st, (uint32_t)Sh::KV_STAGE);
-        mbar_expect_tx(v_full + st, (uint32_t)Sh::KV_STAGE);
-        if (FLAT) {
-          // rows of the map: (sequence, K | V, KV head, key); the second coordinate selects the plane
-          const long long rk = (((long long)seq * 2 + 0) * a.hkv + kvh) * a.flat_rows_per_head + j0;
-          const long long rv = (((long long)seq * 2 + 1) * a.hkv + kvh) * a.flat_rows_per_head + j0;
-          for (int pl = 0; pl < PLANES; ++pl)
-            for (int kp = 0; kp < KP; ++kp) {
-              tma_load_3d(kd + (pl * KP + kp) * AT_KVTILE, &map_k, k_full + st, kp * 64, pl, (int)rk, pol_kv);
-              tma_load_3d(vd + (pl * KP + kp) * AT_KVTILE, &map_v, v_full + st, kp * 64, pl, (int)rv, pol_kv);
-            }
-        } else {
-          for (int sb = 0; sb < n_sub; ++sb) {
-            const int j = min(j0 + sb * sub_rows, a.pages_per_seq * a.page_tokens - 1);
-            const int pg = a.page_table[seq * a.pages_per_seq + (j >> a.page_shift)];
-            const int row = (pg * a.hkv + kvh) * a.page_tokens + (j & (a.page_tokens - 1));
-            for (int kp = 0; kp < KP; ++kp) {
-              tma_load_2d(kd + kp * AT_KVTILE + sb * sub_rows * 128, &map_k, k_full + st, kp * 64, row, pol_kv);
-              tma_load_2d(vd + kp * AT_KVTILE + sb * sub_rows * 128, &map_v, v_full + st, kp * 64, row, pol_kv);
-            }
-          }
-        }
+        issue_kv(it);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && n_blk > 0) {
       // fp32 accumulate, bf16 operands, M = 128; S: N = 64, both K-major; O: N = head_dim, B MN-major
-      const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       const uint32_t o_addr = tmem_base, s_addr0 = tmem_base + HD;
       bool ok = mbar_wait(q_full, 0);
       const int n_groups = (n_blk + GROUP - 1) / GROUP;
       for (int gi = 0; gi < n_groups && ok; ++gi) {
         const int gb = gi * GROUP, ge = min(n_blk, gb + GROUP);
-        for (int it = gb; it < ge && ok; ++it) {                       // S_b = Q K_b^T
+        // S = Q K^T for all keys of the group at once: N = 64 x blocks
+        for (int it = gb; it < ge && ok; ++it) {
           const int st = it % GROUP;
-          if (!mbar_wait(k_full + st, (uint32_t)gi & 1u) || (gi >= 1 && !mbar_wait(s_free + st, (uint32_t)(gi - 1) & 1u))) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d = s_addr0 + (uint32_t)st * 64u;
+          if (!mbar_wait(k_full + st, (uint32_t)gi & 1u) || (gi >= 1 && !mbar_wait(s_free + st, (uint32_t)(gi - 1) & 1u))) ok = false;
+        }
+        if (!ok) break;
+        tc_fence_after();
+        {
+          const uint32_t n_keys_g = (uint32_t)(ge - gb) * 64u;
+          const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((n_keys_g >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
           uint32_t acc = 0u;
           for (int pl = 0; pl < PLANES; ++pl)
             for (int kp = 0; kp < KP; ++kp) {
               const uint64_t ad = smem_desc(smem_u32(q_s + kp * AT_QTILE));
-              const uint64_t bd = smem_desc(smem_u32(k_s + st * Sh::KV_STAGE + (pl * KP + kp) * AT_KVTILE));
+              const uint64_t bd = smem_desc(smem_u32(k_s + (pl * KP + kp) * GROUP * AT_KVTILE));
 #pragma unroll
-              for (int k = 0; k < 4; ++k) { mma_bf16(d, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc_s, acc); acc = 1u; }
+              for (int k = 0; k < 4; ++k) { mma_bf16(s_addr0, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc_s, acc); acc = 1u; }
             }
-          mma_commit(k_empty + st);
-          mma_commit(s_full + st);
+          for (int it = gb; it < ge; ++it) { mma_commit(k_empty + it % GROUP); mma_commit(s_full + it % GROUP); }
         }
         for (int it = gb; it < ge && ok; ++it) {                       // O += P_b V_b
           const int st = it % GROUP, pb = it & 1;
@@ -283,21 +312,37 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         }
       }
     }
-    auto visible = [&](int j) -> bool {
-      if (j < vis_end) return true;
-      const int jt = j - tail0;
-      if (a.mode == AT_PREFILL || jt < 0 || jt >= a.tail_len) return false;
-      const uint32_t w = (jt >> 5) == 0 ? mw[0] : (jt >> 5) == 1 ? mw[1] : (jt >> 5) == 2 ? mw[2] : mw[3];
-      return (w >> (jt & 31)) & 1u;
+    // Everything the loops below read sits in registers (the argument block is read through memory),
+    // and the loops are kept small on purpose: the kernel's code is fetched anew at every launch
+    // (the weight stream has pushed it out of L2 by then), so straight-line code costs its fetch.
+    const float scale = a.scale_log2;
+    const int tail_len = a.mode == AT_PREFILL ? 0 : a.tail_len;
+    const unsigned long long mlo = (unsigned long long)mw[0] | ((unsigned long long)mw[1] << 32),
+                             mhi = (unsigned long long)mw[2] | ((unsigned long long)mw[3] << 32);
+    // visibility of the 32 keys j32 .. j32 + 31 as a bit mask
+    auto vis32 = [=](int j32) -> uint32_t {
+      const int npre = min(32, max(0, vis_end - j32));
+      uint32_t m = npre >= 32 ? 0xffffffffu : (1u << npre) - 1u;
+      if (npre < 32 && tail_len > 0) {
+        const int sh = j32 - tail0;                            // tail key index of bit 0
+        unsigned long long t;
+        if (sh < 0) t = sh > -32 ? mlo << (-sh) : 0ull;
+        else if (sh < 64) t = (mlo >> sh) | (sh ? mhi << (64 - sh) : 0ull);
+        else t = sh < 128 ? mhi >> (sh - 64) : 0ull;
+        m |= (uint32_t)t;
+      }
+      return m;
     };
     float m_run = -INFINITY, l_run = 0.f, u_run = 0.f;       // exp2 domain; u = sum p (s - m) for the entropy
     const bool want_ent = a.ent != nullptr;
     bool ok = n_blk > 0;
     const int n_groups = (n_blk + GROUP - 1) / GROUP;
+#pragma unroll 1
     for (int gi = 0; gi < n_groups && ok; ++gi) {
       const int gb = gi * GROUP, ge = min(n_blk, gb + GROUP);
       // ---- first pass: the row maximum over the group's keys
       float gmax = m_run;
+#pragma unroll 1
       for (int it = gb; it < ge && ok; ++it) {
         const int st = it % GROUP, j0 = (b0 + it) * AT_KBLK;
         int w_ok = 1;
@@ -305,19 +350,25 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
         if (!w_ok || *abort_flag) { ok = false; break; }
         tc_fence_after();
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
+#pragma unroll 1
+        for (int ch = 0; ch < 2; ++ch) {
           uint32_t sr[32];
-          tmem_ld32(lane_addr + (uint32_t)(HD + st * 64 + half * 32), sr);
+          tmem_ld32(lane_addr + (uint32_t)(HD + st * 64 + ch * 32), sr);
+          const uint32_t vm = vis32(j0 + ch * 32);
           tmem_ld_wait();
+          // lanes 2e and 2e+1 hold the products of entry e's high and low query parts: the even lane
+          // keeps keys 0..15 of the chunk and the odd lane 16..31, each sends the partner what it needs
+          const uint32_t vmh = vm >> (part * 16);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            float v = __uint_as_float(sr[c]);
-            v += __shfl_xor_sync(0xffffffffu, v, 1);
-            if (visible(j0 + half * 32 + c)) gmax = fmaxf(gmax, v * a.scale_log2);
+          for (int c = 0; c < 16; ++c) {
+            const float send = __uint_as_float(part ? sr[c] : sr[16 + c]);
+            const float mine = __uint_as_float(part ? sr[16 + c] : sr[c]);
+            const float t = (mine + __shfl_xor_sync(0xffffffffu, send, 1)) * scale;
+            gmax = fmaxf(gmax, ((vmh >> c) & 1u) ? t : -INFINITY);
           }
         }
       }
+      gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
       if (!ok) break;
       const float base = gmax == -INFINITY ? 0.f : gmax;
       const float corr = exp2f(m_run - base);                 // 0 when nothing was seen before
@@ -345,6 +396,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       }
       m_run = gmax;
       // ---- second pass: probabilities, row sum, P's high or low part into shared memory
+#pragma unroll 1
       for (int it = gb; it < ge && ok; ++it) {
         const int st = it % GROUP, pb = it & 1, j0 = (b0 + it) * AT_KBLK;
         if ((it >> 1) >= 1) {
@@ -353,32 +405,34 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
           if (!w_ok || *abort_flag) { ok = false; break; }
         }
-        uint8_t *prow = p_s + pb * AT_PTILE + row * 128;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        uint8_t *prow0 = p_s + pb * AT_PTILE;
+#pragma unroll 1
+        for (int ch = 0; ch < 2; ++ch) {
           uint32_t sr[32];
-          tmem_ld32(lane_addr + (uint32_t)(HD + st * 64 + half * 32), sr);
+          tmem_ld32(lane_addr + (uint32_t)(HD + st * 64 + ch * 32), sr);
+          const uint32_t vm = vis32(j0 + ch * 32);
           tmem_ld_wait();
-          uint32_t packed[16];
+          const uint32_t vmh = vm >> (part * 16);
+          uint32_t ph[8], pl2[8];
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            float v0 = __uint_as_float(sr[c]), v1 = __uint_as_float(sr[c + 1]);
-            v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
-            v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-            const float d0 = v0 * a.scale_log2 - base, d1 = v1 * a.scale_log2 - base;
-            const float p0 = visible(j0 + half * 32 + c) ? exp2f(d0) : 0.f, p1 = visible(j0 + half * 32 + c + 1) ? exp2f(d1) : 0.f;
+          for (int c = 0; c < 16; c += 2) {
+            const float s0 = __uint_as_float(part ? sr[c] : sr[16 + c]), s1 = __uint_as_float(part ? sr[c + 1] : sr[17 + c]);
+            const float m0 = __uint_as_float(part ? sr[16 + c] : sr[c]), m1 = __uint_as_float(part ? sr[17 + c] : sr[c + 1]);
+            const float d0 = (m0 + __shfl_xor_sync(0xffffffffu, s0, 1)) * scale - base;
+            const float d1 = (m1 + __shfl_xor_sync(0xffffffffu, s1, 1)) * scale - base;
+            const float p0 = ((vmh >> c) & 1u) ? exp2f(d0) : 0.f, p1 = ((vmh >> (c + 1)) & 1u) ? exp2f(d1) : 0.f;
             l_run += p0 + p1;
             if (want_ent) u_run += (p0 > 0.f ? p0 * d0 : 0.f) + (p1 > 0.f ? p1 * d1 : 0.f);
-            uint32_t hi, lo;
-            split_pair(p0, p1, hi, lo);
-            packed[c >> 1] = part ? lo : hi;
+            split_pair(p0, p1, ph[c >> 1], pl2[c >> 1]);
           }
-          // 16-byte pieces of the row, swizzled like the MMA expects a K-major operand (piece ^ (row & 7))
+          // this lane's 16 keys: high parts into the entry's even row, low parts into its odd row; 16-byte
+          // pieces swizzled like the MMA expects a K-major operand (piece ^ (row & 7))
+          uint8_t *row_hi = prow0 + (row & ~1) * 128, *row_lo = row_hi + 128;
 #pragma unroll
-          for (int pc = 0; pc < 4; ++pc) {
-            const int piece = half * 4 + pc;
-            *reinterpret_cast<uint4 *>(prow + ((piece ^ (row & 7)) << 4)) =
-                make_uint4(packed[pc * 4], packed[pc * 4 + 1], packed[pc * 4 + 2], packed[pc * 4 + 3]);
+          for (int pc = 0; pc < 2; ++pc) {
+            const int piece = ch * 4 + part * 2 + pc;
+            *reinterpret_cast<uint4 *>(row_hi + ((piece ^ (row & 6)) << 4)) = make_uint4(ph[pc * 4], ph[pc * 4 + 1], ph[pc * 4 + 2], ph[pc * 4 + 3]);
+            *reinterpret_cast<uint4 *>(row_lo + ((piece ^ ((row & 6) | 1)) << 4)) = make_uint4(pl2[pc * 4], pl2[pc * 4 + 1], pl2[pc * 4 + 2], pl2[pc * 4 + 3]);
           }
         }
         fence_proxy_async_smem();
@@ -395,6 +449,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       ok = w_ok != 0;
     }
     if (n_blk > 0 && !ok && lane == 0) { atomicMax(a.status, DREAM_DEV_TIMEOUT); *abort_flag = 1; }
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);           // each lane of a pair summed half of the keys
+    u_run += __shfl_xor_sync(0xffffffffu, u_run, 1);
     pdl_trigger();                                            // the keys are done: the kernel that follows may take the SMs
     if (n_blk == 0 || ok) {
       tc_fence_after();

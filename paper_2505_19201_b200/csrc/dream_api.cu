@@ -685,6 +685,18 @@ static long long prefill_chunk_stride(const dream_ctx *c) {
 template <typename T, int HD> struct AttnLaunch {
   // The output rows are laid out per prefill chunk of ROW_CHUNK rows (the O projection's input).
   static void prefill(dream_ctx *c, int layer, int seq, int n) {
+    if (sizeof(T) == 2) {
+      // causal attention of the n prompt rows on the tensor cores: one CTA per (KV head, 64 entries)
+      // walks all keys up to its last row; row log-sum-exp and entropy (Eq. 2) come out of the same pass
+      AttnTcArgs a = {};
+      a.mode = AT_PREFILL;
+      a.n_keys = n; a.lay = xlay(xmode(c, ROW_CHUNK), c->Hhd);
+      a.out_chunk_rows = ROW_CHUNK; a.out_chunk_stride = prefill_chunk_stride(c);
+      a.lse = c->lse_pre; a.ent = c->ent_pre;
+      c->cur_seq[0] = seq;
+      tc(c, a, layer, nullptr, 1, n, 0, nullptr);
+      return;
+    }
     dim3 grid((n + ATT_WARPS * ATT_PF_ROWS - 1) / (ATT_WARPS * ATT_PF_ROWS), c->cfg.n_heads);
     const XMode m = xmode(c, ROW_CHUNK);
     LAUNCH(c, (k_attn_prefill<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n, c->cfg.n_heads,
@@ -737,6 +749,7 @@ template <typename T, int HD> struct AttnLaunch {
     const int want = imin(imin(AM_MAX_CHUNKS, ng), imax(1, c->tc.n_sms / tiles));
     a.blocks_per_chunk = (ng + want - 1) / want * GROUP;
     a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
+    if (a.mode == AT_PREFILL) { a.n_chunks = 1; a.blocks_per_chunk = 1 << 24; }   // a CTA walks every key its rows see
     a.part_o = c->am_part_o; a.part_ml = c->am_part_ml; a.out = c->attn_out; a.status = c->status;
     a.hkv = f.n_kv_heads;
     CUtensorMap mq, mk, mv;

@@ -33,3 +33,21 @@ def test_single_rank_needs_no_process_group():
     import bench
     assert bench.slowest_rank([3.0, 4.0], 1, "cpu") == [3.0, 4.0]
     assert bench.job_value(1, 4, 61, 10.0) == 4 * 61 / 10e-3
+
+
+def test_gpus_flag_without_a_launcher_starts_that_many_ranks(monkeypatch):
+    """`python bench.py --gpus 4` with no WORLD_SIZE in the environment re-launches itself under
+    torch.distributed.run with four ranks on 127.0.0.1 and its own arguments."""
+    sys.path.insert(0, ROOT)
+    import bench
+    seen = {}
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "7"])
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    bench.main()
+    cmd = seen["cmd"]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "7"] and cmd[-5].endswith("bench.py")
+    assert abs(bench.setup_flops(dict(d_model=4, n_heads=1, n_kv_heads=1, head_dim=4, d_ff=8, vocab=10, n_layers=1,
+                                      n_visual=1, n_prompt=1)) - (2 * (48 + 16 + 96) * 2 + 2 * 2 * 4 * 3 + 2 * 40)) < 1e-9
