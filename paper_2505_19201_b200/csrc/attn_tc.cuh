@@ -6,25 +6,33 @@
 // head and one chunk of keys.  Queries carry ~16 mantissa bits as a high and a low bf16 row, so
 // the tile is the MMA's M = 128: row 2e = high part of entry e, row 2e + 1 = its low part; the two
 // accumulator lanes of an entry are added with one shuffle.  Keys are walked in blocks of 64,
-// GROUP blocks at a time:
-//   S_b = Q K_b^T        tcgen05.mma 128 x 64 x 16 steps over head_dim, A = Q and B = K_b from shared
-//                        memory (K-major, 128-byte swizzle, TMA-fed), fp32 accumulators in TMEM;
-//   softmax              four warps, one TMEM lane (row) per thread: a first pass over the group's
-//                        S_b for the row maximum, a second pass for P = 2^(s - m) (masked), the row
-//                        sum, and P's high or low bf16 part written to shared memory in the
-//                        operand layout; between groups the O accumulator is rescaled in TMEM;
-//   O += P_b V_b         tcgen05.mma 128 x head_dim x 16 steps over the block's keys, A = P_b (K-major)
+// GROUP blocks (one group) at a time:
+//   S = Q K^T            one chain of tcgen05.mma 128 x (64 x blocks) x 16 over head_dim for the whole
+//                        group, A = Q and B = K from shared memory (K-major, 128-byte swizzle,
+//                        TMA-fed; the group's K blocks are contiguous), fp32 accumulators in TMEM;
+//   softmax              four warps, one TMEM lane per thread; the two lanes of an entry split each
+//                        32-key piece between them.  A first pass over the group's S for the row
+//                        maximum, a second pass for P = 2^(s - m) (masked) and the row sum; P's high
+//                        bf16 part goes to the entry's even row and its low part to the odd row of a
+//                        shared-memory tile in the operand layout.  Between groups the O accumulator
+//                        is rescaled in TMEM (tcgen05.ld / tcgen05.st);
+//   O += P_b V_b         tcgen05.mma 128 x head_dim x 16 steps over each block's keys, A = P_b (K-major)
 //                        and B = V_b as stored ([key][head_dim]: an MN-major operand).
-// K/V blocks arrive through two TMA rings; flat draft caches carry a low plane per key, which costs
-// one more MMA per step.  A chunk leaves (m, l, O) partials for k_attn_combine, or the finished
-// rows when it is the only chunk.  Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner,
-// 2..5 = softmax and epilogue.  Every mbarrier wait is bounded; on expiry the kernel raises the
+// K/V blocks arrive through two TMA rings; during verification the blocks below the verified prefix
+// length are requested before the grid dependency resolves.  Flat draft caches carry a low plane
+// per key, which costs one more MMA per step.  A chunk leaves (m, l, O) partials for
+// k_attn_combine, or the finished rows (and, for the prefill, each row's log-sum-exp and entropy)
+// when it is the only chunk.  Warp roles: 0 = TMA producer, 1 = MMA issuer and TMEM owner, 2..5 =
+// softmax and epilogue.  The softmax loops are kept compact on purpose: this kernel's code is
+// fetched anew at almost every launch (the weight stream between two launches pushes it out of the
+// caches), and straight-line code then costs its own fetch (a fully unrolled version of the same
+// loops ran four times slower).  Every mbarrier wait is bounded; on expiry the kernel raises the
 // status word and leaves.
 #pragma once
 #include <map>
 #include <vector>
 
-#include "attn_mma.cuh"
+#include "attn_merge.cuh"
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "rows.cuh"
@@ -217,7 +225,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     }
     pdl_wait();
   }
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) trace_stamp(TR_k_attn_mma);
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) trace_stamp(TR_k_attn_tc);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer

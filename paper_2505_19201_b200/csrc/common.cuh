@@ -51,7 +51,7 @@ enum {
   TR_k_colsum,
   TR_k_attn_tree,
   TR_k_attn_draft,
-  TR_k_attn_mma,
+  TR_k_attn_tc,
   TR_k_attn_combine,
   TR_k_draft_begin,
   TR_k_tree_expand,
@@ -75,7 +75,7 @@ enum {
   TR_k_gemm_tc,
   TR_count
 };
-#define DREAM_TRACE_NAMES {"none", "k_embed", "k_build_prompt", "k_resid_norm", "k_qkv_post_target", "k_qkv_post_draft", "k_gemm_to_q", "k_mem_append", "k_silu_mul", "k_resid_add", "k_gather_rows", "k_topk_lse", "k_attn_prefill", "k_entropy_mean", "k_colsum", "k_attn_tree", "k_attn_draft", "k_attn_mma", "k_attn_combine", "k_draft_begin", "k_tree_expand", "k_tree_finalize", "k_verify_setup", "k_accept", "k_compact_kv", "k_accept_rows", "k_select_tap", "k_select_visual", "k_ctx_rows", "k_gemm_simt", "k_iota_rows", "k_set_seq", "k_set_int", "k_first_token", "k_argmax_out", "k_copy_f32", "k_split_rows", "k_gemm_collect", "k_gemm_tc"}
+#define DREAM_TRACE_NAMES {"none", "k_embed", "k_build_prompt", "k_resid_norm", "k_qkv_post_target", "k_qkv_post_draft", "k_gemm_to_q", "k_mem_append", "k_silu_mul", "k_resid_add", "k_gather_rows", "k_topk_lse", "k_attn_prefill", "k_entropy_mean", "k_colsum", "k_attn_tree", "k_attn_draft", "k_attn_tc", "k_attn_combine", "k_draft_begin", "k_tree_expand", "k_tree_finalize", "k_verify_setup", "k_accept", "k_compact_kv", "k_accept_rows", "k_select_tap", "k_select_visual", "k_ctx_rows", "k_gemm_simt", "k_iota_rows", "k_set_seq", "k_set_int", "k_first_token", "k_argmax_out", "k_copy_f32", "k_split_rows", "k_gemm_collect", "k_gemm_tc"}
 __device__ __forceinline__ void trace_stamp(int id) {
   unsigned long long *tr = g_dream_trace;
   if (tr) {

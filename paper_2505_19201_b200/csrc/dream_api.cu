@@ -12,7 +12,7 @@
 
 #include "../../include/dream.h"
 #include "attn.cuh"
-#include "attn_mma.cuh"
+#include "attn_merge.cuh"
 #include "attn_tc.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
@@ -510,14 +510,6 @@ static const char *attn_tc_setup_all() {
   return w ? w : attn_tc_setup<HD, true>();
 }
 
-template <int HD>
-static const char *attn_mma_setup() {
-  if (cudaFuncSetAttribute(k_attn_mma<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_mma_smem<HD, true>()) != cudaSuccess ||
-      cudaFuncSetAttribute(k_attn_mma<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_mma_smem<HD, false>()) != cudaSuccess)
-    return "cannot raise the attention kernel's shared memory limit";
-  return nullptr;
-}
-
 static void free_host_side(dream_ctx *c) {
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   for (int i = 0; i < SNAP_SLOTS; ++i) if (c->snap_ev[i]) cudaEventDestroy(c->snap_ev[i]);
@@ -584,8 +576,7 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
     if (why) { free_host_side(c); return fail(nullptr, DREAM_E_CUDA, "tensor-core GEMM set-up: %s", why); }
   }
   if (c->use_tc) {
-    const char *why = cfg->head_dim == 64 ? attn_mma_setup<64>() : cfg->head_dim == 128 ? attn_mma_setup<128>() : attn_mma_setup<256>();
-    if (!why) why = cfg->head_dim == 64 ? attn_tc_setup_all<64>() : cfg->head_dim == 128 ? attn_tc_setup_all<128>() : attn_tc_setup_all<256>();
+    const char *why = cfg->head_dim == 64 ? attn_tc_setup_all<64>() : cfg->head_dim == 128 ? attn_tc_setup_all<128>() : attn_tc_setup_all<256>();
     if (why) { free_host_side(c); return fail(nullptr, DREAM_E_CUDA, "%s", why); }
   }
   k_rope_table<<<(cfg->head_dim / 2 + 127) / 128, 128, 0, c->stream>>>(c->rope_inv, cfg->head_dim, cfg->rope_theta);
@@ -710,29 +701,6 @@ template <typename T, int HD> struct AttnLaunch {
            c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, c->ent_pre);
     LAUNCH(c, k_colsum_heads, (v + 255) / 256, 256, 0, (const float *)c->ent_pre, c->cfg.n_heads, v, score);
   }
-  // Split-K plan and launch of the tensor-core attention (bf16 configurations).
-  template <bool PAGED>
-  static void mma(dream_ctx *c, AttnMmaArgs a, int B, int rows_per_seq, int key_ub) {
-    const dream_config &f = c->cfg;
-    constexpr int KBLK = AmShape<HD>::KBLK;
-    for (int b = 0; b < DREAM_MAX_BATCH; ++b) a.slot_seq[b] = b < B ? c->cur_seq[b] : 0;
-    a.q = (const bf16 *)c->qbuf; a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq;
-    a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
-    a.n_rt = (rows_per_seq * a.G + AM_ROWS - 1) / AM_ROWS;
-    int nb_ub = imax(1, (key_ub + KBLK - 1) / KBLK), ctas = f.n_kv_heads * a.n_rt * B;
-    // two CTAs fit an SM: as many key chunks as keep the whole grid in one wave
-    int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, 2 * c->tc.n_sms / ctas));
-    a.blocks_per_chunk = (nb_ub + want - 1) / want;
-    a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
-    a.part_o = c->am_part_o; a.part_ml = c->am_part_ml;
-    a.out = c->attn_out;
-    dim3 grid(a.n_chunks, f.n_kv_heads * a.n_rt, B);
-    LAUNCH(c, (k_attn_mma<HD, PAGED>), grid, AM_THREADS, (attn_mma_smem<HD, PAGED>()), a);
-    if (a.n_chunks > 1) {
-      long long items = (long long)B * rows_per_seq * f.n_heads * (HD / 4);
-      LAUNCH(c, (k_attn_combine<HD>), (unsigned)((items + 255) / 256), 256, 0, a, B * rows_per_seq);
-    }
-  }
   // The tcgen05 attention (bf16 configurations): split-K plan, tensor maps, launch, merge of the chunks.
   // cache: null = the paged target cache of `layer`, else a flat draft cache.
   static void tc(dream_ctx *c, AttnTcArgs a, int layer, const float *cache, int B, int rows_per_seq, int key_ub, const int *row_in) {
@@ -782,7 +750,7 @@ template <typename T, int HD> struct AttnLaunch {
     if (e != cudaSuccess && c->launch_err == cudaSuccess) { c->launch_err = e; c->launch_err_name = "k_attn_tc"; }
     c->launches++;
     if (a.n_chunks > 1) {
-      AttnMmaArgs m = {};
+      AttnMergeArgs m = {};
       m.row_in = row_in; m.rows_per_seq = rows_per_seq; m.H = a.H; m.G = a.G; m.n_chunks = a.n_chunks; m.n_rt = a.n_rt;
       m.part_o = a.part_o; m.part_ml = a.part_ml; m.out = a.out; m.lay = a.lay;
       long long items = (long long)B * rows_per_seq * f.n_heads * (HD / 4);
