@@ -711,12 +711,14 @@ template <typename T, int HD> struct AttnLaunch {
     a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq; a.row_in = row_in;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
     a.n_rt = (rows_per_seq * a.G + 63) / 64;
-    const int nb_ub = imax(1, (key_ub + AT_KBLK - 1) / AT_KBLK), ng = (nb_ub + GROUP - 1) / GROUP;
+    const int nb_ub = imax(1, (key_ub + AT_KBLK - 1) / AT_KBLK);
     const int tiles = f.n_kv_heads * a.n_rt * B;
-    // one CTA per SM: as many key chunks (of whole groups) as keep the grid in one wave
-    const int want = imin(imin(AM_MAX_CHUNKS, ng), imax(1, c->tc.n_sms / tiles));
-    a.blocks_per_chunk = (ng + want - 1) / want * GROUP;
+    // one CTA per SM: as many key chunks as keep the grid in one wave, the blocks dealt out evenly
+    // (a chunk walks its blocks GROUP at a time)
+    const int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, c->tc.n_sms / tiles));
+    a.blocks_per_chunk = (nb_ub + want - 1) / want;
     a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
+    (void)GROUP;
     if (a.mode == AT_PREFILL) { a.n_chunks = 1; a.blocks_per_chunk = 1 << 24; }   // a CTA walks every key its rows see
     a.part_o = c->am_part_o; a.part_ml = c->am_part_ml; a.out = c->attn_out; a.status = c->status;
     a.hkv = f.n_kv_heads;
