@@ -58,13 +58,14 @@ class OracleConfig:
     tap_hi: int = 1
     score_include_self: int = 0
     xattn_full_memory: int = 0
+    draft_blocks: int = 1       # 1: one layer (self-attention, cross-attention, MLP); 3: the paper's three blocks
 
     @staticmethod
     def from_preset(p):
         names = ("n_layers d_model n_heads n_kv_heads head_dim d_ff vocab rms_eps rope_theta "
                  "tree_depth tree_topk tree_beam tree_max_nodes tap_mode tap_layer tap_lo tap_hi "
                  "score_include_self xattn_full_memory").split()
-        return OracleConfig(**{k: p[k] for k in names})
+        return OracleConfig(draft_blocks=int(p.get("draft_blocks", 1)), **{k: p[k] for k in names})
 
 
 # --------------------------------------------------------------------------- primitives
@@ -166,6 +167,12 @@ class SeqState:
     mV: torch.Tensor = None
     new_tokens: list = field(default_factory=list)   # tokens verified since the last draft call
     new_pos: list = field(default_factory=list)
+    # three-block draft only: the final block's self-attention rows, and the position of every
+    # permanent row of the draft's caches and of the memory
+    fK: torch.Tensor = None
+    fV: torch.Tensor = None
+    dpos: torch.Tensor = None
+    mpos: torch.Tensor = None
 
 
 class DreamOracle:
@@ -304,6 +311,9 @@ class DreamOracle:
         st.mK = kv[:, :Hkv * hd].reshape(-1, Hkv, hd)
         st.mV = kv[:, Hkv * hd:].reshape(-1, Hkv, hd)
         st.new_tokens, st.new_pos = [], []
+        st.dpos, st.mpos = C.clone(), M.clone()
+        if c.draft_blocks == 3:
+            self._draft3_context(st)
         return kept, sc, margin
 
     # ------------------------------------------------------------------ O6
@@ -320,25 +330,66 @@ class DreamOracle:
         v = qkv[:, (H + Hkv) * hd:].reshape(-1, Hkv, hd)
         return x, q, k, v
 
+    def _draft_catch_up(self, st):
+        """Permanent draft rows of the tokens the last acceptance emitted (all but the pending one)."""
+        if not st.new_tokens:
+            return
+        if self.cfg.draft_blocks == 3:
+            self._draft3_rows(st, self.embed_rows(st.new_tokens), torch.as_tensor(st.new_pos, dtype=torch.long))
+        else:
+            _, _, k, v = self._draft_rows(st, st.new_tokens, st.new_pos)
+            st.dK, st.dV = torch.cat([st.dK, k], 0), torch.cat([st.dV, v], 0)
+        st.new_tokens, st.new_pos = [], []
+
+    @staticmethod
+    def _tree_mask(n_perm, n_tree, rows, anc, strict):
+        """[rows, n_perm + n_tree]: every permanent row, and in the tree region the row's ancestors
+        (and the row itself unless `strict`)."""
+        mask = torch.zeros(len(rows), n_perm + n_tree, dtype=torch.bool)
+        mask[:, :n_perm] = True
+        for i, r in enumerate(rows):
+            mask[i, [n_perm + a for a in anc[i] if not (strict and a == r)]] = True
+        return mask
+
+    def _draft_pass(self, st, tr, rows, toks, pos, anc):
+        """One pass of the single-block draft over the input nodes `rows`: self-attention, Eq. 1,
+        MLP.  Appends the rows' K/V and memory rows to the tree regions `tr`; returns e^M."""
+        c, dw = self.cfg, self.dw
+        H, Hkv, hd = c.n_heads, c.n_kv_heads, c.head_dim
+        nK, nM = st.dK.shape[0], st.mK.shape[0]
+        x, q, k, v = self._draft_rows(st, toks, pos)
+        tr["K"], tr["V"] = torch.cat([tr["K"], k], 0), torch.cat([tr["V"], v], 0)
+        # self-attention: all permanent rows, plus own ancestors and self in the tree region
+        mask = self._tree_mask(nK, tr["K"].shape[0], rows, anc, strict=False)
+        o, _ = attention(q, torch.cat([st.dK, tr["K"]], 0), torch.cat([st.dV, tr["V"]], 0), mask)
+        h = x + linear(o, dw["wo"])
+        # cross-attention: verified memory rows plus strict ancestors' draft features
+        qx = linear(rmsnorm(h, dw["lnx"], c.rms_eps), dw["xq"]).reshape(-1, H, hd)
+        mask = self._tree_mask(nM, tr["mK"].shape[0], rows, anc, strict=True)
+        o, _ = attention(qx, torch.cat([st.mK, tr["mK"]], 0), torch.cat([st.mV, tr["mV"]], 0), mask)
+        h = h + linear(o, dw["xo"])
+        h = h + mlp(rmsnorm(h, dw["ln2"], c.rms_eps), dw["wgu"], dw["wd"], c.d_ff)
+        # e^M: the draft's final feature joins the memory (raw, unnormalised)
+        kv = linear(h, dw["xkv"])
+        tr["mK"] = torch.cat([tr["mK"], kv[:, :Hkv * hd].reshape(-1, Hkv, hd)], 0)
+        tr["mV"] = torch.cat([tr["mV"], kv[:, Hkv * hd:].reshape(-1, Hkv, hd)], 0)
+        return h
+
     def draft_tree(self, st):
         """Expand the draft token tree from the pending token (Section 3.1, tree drafting).
 
         Returns a dict with tokens, parent, depth, mask (list of ancestor-or-self sets),
         cum (cumulative log-probability), and the decision margins met on the way.
         """
-        c, dw = self.cfg, self.dw
-        H, Hkv, hd, D, K = c.n_heads, c.n_kv_heads, c.head_dim, c.tree_depth, c.tree_topk
-        # tokens verified by the last accept get their permanent draft self-attention rows
-        if st.new_tokens:
-            _, _, k, v = self._draft_rows(st, st.new_tokens, st.new_pos)
-            st.dK, st.dV = torch.cat([st.dK, k], 0), torch.cat([st.dV, v], 0)
-            st.new_tokens, st.new_pos = [], []
+        c = self.cfg
+        Hkv, hd, D, K = c.n_kv_heads, c.head_dim, c.tree_depth, c.tree_topk
+        # tokens verified by the last accept get their permanent rows in the draft's caches
+        self._draft_catch_up(st)
         P = st.P
-        nK, nM = st.dK.shape[0], st.mK.shape[0]
-        # input nodes of the draft: each has a row in the tree regions of both caches
+        # input nodes of the draft: each has a row in the tree regions of the draft's caches
         in_tok, in_depth, in_anc, in_cum, in_cand = [st.pending], [0], [[0]], [0.0], [-1]
-        tK = torch.empty(0, Hkv, hd, dtype=self.dtype)
-        tV, tmK, tmV = tK.clone(), tK.clone(), tK.clone()
+        empty = torch.empty(0, Hkv, hd, dtype=self.dtype)
+        tr = {n: empty.clone() for n in ("K", "V", "mK", "mV", "fK", "fV")}   # tree regions
         cands = []            # (token, parent candidate index or -1 for the root, depth, cum)
         margins = []          # decision margins: top-K cut of a row, adjacent gaps, beam cut
         feats, logp_rows = [], []
@@ -348,30 +399,8 @@ class DreamOracle:
             rows = beam
             toks = [in_tok[r] for r in rows]
             pos = [P + in_depth[r] for r in rows]
-            x, q, k, v = self._draft_rows(st, toks, pos)
-            tK, tV = torch.cat([tK, k], 0), torch.cat([tV, v], 0)
-            nt = tK.shape[0]
-            # self-attention: all permanent rows, plus own ancestors and self in the tree region
-            mask = torch.zeros(len(rows), nK + nt, dtype=torch.bool)
-            mask[:, :nK] = True
-            for i, r in enumerate(rows):
-                mask[i, [nK + a for a in in_anc[r]]] = True
-            o, _ = attention(q, torch.cat([st.dK, tK], 0), torch.cat([st.dV, tV], 0), mask)
-            h = x + linear(o, dw["wo"])
-            # cross-attention: verified memory rows plus strict ancestors' draft features
-            qx = linear(rmsnorm(h, dw["lnx"], c.rms_eps), dw["xq"]).reshape(-1, H, hd)
-            ntm = tmK.shape[0]
-            mask = torch.zeros(len(rows), nM + ntm, dtype=torch.bool)
-            mask[:, :nM] = True
-            for i, r in enumerate(rows):
-                mask[i, [nM + a for a in in_anc[r] if a != r]] = True
-            o, _ = attention(qx, torch.cat([st.mK, tmK], 0), torch.cat([st.mV, tmV], 0), mask)
-            h = h + linear(o, dw["xo"])
-            h = h + mlp(rmsnorm(h, dw["ln2"], c.rms_eps), dw["wgu"], dw["wd"], c.d_ff)
-            # e^M: the draft's final feature joins the memory (raw, unnormalised)
-            kv = linear(h, dw["xkv"])
-            tmK = torch.cat([tmK, kv[:, :Hkv * hd].reshape(-1, Hkv, hd)], 0)
-            tmV = torch.cat([tmV, kv[:, Hkv * hd:].reshape(-1, Hkv, hd)], 0)
+            anc = [in_anc[r] for r in rows]
+            h = (self._draft_pass3 if c.draft_blocks == 3 else self._draft_pass)(st, tr, rows, toks, pos, anc)
             logp = torch.log_softmax(self._logits(h), dim=-1)
             new = []
             for i, r in enumerate(rows):
@@ -419,7 +448,95 @@ class DreamOracle:
             mask.append(mask[parent[i]] | {i})
         return dict(tokens=tokens, parent=parent, depth=depth, mask=mask, cum=cum,
                     margins=margins, min_margin=min(margins) if margins else float("inf"),
-                    cands=cands, feats=feats, logp_rows=logp_rows, in_tok=in_tok, in_depth=in_depth)
+                    cands=cands, feats=feats, logp_rows=logp_rows, in_tok=in_tok, in_depth=in_depth,
+                    in_anc=in_anc)
+
+    # ------------------------------------------------------------------ three-block draft (Section 4)
+    # Reading of "an initial decoder block, an intermediate cross-attention block, and a final decoder
+    # block": each block is pre-norm with a gated MLP behind its attention; the initial and the final
+    # block attend causally to the draft's own rows (rotary positions), the intermediate block is Eq. 1.
+    # Weights: initial = ln1, wqkv, wo, i_ln2, i_wgu, i_wd; intermediate = lnx, xq, xkv, xo, ln2, wgu, wd;
+    # final = f_ln1, f_wqkv, f_wo, f_ln2, f_wgu, f_wd.  A row at position p sees, in the self-attention
+    # caches, every row of a position <= p that is on its own path, and in the memory every row of a
+    # position < p on its path (a target feature s_p already encodes the prediction of token p + 1).
+    def _self_block(self, x, pos, Kc, Vc, mask, names):
+        """One decoder block of the draft on rows x; (Kc, Vc) cached rows, the new rows' K/V are
+        appended behind them and mask [m, cached + m] covers both.  Returns (x, k, v)."""
+        c, dw = self.cfg, self.dw
+        ln1, wqkv, wo, ln2, wgu, wd = (dw[n] for n in names)
+        H, Hkv, hd = c.n_heads, c.n_kv_heads, c.head_dim
+        qkv = linear(rmsnorm(x, ln1, c.rms_eps), wqkv)
+        p = torch.as_tensor(pos, dtype=torch.long)
+        q = rope(qkv[:, :H * hd].reshape(-1, H, hd), p, c.rope_theta)
+        k = rope(qkv[:, H * hd:(H + Hkv) * hd].reshape(-1, Hkv, hd), p, c.rope_theta)
+        v = qkv[:, (H + Hkv) * hd:].reshape(-1, Hkv, hd)
+        o, _ = attention(q, torch.cat([Kc, k], 0), torch.cat([Vc, v], 0), mask)
+        x = x + linear(o, wo)
+        x = x + mlp(rmsnorm(x, ln2, c.rms_eps), wgu, wd, c.d_ff)
+        return x, k, v
+
+    def _cross_block(self, x, MK, MV, mask):
+        """The intermediate block: Eq. 1 over the memory rows the mask admits (a row that sees none
+        gets no attention term), then the block's MLP."""
+        c, dw = self.cfg, self.dw
+        H, hd = c.n_heads, c.head_dim
+        q = linear(rmsnorm(x, dw["lnx"], c.rms_eps), dw["xq"]).reshape(-1, H, hd)
+        o = torch.zeros(x.shape[0], H * hd, dtype=x.dtype)
+        live = mask.any(dim=1)
+        if bool(live.any()):
+            ol, _ = attention(q[live], MK, MV, mask[live])
+            o[live] = ol
+        x = x + linear(o, dw["xo"])
+        return x + mlp(rmsnorm(x, dw["ln2"], c.rms_eps), dw["wgu"], dw["wd"], c.d_ff)
+
+    def _draft3_rows(self, st, x, pos):
+        """Permanent rows of the three-block draft for inputs x at ascending positions `pos` (the
+        compressed context at set-up, then the tokens each acceptance emits): the initial block over
+        its cache, Eq. 1 over the memory rows of an earlier position, the final block over its cache.
+        Appends the K/V rows of both self-attention blocks."""
+        m = x.shape[0]
+        seen = torch.cat([torch.ones(m, st.dK.shape[0], dtype=torch.bool),
+                          torch.ones(m, m, dtype=torch.bool).tril()], 1)
+        h, k1, v1 = self._self_block(x, pos, st.dK, st.dV, seen, self.INITIAL)
+        h = self._cross_block(h, st.mK, st.mV, st.mpos[None, :] < pos[:, None])
+        _, k3, v3 = self._self_block(h, pos, st.fK, st.fV, seen, self.FINAL)
+        st.dK, st.dV = torch.cat([st.dK, k1], 0), torch.cat([st.dV, v1], 0)
+        st.fK, st.fV = torch.cat([st.fK, k3], 0), torch.cat([st.fV, v3], 0)
+        st.dpos = torch.cat([st.dpos, pos])
+
+    def _draft3_context(self, st):
+        """Draft prefill over the compressed context C (Section 3.3: the draft works on the reduced
+        sequence): every block's rows for the inputs at C, from empty caches."""
+        c = self.cfg
+        empty = torch.empty(0, c.n_kv_heads, c.head_dim, dtype=self.dtype)
+        st.dK, st.dV, st.fK, st.fV = empty, empty.clone(), empty.clone(), empty.clone()
+        st.dpos = torch.empty(0, dtype=torch.long)
+        self._draft3_rows(st, st.x0[st.ctx_pos], st.ctx_pos)
+
+    def _draft_pass3(self, st, tr, rows, toks, pos, anc):
+        """One pass of the three-block draft over the input nodes `rows`; the tree regions of the
+        two self-attention caches hold ancestors and self, that of the memory strict ancestors."""
+        c, dw = self.cfg, self.dw
+        Hkv, hd = c.n_kv_heads, c.head_dim
+        x = self.embed_rows(toks)
+        m, nt = len(rows), tr["K"].shape[0] + len(rows)
+        mask = self._tree_mask(st.dK.shape[0], nt, rows, anc, strict=False)
+        h, k, v = self._self_block(x, pos, torch.cat([st.dK, tr["K"]], 0), torch.cat([st.dV, tr["V"]], 0),
+                                   mask, self.INITIAL)
+        tr["K"], tr["V"] = torch.cat([tr["K"], k], 0), torch.cat([tr["V"], v], 0)
+        mask = self._tree_mask(st.mK.shape[0], tr["mK"].shape[0], rows, anc, strict=True)
+        h = self._cross_block(h, torch.cat([st.mK, tr["mK"]], 0), torch.cat([st.mV, tr["mV"]], 0), mask)
+        mask = self._tree_mask(st.fK.shape[0], nt, rows, anc, strict=False)
+        h, k, v = self._self_block(h, pos, torch.cat([st.fK, tr["fK"]], 0), torch.cat([st.fV, tr["fV"]], 0),
+                                   mask, self.FINAL)
+        tr["fK"], tr["fV"] = torch.cat([tr["fK"], k], 0), torch.cat([tr["fV"], v], 0)
+        kv = linear(h, dw["xkv"])
+        tr["mK"] = torch.cat([tr["mK"], kv[:, :Hkv * hd].reshape(-1, Hkv, hd)], 0)
+        tr["mV"] = torch.cat([tr["mV"], kv[:, Hkv * hd:].reshape(-1, Hkv, hd)], 0)
+        return h
+
+    INITIAL = ("ln1", "wqkv", "wo", "i_ln2", "i_wgu", "i_wd")
+    FINAL = ("f_ln1", "f_wqkv", "f_wo", "f_ln2", "f_wgu", "f_wd")
 
     # ------------------------------------------------------------------ O7
     def verify_tree(self, st, tree):
@@ -535,6 +652,8 @@ class DreamOracle:
         st.mV = torch.cat([st.mV, kv[:, Hkv * hd:].reshape(-1, Hkv, hd)], 0)
         st.new_tokens = [tree["tokens"][i] for i in path]
         st.new_pos = [P + j for j in range(A1)]
+        if st.mpos is not None:
+            st.mpos = torch.cat([st.mpos, torch.arange(P, P + A1)])
         st.P = P + A1
         st.pending = out_tokens[-1]
         return path

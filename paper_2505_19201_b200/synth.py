@@ -111,15 +111,23 @@ def target_weights(p, seed=0, device="cpu"):
 
 
 def draft_weights(p, seed=0, device="cpu"):
-    """Random-init weights of the one-layer draft (self-attention, cross-attention, MLP)."""
+    """Random-init weights of the draft: one layer (self-attention, cross-attention, MLP), or with
+    draft_blocks = 3 the three blocks of Section 4."""
     dt = torch_dtype(p["dtype"])
     d, H, Hkv, hd, ff = (p[k] for k in ("d_model", "n_heads", "n_kv_heads", "head_dim", "d_ff"))
     one = lambda: torch.ones(d, dtype=dt, device=device)
     nrm = lambda shape, j: normal(shape, 0.02, stream_id(seed, 20, j), dt, device)
-    return {"ln1": one(), "wqkv": nrm(((H + 2 * Hkv) * hd, d), 0), "wo": nrm((d, H * hd), 1),
-            "lnx": one(), "xq": nrm((H * hd, d), 2), "xkv": nrm((2 * Hkv * hd, d), 3),
-            "xo": nrm((d, H * hd), 4),
-            "ln2": one(), "wgu": nrm((2 * ff, d), 5), "wd": nrm((d, ff), 6)}
+    w = {"ln1": one(), "wqkv": nrm(((H + 2 * Hkv) * hd, d), 0), "wo": nrm((d, H * hd), 1),
+         "lnx": one(), "xq": nrm((H * hd, d), 2), "xkv": nrm((2 * Hkv * hd, d), 3),
+         "xo": nrm((d, H * hd), 4),
+         "ln2": one(), "wgu": nrm((2 * ff, d), 5), "wd": nrm((d, ff), 6)}
+    if int(p.get("draft_blocks", 1)) == 3:
+        # the paper's three blocks: the tensors above are the initial block's attention and the
+        # intermediate (cross-attention) block; these are the initial block's MLP and the final block
+        w.update({"i_ln2": one(), "i_wgu": nrm((2 * ff, d), 7), "i_wd": nrm((d, ff), 8),
+                  "f_ln1": one(), "f_wqkv": nrm(((H + 2 * Hkv) * hd, d), 9), "f_wo": nrm((d, H * hd), 10),
+                  "f_ln2": one(), "f_wgu": nrm((2 * ff, d), 11), "f_wd": nrm((d, ff), 12)})
+    return w
 
 
 def request_inputs(p, seq_seed=0, device="cpu"):
