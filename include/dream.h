@@ -68,6 +68,8 @@ typedef struct {
   int32_t tap_mode, tap_layer, tap_lo, tap_hi;   /* 1-based layers; [lo,hi] = entropy search range */
   int32_t score_include_self;    /* 1: a token's attention to itself counts in its importance */
   int32_t xattn_full_memory;     /* 1: cross-attention memory keeps all n prompt positions */
+  int32_t draft_blocks;          /* 0 or 1: one draft layer (self-attention, Eq. 1, MLP); 3: the three
+                                    blocks of Section 4 (initial decoder block, Eq. 1 block, final decoder block) */
 } dream_config;
 
 /* Target weights (device, borrowed).  Arrays of n_layers device pointers live on the HOST. */
@@ -84,11 +86,18 @@ typedef struct {
 } dream_target_weights;
 
 /* Draft weights (device, borrowed): one layer = self-attention, cross-attention, MLP.
- * The draft shares the target's embedding, final norm and LM head. */
+ * The draft shares the target's embedding, final norm and LM head.
+ * With draft_blocks = 3 (Section 4: an initial decoder block, an intermediate cross-attention
+ * block, a final decoder block, each pre-norm with a gated MLP) the first group is the initial
+ * block's attention and i_* its MLP; lnx..xo and ln2, wgu, wd are the intermediate block; f_* is the
+ * final block.  The i_* and f_* pointers are ignored (may be NULL) otherwise. */
 typedef struct {
   const void *ln1, *wqkv, *wo;           /* self-attention, shapes as in the target */
   const void *lnx, *xq, *xkv, *xo;       /* cross-attention (Eq. 1): xq [H hd, d], xkv [2 H_kv hd, d] (K rows then V rows), xo [d, H hd] */
   const void *ln2, *wgu, *wd;            /* fusion MLP */
+  const void *i_ln2, *i_wgu, *i_wd;      /* draft_blocks = 3: MLP of the initial block */
+  const void *f_ln1, *f_wqkv, *f_wo;     /* draft_blocks = 3: self-attention of the final block */
+  const void *f_ln2, *f_wgu, *f_wd;      /* draft_blocks = 3: MLP of the final block */
 } dream_draft_weights;
 
 /* A token tree, caller-allocated DEVICE buffers of capacity tree_nodes = dream_tree_nodes().
@@ -141,16 +150,21 @@ dream_status dream_set_tap(dream_ctx *ctx, int32_t seq, int32_t tap_layer);
 /* Visual-token compression (Section 3.3): importance of visual token j = attention it
  * receives at layer l* summed over query rows and heads; the k highest are kept.  Builds
  * the draft's compressed context (self-attention K/V from input embeddings, cross-attention
- * memory from the tapped features S^{l*}, Eq. 1).  forced_idx (device int32[k], ascending,
- * or NULL) replaces the selection.  Outputs (device, may be NULL): kept_idx int32[k]
- * ascending, scores float[v]. */
+ * memory from the tapped features S^{l*}, Eq. 1).  With draft_blocks = 3 the draft then runs
+ * over the compressed context (the reduced sequence of Section 3.3): a row at position p attends
+ * causally in both decoder blocks and, in the Eq. 1 block, to the memory rows of positions < p;
+ * what stays are the K/V rows of the initial and of the final block.  forced_idx (device
+ * int32[k], ascending, or NULL) replaces the selection.  Outputs (device, may be NULL): kept_idx
+ * int32[k] ascending, scores float[v]. */
 dream_status dream_compress_visual(dream_ctx *ctx, int32_t seq, int32_t k,
                                    const int32_t *forced_idx, int32_t *kept_idx, float *scores);
 
 /* Draft a token tree for each listed sequence (Section 3.1): D passes of the draft layer
  * (self-attention over the draft cache, cross-attention over target features plus the
  * draft's own earlier features, fusion MLP), top-K expansion per pass, beam selection, and
- * a final re-rank to T nodes.  seqs: HOST int32[n_seqs], distinct.  trees: HOST array of
+ * a final re-rank to T nodes.  With draft_blocks = 3 a pass is the three blocks of Section 4, and
+ * the tokens the last acceptance emitted run through them first (with the memory rows of earlier
+ * positions) to leave their K/V rows in both decoder blocks' caches.  seqs: HOST int32[n_seqs], distinct.  trees: HOST array of
  * n_seqs dream_tree structs whose members are DEVICE buffers that receive the trees. */
 dream_status dream_draft_tree(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs,
                               const dream_tree *trees);
@@ -215,7 +229,8 @@ dream_status dream_seq_state(dream_ctx *ctx, int32_t seq, int32_t *verified_len,
  * 1 = target V row, 2 = cross-memory K row (index = memory row), 3 = cross-memory V row,
  * 4 = draft self-attention K row, 5 = draft self-attention V row,
  * 6 = tapped features of tree node `index` from the last verify [d_model],
- * 7 = final hidden state of tree node `index` from the last verify [d_model].
+ * 7 = final hidden state of tree node `index` from the last verify [d_model],
+ * 8 = K row of the draft's final decoder block (draft_blocks = 3), 9 = its V row.
  * dst: HOST float buffer. */
 dream_status dream_debug_read(dream_ctx *ctx, int32_t seq, int32_t what, int32_t layer,
                               int32_t index, float *dst);

@@ -33,7 +33,7 @@ class dream_config(C.Structure):
                [(n, C.c_int32) for n in ("max_batch", "max_seq", "max_prompt", "max_visual", "page_tokens",
                                           "tree_depth", "tree_topk", "tree_beam", "tree_max_nodes",
                                           "tap_mode", "tap_layer", "tap_lo", "tap_hi",
-                                          "score_include_self", "xattn_full_memory")]
+                                          "score_include_self", "xattn_full_memory", "draft_blocks")]
 
 
 class dream_target_weights(C.Structure):
@@ -42,8 +42,12 @@ class dream_target_weights(C.Structure):
                [("ln_f", C.c_void_p), ("lm_head", C.c_void_p)]
 
 
+DRAFT_TENSORS = ("ln1", "wqkv", "wo", "lnx", "xq", "xkv", "xo", "ln2", "wgu", "wd")
+DRAFT_TENSORS_3 = ("i_ln2", "i_wgu", "i_wd", "f_ln1", "f_wqkv", "f_wo", "f_ln2", "f_wgu", "f_wd")   # draft_blocks = 3 only
+
+
 class dream_draft_weights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("ln1", "wqkv", "wo", "lnx", "xq", "xkv", "xo", "ln2", "wgu", "wd")]
+    _fields_ = [(n, C.c_void_p) for n in DRAFT_TENSORS + DRAFT_TENSORS_3]
 
 
 class dream_tree(C.Structure):
@@ -106,6 +110,7 @@ def make_config(p, max_batch=None, max_seq=None, page_tokens=64):
               "tree_topk", "tree_beam", "tree_max_nodes", "tap_mode", "tap_layer", "tap_lo", "tap_hi",
               "score_include_self", "xattn_full_memory"):
         setattr(c, k, int(p[k]))
+    c.draft_blocks = int(p.get("draft_blocks", 1))
     c.dtype = DREAM_BF16 if p["dtype"] == "bf16" else DREAM_F32
     c.rms_eps, c.rope_theta = p["rms_eps"], p["rope_theta"]
     n = p["n_visual"] + p["n_prompt"]
@@ -200,7 +205,8 @@ class Context:
             arr = (C.c_void_p * L)(*(w.data_ptr() for w in tw[name]))
             self._arrs[name] = arr
             setattr(t, name, arr)
-        d = dream_draft_weights(*(dw[n].data_ptr() for n in ("ln1", "wqkv", "wo", "lnx", "xq", "xkv", "xo", "ln2", "wgu", "wd")))
+        d = dream_draft_weights(*(dw[n].data_ptr() for n in DRAFT_TENSORS),
+                                *(dw[n].data_ptr() if n in dw else None for n in DRAFT_TENSORS_3))
         self.arena_bytes = dream_arena_bytes(cfg)
         self.arena = torch.empty(self.arena_bytes + 256, dtype=torch.uint8, device=self.device)
         base = (self.arena.data_ptr() + 255) & ~255
@@ -279,7 +285,7 @@ class Context:
         return P.value, t.value, tap.value
 
     def dream_debug_read(self, seq, what, layer, index):
-        n = self.cfg.n_kv_heads * self.cfg.head_dim if what <= 5 else self.cfg.d_model
+        n = self.cfg.n_kv_heads * self.cfg.head_dim if what <= 5 or what >= 8 else self.cfg.d_model
         out = torch.empty(n, dtype=torch.float32)
         _check(self.h, lib().dream_debug_read(self.h, seq, what, layer, index, C.c_void_p(out.data_ptr())))
         return out

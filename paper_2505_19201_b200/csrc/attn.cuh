@@ -255,11 +255,12 @@ k_attn_tree(const void *__restrict__ qbuf, PagedKV kv, const int *__restrict__ r
 // Draft attention over a flat cache: permanent rows [0, nperm[seq]) are all visible, then
 // tree-region rows nperm + j for each j in the row's ancestor set (self excluded when
 // strict: cross-attention reads the draft features of strict ancestors only, Section 3.1).
-// Rows with row_in < 0 are idle.  grid (ceil(R/8), H).
+// Rows with row_in < 0 are idle, unless row_vis is given and holds v >= 0 for the row: such a row
+// sees the rows [0, v) and nothing else (none at all when v = 0: its output is zero).  grid (ceil(R/8), H).
 template <typename T, int HD>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_draft(const void *__restrict__ qbuf, FlatKV kv, const int *__restrict__ row_seq,
-             const int *__restrict__ row_in, const int *__restrict__ nperm,
+             const int *__restrict__ row_in, const int *__restrict__ row_vis, const int *__restrict__ nperm,
              const unsigned long long *__restrict__ anc, int anc_stride, int strict, int R, int H,
              float scale, T *attn_out, XLayout lay) {
   constexpr int EPL = HD / 32;
@@ -267,9 +268,10 @@ k_attn_draft(const void *__restrict__ qbuf, FlatKV kv, const int *__restrict__ r
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int r = blockIdx.x * ATT_WARPS + w, h = blockIdx.y;
   if (r >= R) return;
-  int in = row_in[r];
-  if (in < 0) return;
-  int seq = row_seq[r], np = nperm[seq];
+  int in = row_in ? row_in[r] : 0;
+  const int rv = row_vis ? row_vis[r] : -1;
+  if (in < 0 && rv < 0) return;
+  int seq = row_seq[r], np = rv >= 0 ? rv : nperm[seq];
   int kvh = h / (H / kv.hkv);
   const float *base = (const float *)kv.base;          // fp32 configurations only
   long long ok = kv.off(seq, 0, kvh, 0), ov = kv.off(seq, 1, kvh, 0);
@@ -284,8 +286,8 @@ k_attn_draft(const void *__restrict__ qbuf, FlatKV kv, const int *__restrict__ r
     RowLoad<EPL, float>::ld(base + ov + (long long)j * HD, lane, v);
     st.template push<false>(dot_lane<EPL>(q, k), v);
   }
-  unsigned long long bits = anc[(long long)seq * anc_stride + in];
-  if (strict) bits &= ~(1ull << in);
+  unsigned long long bits = rv >= 0 ? 0ull : anc[(long long)seq * anc_stride + in];
+  if (strict && rv < 0) bits &= ~(1ull << in);
   while (bits) {
     int j = __ffsll((long long)bits) - 1;
     bits &= bits - 1;
@@ -293,7 +295,7 @@ k_attn_draft(const void *__restrict__ qbuf, FlatKV kv, const int *__restrict__ r
     RowLoad<EPL, float>::ld(base + ov + (long long)(np + j) * HD, lane, v);
     st.template push<false>(dot_lane<EPL>(q, k), v);
   }
-  float inv = 1.f / st.z;
+  float inv = st.z > 0.f ? 1.f / st.z : 0.f;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
     store_split<T>(attn_out + r * lay.row_stride + h * HD + lane * EPL + e, lay.lo_delta, st.acc[e] * inv);

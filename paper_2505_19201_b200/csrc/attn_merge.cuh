@@ -21,7 +21,8 @@ __device__ __forceinline__ void split_pair(float x, float y, uint32_t &hi, uint3
 
 // What the merge kernel needs to know about the partials and the output rows.
 struct AttnMergeArgs {
-  const int *row_in;                // [R] or null: rows with a negative entry are idle
+  const int *row_in;                // [R] or null: rows with a negative entry are idle ...
+  const int *row_vis;               // ... unless this one is given and holds an entry >= 0 for the row
   int rows_per_seq, H, G;           // query rows per sequence slot, query heads, heads per KV head
   int n_chunks, n_rt;               // key chunks, 64-entry tiles per KV head
   float *part_o, *part_ml;          // [slot][chunk][kvh][rt][64][hd], [..][64][2]
@@ -42,7 +43,7 @@ k_attn_combine(AttnMergeArgs a, int R) {
   int c4 = (int)(idx % Q4);
   long long rh = idx / Q4;
   int h = (int)(rh % a.H), r = (int)(rh / a.H);
-  if (a.row_in && a.row_in[r] < 0) return;
+  if (a.row_in && a.row_in[r] < 0 && !(a.row_vis && a.row_vis[r] >= 0)) return;
   const int Hkv = a.H / a.G;
   int slot = r / a.rows_per_seq, node = r - slot * a.rows_per_seq;
   int kvh = h / a.G, rr = node * a.G + (h - kvh * a.G);

@@ -61,6 +61,7 @@ struct AttnTcArgs {
   int slot_seq[DREAM_MAX_BATCH];    // sequence of each grid-z slot
   const int *prefix_len;            // by sequence: keys [0, prefix) are visible to every row (verify, draft)
   const int *row_in;                // [R] or null: rows with a negative entry are idle; index into anc (draft)
+  const int *row_vis;               // [R] or null (draft): an entry >= 0 makes the row see keys [0, entry) and no tail key
   const uint32_t *mask;             // [R][4] visible tail keys (verify)
   const unsigned long long *anc;    // [seq][anc_stride] ancestor-or-self bits over tail keys (draft)
   int anc_stride, strict;
@@ -311,7 +312,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           for (int wd = 0; wd < 4; ++wd) mw[wd] = a.mask[(long long)r * 4 + wd];
         } else {
           const int in = a.row_in ? a.row_in[r] : 0;
-          if (in < 0) r = -1;
+          const int rv = a.row_vis ? a.row_vis[r] : -1;
+          if (rv >= 0) vis_end = rv;
+          else if (in < 0) r = -1;
           else {
             unsigned long long bits = a.anc[(long long)seq * a.anc_stride + in];
             if (a.strict) bits &= ~(1ull << in);

@@ -51,6 +51,8 @@ struct dream_ctx {
   int *page_table, *status;
   SeqDev sd;
   float *dself, *dmem;
+  float *dself2;                       // three-block draft: K/V rows of the final decoder block (else null)
+  bool three;                          // cfg.draft_blocks == 3
   DraftTreeDev dt;
   TreePtrs itree[DREAM_MAX_BATCH];
   RowMeta rm[2];
@@ -243,6 +245,8 @@ static dream_status check_config(const dream_config *c, TreeShape *ts) {
   } else if (c->tap_mode == DREAM_TAP_ENTROPY_MIN || c->tap_mode == DREAM_TAP_ENTROPY_MAX) {
     if (c->tap_lo < 1 || c->tap_hi > c->n_layers || c->tap_lo > c->tap_hi) return fail(nullptr, DREAM_E_ARG, "tap range");
   } else return fail(nullptr, DREAM_E_ARG, "tap_mode");
+  if (c->draft_blocks != 0 && c->draft_blocks != 1 && c->draft_blocks != 3)
+    return fail(nullptr, DREAM_E_ARG, "draft_blocks must be 1 (or 0) or 3");
   return DREAM_OK;
 }
 
@@ -275,6 +279,7 @@ static void derive(dream_ctx *c) {
   c->chunk = f.dtype == DREAM_BF16 ? TC_ROWS_SPLIT_1MMA : ROW_CHUNK;
   c->RM = (imax(ROW_CHUNK, f.max_prompt) + 15) & ~15;
   c->XR = c->RM;
+  c->three = f.draft_blocks == 3;
 }
 
 static size_t carve(dream_ctx *c, char *base) {
@@ -298,6 +303,7 @@ static size_t carve(dream_ctx *c, char *base) {
   size_t flat = (size_t)MB * 2 * f.n_kv_heads * c->cap_rows * f.head_dim;
   c->dself = a.take<float>(flat);
   c->dmem = a.take<float>(flat);
+  c->dself2 = c->three ? a.take<float>(flat) : nullptr;
   c->dt.in_tok = a.take<int>((size_t)MB * NI); c->dt.in_depth = a.take<int>((size_t)MB * NI);
   c->dt.in_cand = a.take<int>((size_t)MB * NI); c->dt.in_cum = a.take<float>((size_t)MB * NI);
   c->dt.in_anc = a.take<unsigned long long>((size_t)MB * NI);
@@ -313,6 +319,7 @@ static size_t carve(dream_ctx *c, char *base) {
   for (int i = 0; i < 2; ++i) {
     c->rm[i].seq = a.take<int>(c->RM); c->rm[i].tok = a.take<int>(c->RM); c->rm[i].pos = a.take<int>(c->RM);
     c->rm[i].slot = a.take<int>(c->RM); c->rm[i].dst = a.take<int>(c->RM); c->rm[i].in = a.take<int>(c->RM);
+    c->rm[i].vis_d = a.take<int>(c->RM); c->rm[i].vis_m = a.take<int>(c->RM);
   }
   c->gather_idx = a.take<int>(c->RM);
   c->ctx_pos = a.take<int>(f.max_prompt);
@@ -538,6 +545,10 @@ extern "C" dream_status dream_init(const dream_config *cfg, const dream_target_w
   const void *dptr[] = {dw->ln1, dw->wqkv, dw->wo, dw->lnx, dw->xq, dw->xkv, dw->xo, dw->ln2, dw->wgu, dw->wd,
                         tw->embed, tw->ln_f, tw->lm_head};
   for (const void *p : dptr) if (!p) { delete c; return fail(nullptr, DREAM_E_ARG, "null weight pointer"); }
+  if (c->three) {
+    const void *d3[] = {dw->i_ln2, dw->i_wgu, dw->i_wd, dw->f_ln1, dw->f_wqkv, dw->f_wo, dw->f_ln2, dw->f_wgu, dw->f_wd};
+    for (const void *p : d3) if (!p) { delete c; return fail(nullptr, DREAM_E_ARG, "draft_blocks = 3: null i_* or f_* weight pointer"); }
+  }
   for (int l = 0; l < cfg->n_layers; ++l) {
     if (!tw->ln1[l] || !tw->wqkv[l] || !tw->wo[l] || !tw->ln2[l] || !tw->wgu[l] || !tw->wd[l]) {
       delete c; return fail(nullptr, DREAM_E_ARG, "null weight pointer in layer %d", l);
@@ -703,12 +714,13 @@ template <typename T, int HD> struct AttnLaunch {
   }
   // The tcgen05 attention (bf16 configurations): split-K plan, tensor maps, launch, merge of the chunks.
   // cache: null = the paged target cache of `layer`, else a flat draft cache.
-  static void tc(dream_ctx *c, AttnTcArgs a, int layer, const float *cache, int B, int rows_per_seq, int key_ub, const int *row_in) {
+  static void tc(dream_ctx *c, AttnTcArgs a, int layer, const float *cache, int B, int rows_per_seq, int key_ub, const int *row_in,
+                 const int *row_vis = nullptr) {
     const dream_config &f = c->cfg;
     const bool flat_kv = cache != nullptr;
     const int GROUP = flat_kv ? AtShape<HD, true>::GROUP : AtShape<HD, false>::GROUP;
     for (int b = 0; b < DREAM_MAX_BATCH; ++b) a.slot_seq[b] = b < B ? c->cur_seq[b] : 0;
-    a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq; a.row_in = row_in;
+    a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads; a.rows_per_seq = rows_per_seq; a.row_in = row_in; a.row_vis = row_vis;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
     a.n_rt = (rows_per_seq * a.G + 63) / 64;
     const int nb_ub = imax(1, (key_ub + AT_KBLK - 1) / AT_KBLK);
@@ -719,7 +731,8 @@ template <typename T, int HD> struct AttnLaunch {
     a.blocks_per_chunk = (nb_ub + want - 1) / want;
     a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
     (void)GROUP;
-    if (a.mode == AT_PREFILL) { a.n_chunks = 1; a.blocks_per_chunk = 1 << 24; }   // a CTA walks every key its rows see
+    // a CTA walks every key its rows see: prefill, and row sets wider than the partials were sized for
+    if (a.mode == AT_PREFILL || a.n_rt > c->am_rt_max) { a.n_chunks = 1; a.blocks_per_chunk = 1 << 24; }
     a.part_o = c->am_part_o; a.part_ml = c->am_part_ml; a.out = c->attn_out; a.status = c->status;
     a.hkv = f.n_kv_heads;
     CUtensorMap mq, mk, mv;
@@ -753,7 +766,7 @@ template <typename T, int HD> struct AttnLaunch {
     c->launches++;
     if (a.n_chunks > 1) {
       AttnMergeArgs m = {};
-      m.row_in = row_in; m.rows_per_seq = rows_per_seq; m.H = a.H; m.G = a.G; m.n_chunks = a.n_chunks; m.n_rt = a.n_rt;
+      m.row_in = row_in; m.row_vis = row_vis; m.rows_per_seq = rows_per_seq; m.H = a.H; m.G = a.G; m.n_chunks = a.n_chunks; m.n_rt = a.n_rt;
       m.part_o = a.part_o; m.part_ml = a.part_ml; m.out = a.out; m.lay = a.lay;
       long long items = (long long)B * rows_per_seq * f.n_heads * (HD / 4);
       LAUNCH(c, (k_attn_combine<HD>), (unsigned)((items + 255) / 256), 256, 0, m, B * rows_per_seq);
@@ -772,18 +785,20 @@ template <typename T, int HD> struct AttnLaunch {
     LAUNCH(c, (k_attn_tree<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
            c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
   }
+  // row_vis: null, or per row the number of leading cache rows a permanent row sees (RowMeta::vis_d / vis_m).
+  // tail: false when no row of the launch reads the tree region (the draft's run over the context).
   static void draft(dream_ctx *c, const RowMeta &rm, float *cache, const int *nperm, int strict, int R, XMode m, int B,
-                    int rows_per_seq, int key_ub) {
+                    int rows_per_seq, int key_ub, const int *row_vis = nullptr, bool tail = true) {
     if (sizeof(T) == 2) {
       AttnTcArgs a = {};
       a.mode = AT_DRAFT;
-      a.prefix_len = nperm; a.anc = c->dt.in_anc; a.anc_stride = c->ts.NI; a.strict = strict; a.tail_len = c->ts.NI;
+      a.prefix_len = nperm; a.anc = c->dt.in_anc; a.anc_stride = c->ts.NI; a.strict = strict; a.tail_len = tail ? c->ts.NI : 0;
       a.lay = xlay(m, c->Hhd);
-      tc(c, a, 0, cache, B, rows_per_seq, key_ub, rm.in);
+      tc(c, a, 0, cache, B, rows_per_seq, key_ub, rm.in, row_vis);
       return;
     }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
-    LAUNCH(c, (k_attn_draft<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, flat(c, cache), rm.seq, rm.in, nperm,
+    LAUNCH(c, (k_attn_draft<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, flat(c, cache), rm.seq, rm.in, row_vis, nperm,
            c->dt.in_anc, c->ts.NI, strict, R, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
   }
 };
@@ -912,6 +927,48 @@ extern "C" dream_status dream_set_tap(dream_ctx *c, int32_t seq, int32_t tap_lay
 
 // ------------------------------------------------------------------------------------- compression
 
+// One pass of the draft over R rows whose inputs sit in c->x (Section 3.1; Section 4 for the three
+// blocks): everything up to the last MLP's down projection, whose output (still to be added to c->x)
+// is returned.  vis: the row set holds permanent rows (context or catch-up rows, RowMeta::vis_d/vis_m).
+// tail: rows of the tree region exist.  context: the rows are the compressed context itself, which
+// needs nothing behind the final block's K/V rows.
+template <typename T>
+static GemmOut draft_rows(dream_ctx *c, const RowMeta &rm, int R, XMode xm, int B, int m, int key_ub, bool vis, bool tail,
+                          bool context, const float2 *rope_tab) {
+  const dream_config &f = c->cfg;
+  const int d = f.d_model;
+  const dream_draft_weights &w = c->dw;
+  const int *vd = vis ? rm.vis_d : nullptr, *vm = vis ? rm.vis_m : nullptr;
+  GemmOut g;
+  norm_rows<T>(c, c->x, NO_GEMM, false, w.ln1, R, xm);
+  g = gemm<T>(c, w.wqkv, c->xn, xm, R, c->qkvN, d);
+  LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv, rope_tab);
+  HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub, vd, tail));
+  g = gemm<T>(c, w.wo, c->attn_out, xm, R, d, c->Hhd);
+  if (c->three) {
+    norm_rows<T>(c, c->x, g, true, w.i_ln2, R, xm);
+    g = mlp_rows<T>(c, w.i_wgu, w.i_wd, R, xm);
+  }
+  norm_rows<T>(c, c->x, g, true, w.lnx, R, xm);
+  g = gemm<T>(c, w.xq, c->xn, xm, R, c->Hhd, d);
+  LAUNCH(c, k_gemm_to_q, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, f.n_heads, f.head_dim, sizeof(T) == 2 ? 1 : 0);
+  HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm, B, m, key_ub, vm, tail));
+  g = gemm<T>(c, w.xo, c->attn_out, xm, R, d, c->Hhd);
+  norm_rows<T>(c, c->x, g, true, w.ln2, R, xm);
+  g = mlp_rows<T>(c, w.wgu, w.wd, R, xm);
+  if (c->three) {
+    norm_rows<T>(c, c->x, g, true, w.f_ln1, R, xm);
+    g = gemm<T>(c, w.f_wqkv, c->xn, xm, R, c->qkvN, d);
+    LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself2), f.n_heads, c->rope_inv, rope_tab);
+    if (context) return g;
+    HD_DISPATCH(c, T, draft(c, rm, c->dself2, c->sd.nperm_d, 0, R, xm, B, m, key_ub, vd, tail));
+    g = gemm<T>(c, w.f_wo, c->attn_out, xm, R, d, c->Hhd);
+    norm_rows<T>(c, c->x, g, true, w.f_ln2, R, xm);
+    g = mlp_rows<T>(c, w.f_wgu, w.f_wd, R, xm);
+  }
+  return g;
+}
+
 template <typename T>
 static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *forced, int *kept, float *scores) {
   const dream_config &f = c->cfg;
@@ -921,9 +978,9 @@ static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *force
   // draft self-attention K/V of the compressed context, from the input embeddings
   const char *wkv = (const char *)c->dw.wqkv + (size_t)c->Hhd * d * c->esz;
   const XMode m1 = xmode(c, 1);
-  for (int r0 = 0; r0 < nc; r0 += CH) {
+  for (int r0 = 0; r0 < nc && !c->three; r0 += CH) {
     int rows = imin(CH, nc - r0);
-    LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, 0, seq, c->rm[0], c->gather_idx, r0);
+    LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, 0, seq, c->rm[0], c->gather_idx, r0, 0);
     LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL, XLayout{d, 0});
     norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, rows, m1);
     GemmOut g = gemm<T>(c, wkv, c->xn, m1, rows, c->kvN, d);
@@ -934,13 +991,27 @@ static dream_status compress_impl(dream_ctx *c, int seq, int k, const int *force
   int nm = f.xattn_full_memory ? n : nc;
   for (int r0 = 0; r0 < nm; r0 += CH) {
     int rows = imin(CH, nm - r0);
-    LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, f.xattn_full_memory, seq, c->rm[0], c->gather_idx, r0);
+    LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, f.xattn_full_memory, seq, c->rm[0], c->gather_idx, r0, 0);
     LAUNCH(c, (k_gather_rows<T>), rows, 256, 0, c->taps_store, c->gather_idx, (T *)c->raw, d, c->sd.tap + seq, c->tap_lo_eff,
            (long long)f.max_prompt * d, xlay(m1, d));
     GemmOut g = gemm<T>(c, c->dw.xkv, c->raw, m1, rows, c->kvN, d);
     LAUNCH(c, k_mem_append, dim3(rows, (c->kvN + 1023) / 1024), 256, 0, g, c->rm[0].seq, c->rm[0].dst, (const int *)nullptr, (const int *)nullptr, 0, flat(c, c->dmem));
   }
   LAUNCH(c, k_set_seq, 1, 32, 0, c->sd, seq, -1, (const int *)nullptr, nc, nm);
+  if (c->three) {
+    // The three-block draft runs over its compressed context (the memory above is complete by now):
+    // a chunk of rows at a time, each row seeing the rows up to itself in the decoder blocks' caches
+    // and the memory rows of earlier positions.  The cache rows behind a chunk are not written yet;
+    // no row of the chunk sees them.
+    c->cur_seq[0] = seq;
+    for (int r0 = 0; r0 < nc; r0 += CH) {
+      int rows = imin(CH, nc - r0);
+      const XMode xm = xmode(c, rows);
+      LAUNCH(c, k_ctx_rows, (rows + 255) / 256, 256, 0, c->ctx_pos + r0, rows, 0, seq, c->rm[0], c->gather_idx, r0, f.xattn_full_memory);
+      LAUNCH(c, (k_gather_rows<float>), rows, 256, 0, c->x0, c->gather_idx, c->x, d, (const int *)nullptr, 0, 0LL, XLayout{d, 0});
+      draft_rows<T>(c, c->rm[0], rows, xm, 1, rows, imax(nc, nm), true, false, true, (const float2 *)nullptr);
+    }
+  }
   return DREAM_OK;
 }
 
@@ -1003,19 +1074,8 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     if (p == 1) LAUNCH(c, k_draft_begin, 1, 32, 0, tb, B, c->sd, c->dt, ts, rm, m, c->cap_rows, c->status);
     LAUNCH(c, (k_embed<T>), dim3(R, (d + 1023) / 1024), 256, 0, (const T *)c->embed, rm.tok, c->x, d, f.vocab, c->status,
            (const int *)rm.pos, (const double *)c->rope_inv, c->rope_tab, f.head_dim / 2);
-    GemmOut g;
-    norm_rows<T>(c, c->x, NO_GEMM, false, c->dw.ln1, R, xm);
-    g = gemm<T>(c, c->dw.wqkv, c->xn, xm, R, c->qkvN, d);
-    LAUNCH(c, k_qkv_post_draft, dim3(R, (c->qkvN / 8 + 255) / 256), 256, 0, g, rm.seq, rm.pos, rm.dst, 0, 1, c->qbuf, flat(c, c->dself), f.n_heads, c->rope_inv, (const float2 *)c->rope_tab);
-    HD_DISPATCH(c, T, draft(c, rm, c->dself, c->sd.nperm_d, 0, R, xm, B, m, key_ub));
-    g = gemm<T>(c, c->dw.wo, c->attn_out, xm, R, d, c->Hhd);
-    norm_rows<T>(c, c->x, g, true, c->dw.lnx, R, xm);
-    g = gemm<T>(c, c->dw.xq, c->xn, xm, R, c->Hhd, d);
-    LAUNCH(c, k_gemm_to_q, dim3(R, (c->Hhd + 1023) / 1024), 256, 0, g, c->qbuf, f.n_heads, f.head_dim, sizeof(T) == 2 ? 1 : 0);
-    HD_DISPATCH(c, T, draft(c, rm, c->dmem, c->sd.nperm_m, 1, R, xm, B, m, key_ub));
-    g = gemm<T>(c, c->dw.xo, c->attn_out, xm, R, d, c->Hhd);
-    norm_rows<T>(c, c->x, g, true, c->dw.ln2, R, xm);
-    g = mlp_rows<T>(c, c->dw.wgu, c->dw.wd, R, xm);
+    // pass 1 of the three-block draft carries the catch-up rows through every block
+    GemmOut g = draft_rows<T>(c, rm, R, xm, B, m, key_ub, c->three && p == 1, true, false, (const float2 *)c->rope_tab);
     // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
     norm_rows<T>(c, c->x, g, true, c->ln_f, R, xm, nullptr, nullptr, nullptr, 0, true);
     g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
@@ -1212,7 +1272,7 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
   const dream_config &f = c->cfg;
   int w = f.n_kv_heads * f.head_dim, d = f.d_model;
   float *tmp = c->gout;     // scratch: idle between calls
-  int count = what <= 5 ? w : d;
+  int count = what <= 5 || what >= 8 ? w : d;
   CUDA_OK(c, cudaStreamSynchronize(c->stream));
   if (what == 0 || what == 1) {
     if (layer < 0 || layer >= f.n_layers || index < 0 || index >= f.max_seq) return fail(c, DREAM_E_ARG, "layer/position out of range");
@@ -1221,9 +1281,10 @@ static dream_status debug_read_impl(dream_ctx *c, int seq, int what, int layer, 
     const T *base = (const T *)c->kv_pool + (size_t)layer * c->layer_stride + (size_t)what * c->kv_stride;
     const T *src = base + (((size_t)pg * f.n_kv_heads) * f.page_tokens + in) * f.head_dim;
     k_read_row<T><<<f.n_kv_heads, 256, 0, c->stream>>>(src, (long long)f.page_tokens * f.head_dim, tmp, f.head_dim, 0);
-  } else if (what >= 2 && what <= 5) {
+  } else if ((what >= 2 && what <= 5) || what == 8 || what == 9) {
     if (index < 0 || index >= c->cap_rows) return fail(c, DREAM_E_ARG, "row out of range");
-    const float *base = what <= 3 ? c->dmem : c->dself;
+    if (what >= 8 && !c->three) return fail(c, DREAM_E_STATE, "no final decoder block: draft_blocks is not 3");
+    const float *base = what <= 3 ? c->dmem : (what <= 5 ? c->dself : c->dself2);
     int kvsel = (what - 2) & 1;
     // a row holds head_dim floats, or head_dim high then head_dim low bf16 parts: 4 bytes per element either way
     const float *src = base + (((size_t)seq * 2 + kvsel) * f.n_kv_heads * c->cap_rows + index) * f.head_dim;

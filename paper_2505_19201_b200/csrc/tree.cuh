@@ -43,6 +43,9 @@ struct DraftTreeDev {
 // Row metadata of the current launch set.
 struct RowMeta {
   int *seq, *tok, *pos, *slot, *dst, *in;
+  // Three-block draft: a row with vis_d >= 0 is a permanent row (context or catch-up): it sees the
+  // first vis_d rows of the self-attention caches and the first vis_m memory rows, nothing else.
+  int *vis_d, *vis_m;
 };
 
 struct TreePtrs {                       // device buffers of one caller-visible tree
@@ -58,6 +61,9 @@ struct TreeBatch { TreePtrs t[DREAM_MAX_BATCH]; int seq[DREAM_MAX_BATCH]; };
 // draft self-attention K/V rows.  One thread per sequence slot b.
 __global__ void k_draft_begin(TreeBatch tb, int B, SeqDev s, DraftTreeDev dt, TreeShape ts,
                               RowMeta rm, int rows_per_seq, int cap_rows, int *status) {
+  // Visibility of the catch-up rows (read by the three-block draft only): catch-up row j sits at
+  // position P_old + j, behind np + j rows of the self-attention caches; the acceptance appended one
+  // memory row per catch-up token, so the memory rows of earlier positions are the first nm - nn + j.
   kernel_entry(TR_k_draft_begin);
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
@@ -71,12 +77,14 @@ __global__ void k_draft_begin(TreeBatch tb, int B, SeqDev s, DraftTreeDev dt, Tr
   for (int j = 0; j < rows_per_seq; ++j) {
     int r = base + j;
     rm.seq[r] = seq;
+    rm.vis_d[r] = -1; rm.vis_m[r] = -1;
     if (j == 0) {
       rm.tok[r] = s.pending[seq]; rm.pos[r] = P; rm.dst[r] = np + nn; rm.in[r] = 0;
     } else if (j - 1 < nn) {
       rm.tok[r] = s.new_tok[seq * (DREAM_MAX_DEPTH + 1) + j - 1];
       rm.pos[r] = s.new_pos[seq * (DREAM_MAX_DEPTH + 1) + j - 1];
       rm.dst[r] = np + j - 1; rm.in[r] = -1;
+      rm.vis_d[r] = np + j; rm.vis_m[r] = max(0, s.nperm_m[seq] - nn + j - 1);
     } else {
       rm.tok[r] = -1; rm.pos[r] = 0; rm.dst[r] = -1; rm.in[r] = -1;
     }
@@ -528,11 +536,14 @@ __global__ void k_select_visual(const float *__restrict__ scores_all, long long 
 
 // Row maps of the context-building GEMMs after compression: row i <-> context position
 // ctx_pos[i] (or position i when the memory keeps every prompt position).
+// mem_all_positions: the memory keeps every prompt position, so a context row at position p has p
+// memory rows of earlier positions; otherwise the memory rows are the context rows themselves.
 __global__ void k_ctx_rows(const int *__restrict__ ctx_pos, int count, int identity, int seq,
-                           RowMeta rm, int *gather_idx, int row0) {
+                           RowMeta rm, int *gather_idx, int row0, int mem_all_positions) {
   kernel_entry(TR_k_ctx_rows);
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
   int p = identity ? row0 + i : ctx_pos[i];
   rm.seq[i] = seq; rm.pos[i] = p; rm.dst[i] = row0 + i; gather_idx[i] = p;
+  rm.in[i] = -1; rm.vis_d[i] = row0 + i + 1; rm.vis_m[i] = mem_all_positions ? p : row0 + i;
 }
