@@ -40,18 +40,22 @@ UNIT = "tokens/s"
 
 
 def step_bytes(p, T, P0):
-    """Algorithmic bytes of one step (weights + KV read), bf16 storage, one-layer draft."""
+    """Algorithmic bytes of one step (weights + KV read), bf16 storage; the draft is one layer, or
+    with draft_blocks = 3 two decoder blocks around the cross-attention block (three caches)."""
     e = 2 if p["dtype"] == "bf16" else 4
     d, H, Hkv, hd, ff, V, L = (p[k] for k in ("d_model", "n_heads", "n_kv_heads", "head_dim", "d_ff", "vocab", "n_layers"))
     Hhd, kvw = H * hd, 2 * Hkv * hd
     layer = (Hhd + kvw) * d + d * Hhd + 3 * d * ff
     head = V * d
+    three = int(p.get("draft_blocks", 1)) == 3
     draft_layer = layer + Hhd * d + kvw * d + d * Hhd      # + cross-attention q, kv, o
+    if three:
+        draft_layer += 3 * d * ff + layer                   # the initial block's MLP, the final block
     kv_tok = L * kvw
     B = p["batch"]
     verify = (L * layer + head) * e + B * P0 * kv_tok * e
     n_ctx = p["n_prompt"] + p["k_visual"]
-    draft_pass = (draft_layer + head) * e + B * 2 * n_ctx * kvw * 4   # draft caches are fp32
+    draft_pass = (draft_layer + head) * e + B * (3 if three else 2) * n_ctx * kvw * 4   # draft caches are fp32
     draft = p["tree_depth"] * draft_pass
     accept = kvw * d * e
     return dict(verify=verify, draft=draft, accept=accept, total=verify + draft + accept,
@@ -144,6 +148,9 @@ def oracle_sample(p, twg, dwg, T, budget_s=12.0, max_steps=8):
     st.K = [rnd(n) for _ in range(p["n_layers"])]
     st.V = [rnd(n) for _ in range(p["n_layers"])]
     st.dK, st.dV, st.mK, st.mV = rnd(nc), rnd(nc), rnd(nc), rnd(nc)
+    if int(p.get("draft_blocks", 1)) == 3:
+        st.fK, st.fV = rnd(nc), rnd(nc)
+        st.dpos, st.mpos = torch.arange(nc), torch.arange(nc)
     t0 = time.perf_counter()
     done = 0
     while done < max_steps and (done == 0 or time.perf_counter() - t0 < budget_s):
@@ -241,6 +248,9 @@ def main():
     ap.add_argument("--chain", action="store_true",
                     help="sweep aid: a chain-shaped draft (one child per node, depth D) instead of the tree")
     ap.add_argument("--batch", type=int, default=0, help="sweep aid: number of sequences per step")
+    ap.add_argument("--draft-blocks", type=int, default=1, choices=(1, 3),
+                    help="3: the draft is an initial decoder block, a cross-attention block and a final decoder "
+                         "block; 1: one layer of self-attention, cross-attention and MLP")
     ap.add_argument("--temp", type=float, default=0.0,
                     help="acceptance by the sampling rule at this temperature (greedy otherwise); the verify "
                          "call then also writes the logits")
@@ -265,6 +275,9 @@ def main():
         p["name"] = "%s[batch=%d]" % (p["name"], args.batch)
     if args.temp > 0:
         p["name"] = "%s[temp=%g]" % (p["name"], args.temp)
+    if args.draft_blocks == 3:
+        p["draft_blocks"] = 3
+        p["name"] = "%s[draft_blocks=3]" % p["name"]
     if args.impl == "reference":
         return run_reference(args, p)
 
