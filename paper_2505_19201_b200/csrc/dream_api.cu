@@ -14,6 +14,7 @@
 #include "attn.cuh"
 #include "attn_merge.cuh"
 #include "attn_tc.cuh"
+#include "colsum_tc.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
@@ -514,7 +515,8 @@ static void refresh_bounds(dream_ctx *c) {
 template <int HD>
 static const char *attn_tc_setup_all() {
   const char *w = attn_tc_setup<HD, false>();
-  return w ? w : attn_tc_setup<HD, true>();
+  if (!w) w = attn_tc_setup<HD, true>();
+  return w ? w : colsum_tc_setup<HD>();
 }
 
 static void free_host_side(dream_ctx *c) {
@@ -708,6 +710,40 @@ template <typename T, int HD> struct AttnLaunch {
     if (v == 0) return;
     // the per-head sums land in the entropy buffer, which is idle between this layer's entropy mean
     // and the next layer's attention ([H][n] floats, v <= n)
+    if (sizeof(T) == 2) {
+      // tensor cores: 128 keys of one head per CTA, the query rows stream past (colsum_tc.cuh)
+      const dream_config &f = c->cfg;
+      ColsumTcArgs a = {};
+      a.seq = seq; a.n = n; a.H = f.n_heads; a.G = f.n_heads / f.n_kv_heads;
+      a.vis_start = vis_start; a.v = v; a.include_self = f.score_include_self;
+      a.key0 = vis_start & ~63;
+      a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+      a.lse = c->lse_pre; a.part = c->ent_pre; a.status = c->status;
+      const PagedKV kv = paged(c, layer);
+      a.page_table = kv.page_table; a.pages_per_seq = kv.pages_per_seq; a.page_tokens = kv.page_tokens; a.page_shift = kv.page_shift;
+      a.hkv = f.n_kv_heads;
+      CUtensorMap mq, mk;
+      bool ok;
+      {
+        const unsigned long long dims[4] = {(unsigned long long)HD, 2ull, (unsigned long long)f.n_heads, (unsigned long long)c->XR};
+        const unsigned long long st[3] = {(unsigned long long)HD * 2, (unsigned long long)HD * 4, (unsigned long long)f.n_heads * HD * 4};
+        const unsigned box[4] = {64u, 1u, 1u, (unsigned)CsShape<HD>::NQ};
+        ok = at_map(&c->tc, &c->at_maps, c->qbuf, 4, dims, st, box, &mq);
+      }
+      {
+        const unsigned long long dims[2] = {(unsigned long long)HD, (unsigned long long)c->n_pages * f.n_kv_heads * f.page_tokens};
+        const unsigned long long st[1] = {(unsigned long long)HD * 2};
+        const unsigned box[2] = {64u, (unsigned)imin(64, f.page_tokens)};
+        ok = ok && at_map(&c->tc, &c->at_maps, kv.base, 2, dims, st, box, &mk);
+      }
+      if (!ok) { c->gemm_failed = 1; return; }
+      const int n_tiles = (vis_start + v - a.key0 + CS_KEYS - 1) / CS_KEYS;
+      cudaError_t e = colsum_tc_launch<HD>(c->stream, c->use_pdl, mq, mk, a, n_tiles);
+      if (e != cudaSuccess && c->launch_err == cudaSuccess) { c->launch_err = e; c->launch_err_name = "k_colsum_tc"; }
+      c->launches++;
+      LAUNCH(c, k_colsum_heads, (v + 255) / 256, 256, 0, (const float *)c->ent_pre, c->cfg.n_heads, v, score);
+      return;
+    }
     LAUNCH(c, (k_colsum<T, HD>), dim3((v + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads), ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), seq, n,
            c->cfg.n_heads, 1.f / sqrtf((float)HD), c->lse_pre, vis_start, v, c->cfg.score_include_self, c->ent_pre);
     LAUNCH(c, k_colsum_heads, (v + 255) / 256, 256, 0, (const float *)c->ent_pre, c->cfg.n_heads, v, score);
