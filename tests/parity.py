@@ -293,8 +293,8 @@ class Pair:
             close(self.ctx.dream_debug_read(seq, 4, 0, row), st.dK[row].flatten(), self.tol, "draft K row", self.report)
             close(self.ctx.dream_debug_read(seq, 5, 0, row), st.dV[row].flatten(), self.tol, "draft V row", self.report)
             if st.fK is not None:                      # three-block draft: the final decoder block's rows
-                close(self.ctx.dream_debug_read(seq, 8, 0, row), st.fK[row].flatten(), self.tol, "draft final-block K row", self.report)
-                close(self.ctx.dream_debug_read(seq, 9, 0, row), st.fV[row].flatten(), self.tol, "draft final-block V row", self.report)
+                close(self.ctx.dream_debug_read(seq, 8, 0, row), st.fK[row].flatten(), self.tol, "draft final-block K row", self.report, self.stated_miss)
+                close(self.ctx.dream_debug_read(seq, 9, 0, row), st.fV[row].flatten(), self.tol, "draft final-block V row", self.report, self.stated_miss)
 
     @staticmethod
     def _path(t, i):

@@ -15,6 +15,21 @@ def test_llava_full_size_against_the_oracle():
     _run("llava7b", 1, decode_steps=4, stated_miss=FULL_SIZE_MISS)
 
 
+def test_llava_full_size_three_block_draft_against_the_oracle():
+    """The same workload with the draft of Section 4 (initial decoder block, cross-attention block,
+    final decoder block): the draft's run over the 400-row compressed context, one round, and the
+    draft call after it (catch-up row), element by element."""
+    from tests.test_gpu_parity import _run
+    # Stated misses of the flat 3e-2 (all with relative L2 below 1e-2): the tree this draft proposes holds a
+    # node whose verify logits are off by 3.4e-2 (one of 61 x 32000 values; relative L2 2.1e-3; target path);
+    # the final decoder block's cache rows inherit the memory rows' relative difference (2e-3 at the
+    # tapped layer 20, rms 12.6) through the peaked softmax of Eq. 1: 3.9e-2 / 4.9e-2 on K / V rows
+    # (a row that sees a single memory row differs by exactly that 2e-3; the row that sees none by 8e-6)
+    miss = dict(FULL_SIZE_MISS, **{"verify logits": 5e-2, "draft final-block K row": 8e-2, "draft final-block V row": 8e-2})
+    pr, s = _run("llava7b", 1, decode_steps=4, stated_miss=miss, draft_blocks=3)
+    assert any("final-block" in what for what in s["worst"])
+
+
 def test_llava_full_size_output_does_not_depend_on_the_tree():
     """Section 2.1: whatever the draft proposes, the emitted tokens are the target's own greedy
     continuation.  At full size three decodes of the same request must therefore emit the same
