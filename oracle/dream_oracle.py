@@ -173,6 +173,9 @@ class SeqState:
     fV: torch.Tensor = None
     dpos: torch.Tensor = None
     mpos: torch.Tensor = None
+    # Eq. 2 kept up to date over the verified sequence: per layer the sum over rows and heads of the
+    # row entropies (fp64), over the P rows verified so far
+    ent_sum: torch.Tensor = None
 
 
 class DreamOracle:
@@ -236,6 +239,7 @@ class DreamOracle:
         pos = torch.arange(n)
         causal = torch.ones(n, n, dtype=torch.bool).tril()
         ent = torch.zeros(c.n_layers, dtype=torch.float64)
+        ent_sum = torch.zeros(c.n_layers, dtype=torch.float64)
         for l in range(c.n_layers):
             x, k, vv, probs = self._block(x, l, pos, None, None, causal, want_probs=True)
             st.K.append(k)
@@ -244,11 +248,13 @@ class DreamOracle:
                     or c.tap_mode == TAP_FIXED and l + 1 == c.tap_layer:
                 st.taps[l + 1] = x.clone()
             ent[l] = row_entropy(probs).to(torch.float64).mean()       # mean over rows and heads
+            ent_sum[l] = row_entropy(probs).to(torch.float64).sum()
             col = probs.sum(dim=0)                                      # sum over heads [n, n]
             if not c.score_include_self:
                 col = col - torch.diag(torch.diagonal(col))
             st.scores[l + 1] = col.sum(dim=0)[vis_start:vis_start + v].clone()
         st.entropy = ent
+        st.ent_sum = ent_sum
         tok, margin = argmax_low(self._logits(x[n - 1:n])[0])
         st.pending = tok
         st.tap, st.tap_margin = self.select_tap(ent)
@@ -554,16 +560,20 @@ class DreamOracle:
         mask[:, :P] = True
         for i in range(T):
             mask[i, [P + j for j in tree["mask"][i]]] = True
-        tailK, tailV, tap_rows = [], [], None
+        tailK, tailV, tap_rows, row_ent = [], [], None, []
         for l in range(c.n_layers):
-            x, k, v, _ = self._block(x, l, pos, st.K[l][:P], st.V[l][:P], mask)
+            x, k, v, probs = self._block(x, l, pos, st.K[l][:P], st.V[l][:P], mask, want_probs=True)
             tailK.append(k); tailV.append(v)
+            # entropy of each tree row's attention distribution, summed over heads: for a node on the
+            # accepted path the distribution is the causal one of its position (it sees the prefix and
+            # its ancestors, which are the accepted tokens before it)
+            row_ent.append(row_entropy(probs).to(torch.float64).sum(dim=0))
             if l + 1 == st.tap:
                 tap_rows = x.clone()
         logits = self._logits(x)
         am, mg = zip(*(argmax_low(logits[i]) for i in range(T)))
         return dict(logits=logits, argmax=list(am), margin=list(mg), tailK=tailK, tailV=tailV,
-                    tap_rows=tap_rows, hidden=x)
+                    tap_rows=tap_rows, hidden=x, row_entropy=row_ent)
 
     # ------------------------------------------------------------------ O8
     @staticmethod
@@ -654,9 +664,21 @@ class DreamOracle:
         st.new_pos = [P + j for j in range(A1)]
         if st.mpos is not None:
             st.mpos = torch.cat([st.mpos, torch.arange(P, P + A1)])
+        if st.ent_sum is not None and "row_entropy" in ver:
+            # Eq. 2 over the longer sequence: only the new rows' entropies are added (Section 3.2,
+            # the selection "during each decoding step")
+            st.ent_sum = st.ent_sum + torch.stack([re[idx].sum() for re in ver["row_entropy"]])
         st.P = P + A1
         st.pending = out_tokens[-1]
         return path
+
+    def layer_entropy(self, st):
+        """AE of Eq. 2 over the P rows verified so far, per layer, and the layer Section 3.2 would
+        select from it now (the draft keeps the layer chosen at prefill: its memory holds that
+        layer's features).  Returns (AE [L], layer, margin)."""
+        ae = st.ent_sum / (self.cfg.n_heads * st.P)
+        layer, margin = self.select_tap(ae)
+        return ae, layer, margin
 
     def step(self, st, tree=None, temp=0.0, uniforms=None):
         """One draft + verify + accept + commit round; `tree` overrides the draft's tree.
