@@ -248,6 +248,9 @@ def main():
     ap.add_argument("--chain", action="store_true",
                     help="sweep aid: a chain-shaped draft (one child per node, depth D) instead of the tree")
     ap.add_argument("--batch", type=int, default=0, help="sweep aid: number of sequences per step")
+    ap.add_argument("--track-entropy", action="store_true",
+                    help="keep the layer entropies of Eq. 2 up to date while decoding (row entropies out of the "
+                         "verify attention, added up by the acceptance)")
     ap.add_argument("--draft-blocks", type=int, default=1, choices=(1, 3),
                     help="3: the draft is an initial decoder block, a cross-attention block and a final decoder "
                          "block; 1: one layer of self-attention, cross-attention and MLP")
@@ -275,6 +278,9 @@ def main():
         p["name"] = "%s[batch=%d]" % (p["name"], args.batch)
     if args.temp > 0:
         p["name"] = "%s[temp=%g]" % (p["name"], args.temp)
+    if args.track_entropy:
+        p["track_entropy"] = 1
+        p["name"] = "%s[track_entropy]" % p["name"]
     if args.draft_blocks == 3:
         p["draft_blocks"] = 3
         p["name"] = "%s[draft_blocks=3]" % p["name"]

@@ -70,6 +70,7 @@ typedef struct {
   int32_t xattn_full_memory;     /* 1: cross-attention memory keeps all n prompt positions */
   int32_t draft_blocks;          /* 0 or 1: one draft layer (self-attention, Eq. 1, MLP); 3: the three
                                     blocks of Section 4 (initial decoder block, Eq. 1 block, final decoder block) */
+  int32_t track_entropy;         /* 1: keep Eq. 2 up to date while decoding (dream_layer_entropy); 0: prefill only */
 } dream_config;
 
 /* Target weights (device, borrowed).  Arrays of n_layers device pointers live on the HOST. */
@@ -223,6 +224,17 @@ dream_status dream_step_host(dream_ctx *ctx, const int32_t *seqs, int32_t n_seqs
  * the bound exact again, so DREAM_E_CAPACITY is only reported when max_seq is really reached. */
 dream_status dream_seq_state(dream_ctx *ctx, int32_t seq, int32_t *verified_len,
                              int32_t *pending_token, int32_t *tap_layer);
+
+/* Eq. 2 over the rows verified so far (Section 3.2 speaks of selecting the layer "during each
+ * decoding step"): with config.track_entropy = 1 the verification also leaves every tree row's
+ * attention entropy per layer and head, and dream_accept adds those of the accepted path to the
+ * per-layer sums of the prefill, so nothing is recomputed.  Outputs (HOST, may be NULL):
+ * layer_entropy float[n_layers] = AE(l) over the verified_len rows; layer_now = the layer
+ * config.tap_mode would select from it now (1-based; the fixed layer for DREAM_TAP_FIXED).  The
+ * draft keeps the layer chosen at prefill (its memory holds that layer's features); this call only
+ * reports.  Synchronises the stream.  DREAM_E_STATE when track_entropy is 0 or the sequence has no
+ * prefill. */
+dream_status dream_layer_entropy(dream_ctx *ctx, int32_t seq, float *layer_entropy, int32_t *layer_now);
 
 /* Debug read-back of internal device buffers for parity tests (synchronises).  what:
  * 0 = target K row [n_kv_heads*head_dim] of (layer, position) as float,

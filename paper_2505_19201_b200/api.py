@@ -33,7 +33,7 @@ class dream_config(C.Structure):
                [(n, C.c_int32) for n in ("max_batch", "max_seq", "max_prompt", "max_visual", "page_tokens",
                                           "tree_depth", "tree_topk", "tree_beam", "tree_max_nodes",
                                           "tap_mode", "tap_layer", "tap_lo", "tap_hi",
-                                          "score_include_self", "xattn_full_memory", "draft_blocks")]
+                                          "score_include_self", "xattn_full_memory", "draft_blocks", "track_entropy")]
 
 
 class dream_target_weights(C.Structure):
@@ -79,6 +79,7 @@ def lib():
             "dream_accept_sample": [vp, i32p, i32, C.POINTER(dream_tree), vp, C.c_float, vp, vp, vp, vp],
             "dream_step_host": [vp, i32p, i32, vp, vp],
             "dream_seq_state": [vp, i32, i32p, i32p, i32p],
+            "dream_layer_entropy": [vp, i32, vp, i32p],
             "dream_debug_read": [vp, i32, i32, i32, i32, vp],
             "dream_seq_reset": [vp, i32],
             "dream_debug_gemm": [vp, vp, vp, i32, i32, i32, i32, vp],
@@ -111,6 +112,7 @@ def make_config(p, max_batch=None, max_seq=None, page_tokens=64):
               "score_include_self", "xattn_full_memory"):
         setattr(c, k, int(p[k]))
     c.draft_blocks = int(p.get("draft_blocks", 1))
+    c.track_entropy = int(p.get("track_entropy", 0))
     c.dtype = DREAM_BF16 if p["dtype"] == "bf16" else DREAM_F32
     c.rms_eps, c.rope_theta = p["rms_eps"], p["rope_theta"]
     n = p["n_visual"] + p["n_prompt"]
@@ -283,6 +285,13 @@ class Context:
         P, t, tap = C.c_int32(), C.c_int32(), C.c_int32()
         _check(self.h, lib().dream_seq_state(self.h, seq, C.byref(P), C.byref(t), C.byref(tap)))
         return P.value, t.value, tap.value
+
+    def dream_layer_entropy(self, seq):
+        """(AE per layer over the rows verified so far [L] float32, the layer that would be selected now)."""
+        ae = torch.empty(self.cfg.n_layers, dtype=torch.float32)
+        layer = C.c_int32()
+        _check(self.h, lib().dream_layer_entropy(self.h, seq, C.c_void_p(ae.data_ptr()), C.byref(layer)))
+        return ae, layer.value
 
     def dream_debug_read(self, seq, what, layer, index):
         n = self.cfg.n_kv_heads * self.cfg.head_dim if what <= 5 or what >= 8 else self.cfg.d_model

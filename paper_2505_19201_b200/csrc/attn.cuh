@@ -146,14 +146,16 @@ k_attn_prefill(const void *__restrict__ qbuf, PagedKV kv, int seq, int n, int H,
 }
 
 // AE(l) = mean over rows and heads of the row entropies (Eq. 2).  One block, fixed order.
-__global__ void k_entropy_mean(const float *__restrict__ ent, int count, float *out) {
+// sum_out (may be null) receives the sum itself: the start of the running form of Eq. 2.
+__global__ void k_entropy_mean(const float *__restrict__ ent, int count, float *out, float *sum_out) {
   __shared__ float sh[33];
   kernel_entry(TR_k_entropy_mean);
   float s = 0.f;
   for (int i = threadIdx.x; i < count; i += blockDim.x) s += ent[i];
   float t = block_sum(s, sh);
-  if (threadIdx.x == 0) *out = t / (float)count;
+  if (threadIdx.x == 0) { *out = t / (float)count; if (sum_out) *sum_out = t; }
 }
+
 
 // Importance of visual token j at this layer (Section 3.3): the attention weight it receives,
 // summed over the later query rows (and its own row when include_self) and over heads.
@@ -210,12 +212,13 @@ __global__ void k_colsum_heads(const float *__restrict__ part, int H, int v, flo
 // Tree-masked verification attention (Section 3.1).  Row r = tree node of sequence
 // row_seq[r]; it sees prefix slots [0, P) and tail slots P + j for every j in its
 // ancestor-or-self bit set.  grid (ceil(R/8), H).
-template <typename T, int HD>
+// row_ent (ENT only): [R][H] entropy of the row's attention distribution.
+template <typename T, int HD, bool ENT>
 __global__ void __launch_bounds__(ATT_WARPS * 32)
 k_attn_tree(const void *__restrict__ qbuf, PagedKV kv, const int *__restrict__ row_seq,
             const int *__restrict__ row_node, const int *__restrict__ P_state,
             const uint32_t *__restrict__ mask, int R, int T_nodes, int H, float scale, T *attn_out,
-            XLayout lay) {
+            XLayout lay, float *row_ent) {
   constexpr int EPL = HD / 32;
   kernel_entry(TR_k_attn_tree);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -234,7 +237,7 @@ k_attn_tree(const void *__restrict__ qbuf, PagedKV kv, const int *__restrict__ r
     long long o = kv.off(seq, j, kvh);
     RowLoad<EPL, T>::ld(Kp + o, lane, k);
     RowLoad<EPL, T>::ld(Vp + o, lane, v);
-    st.template push<false>(dot_lane<EPL>(q, k), v);
+    st.template push<ENT>(dot_lane<EPL>(q, k), v);
   }
   const uint32_t *mr = mask + (long long)r * 4;
   for (int j = 0; j < T_nodes; ++j) {
@@ -242,10 +245,11 @@ k_attn_tree(const void *__restrict__ qbuf, PagedKV kv, const int *__restrict__ r
     long long o = kv.off(seq, P + j, kvh);
     RowLoad<EPL, T>::ld(Kp + o, lane, k);
     RowLoad<EPL, T>::ld(Vp + o, lane, v);
-    st.template push<false>(dot_lane<EPL>(q, k), v);
+    st.template push<ENT>(dot_lane<EPL>(q, k), v);
   }
   (void)row_node;
   float inv = 1.f / st.z;
+  if (ENT && lane == 0) row_ent[(long long)r * H + h] = logf(st.z) - st.u * inv;
 #pragma unroll
   for (int e = 0; e < EPL; ++e)
     store_split<T>(attn_out + r * lay.row_stride + h * HD + lane * EPL + e, lay.lo_delta, st.acc[e] * inv);

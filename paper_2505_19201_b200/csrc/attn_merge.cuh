@@ -26,6 +26,8 @@ struct AttnMergeArgs {
   int rows_per_seq, H, G;           // query rows per sequence slot, query heads, heads per KV head
   int n_chunks, n_rt;               // key chunks, 64-entry tiles per KV head
   float *part_o, *part_ml;          // [slot][chunk][kvh][rt][64][hd], [..][64][2]
+  const float *part_u;              // [..][64] the chunks' u = sum p (s - m) (exp2 domain), with row_ent
+  float *row_ent;                   // [R][H] entropy of each row's attention distribution, or null
   void *out;                        // [R][H*hd] rows in GEMM-input layout
   XLayout lay;
 };
@@ -52,7 +54,8 @@ k_attn_combine(AttnMergeArgs a, int R) {
   const long long p0 = (((long long)slot * a.n_chunks * Hkv + kvh) * a.n_rt + rt) * 64 + lr;
   // chunks in rounds of four: (m, l) pairs and output vectors are fetched together, the running
   // maximum rescales what has been accumulated (same result as a two-pass merge up to rounding)
-  float M = -INFINITY, L = 0.f;
+  float M = -INFINITY, L = 0.f, U = 0.f;
+  const bool want_ent = a.row_ent != nullptr && c4 == 0;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int c0 = 0; c0 < a.n_chunks; c0 += 4) {
     float2 ml[4];
@@ -69,6 +72,8 @@ k_attn_combine(AttnMergeArgs a, int R) {
       if (ml[k].x == -INFINITY) continue;
       float Mn = fmaxf(M, ml[k].x);
       float sc = exp2f(M - Mn), w = exp2f(ml[k].x - Mn);       // exp2(-inf) = 0 on the first live chunk
+      // u relative to the new maximum: sum p' (s - Mn) with p' = p 2^(m - Mn)
+      if (want_ent) U = (L > 0.f ? sc * (U + (M - Mn) * L) : 0.f) + w * (a.part_u[p0 + (long long)(c0 + k) * cstride] + (ml[k].x - Mn) * ml[k].y);
       L = L * sc + ml[k].y * w;
       acc.x = acc.x * sc + o[k].x * w; acc.y = acc.y * sc + o[k].y * w;
       acc.z = acc.z * sc + o[k].z * w; acc.w = acc.w * sc + o[k].w * w;
@@ -76,6 +81,7 @@ k_attn_combine(AttnMergeArgs a, int R) {
     }
   }
   float inv = L > 0.f ? 1.f / L : 0.f;
+  if (want_ent) a.row_ent[(long long)r * a.H + h] = L > 0.f ? logf(L) - U * 0.6931471805599453f * inv : 0.f;
   store_split4<bf16>(reinterpret_cast<bf16 *>(a.out) + r * a.lay.row_stride + h * HD + c4 * 4, a.lay.lo_delta,
                      make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
 }

@@ -75,6 +75,8 @@ struct AttnTcArgs {
   int out_chunk_rows;               // prefill: the output rows are laid out per chunk of this many rows ...
   long long out_chunk_stride;       // ... this many elements apart (0: one chunk)
   float *lse, *ent;                 // prefill: [H][n] row log-sum-exp and entropy, or null
+  float *row_ent;                   // verify: [R][H] entropy of every tree row's attention distribution, or null
+  float *part_u;                    // ... and, with several chunks, the chunks' u = sum p (s - m) beside part_ml
   L2Prefetch next_w;
   // where the K/V blocks live, as rows of the K and V tensor maps
   const int *page_table;            // paged: [max_batch][pages_per_seq]
@@ -345,7 +347,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
       return m;
     };
     float m_run = -INFINITY, l_run = 0.f, u_run = 0.f;       // exp2 domain; u = sum p (s - m) for the entropy
-    const bool want_ent = a.ent != nullptr;
+    const bool want_ent = a.ent != nullptr || a.row_ent != nullptr;
     bool ok = n_blk > 0;
     const int n_groups = (n_blk + GROUP - 1) / GROUP;
 #pragma unroll 1
@@ -500,7 +502,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         }
       }
       if (r >= 0 && part == 0) {
-        if (a.n_chunks > 1) *reinterpret_cast<float2 *>(a.part_ml + pbase * 2) = make_float2(m_run, l_run);
+        if (a.n_chunks > 1) {
+          *reinterpret_cast<float2 *>(a.part_ml + pbase * 2) = make_float2(m_run, l_run);
+          if (a.row_ent) a.part_u[pbase] = u_run;
+        } else if (a.row_ent) {
+          a.row_ent[(long long)r * a.H + h] = l_run > 0.f ? logf(l_run) - u_run * 0.6931471805599453f / l_run : 0.f;
+        }
         if (a.lse) {
           // natural-log units: lse = m ln 2 + ln l;  H = ln l - u ln 2 / l
           const int node = r - slot * a.rows_per_seq;

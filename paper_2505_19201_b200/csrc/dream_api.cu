@@ -65,6 +65,9 @@ struct dream_ctx {
   float *top_val, *lse_rows, *margin_i;
   TopkScratch tks;
   float *am_part_o, *am_part_ml;       // split-K attention partials
+  // track_entropy: the chunks' u beside am_part_ml, every tree row's entropy [layer][ROW_CHUNK][H] from
+  // the last verification, and the per-layer sums over the verified rows [seq][layer]
+  float *am_part_u, *row_ent, *ent_sum;
   int am_rt_max;
   int key_ub0[DREAM_MAX_BATCH];        // permanent rows of the draft caches right after compression
   // Verified lengths as the host knows them.  The device advances P by A + 1 per accept and the host
@@ -248,6 +251,7 @@ static dream_status check_config(const dream_config *c, TreeShape *ts) {
   } else return fail(nullptr, DREAM_E_ARG, "tap_mode");
   if (c->draft_blocks != 0 && c->draft_blocks != 1 && c->draft_blocks != 3)
     return fail(nullptr, DREAM_E_ARG, "draft_blocks must be 1 (or 0) or 3");
+  if (c->track_entropy != 0 && c->track_entropy != 1) return fail(nullptr, DREAM_E_ARG, "track_entropy must be 0 or 1");
   return DREAM_OK;
 }
 
@@ -375,7 +379,10 @@ static size_t carve(dream_ctx *c, char *base) {
     size_t prow = (size_t)MB * AM_MAX_CHUNKS * f.n_kv_heads * c->am_rt_max * AM_ROWS;
     c->am_part_o = a.take<float>(prow * f.head_dim);
     c->am_part_ml = a.take<float>(prow * 2);
-  } else { c->am_part_o = nullptr; c->am_part_ml = nullptr; }
+    c->am_part_u = f.track_entropy ? a.take<float>(prow) : nullptr;
+  } else { c->am_part_o = nullptr; c->am_part_ml = nullptr; c->am_part_u = nullptr; }
+  c->row_ent = f.track_entropy ? a.take<float>((size_t)f.n_layers * ROW_CHUNK * f.n_heads) : nullptr;
+  c->ent_sum = f.track_entropy ? a.take<float>((size_t)MB * f.n_layers) : nullptr;
   // small blocks (1024 columns) while the merge of the blocks' lists stays within 1024 candidates
   c->tk_nv = (f.vocab + 1023) / 1024 * TOPK_MAX <= 1024 ? 4 : 16;
   c->tk_nsplit = (f.vocab + c->tk_nv * TOPK_THREADS - 1) / (c->tk_nv * TOPK_THREADS);
@@ -804,6 +811,7 @@ template <typename T, int HD> struct AttnLaunch {
       AttnMergeArgs m = {};
       m.row_in = row_in; m.row_vis = row_vis; m.rows_per_seq = rows_per_seq; m.H = a.H; m.G = a.G; m.n_chunks = a.n_chunks; m.n_rt = a.n_rt;
       m.part_o = a.part_o; m.part_ml = a.part_ml; m.out = a.out; m.lay = a.lay;
+      m.part_u = a.part_u; m.row_ent = a.row_ent;
       long long items = (long long)B * rows_per_seq * f.n_heads * (HD / 4);
       LAUNCH(c, (k_attn_combine<HD>), (unsigned)((items + 255) / 256), 256, 0, m, B * rows_per_seq);
     }
@@ -814,12 +822,18 @@ template <typename T, int HD> struct AttnLaunch {
       a.mode = AT_VERIFY;
       a.next_w.ptr = (const char *)c->wo[layer]; a.next_w.bytes = (unsigned long long)c->cfg.d_model * c->Hhd * 2;
       a.prefix_len = c->sd.P; a.mask = c->vmask; a.tail_len = c->T; a.lay = xlay(m, c->Hhd);
+      if (c->row_ent) { a.row_ent = c->row_ent + (size_t)layer * ROW_CHUNK * c->cfg.n_heads; a.part_u = c->am_part_u; }
       tc(c, a, layer, nullptr, B, c->T, key_ub, nullptr);
       return;
     }
     dim3 grid((R + ATT_WARPS - 1) / ATT_WARPS, c->cfg.n_heads);
-    LAUNCH(c, (k_attn_tree<T, HD>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
-           c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd));
+    if (c->row_ent)
+      LAUNCH(c, (k_attn_tree<T, HD, true>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
+             c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd),
+             c->row_ent + (size_t)layer * ROW_CHUNK * c->cfg.n_heads);
+    else
+      LAUNCH(c, (k_attn_tree<T, HD, false>), grid, ATT_WARPS * 32, 0, c->qbuf, paged(c, layer), c->rm[0].seq, c->rm[0].in,
+             c->sd.P, c->vmask, R, c->T, c->cfg.n_heads, 1.f / sqrtf((float)HD), (T *)c->attn_out, xlay(m, c->Hhd), (float *)nullptr);
   }
   // row_vis: null, or per row the number of leading cache rows a permanent row sees (RowMeta::vis_d / vis_m).
   // tail: false when no row of the launch reads the tree region (the draft's run over the context).
@@ -895,7 +909,8 @@ static dream_status prefill_impl(dream_ctx *c, int seq, const void *visual, int 
              paged(c, l), f.n_heads, c->rope_inv, (const float2 *)nullptr);
     }
     HD_DISPATCH(c, T, prefill(c, l, seq, n));
-    LAUNCH(c, k_entropy_mean, 1, 1024, 0, c->ent_pre, f.n_heads * n, c->ae + l);
+    LAUNCH(c, k_entropy_mean, 1, 1024, 0, c->ent_pre, f.n_heads * n, c->ae + l,
+           c->ent_sum ? c->ent_sum + (size_t)seq * L + l : (float *)nullptr);
     int cand = l + 1 - c->tap_lo_eff;
     bool is_cand = cand >= 0 && cand < c->n_cand;
     if (is_cand) HD_DISPATCH(c, T, colsum(c, l, seq, n, vis_start, v, c->scores_all + (size_t)cand * imax(f.max_visual, 1)));
@@ -1217,6 +1232,7 @@ static dream_status accept_impl(dream_ctx *c, const TreeBatch &tb, int B, const 
   else if (logits) LAUNCH(c, k_accept_sample<false>, B, 1024, 0, tb, B, c->T, D, f.vocab, c->sd, logits, temp, uniforms, accept_len, out_tokens, comp_src, c->status);
   else LAUNCH(c, k_accept, B, 32, 0, tb, B, c->T, D, c->sd, argmax, accept_len, out_tokens, comp_src);
   LAUNCH(c, (k_compact_kv<T>), dim3(f.n_layers * 2, B), 256, 0, tb, c->sd, c->kv_pool, c->layer_stride, c->kv_stride, paged(c, 0));
+  if (c->ent_sum) LAUNCH(c, k_accept_entropy, B, 64, 0, tb, c->T, f.n_layers, f.n_heads, ROW_CHUNK, c->sd, (const float *)c->row_ent, c->ent_sum);
   LAUNCH(c, k_accept_rows, 1, 32, 0, tb, B, c->T, D, c->sd, c->gather_idx, rm, c->cap_rows - c->ts.NI, c->status);
   const XMode xm = xmode(c, R);
   LAUNCH(c, (k_gather_rows<T>), R, 256, 0, c->tapbuf, c->gather_idx, (T *)c->raw, d, (const int *)nullptr, 0, 0LL, xlay(xm, d));
@@ -1300,6 +1316,35 @@ extern "C" dream_status dream_seq_state(dream_ctx *c, int32_t seq, int32_t *veri
   if (verified_len) *verified_len = P_now;
   if (pending) CUDA_OK(c, cudaMemcpy(pending, c->sd.pending + seq, sizeof(int), cudaMemcpyDeviceToHost));
   if (tap) CUDA_OK(c, cudaMemcpy(tap, c->sd.tap + seq, sizeof(int), cudaMemcpyDeviceToHost));
+  return DREAM_OK;
+}
+
+extern "C" dream_status dream_layer_entropy(dream_ctx *c, int32_t seq, float *layer_entropy, int32_t *layer_now) {
+  dream_status s = check_seq(c, seq);
+  if (s) return s;
+  const dream_config &f = c->cfg;
+  if (!c->ent_sum) return fail(c, DREAM_E_STATE, "config.track_entropy is 0");
+  if (c->phase[seq] == PH_EMPTY) return fail(c, DREAM_E_STATE, "sequence %d has no prefill", seq);
+  std::vector<float> sum(f.n_layers);
+  int P = 0;
+  CUDA_OK(c, cudaStreamSynchronize(c->stream));
+  CUDA_OK(c, cudaMemcpy(sum.data(), c->ent_sum + (size_t)seq * f.n_layers, sizeof(float) * f.n_layers, cudaMemcpyDeviceToHost));
+  CUDA_OK(c, cudaMemcpy(&P, c->sd.P + seq, sizeof(int), cudaMemcpyDeviceToHost));
+  if (P < 1) return fail(c, DREAM_E_STATE, "sequence %d has no verified row", seq);
+  const float denom = (float)f.n_heads * (float)P;
+  for (int l = 0; l < f.n_layers; ++l) sum[l] /= denom;
+  if (layer_entropy) memcpy(layer_entropy, sum.data(), sizeof(float) * f.n_layers);
+  if (layer_now) {
+    int best = f.tap_layer;
+    if (f.tap_mode != DREAM_TAP_FIXED) {
+      best = f.tap_lo;                                         // ties go to the lower layer
+      for (int l = f.tap_lo + 1; l <= f.tap_hi; ++l) {
+        const float a = sum[l - 1], b = sum[best - 1];
+        if (f.tap_mode == DREAM_TAP_ENTROPY_MIN ? a < b : a > b) best = l;
+      }
+    }
+    *layer_now = best;
+  }
   return DREAM_OK;
 }
 

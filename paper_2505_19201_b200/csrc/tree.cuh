@@ -534,6 +534,25 @@ __global__ void k_select_visual(const float *__restrict__ scores_all, long long 
   }
 }
 
+// Eq. 2 over the longer sequence (Section 3.2, "during each decoding step"): the entropies of the
+// rows an acceptance commits (tree nodes path[0..A] of the sequence in batch slot b) are added to
+// the per-layer sums, heads in ascending order inside a row, rows in path order.
+// row_ent [L][rows_cap][H] from the last verification; ent_sum [seq][L].  grid (slots), a thread per layer.
+__global__ void k_accept_entropy(TreeBatch tb, int T, int L, int H, int rows_cap, SeqDev s,
+                                 const float *__restrict__ row_ent, float *ent_sum) {
+  kernel_entry(TR_k_accept);
+  const int b = blockIdx.x, seq = tb.seq[b], A = s.last_A[seq];
+  const int *path = s.path + seq * (DREAM_MAX_DEPTH + 1);
+  for (int l = threadIdx.x; l < L; l += blockDim.x) {
+    float sum = 0.f;
+    for (int j = 0; j <= A; ++j) {
+      const float *e = row_ent + ((long long)l * rows_cap + b * T + path[j]) * H;
+      for (int h = 0; h < H; ++h) sum += e[h];
+    }
+    ent_sum[(long long)seq * L + l] += sum;
+  }
+}
+
 // Row maps of the context-building GEMMs after compression: row i <-> context position
 // ctx_pos[i] (or position i when the memory keeps every prompt position).
 // mem_all_positions: the memory keeps every prompt position, so a context row at position p has p
