@@ -371,6 +371,9 @@ def main():
     verify_us = statistics.median(e[1].elapsed_time(e[2]) for e in evs) * 1e3
     accept_us = statistics.median(e[2].elapsed_time(e[3]) for e in evs) * 1e3
     per_step_ms = [e[0].elapsed_time(e[3]) for e in evs]
+    srt = sorted(per_step_ms)
+    pct = lambda q: srt[min(len(srt) - 1, int(q * len(srt)))]
+    step_ms = dict(median=statistics.median(per_step_ms), p10=pct(0.10), p90=pct(0.90))
     k50 = min(50, len(per_step_ms))
     first_ms, last_ms = statistics.median(per_step_ms[:k50]), statistics.median(per_step_ms[-k50:])
     ctx.dream_poll()
@@ -415,7 +418,7 @@ def main():
                 config=dict(workload=p["name"], batch=B, tree_nodes=T, prefix=P0, parallelism=f"replicas{world}",
                             l2="step working set (weights, %.1f GB) exceeds the 126 MB L2" % (sb["gemm_weights"] / 1e9)),
                 draft_us=draft_us, verify_us=verify_us, accept_us=accept_us,
-                first_steps_ms=first_ms, last_steps_ms=last_ms,
+                step_ms=step_ms, first_steps_ms=first_ms, last_steps_ms=last_ms,
                 setup_ms_per_sequence=statistics.median(setup_ms),
                 setup_tflops=setup_flops(p) / (statistics.median(setup_ms) / 1e3) / 1e12,
                 setup_frac_of_bf16_sustained=(setup_flops(p) / (statistics.median(setup_ms) / 1e3) / 1e12 / pk["bf16_tflops_sustained"]
