@@ -49,7 +49,11 @@ enum { AT_VERIFY = 0, AT_DRAFT = 1, AT_PREFILL = 2 };
 // the 512 TMEM columns (head_dim for O, 64 per S_b) hold.
 template <int HD, bool FLAT> struct AtShape {
   static constexpr int PLANES = FLAT ? 2 : 1;
-  static constexpr int GROUP = HD == 64 ? 4 : (HD == 128 ? (FLAT ? 2 : 4) : (FLAT ? 1 : 2));
+  // head_dim 64 over the paged cache takes three blocks, so that O and S fit 256 TMEM columns and two
+  // CTAs share an SM (98 KB of shared memory each): twice the key chunks in flight per layer
+  static constexpr int GROUP = HD == 64 ? (FLAT ? 4 : 3) : (HD == 128 ? (FLAT ? 2 : 4) : (FLAT ? 1 : 2));
+  static constexpr int TMEM_COLS = HD + GROUP * 64 <= 256 ? 256 : 512;
+  static constexpr int CTAS_PER_SM = HD == 64 && !FLAT ? 2 : 1;
   static constexpr int KP = HD / 64;                                 // 64-column panels per row
   static constexpr int KV_STAGE = PLANES * KP * AT_KVTILE;           // one block of K (or of V)
   static constexpr int Q_BYTES = KP * AT_QTILE;
@@ -129,7 +133,7 @@ __device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr, uint32_t lbo_by
 }
 
 template <int HD, bool FLAT>
-__global__ void __launch_bounds__(AT_THREADS, 1)
+__global__ void __launch_bounds__(AT_THREADS, (AtShape<HD, FLAT>::CTAS_PER_SM))
 k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
           const __grid_constant__ AttnTcArgs a) {
   using Sh = AtShape<HD, FLAT>;
@@ -158,7 +162,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_p)), "r"(512u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_p)), "r"((uint32_t)Sh::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   l2_prefetch_slice(a.next_w, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z), gridDim.x * gridDim.y * gridDim.z);
@@ -522,7 +526,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Sh::TMEM_COLS) : "memory");
   }
 }
 

@@ -768,9 +768,10 @@ template <typename T, int HD> struct AttnLaunch {
     a.n_rt = (rows_per_seq * a.G + 63) / 64;
     const int nb_ub = imax(1, (key_ub + AT_KBLK - 1) / AT_KBLK);
     const int tiles = f.n_kv_heads * a.n_rt * B;
-    // one CTA per SM: as many key chunks as keep the grid in one wave, the blocks dealt out evenly
+    // as many key chunks as keep the grid in one wave of resident CTAs, the blocks dealt out evenly
     // (a chunk walks its blocks GROUP at a time)
-    const int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, c->tc.n_sms / tiles));
+    const int per_sm = flat_kv ? AtShape<HD, true>::CTAS_PER_SM : AtShape<HD, false>::CTAS_PER_SM;
+    const int want = imin(imin(AM_MAX_CHUNKS, nb_ub), imax(1, c->tc.n_sms * per_sm / tiles));
     a.blocks_per_chunk = (nb_ub + want - 1) / want;
     a.n_chunks = (nb_ub + a.blocks_per_chunk - 1) / a.blocks_per_chunk;
     (void)GROUP;
