@@ -56,10 +56,10 @@ def step_bytes(p, T, P0):
     verify = (L * layer + head) * e + B * P0 * kv_tok * e
     n_ctx = p["n_prompt"] + p["k_visual"]
     draft_pass = (draft_layer + head) * e + B * (3 if three else 2) * n_ctx * kvw * 4   # draft caches are fp32
-    draft = p["tree_depth"] * draft_pass
+    draft = p["tree_depth"] * draft_pass - kvw * d * e       # the last pass projects no memory rows (nothing reads them)
     accept = kvw * d * e
     return dict(verify=verify, draft=draft, accept=accept, total=verify + draft + accept,
-                gemm_weights=(L * layer + head + p["tree_depth"] * (draft_layer + head) + kvw * d) * e)
+                gemm_weights=(L * layer + head + p["tree_depth"] * (draft_layer + head)) * e)
 
 
 class ClockSampler:

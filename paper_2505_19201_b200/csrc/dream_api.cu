@@ -1130,8 +1130,10 @@ static dream_status draft_impl(dream_ctx *c, const TreeBatch &tb, int B) {
     GemmOut g = draft_rows<T>(c, rm, R, xm, B, m, key_ub, c->three && p == 1, true, false, (const float2 *)c->rope_tab);
     // e^M = x: the raw copy feeds the memory projection, the normalised copy the LM head
     norm_rows<T>(c, c->x, g, true, c->ln_f, R, xm, nullptr, nullptr, nullptr, 0, true);
-    g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
-    LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
+    if (p < ts.D) {     // the last pass's features have no descendants to attend to them
+      g = gemm<T>(c, c->dw.xkv, c->raw, xm, R, c->kvN, d);
+      LAUNCH(c, k_mem_append, dim3(R, (c->kvN + 1023) / 1024), 256, 0, g, rm.seq, rm.dst, rm.in, c->sd.nperm_m, 0, flat(c, c->dmem));
+    }
     g = gemm<T>(c, c->lm_head, c->xn, xm, R, f.vocab, d);
     TOPK_LAUNCH(c, dim3(R, c->tk_nsplit), g, f.vocab, ts.K, c->tk_nsplit, c->tks, c->top_val, c->top_id, c->lse_rows, (float *)nullptr);
     int next_m = p < ts.D ? ts.beam[p] : 1;
