@@ -95,3 +95,26 @@ def test_two_sequences():
         print(json.dumps(pr.summary(), default=float))
     finally:
         pr.close()
+
+
+def test_chain_shaped_three_block_draft_with_running_entropy_and_sampling():
+    """The options together: one child per node (a chain of depth D), Eq. 2 kept up to date, and an
+    acceptance by the sampling rule at temperature 1 after a greedy one."""
+    import torch
+    from tests.parity import Pair
+    from tests.test_gpu_accept import continuation_tree
+    pr = Pair("llava7b", draft_blocks=3, track_entropy=1, tree_topk=1, tree_beam=1, tree_max_nodes=6,
+              n_layers=2, n_visual=96, k_visual=24, n_prompt=40, decode_steps=8)
+    try:
+        pr.prefill()
+        gen = torch.Generator().manual_seed(5)
+        got = [pr.step(inject={0: continuation_tree(pr, 0, 2)})[0]["A"]]
+        got.append(pr.step(inject={0: continuation_tree(pr, 0, 3)}, temp=1.0, gen=gen)[0]["A"])
+        pr.step()
+        pr.check_draft_cache()
+        ae_g, _ = pr.ctx.dream_layer_entropy(0)
+        ae_o, _, _ = pr.orc.layer_entropy(pr.st[0])
+        assert float((ae_g.double() - ae_o.double()).abs().max()) <= 1e-3
+        print(json.dumps(dict(pr.summary(), accepted=got), default=float))
+    finally:
+        pr.close()
