@@ -51,7 +51,9 @@ template <int HD, bool FLAT> struct AtShape {
   static constexpr int PLANES = FLAT ? 2 : 1;
   // head_dim 64 over the paged cache takes three blocks, so that O and S fit 256 TMEM columns and two
   // CTAs share an SM (98 KB of shared memory each): twice the key chunks in flight per layer
-  static constexpr int GROUP = HD == 64 ? (FLAT ? 4 : 3) : (HD == 128 ? (FLAT ? 2 : 4) : (FLAT ? 1 : 2));
+  // head_dim 128 over the paged cache takes five (231 KB of the 227 KiB a CTA may hold, 448 TMEM columns):
+  // prefixes up to 1280 keys then stay one group per chunk when the sequence is cut four ways
+  static constexpr int GROUP = HD == 64 ? (FLAT ? 4 : 3) : (HD == 128 ? (FLAT ? 2 : 5) : (FLAT ? 1 : 2));
   static constexpr int TMEM_COLS = HD + GROUP * 64 <= 256 ? 256 : 512;
   static constexpr int CTAS_PER_SM = HD == 64 && !FLAT ? 2 : 1;
   static constexpr int KP = HD / 64;                                 // 64-column panels per row
@@ -142,8 +144,8 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   uint8_t *smem = (uint8_t *)(((uintptr_t)at_smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t *q_s = smem, *k_s = q_s + Sh::Q_BYTES, *v_s = k_s + GROUP * Sh::KV_STAGE, *p_s = v_s + GROUP * Sh::KV_STAGE;
   uint64_t *bars = (uint64_t *)(p_s + 2 * AT_PTILE);
-  uint64_t *q_full = bars, *k_full = q_full + 1, *k_empty = k_full + 4, *v_full = k_empty + 4, *v_empty = v_full + 4;
-  uint64_t *s_full = v_empty + 4, *s_free = s_full + 4, *p_full = s_free + 4, *p_empty = p_full + 2, *o_done = p_empty + 2;
+  uint64_t *q_full = bars, *k_full = q_full + 1, *k_empty = k_full + 8, *v_full = k_empty + 8, *v_empty = v_full + 8;
+  uint64_t *s_full = v_empty + 8, *s_free = s_full + 8, *p_full = s_free + 8, *p_empty = p_full + 2, *o_done = p_empty + 2;
   uint32_t *tmem_base_p = (uint32_t *)(o_done + 1);
   volatile int *abort_flag = (volatile int *)(tmem_base_p + 1);
 
@@ -152,7 +154,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const int seq = a.slot_seq[slot];
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int s = 0; s < 4; ++s) {
+    for (int s = 0; s < GROUP; ++s) {
       mbar_init(k_full + s, 1); mbar_init(k_empty + s, 1); mbar_init(v_full + s, 1); mbar_init(v_empty + s, 1);
       mbar_init(s_full + s, 1); mbar_init(s_free + s, 4);
     }
@@ -269,19 +271,20 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         }
         if (!ok) break;
         tc_fence_after();
-        {
-          const uint32_t n_keys_g = (uint32_t)(ge - gb) * 64u;
+        // (an MMA's N ends at 256: a group of five blocks takes a chain of four blocks and one of one)
+        for (int b0 = 0; b0 < ge - gb; b0 += 4) {
+          const uint32_t n_keys_g = (uint32_t)min(4, ge - gb - b0) * 64u;
           const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((n_keys_g >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
           uint32_t acc = 0u;
           for (int pl = 0; pl < PLANES; ++pl)
             for (int kp = 0; kp < KP; ++kp) {
               const uint64_t ad = smem_desc(smem_u32(q_s + kp * AT_QTILE));
-              const uint64_t bd = smem_desc(smem_u32(k_s + (pl * KP + kp) * GROUP * AT_KVTILE));
+              const uint64_t bd = smem_desc(smem_u32(k_s + ((pl * KP + kp) * GROUP + b0) * AT_KVTILE));
 #pragma unroll
-              for (int k = 0; k < 4; ++k) { mma_bf16(s_addr0, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc_s, acc); acc = 1u; }
+              for (int k = 0; k < 4; ++k) { mma_bf16(s_addr0 + (uint32_t)(b0 * 64), ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc_s, acc); acc = 1u; }
             }
-          for (int it = gb; it < ge; ++it) { mma_commit(k_empty + it % GROUP); mma_commit(s_full + it % GROUP); }
         }
+        for (int it = gb; it < ge; ++it) { mma_commit(k_empty + it % GROUP); mma_commit(s_full + it % GROUP); }
         for (int it = gb; it < ge && ok; ++it) {                       // O += P_b V_b
           const int st = it % GROUP, pb = it & 1;
           if (!mbar_wait(p_full + pb, (uint32_t)(it >> 1) & 1u) || !mbar_wait(v_full + st, (uint32_t)gi & 1u)) { ok = false; break; }
