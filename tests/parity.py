@@ -82,7 +82,7 @@ class Pair:
     """One model on both sides: the oracle on the CPU and a library context on the GPU."""
 
     def __init__(self, preset, oracle_dtype=None, device="cuda:0", seed=0, max_batch=None, oracle_kv="bf16",
-                 stated_miss=None, **over):
+                 stated_miss=None, page_tokens=64, **over):
         """oracle_kv: "bf16" = the oracle keeps its target K/V cache as a bf16 store like the GPU
         (the reading of Section 4's "KV caching enabled" for bf16 models); "plain" = the oracle keeps
         K/V in its arithmetic type, which shows how much that reading absorbs.
@@ -99,7 +99,7 @@ class Pair:
                                kv_dtype=torch.bfloat16 if p["dtype"] == "bf16" and oracle_kv == "bf16" else None)
         self.odt = odt
         self.stated_miss = stated_miss or {}
-        self.cfg = api.make_config(p, max_batch=max_batch)
+        self.cfg = api.make_config(p, max_batch=max_batch, page_tokens=page_tokens)
         self.ctx = api.Context(self.cfg, self.twg, self.dwg, device)
         self.T = self.ctx.T
         self.report = dict(exempt=0, decisions=0)

@@ -95,6 +95,16 @@ def test_two_sequences_with_different_prompt_lengths():
         pr.close()
 
 
+@pytest.mark.parametrize("page_tokens", [16, 32, 128, 256])
+@pytest.mark.parametrize("preset", ["toy", "llava7b", "smolvlm2b"])
+def test_page_sizes_of_the_target_cache(preset, page_tokens):
+    """The paged target cache with 16 to 256 tokens per page: a 64-key block of the attention spans
+    four pages or a quarter of one; prefill, importance sums, verification and compaction all
+    address keys through the page table.  The prompt (136 tokens) ends inside a page at every size."""
+    over = {} if preset == "toy" else dict(SMALL, n_layers=2)
+    _run(preset, 2, pair=dict(page_tokens=page_tokens), **over)
+
+
 @pytest.mark.parametrize("preset,over", [("smolvlm2b", {}), ("llava7b", dict(n_layers=4, decode_steps=6))])
 def test_against_the_oracle_without_a_bf16_cache(preset, over):
     """The same GPU run compared with the oracle that keeps K/V in fp32.  The library stores the
