@@ -95,6 +95,27 @@ def test_two_sequences_with_different_prompt_lengths():
         pr.close()
 
 
+def test_model_width_above_8192():
+    """d_model 8448: the residual-norm kernel takes four vectors per thread (two at 4097..8192 columns,
+    one below), the widest form the configuration check admits short of 16384."""
+    _run("llava7b", 1, **dict(SMALL, d_model=8448, n_heads=4, n_kv_heads=2, head_dim=64, d_ff=512, vocab=2048, n_layers=2))
+
+
+def test_eight_sequences_in_one_call():
+    """max_batch = 8 (the most a context holds): the toy tree has 15 nodes, so a verification has 120 rows."""
+    from tests.parity import Pair
+    pr = Pair("toy", max_batch=8)
+    try:
+        for s in range(8):
+            pr.prefill(seq=s, seq_seed=s)
+        for _ in range(3):
+            pr.step(seqs=tuple(range(8)))
+        pr.step(seqs=(7, 2, 5))
+        print(json.dumps(pr.summary(), default=float))
+    finally:
+        pr.close()
+
+
 @pytest.mark.parametrize("page_tokens", [16, 32, 128, 256])
 @pytest.mark.parametrize("preset", ["toy", "llava7b", "smolvlm2b"])
 def test_page_sizes_of_the_target_cache(preset, page_tokens):
