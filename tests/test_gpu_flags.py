@@ -95,6 +95,17 @@ def test_two_sequences_with_different_prompt_lengths():
         pr.close()
 
 
+def test_tree_of_121_rows():
+    """The largest tree the mask words hold is 128 nodes: 120 drafted nodes and the root use all four
+    mask words of a row and two row tiles of the verification attention."""
+    s = _run("llava7b", 2, **dict(SMALL, tree_depth=6, tree_topk=10, tree_beam=10, tree_max_nodes=120))
+
+
+def test_deep_narrow_tree():
+    """Depth 12 with two children per node and a beam of three: 12 draft passes, 37 rows."""
+    s = _run("llava7b", 2, **dict(SMALL, tree_depth=12, tree_topk=2, tree_beam=3, tree_max_nodes=36, decode_steps=30))
+
+
 def test_model_width_above_8192():
     """d_model 8448: the residual-norm kernel takes four vectors per thread (two at 4097..8192 columns,
     one below), the widest form the configuration check admits short of 16384."""
