@@ -56,6 +56,23 @@ def test_configurations_the_kernels_cannot_hold_are_refused():
         raise AssertionError("256 vocabulary blocks x 16 candidates was accepted")
 
 
+def test_draft_shape_and_entropy_switch_are_validated_and_sized():
+    """draft_blocks is 0, 1 or 3 and track_entropy 0 or 1; the three-block draft's second cache and the
+    entropy buffers show in the arena size."""
+    from paper_2505_19201_b200 import api, configs
+    p = configs.scaled("llava7b", n_layers=2)
+    base = api.dream_arena_bytes(api.make_config(p))
+    assert api.dream_arena_bytes(api.make_config(dict(p, draft_blocks=3))) > base
+    assert api.dream_arena_bytes(api.make_config(dict(p, track_entropy=1))) > base
+    for bad in (dict(draft_blocks=2), dict(draft_blocks=-1), dict(track_entropy=2)):
+        try:
+            api.dream_arena_bytes(api.make_config(dict(p, **bad)))
+        except api.DreamError as e:
+            assert e.code == -1, bad
+        else:
+            raise AssertionError(f"{bad} was accepted")
+
+
 def test_tree_from_parents_checks_its_input():
     import ctypes as C
     import torch
