@@ -152,15 +152,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x, kvh = blockIdx.y / a.n_rt, rt = blockIdx.y - kvh * a.n_rt, slot = blockIdx.z;
   const int seq = a.slot_seq[slot];
-  if (threadIdx.x == 0) {
-    mbar_init(q_full, 1);
-    for (int s = 0; s < GROUP; ++s) {
-      mbar_init(k_full + s, 1); mbar_init(k_empty + s, 1); mbar_init(v_full + s, 1); mbar_init(v_empty + s, 1);
-      mbar_init(s_full + s, 1); mbar_init(s_free + s, 4);
-    }
-    for (int s = 0; s < 2; ++s) { mbar_init(p_full + s, 4); mbar_init(p_empty + s, 1); }
-    mbar_init(o_done, 1);
-    *abort_flag = 0;
+  if (warp == 0) {      // a lane per ring stage: the set-up is a few instructions deep instead of a loop
+    if (lane < GROUP) {
+      mbar_init(k_full + lane, 1); mbar_init(k_empty + lane, 1); mbar_init(v_full + lane, 1); mbar_init(v_empty + lane, 1);
+      mbar_init(s_full + lane, 1); mbar_init(s_free + lane, 4);
+    } else if (lane >= 8 && lane < 10) { mbar_init(p_full + lane - 8, 4); mbar_init(p_empty + lane - 8, 1); }
+    else if (lane == 16) { mbar_init(q_full, 1); mbar_init(o_done, 1); *abort_flag = 0; }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {

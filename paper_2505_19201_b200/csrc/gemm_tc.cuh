@@ -153,11 +153,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (blockIdx.x == 0 && threadIdx.x == 0) trace_stamp(TR_none);     // CTA start, before any dependency
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < p.w_stages; ++s) { mbar_init(full_w + s, 1); mbar_init(empty_w + s, 1); }
-    for (int s = 0; s < p.x_stages; ++s) { mbar_init(full_x + s, 1); mbar_init(empty_x + s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 8); }
-    *abort_flag = 0;
+  if (warp == 0) {      // one barrier pair per lane: the set-up is a few instructions deep instead of a loop
+    if (lane < p.w_stages) { mbar_init(full_w + lane, 1); mbar_init(empty_w + lane, 1); }
+    else if (lane >= 8 && lane < 8 + p.x_stages) { mbar_init(full_x + lane - 8, 1); mbar_init(empty_x + lane - 8, 1); }
+    else if (lane >= 16 && lane < 18) { mbar_init(acc_full + lane - 16, 1); mbar_init(acc_empty + lane - 16, 8); }
+    else if (lane == 31) *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {      // all 512 TMEM columns (two accumulators of 256), allocated by one full warp
